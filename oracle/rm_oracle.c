@@ -1,0 +1,309 @@
+/*
+ * CPU oracle for the activation-masked gated MLP of the action expert (the paper's Action Cache compute).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the path computes; it exists so
+ * that the CUDA library can be checked against something written independently from the paper.  Nothing in
+ * the product (the package, its C-ABI library) may include, link or call it.  It shares no code, header,
+ * table or helper with the CUDA sources.
+ *
+ * Conventions (all sizes in elements):
+ *   x      [T,H]  bf16 bit patterns (uint16), the FFN input after RMSNorm (Sec. 4.1, "FFN input after RMSNorm")
+ *   Wg, Wu [I,H]  bf16, row n = gate / up weights of intermediate neuron n
+ *   Wd     [H,I]  bf16, column n = down-projection weights of neuron n
+ *   r      [T,H]  fp32 residual (nullable => 0);  y [T,H] fp32
+ *   idx    [K]    int32, strictly ascending neuron indices (the mask M stored as indices, Sec. 4.1)
+ * Arithmetic: every dot product is accumulated in double and rounded once to fp32, so the result does not
+ * depend on loop order or thread count.  The hidden activation h is kept in fp32 (never rounded to bf16).
+ *
+ * Pins (tests/test_oracle_pins.py): printed GeLU values and the odd-part identity; all-ones mask == the
+ * separately written dense loop; masked == dense with h zeroed outside the set; empty mask returns r
+ * bit-exactly; a pure-Python brute-force loop on tiny shapes; an exact-integer closed form with |g| >= 10
+ * (GeLU-tanh degenerates to ReLU); a library-matmul special case; additivity over disjoint sets; neuron
+ * permutation invariance; linearity in W_down and r; RMSNorm unit RMS and scale invariance; compaction round
+ * trips, top-k order properties and vote identities; Eq. 4 special cases.
+ * Parity unpinned: the L-layer stack (orc_step) has no closed form; it is pinned only as the composition of
+ * pinned single layers and by L=1 equalling the single-layer routine.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static inline float bf16_to_f32(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* round-to-nearest-even fp32 -> bf16 (inputs here are finite) */
+static inline uint16_t f32_to_bf16(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+/* GeLU, tanh form: 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3))).  The paper only says "post-GeGLU
+ * activation" (Eq. 1); the tanh form is the reading fixed by the workload definition. */
+double orc_gelu_tanh(double g) {
+    return 0.5 * g * (1.0 + tanh(0.7978845608028654 * (g + 0.044715 * g * g * g)));
+}
+
+/* One neuron's hidden activation for one token: h = gelu_tanh(g) * u with g = <x_t, Wg_n>, u = <x_t, Wu_n>
+ * (Sec. 4.1: "compute only the selected neurons' hidden activations").  g and u are rounded to fp32 once,
+ * the activation is evaluated in double on those, and h is rounded to fp32 once. */
+static float hidden_one(const uint16_t* xt, const uint16_t* wg, const uint16_t* wu, int H) {
+    double g = 0.0, u = 0.0;
+    for (int k = 0; k < H; ++k) {
+        double xv = (double)bf16_to_f32(xt[k]);
+        g += xv * (double)bf16_to_f32(wg[k]);
+        u += xv * (double)bf16_to_f32(wu[k]);
+    }
+    float gf = (float)g, uf = (float)u;
+    return (float)(orc_gelu_tanh((double)gf) * (double)uf);
+}
+
+/* Masked gated MLP, zero-fill form: y = r + W_down[:,S] (act(W_gate[S,:] x) * W_up[S,:] x).
+ * h_out (nullable) receives the compact activations [T,K], column j = neuron idx[j]. */
+void orc_masked_mlp(const uint16_t* x, const uint16_t* Wg, const uint16_t* Wu, const uint16_t* Wd,
+                    const float* r, const int32_t* idx, int K, int T, int H, int I, float* y, float* h_out) {
+    float* h = (float*)malloc(sizeof(float) * (size_t)(T > 0 ? T : 1) * (size_t)(K > 0 ? K : 1));
+#pragma omp parallel for schedule(static)
+    for (int j = 0; j < K; ++j) {
+        size_t n = (size_t)idx[j];
+        for (int t = 0; t < T; ++t)
+            h[(size_t)t * K + j] = hidden_one(x + (size_t)t * H, Wg + n * H, Wu + n * H, H);
+    }
+#pragma omp parallel for schedule(static)
+    for (int c = 0; c < H; ++c) {
+        for (int t = 0; t < T; ++t) {
+            double acc = 0.0;
+            for (int j = 0; j < K; ++j)
+                acc += (double)h[(size_t)t * K + j] * (double)bf16_to_f32(Wd[(size_t)c * I + (size_t)idx[j]]);
+            double base = r ? (double)r[(size_t)t * H + c] : 0.0;
+            y[(size_t)t * H + c] = (float)(base + acc);
+        }
+    }
+    if (h_out) memcpy(h_out, h, sizeof(float) * (size_t)T * (size_t)K);
+    free(h);
+}
+
+/* Dense gated MLP over all I neurons, written as its own loop nest (it does not call the masked routine), with
+ * the optional activation record of Eq. 1: A[n] = sum_t |h[t,n]|, times scale[n] when a scale is given
+ * (scale[n] = ||W_down[:,n]||_2 reproduces Eq. 1).  h_out (nullable) is [T,I]. */
+void orc_dense_mlp(const uint16_t* x, const uint16_t* Wg, const uint16_t* Wu, const uint16_t* Wd,
+                   const float* r, int T, int H, int I, float* y, float* h_out, float* record,
+                   const float* scale) {
+    float* h = (float*)malloc(sizeof(float) * (size_t)(T > 0 ? T : 1) * (size_t)I);
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < I; ++n) {
+        double a = 0.0;
+        for (int t = 0; t < T; ++t) {
+            float hv = hidden_one(x + (size_t)t * H, Wg + (size_t)n * H, Wu + (size_t)n * H, H);
+            h[(size_t)t * I + n] = hv;
+            a += fabs((double)hv);
+        }
+        if (record) {
+            float af = (float)a;
+            record[n] = scale ? af * scale[n] : af;
+        }
+    }
+#pragma omp parallel for schedule(static)
+    for (int c = 0; c < H; ++c) {
+        const uint16_t* wrow = Wd + (size_t)c * I;
+        for (int t = 0; t < T; ++t) {
+            const float* ht = h + (size_t)t * I;
+            double acc = 0.0;
+            for (int n = 0; n < I; ++n) acc += (double)ht[n] * (double)bf16_to_f32(wrow[n]);
+            double base = r ? (double)r[(size_t)t * H + c] : 0.0;
+            y[(size_t)t * H + c] = (float)(base + acc);
+        }
+    }
+    if (h_out) memcpy(h_out, h, sizeof(float) * (size_t)T * (size_t)I);
+    free(h);
+}
+
+/* Anchor-relative local update (Eq. 4): y_hat = y_anchor + (h_t^M - h_anchor^M) W_down[:,M], followed by the
+ * residual addition out = r + y_hat.  y_anchor [T,H] is the anchor step's pre-residual FFN output, h_anchor
+ * [T,K] its activations on the mask.  With y_anchor = 0 and h_anchor = 0 this is the zero-fill form. */
+void orc_anchor_mlp(const uint16_t* x, const uint16_t* Wg, const uint16_t* Wu, const uint16_t* Wd,
+                    const float* r, const int32_t* idx, int K, int T, int H, int I,
+                    const float* y_anchor, const float* h_anchor, float* out) {
+    float* d = (float*)malloc(sizeof(float) * (size_t)(T > 0 ? T : 1) * (size_t)(K > 0 ? K : 1));
+#pragma omp parallel for schedule(static)
+    for (int j = 0; j < K; ++j) {
+        size_t n = (size_t)idx[j];
+        for (int t = 0; t < T; ++t) {
+            float hv = hidden_one(x + (size_t)t * H, Wg + n * H, Wu + n * H, H);
+            float ha = h_anchor ? h_anchor[(size_t)t * K + j] : 0.0f;
+            d[(size_t)t * K + j] = (float)((double)hv - (double)ha);
+        }
+    }
+#pragma omp parallel for schedule(static)
+    for (int c = 0; c < H; ++c) {
+        for (int t = 0; t < T; ++t) {
+            double acc = 0.0;
+            for (int j = 0; j < K; ++j)
+                acc += (double)d[(size_t)t * K + j] * (double)bf16_to_f32(Wd[(size_t)c * I + (size_t)idx[j]]);
+            double base = (r ? (double)r[(size_t)t * H + c] : 0.0) +
+                          (y_anchor ? (double)y_anchor[(size_t)t * H + c] : 0.0);
+            out[(size_t)t * H + c] = (float)(base + acc);
+        }
+    }
+    free(d);
+}
+
+/* Parameter-free RMSNorm followed by the bf16 rounding of the FFN input:
+ * x[t,k] = bf16( r[t,k] / sqrt(mean_k r[t,k]^2 + 1e-6) ).  Mean and quotient in double. */
+void orc_rmsnorm_bf16(const float* r, int T, int H, uint16_t* x) {
+    for (int t = 0; t < T; ++t) {
+        double ss = 0.0;
+        for (int k = 0; k < H; ++k) ss += (double)r[(size_t)t * H + k] * (double)r[(size_t)t * H + k];
+        double inv = 1.0 / sqrt(ss / (double)H + 1e-6);
+        for (int k = 0; k < H; ++k) x[(size_t)t * H + k] = f32_to_bf16((float)((double)r[(size_t)t * H + k] * inv));
+    }
+}
+
+/* One denoising step through L layers: r_0 = r_in; x_l = bf16(RMSNorm(r_l)); r_{l+1} = r_l + MLP_l(x_l; S_l);
+ * output r_L.  The residual stream stays fp32 between layers.  Attention, time conditioning and the adaptive
+ * gate are identity here.  idx == NULL runs every layer densely; records (nullable) is [L,I]; scale (nullable)
+ * is [L,I].  Weight pointers are arrays of L per-layer pointers. */
+void orc_step(const uint16_t* const* Wg, const uint16_t* const* Wu, const uint16_t* const* Wd,
+              const float* r_in, const int32_t* idx, const int32_t* count, int64_t stride,
+              int L, int T, int H, int I, float* r_out, float* records, const float* scale) {
+    size_t n = (size_t)T * (size_t)H;
+    float* cur = (float*)malloc(sizeof(float) * (n ? n : 1));
+    float* nxt = (float*)malloc(sizeof(float) * (n ? n : 1));
+    uint16_t* x = (uint16_t*)malloc(sizeof(uint16_t) * (n ? n : 1));
+    memcpy(cur, r_in, sizeof(float) * n);
+    for (int l = 0; l < L; ++l) {
+        orc_rmsnorm_bf16(cur, T, H, x);
+        if (idx)
+            orc_masked_mlp(x, Wg[l], Wu[l], Wd[l], cur, idx + (size_t)l * (size_t)stride, count[l], T, H, I, nxt,
+                           NULL);
+        else
+            orc_dense_mlp(x, Wg[l], Wu[l], Wd[l], cur, T, H, I, nxt, NULL,
+                          records ? records + (size_t)l * I : NULL, scale ? scale + (size_t)l * I : NULL);
+        float* tmp = cur; cur = nxt; nxt = tmp;
+    }
+    memcpy(r_out, cur, sizeof(float) * n);
+    free(cur); free(nxt); free(x);
+}
+
+/* ---------------------------------------------------------------- mask compaction (important-neuron sets) */
+
+/* Boolean mask -> ascending index list.  Returns the count. */
+int orc_compact_bool(const uint8_t* m, int I, int32_t* idx_out) {
+    int c = 0;
+    for (int n = 0; n < I; ++n)
+        if (m[n] != 0) idx_out[c++] = n;
+    return c;
+}
+
+/* Selection flags of one record under a rule.  rule 1: score > threshold (strict).  rule 2: the k neurons with
+ * the largest score, ties going to the lower index ("rank all neurons by c in descending order", Eq. 1 text;
+ * K_l = ceil(rho_n * I) is computed by the caller).  score = record[n] * scale[n] (one fp32 multiply) when a
+ * scale is given.  NaN ranks below every number; -0 equals +0. */
+typedef struct { float s; int32_t n; } orc_pair;
+
+static int pair_cmp(const void* a, const void* b) {
+    const orc_pair* p = (const orc_pair*)a;
+    const orc_pair* q = (const orc_pair*)b;
+    int pn = isnan(p->s), qn = isnan(q->s);
+    if (pn != qn) return pn ? 1 : -1;            /* NaN last */
+    if (!pn) {
+        if (p->s > q->s) return -1;
+        if (p->s < q->s) return 1;
+    }
+    return (p->n > q->n) - (p->n < q->n);        /* equal score: lower index first */
+}
+
+static void select_flags(const float* record, const float* scale, int I, int rule, float threshold, int k,
+                         uint8_t* flag) {
+    memset(flag, 0, (size_t)I);
+    if (rule == 1) {
+        for (int n = 0; n < I; ++n) {
+            float s = scale ? record[n] * scale[n] : record[n];
+            flag[n] = (s > threshold) ? 1 : 0;
+        }
+    } else {
+        orc_pair* p = (orc_pair*)malloc(sizeof(orc_pair) * (size_t)(I > 0 ? I : 1));
+        for (int n = 0; n < I; ++n) {
+            p[n].s = scale ? record[n] * scale[n] : record[n];
+            p[n].n = n;
+        }
+        qsort(p, (size_t)I, sizeof(orc_pair), pair_cmp);   /* the comparator is a total order: no stability needed */
+        int kk = k < I ? k : I;
+        for (int j = 0; j < kk; ++j) flag[p[j].n] = 1;
+        free(p);
+    }
+}
+
+/* W records -> one index list.  Each record is reduced to a set by `rule` (1 threshold, 2 top-k); a neuron is
+ * kept when at least min_votes of the W sets contain it (W = 1, min_votes = 1: the plain single-record case).
+ * records is an array of W pointers to [I] floats.  Returns the count; the list is ascending. */
+int orc_compact_scores(const float* const* records, int W, const float* scale, int I, int rule,
+                       float threshold, int k, int min_votes, int32_t* idx_out) {
+    uint8_t* flag = (uint8_t*)malloc((size_t)(I > 0 ? I : 1));
+    int* votes = (int*)calloc((size_t)(I > 0 ? I : 1), sizeof(int));
+    for (int w = 0; w < W; ++w) {
+        select_flags(records[w], scale, I, rule, threshold, k, flag);
+        for (int n = 0; n < I; ++n) votes[n] += flag[n];
+    }
+    int c = 0;
+    for (int n = 0; n < I; ++n)
+        if (votes[n] >= min_votes) idx_out[c++] = n;
+    free(flag); free(votes);
+    return c;
+}
+
+/* Group mask (Sec. 5, "Constructing Group Neuron Masks"): take each record's top-k set, form the union, rank
+ * the union by the summed score over the W records, keep the top k.  Ties: lower index.  Returns the count. */
+int orc_compact_group(const float* const* records, int W, const float* scale, int I, int k, int32_t* idx_out) {
+    uint8_t* flag = (uint8_t*)malloc((size_t)(I > 0 ? I : 1));
+    uint8_t* in_union = (uint8_t*)calloc((size_t)(I > 0 ? I : 1), 1);
+    for (int w = 0; w < W; ++w) {
+        select_flags(records[w], scale, I, 2, 0.0f, k, flag);
+        for (int n = 0; n < I; ++n) in_union[n] |= flag[n];
+    }
+    orc_pair* p = (orc_pair*)malloc(sizeof(orc_pair) * (size_t)(I > 0 ? I : 1));
+    int m = 0;
+    for (int n = 0; n < I; ++n) {
+        if (!in_union[n]) continue;
+        float sum = 0.0f;                       /* fp32 sum in record order: the decision is taken in fp32 */
+        for (int w = 0; w < W; ++w) sum += scale ? records[w][n] * scale[n] : records[w][n];
+        p[m].s = sum; p[m].n = n; ++m;
+    }
+    qsort(p, (size_t)m, sizeof(orc_pair), pair_cmp);
+    int kk = k < m ? k : m;
+    memset(flag, 0, (size_t)I);
+    for (int j = 0; j < kk; ++j) flag[p[j].n] = 1;
+    int c = 0;
+    for (int n = 0; n < I; ++n)
+        if (flag[n]) idx_out[c++] = n;
+    free(flag); free(in_union); free(p);
+    return c;
+}
+
+/* ||W_down[:,n]||_2 for every neuron (the weight factor of Eq. 1), double accumulate -> fp32. */
+void orc_down_colnorm(const uint16_t* Wd, int H, int I, float* out) {
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < I; ++n) {
+        double s = 0.0;
+        for (int c = 0; c < H; ++c) {
+            double v = (double)bf16_to_f32(Wd[(size_t)c * I + n]);
+            s += v * v;
+        }
+        out[n] = (float)sqrt(s);
+    }
+}
+
+#ifdef _OPENMP
+#include <omp.h>
+int orc_num_threads(void) { return omp_get_max_threads(); }
+void orc_set_threads(int n) { omp_set_num_threads(n); }
+#else
+int orc_num_threads(void) { return 1; }
+void orc_set_threads(int n) { (void)n; }
+#endif

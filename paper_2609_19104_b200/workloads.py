@@ -1,0 +1,228 @@
+"""Seeded synthetic inputs for the masked gated-MLP path.
+
+This module only *draws numbers*: a counter-based generator (SplitMix64 of
+(seed, tensor id, element index) followed by Box-Muller), bf16 bit packing, and
+the recipes that turn those draws into the five workloads (weights, step
+inputs, reference inputs, boolean masks, run-structured scales).  It holds none
+of the method's arithmetic (no MLP, no normalisation, no mask selection), so it
+can feed the CUDA path and the CPU oracle alike without coupling them.
+
+The shapes follow the action expert the paper analyses (Table 1: one 1024x4096
+projection on 32 tokens; Table 2: 10 denoising steps, chunk 32) and its larger
+variant with a 2048/16384 denoiser (model-scaling experiment).  The paper's own
+inputs come from trained checkpoints and simulator episodes; these draws stand
+in for them.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+
+BASE_SEED = 20260919
+
+_U64 = np.uint64
+_GOLDEN = _U64(0x9E3779B97F4A7C15)
+_M1 = _U64(0xBF58476D1CE4E5B9)
+_M2 = _U64(0x94D049BB133111EB)
+
+# tensor roles (part of the tensor id)
+ROLE_WG, ROLE_WU, ROLE_WD = 1, 2, 3
+ROLE_X0, ROLE_REF_NOISE, ROLE_STEP_DIR, ROLE_RESIDUAL = 4, 5, 6, 7
+ROLE_BOOL_MASK, ROLE_RUNS = 8, 9
+
+
+def _mix(z: np.ndarray) -> np.ndarray:
+    with np.errstate(over="ignore"):
+        z = z + _GOLDEN
+        z = (z ^ (z >> _U64(30))) * _M1
+        z = (z ^ (z >> _U64(27))) * _M2
+        return z ^ (z >> _U64(31))
+
+
+def tensor_key(seed: int, config: int, layer: int, role: int, extra: int = 0) -> np.uint64:
+    """A 64-bit stream key for one tensor; every (config, layer, role, extra) gets its own."""
+    tid = ((config & 0xFF) << 48) | ((layer & 0xFFFF) << 32) | ((role & 0xFF) << 24) | (extra & 0xFFFFFF)
+    k = _mix(np.array([seed & 0xFFFFFFFFFFFFFFFF], dtype=_U64))
+    k = _mix(k ^ np.array([tid], dtype=_U64))
+    return k[0]
+
+
+def _hash_range(key: np.uint64, start: int, n: int) -> np.ndarray:
+    with np.errstate(over="ignore"):
+        idx = np.arange(start, start + n, dtype=_U64)
+        return _mix(idx * _GOLDEN + key)
+
+
+def uniform(key: np.uint64, n: int, start: int = 0) -> np.ndarray:
+    """n doubles in [0, 1): element i depends only on (key, start + i)."""
+    h = _hash_range(key, start, n)
+    return (h >> _U64(11)).astype(np.float64) * (1.0 / 9007199254740992.0)
+
+
+def normal(key: np.uint64, n: int, start: int = 0, chunk: int = 1 << 22) -> np.ndarray:
+    """n standard normals as float32 (Box-Muller on the two 32-bit halves of one hash)."""
+    out = np.empty(n, dtype=np.float32)
+    for s in range(0, n, chunk):
+        m = min(chunk, n - s)
+        h = _hash_range(key, start + s, m)
+        u1 = ((h >> _U64(32)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
+        u2 = ((h & _U64(0xFFFFFFFF)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
+        out[s:s + m] = (np.sqrt(-2.0 * np.log(u1)) * np.cos((2.0 * math.pi) * u2)).astype(np.float32)
+    return out
+
+
+def randint(key: np.uint64, n: int, lo: int, hi: int, start: int = 0) -> np.ndarray:
+    """n integers uniform on [lo, hi] (inclusive)."""
+    u = uniform(key, n, start)
+    return (lo + np.floor(u * (hi - lo + 1))).astype(np.int64)
+
+
+# ----------------------------------------------------------------------------- bf16 bits
+def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even fp32 -> bf16, returned as uint16 bit patterns."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    bias = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
+    return ((u + bias) >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+# ----------------------------------------------------------------------------- workloads
+@dataclass(frozen=True)
+class Workload:
+    """Shape and recipe of one of the five configurations."""
+    config: int
+    name: str
+    L: int
+    H: int
+    I: int
+    T: int
+    sigma: float
+    steps: int
+    density: float
+    B: int = 1
+    seed: int = BASE_SEED
+    extra: dict = field(default_factory=dict)
+
+    @property
+    def K(self) -> int:
+        return topk_count(self.density, self.I)
+
+
+def topk_count(rho: float, I: int) -> int:
+    """K = ceil(rho * I), the per-layer number of retained neurons (Sec. 5, mask construction)."""
+    return int(min(I, max(0, math.ceil(rho * I - 1e-9))))
+
+
+def config0(seed: int = BASE_SEED) -> Workload:
+    return Workload(0, "single-layer-bernoulli30", 1, 1024, 4096, 51, 0.02, 1, 0.30, seed=seed)
+
+
+def config1(seed: int = BASE_SEED, L: int = 18) -> Workload:
+    return Workload(1, "pi0-stack-top25", L, 1024, 4096, 51, 0.02, 10, 0.25, seed=seed)
+
+
+def config2(seed: int = BASE_SEED, L: int = 18) -> Workload:
+    return Workload(2, "large-stack-top20-refresh2", L, 2048, 16384, 51, 0.015, 10, 0.20, seed=seed,
+                    extra={"refresh_every": 2})
+
+
+def config3(density: float, B: int = 1, seed: int = BASE_SEED, L: int = 18) -> Workload:
+    return Workload(3, f"sweep-rho{density:g}-B{B}", L, 1024, 4096, 51, 0.02, 10, density, B=B, seed=seed)
+
+
+def config4(seed: int = BASE_SEED, L: int = 18) -> Workload:
+    return Workload(4, "runs-vote-window4", L, 1024, 4096, 32, 0.02, 10, 0.15, seed=seed,
+                    extra={"window": 4, "min_votes": 3, "run_lo": 8, "run_hi": 64, "gap_lo": 8, "gap_hi": 400,
+                           "in_run_scale": 4.0})
+
+
+def scaled(w: Workload, **kw) -> Workload:
+    """A smaller (or otherwise altered) copy of a workload for tests; same recipe, same seed stream."""
+    d = dict(config=w.config, name=w.name + "-scaled", L=w.L, H=w.H, I=w.I, T=w.T, sigma=w.sigma, steps=w.steps,
+             density=w.density, B=w.B, seed=w.seed, extra=dict(w.extra))
+    d.update(kw)
+    return Workload(**d)
+
+
+def layer_weights(w: Workload, layer: int):
+    """(W_gate [I,H], W_up [I,H], W_down [H,I]) as bf16 bit patterns, N(0, sigma^2) rounded to bf16."""
+    out = []
+    for role, shape in ((ROLE_WG, (w.I, w.H)), (ROLE_WU, (w.I, w.H)), (ROLE_WD, (w.H, w.I))):
+        v = normal(tensor_key(w.seed, w.config, layer, role), w.I * w.H) * np.float32(w.sigma)
+        out.append(f32_to_bf16_bits(v).reshape(shape))
+    return tuple(out)
+
+
+def base_input(w: Workload, episode: int = 0) -> np.ndarray:
+    """X0 [T,H]: fp32 standard normals (not yet rounded)."""
+    return normal(tensor_key(w.seed, w.config, 0, ROLE_X0, episode), w.T * w.H).reshape(w.T, w.H)
+
+
+def step_input(w: Workload, s: int, episode: int = 0) -> np.ndarray:
+    """Open-loop input of denoising step s as bf16 bits [T,H]: X_s = cos(theta s) X0 + sin(theta s) D with
+    theta = acos(0.9)/9, so steps 0 and 9 have expected cosine similarity 0.9."""
+    x0 = base_input(w, episode)
+    d = normal(tensor_key(w.seed, w.config, 0, ROLE_STEP_DIR, episode), w.T * w.H).reshape(w.T, w.H)
+    th = math.acos(0.9) / 9.0 * s
+    return f32_to_bf16_bits(np.float32(math.cos(th)) * x0 + np.float32(math.sin(th)) * d)
+
+
+def reference_input(w: Workload, record: int = 0, episode: int = 0, cosine: float = 0.95) -> np.ndarray:
+    """A 'similar earlier execution' input as bf16 bits [T,H]: cosine*X0 + sqrt(1-cosine^2)*E_record."""
+    x0 = base_input(w, episode)
+    e = normal(tensor_key(w.seed, w.config, 0, ROLE_REF_NOISE, episode * 64 + record), w.T * w.H).reshape(w.T, w.H)
+    return f32_to_bf16_bits(np.float32(cosine) * x0 + np.float32(math.sqrt(1.0 - cosine * cosine)) * e)
+
+
+def residual_input(w: Workload, episode: int = 0) -> np.ndarray:
+    """r [T,H] fp32 with bf16-representable values, independent of the step inputs (single-layer case)."""
+    v = normal(tensor_key(w.seed, w.config, 0, ROLE_RESIDUAL, episode), w.T * w.H).reshape(w.T, w.H)
+    return bf16_bits_to_f32(f32_to_bf16_bits(v))
+
+
+def bernoulli_mask(w: Workload, layer: int = 0, episode: int = 0) -> np.ndarray:
+    """uint8 [I]: neuron n active iff uniform(seed, n) < density."""
+    u = uniform(tensor_key(w.seed, w.config, layer, ROLE_BOOL_MASK, episode), w.I)
+    return (u < w.density).astype(np.uint8)
+
+
+def run_structure(w: Workload, layer: int, max_tries: int = 64):
+    """Run-structured neuron set for the sliding-window workload: alternating gaps ~U{gap_lo..gap_hi} and runs
+    ~U{run_lo..run_hi} until I is covered; redrawn (seed advanced) until the realised density lies within
+    +-0.02 of the target.  Returns (member uint8 [I], scale float32 [I]) with scale = in_run_scale inside a
+    run and 1 elsewhere."""
+    ex = w.extra
+    for attempt in range(max_tries):
+        key = tensor_key(w.seed, w.config, layer, ROLE_RUNS, attempt)
+        n_draw = 2 * (w.I // max(1, ex["gap_lo"] + ex["run_lo"]) + 2)
+        gaps = randint(key, n_draw, ex["gap_lo"], ex["gap_hi"], start=0)
+        runs = randint(key, n_draw, ex["run_lo"], ex["run_hi"], start=n_draw)
+        member = np.zeros(w.I, dtype=np.uint8)
+        pos = 0
+        for g, r in zip(gaps, runs):
+            pos += int(g)
+            if pos >= w.I:
+                break
+            member[pos:min(w.I, pos + int(r))] = 1
+            pos += int(r)
+        dens = float(member.mean())
+        if abs(dens - w.density) <= 0.02:
+            scale = np.where(member != 0, np.float32(ex["in_run_scale"]), np.float32(1.0)).astype(np.float32)
+            return member, scale
+    raise RuntimeError("run_structure: no draw met the density band")
+
+
+# ----------------------------------------------------------------------------- byte / flop accounting
+def algorithmic_bytes_per_layer(H: int, T: int, K: int) -> int:
+    """Bytes one masked layer call must move: active weights K*3H bf16, x bf16, residual in + y out fp32,
+    and the K int32 indices.  The compact intermediate h is excluded (it can stay on chip)."""
+    return K * 3 * H * 2 + T * H * 2 + 2 * T * H * 4 + 4 * K
+
+
+def algorithmic_flops_per_layer(H: int, T: int, K: int) -> int:
+    return 2 * T * K * 3 * H
