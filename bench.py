@@ -1,0 +1,330 @@
+#!/usr/bin/env python
+"""Benchmark of the activation-masked gated-MLP path on B200.
+
+One "step" is one denoising step of the pi0-style action expert (18 layers, H=1024, I=4096, T=51, top-25 % masks
+reused across steps): `rm_action_expert_step` with the device-resident index lists, plus -- once every 10 steps,
+which is how often the workload derives its masks -- `rm_mask_compact` (top-k over the resident reference
+records).  Inputs are resident in HBM for `value`; `e2e` goes through `rm_action_expert_step_host` with pinned host
+buffers.  L2 is flushed (a 512 MB fill) before every timed step, outside the timed interval, because one step's
+active weights (113 MB) would otherwise stay in the 126 MB L2.
+
+`--impl reference` times the CPU oracle (a deliberately plain program) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_19104_b200 import workloads as wl  # noqa: E402
+
+METRIC = "masked_mlp_us_per_denoise_step"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def pick_workload(name: str) -> wl.Workload:
+    if name == "config1":
+        return wl.config1()
+    if name == "config2":
+        return wl.config2()
+    if name == "config4":
+        return wl.config4()
+    if name.startswith("config3"):
+        parts = name.split(":")
+        rho = float(parts[1]) if len(parts) > 1 else 0.25
+        B = int(parts[2]) if len(parts) > 2 else 1
+        return wl.config3(rho, B=B)
+    raise SystemExit(f"unknown workload {name}")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100", "-i",
+                 str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                for n, v in zip(names, r[2:6]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------ reference arm
+def oracle_sample(w: wl.Workload, sample_layers: int):
+    """Inputs of the bounded CPU sample: the first `sample_layers` layers of the stack, top-K lists drawn from the
+    oracle's own dense records of those layers."""
+    import oracle
+    ws = wl.scaled(w, L=sample_layers)
+    Wg, Wu, Wd = zip(*[wl.layer_weights(ws, l) for l in range(sample_layers)])
+    r_ref = wl.bf16_bits_to_f32(wl.reference_input(w))
+    _, rec = oracle.step(Wg, Wu, Wd, r_ref, return_records=True)
+    idx = np.zeros((sample_layers, w.I), np.int32)
+    cnt = np.zeros(sample_layers, np.int32)
+    for l in range(sample_layers):
+        s = oracle.compact_scores(rec[l], oracle.RULE_TOPK, k=w.K)
+        idx[l, :s.size] = s
+        cnt[l] = s.size
+    return (Wg, Wu, Wd), idx, cnt
+
+
+def time_oracle(w: wl.Workload, steps: int, warmup: int, sample_layers: int = 3):
+    import oracle
+    (Wg, Wu, Wd), idx, cnt = oracle_sample(w, sample_layers)
+    scale_up = w.L / sample_layers
+    times = []
+    for s in range(warmup + steps):
+        r0 = wl.bf16_bits_to_f32(wl.step_input(w, s % w.steps))
+        t0 = time.perf_counter()
+        oracle.step(Wg, Wu, Wd, r0, idx, cnt)
+        dt = time.perf_counter() - t0
+        if s >= warmup:
+            times.append(dt)
+    us = float(np.mean(times)) * 1e6 * scale_up
+    return us, oracle.num_threads(), (f"{sample_layers} of {w.L} layers of one masked denoising step per timed step "
+                                      f"(K={w.K} per layer), scaled by {scale_up:g}")
+
+
+def run_reference(args, w: wl.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    us, cores, sample = time_oracle(w, args.steps, args.warmup)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64-accumulate/f32", "data": "synthetic",
+        "config": {"workload": w.name, "L": w.L, "H": w.H, "I": w.I, "T": w.T, "K_per_layer": w.K},
+        "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ GPU arm
+def run_gpu(args, w: wl.Workload):
+    import torch
+    import torch.distributed as dist
+    import paper_2609_19104_b200 as rm
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    B = w.B
+    ctx = rm.Context(w.L, w.H, w.I, T_max=w.T, B_max=B)
+    # weights: the workload's seeded draws (same on every rank: replicas of one model)
+    packed = []
+    for l in range(w.L):
+        g, u, d = wl.layer_weights(w, l)
+        to = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+        packed.append(ctx.rm_pack_weights(to(g), to(u), to(d)))
+    torch.cuda.synchronize()
+
+    # every rank runs its own episodes (replicas; no data-path collective)
+    ep0 = rank * B
+    f32 = lambda bits: torch.from_numpy(wl.bf16_bits_to_f32(bits))
+    refs = torch.stack([f32(wl.reference_input(w, episode=ep0 + b)) for b in range(B)]).cuda()
+    step_inputs = [torch.stack([f32(wl.step_input(w, s, episode=ep0 + b)) for b in range(B)]) for s in range(w.steps)]
+    dev_inputs = [t.cuda() for t in step_inputs]
+    pinned_in = [t.pin_memory() for t in step_inputs]
+    pinned_out = torch.empty(B, w.T, w.H, dtype=torch.float32).pin_memory()
+    r_out = torch.empty(B, w.T, w.H, dtype=torch.float32, device="cuda")
+    records = torch.zeros(B, w.L, w.I, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(B * w.L, w.I, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(B * w.L, dtype=torch.int32, device="cuda")
+    n_lists = B * w.L
+    rec_flat = records.view(n_lists, w.I)
+
+    # reference pass (dense, emits the activation records), then the masks
+    ctx.rm_action_expert_step(packed, refs, None, None, 0, r_out, records_out=records, B=B, T=w.T)
+
+    def compact():
+        ctx.rm_mask_compact([rec_flat], rm.RM_SRC_SCORE_F32, rm.RM_REDUCE_TOPK, idx, cnt, w.I, n_lists=n_lists, k=w.K)
+
+    compact()
+    torch.cuda.synchronize()
+    K_mean = float(cnt.float().mean().item())
+
+    flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def one_step(s, timed_events=None):
+        flush.fill_(s & 0xFF)
+        if timed_events is not None:
+            timed_events[0].record(stream)
+        if s % w.steps == 0:
+            compact()
+        ctx.rm_action_expert_step(packed, dev_inputs[s % w.steps], idx, cnt, w.I, r_out, B=B, T=w.T)
+        if timed_events is not None:
+            timed_events[1].record(stream)
+
+    for s in range(args.warmup):
+        one_step(s)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.launch_count()
+    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for s in range(args.steps):
+        one_step(s, events[s])
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches = ctx.launch_count() - launches0
+    step_ms = [a.elapsed_time(b) for a, b in events]
+    total_ms = float(sum(step_ms))
+
+    # end to end through the host-buffer entry point (H2D of the step input, step, D2H of the result, sync)
+    e2e_times = []
+    for s in range(args.warmup + args.steps):
+        flush.fill_(s & 0xFF)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ctx.rm_action_expert_step_host(packed, pinned_in[s % w.steps], idx, cnt, w.I, pinned_out, B=B, T=w.T)
+        dt = time.perf_counter() - t0
+        if s >= args.warmup:
+            e2e_times.append(dt)
+    e2e_total_ms = float(sum(e2e_times)) * 1e3
+
+    # per-layer launch durations for the roofline: CUDA events around single-layer calls of the same kernels on the
+    # same stream (cold L2 each time), layer by layer through the stack
+    layer_ms = []
+    x_bf16 = torch.empty(w.T, w.H, dtype=torch.bfloat16, device="cuda")
+    y_tmp = torch.empty(w.T, w.H, dtype=torch.float32, device="cuda")
+    res = dev_inputs[0][0].contiguous()
+    x_bf16.copy_(res)
+    reps = max(1, min(args.steps, 10))
+    for rep in range(reps):
+        for l in range(w.L):
+            flush.fill_(l & 0xFF)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            ctx.rm_sparse_mlp(packed[l], x_bf16, res, idx[l], cnt[l:l + 1], y_tmp, T=w.T)
+            b.record(stream)
+            layer_ms.append((a, b))
+    torch.cuda.synchronize()
+    layer_us = float(np.mean([a.elapsed_time(b) for a, b in layer_ms])) * 1e3
+    clocks = sampler.stop() if rank == 0 else None
+
+    t = torch.tensor([total_ms, e2e_total_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_total_ms = float(t[0].item()), float(t[1].item())
+
+    if rank == 0:
+        units = args.steps * world * B                      # denoising steps of one episode, whole job
+        us_per_step = total_ms * 1e3 / units
+        e2e_us = e2e_total_ms * 1e3 / units
+        peak, peak_kind = measured_hbm_peak()
+        bytes_layer = wl.algorithmic_bytes_per_layer(w.H, w.T, int(round(K_mean))) * B
+        bytes_step = bytes_layer * w.L
+        achieved = bytes_layer / (layer_us * 1e-6) / 1e9
+        io_bytes = B * w.T * w.H * 4
+        cpu_us, cores, sample = time_oracle(w, steps=3, warmup=1) if world == 1 else (None, None, None)
+        line = {
+            "metric": METRIC, "value": us_per_step, "unit": "us", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (fp32 accumulate)", "data": "synthetic",
+            "config": {"workload": w.name, "L": w.L, "H": w.H, "I": w.I, "T": w.T, "B": B,
+                       "K_per_layer": K_mean, "mask": "top-k of dense reference records, rebuilt every 10 steps",
+                       "l2": "flushed before every timed step (512 MB fill, outside the timed interval)",
+                       "multi_gpu": "replicas: each rank runs its own episodes, no collective on the data path"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_kind": f"{peak_kind} copy bandwidth",
+                         "kernel": "one layer of the masked MLP (rm_sparse_mlp launch sequence)",
+                         "bytes_per_launch": bytes_layer, "us_per_launch": layer_us,
+                         "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+                         "step_effective_gbs": bytes_step / (us_per_step * B * 1e-6) / 1e9},
+            "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if cpu_us is not None:
+            line["cpu_baseline"] = {"value": cpu_us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config1")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = pick_workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_gpu(args, w)
+
+
+if __name__ == "__main__":
+    main()

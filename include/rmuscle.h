@@ -1,0 +1,146 @@
+/*
+ * rmuscle.h -- C ABI of the activation-masked gated MLP of a diffusion action expert (the compute side of the
+ * paper's Action Cache, Sec. 4.1 "Action Cache", Eq. 1 and Eq. 4), implemented as CUDA kernels for sm_100a.
+ *
+ * Notation (paper / this header): L layers, H model width, I intermediate neurons per layer, T tokens per
+ * episode, B independent episodes per call, S_l the active neuron set of layer l (the mask M stored as indices),
+ * K_l = |S_l|.  bf16 tensors are passed as raw 2-byte elements.
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".  The caller allocates and owns every
+ *     buffer, including packed weights and workspace; the library allocates only its small context in rm_create.
+ *   - Device buffers must be 16-byte aligned (RM_ERR_ALIGN otherwise).  Inputs are never written.
+ *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it; no call synchronises the host
+ *     unless its comment says so.  Argument validation is synchronous and returns a negative rm_status.
+ *   - Conditions detected on the device (index >= I, count > stride) never trap: the kernel clamps or skips,
+ *     records the code in the context's status word, and rm_device_status reports it.
+ *   - Index lists are strictly ascending int32.  The number of valid entries is read from DEVICE memory, so a
+ *     list built by rm_mask_compact can be consumed without a host round trip.  A count of 0 is legal.
+ */
+#ifndef RMUSCLE_H
+#define RMUSCLE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rm_ctx rm_ctx;      /* opaque */
+typedef void* rm_stream_t;         /* a cudaStream_t */
+
+typedef enum {
+    RM_OK = 0,
+    RM_ERR_INVALID_ARG = -1,       /* NULL where a pointer is required, negative size, bad enum           */
+    RM_ERR_SHAPE = -2,             /* size outside what the context was created for                       */
+    RM_ERR_ALIGN = -3,             /* a device pointer is not 16-byte aligned                             */
+    RM_ERR_WORKSPACE = -4,         /* workspace NULL or smaller than rm_workspace_bytes                   */
+    RM_ERR_CUDA = -5,              /* a CUDA runtime call failed (launch error, no device)                */
+    RM_ERR_INDEX = -6,             /* device status: a neuron index was out of range or count > stride    */
+    RM_ERR_TIMEOUT = -7,           /* device status: a bounded wait expired                               */
+    RM_ERR_UNSUPPORTED = -8        /* valid request that this build does not implement                    */
+} rm_status;
+
+enum { RM_ACT_GELU_TANH = 0 };     /* the gated unit's activation ("post-GeGLU activation", Eq. 1)        */
+
+/* Model geometry fixed at context creation.  H must be a multiple of 64, I >= 1, L >= 1.
+ * T_max / B_max bound the T and B of later calls (they size rm_workspace_bytes). */
+typedef struct {
+    int32_t L, H, I, T_max, B_max;
+    int32_t act;                   /* RM_ACT_GELU_TANH */
+} rm_model_desc;
+
+/* Creates a context on the CURRENT CUDA device.  Allocates a few hundred bytes of device memory (the status
+ * word and per-call parameter blocks).  Host-synchronous.  *out is NULL on failure. */
+int rm_create(rm_ctx** out, const rm_model_desc* desc);
+int rm_destroy(rm_ctx* ctx);
+
+/* Bytes of one layer in the library's private neuron-major layout (3*H bf16 per neuron: the neuron's gate row,
+ * up row and down column stored next to one another so that one active neuron is one contiguous read). */
+size_t rm_packed_layer_bytes(const rm_ctx* ctx);
+
+/* Bytes of scratch that rm_sparse_mlp / rm_action_expert_step need for B episodes of T tokens. */
+size_t rm_workspace_bytes(const rm_ctx* ctx, int B, int T);
+
+/* One-off repacking of a layer (not on the timed path).
+ *   Wg, Wu [I,H] bf16 row-major (row n = neuron n);  Wd [H,I] bf16 row-major (column n = neuron n).
+ *   packed_out: rm_packed_layer_bytes bytes.  down_colnorm (nullable) [I] fp32 receives ||Wd[:,n]||_2, the weight
+ *   factor of the contribution score (Eq. 1). */
+int rm_pack_weights(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, void* packed_out,
+                    float* down_colnorm, rm_stream_t stream);
+
+/* ---- rm_mask_compact: important-neuron selection (Sec. 3.4 Eq. 1 ranking; Sec. 5 "Constructing Group Neuron
+ * Masks": K_l = ceil(rho_n * I) is computed by the caller and passed as k). */
+enum { RM_SRC_BOOL_U8 = 0,         /* records are uint8 [n_lists, I]; nonzero = selected                  */
+       RM_SRC_SCORE_F32 = 1 };     /* records are fp32 activation records [n_lists, I]                    */
+enum { RM_REDUCE_NONE = 0,         /* boolean source only                                                 */
+       RM_REDUCE_THRESHOLD = 1,    /* score > threshold (strict)                                          */
+       RM_REDUCE_TOPK = 2,         /* the k largest scores; equal scores: lower index first               */
+       RM_REDUCE_GROUP = 3 };      /* union of the records' top-k sets, ranked by the fp32 sum of the
+                                      records' scores (added in record order), top k kept                 */
+typedef struct {
+    int32_t kind;                  /* RM_SRC_*                                                            */
+    int32_t reduce;                /* RM_REDUCE_*                                                         */
+    float   threshold;
+    int32_t k;
+    int32_t n_records;             /* W >= 1 (at most 16) records per list                                */
+    int32_t min_votes;             /* a neuron is kept when >= min_votes of the W per-record sets hold it
+                                      (1 = union, W = intersection); ignored by RM_REDUCE_GROUP           */
+    const void* const* records;    /* HOST array of W device pointers, each [n_lists, I]                  */
+    const float* scale;            /* nullable; score = record * scale (one fp32 multiply)                */
+    int32_t scale_per_list;        /* 0: scale is [I];  1: scale is [n_lists, I]                          */
+    int32_t n_lists;
+    int32_t I;
+} rm_mask_src;
+
+/* Writes, for every list, the selected indices in ascending order to idx_out[list*stride ...] and their number
+ * to count_out[list] (both device).  stride >= I is always sufficient; a list longer than stride is truncated
+ * and RM_ERR_INDEX is recorded.  Float ordering: -0 == +0, NaN ranks below every number. */
+int rm_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out, int64_t stride,
+                    rm_stream_t stream);
+
+/* ---- rm_sparse_mlp: one layer, zero-fill form of the masked evaluation (Sec. 4.1: "compute only the selected
+ * neurons' hidden activations and update the output using their down-projection weights"):
+ *     y[t,:] = residual[t,:] + sum_{n in S} gelu_tanh(<x_t, Wg_n>) * <x_t, Wu_n> * Wd[:,n]
+ *   packed_layer: output of rm_pack_weights.   x [T,H] bf16.   residual [T,H] fp32, nullable (=> 0).
+ *   idx [>= count] int32 ascending, nullable => every neuron (dense);  count_dev [1] int32 on the device
+ *   (ignored when idx is NULL).   y [T,H] fp32; may equal residual (in place).
+ *   record_out (nullable) [I] fp32: dense mode only; receives A[n] = sum_t |h[t,n]| (* record_scale[n] when
+ *   record_scale is given) -- the activation part of Eq. 1, or Eq. 1 itself with record_scale = down_colnorm.
+ *   ws / ws_bytes: scratch of at least rm_workspace_bytes(ctx, 1, T). */
+int rm_sparse_mlp(rm_ctx* ctx, const void* packed_layer, const void* x, const float* residual,
+                  const int32_t* idx, const int32_t* count_dev, float* y, float* record_out,
+                  const float* record_scale, int T, void* ws, size_t ws_bytes, rm_stream_t stream);
+
+/* ---- rm_action_expert_step: the L-layer stack for one denoising step of B independent episodes, with masks
+ * reused from an earlier step (Sec. 4.1 "Group-Shared Neuron Masks"):
+ *     r_0 = r_in;  x_l = bf16(r_l / sqrt(mean_k r_l[t,k]^2 + 1e-6));  r_{l+1} = r_l + MLP_l(x_l; S_l);  r_out = r_L
+ *   The residual stream stays fp32.  Attention, conditioning and the adaptive gate are not part of this path.
+ *   packed_layers: HOST array of L device pointers.   r_in, r_out [B,T,H] fp32 (r_out may equal r_in).
+ *   idx [B,L,stride] int32, nullable => dense;  count_dev [B,L] int32 (device).
+ *   records_out (nullable, dense only) [B,L,I] fp32;  record_scale (nullable) [L,I] fp32. */
+int rm_action_expert_step(rm_ctx* ctx, const void* const* packed_layers, const float* r_in, const int32_t* idx,
+                          const int32_t* count_dev, int64_t stride, float* r_out, float* records_out,
+                          const float* record_scale, int B, int T, void* ws, size_t ws_bytes, rm_stream_t stream);
+
+/* The same step for callers whose activations live in HOST memory: copies r_in_host [B,T,H] fp32 to the device,
+ * runs the step, copies the result to r_out_host and waits for the stream (host-synchronous).  Pinned host
+ * memory makes the copies asynchronous with respect to other streams.  Needs rm_workspace_bytes(ctx,B,T) of
+ * workspace like the device variant (the staging buffer is part of it). */
+int rm_action_expert_step_host(rm_ctx* ctx, const void* const* packed_layers, const float* r_in_host,
+                               const int32_t* idx, const int32_t* count_dev, int64_t stride, float* r_out_host,
+                               int B, int T, void* ws, size_t ws_bytes, rm_stream_t stream);
+
+/* Reads and clears the device status word (0 or the first RM_ERR_* a kernel recorded).  Synchronises `stream`. */
+int rm_device_status(rm_ctx* ctx, int* host_out, rm_stream_t stream);
+
+/* Number of kernels the library has launched through this context since creation (host counter). */
+int64_t rm_launch_count(const rm_ctx* ctx);
+
+const char* rm_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RMUSCLE_H */

@@ -1,0 +1,76 @@
+// Shared declarations of the CUDA library: context, packed-weight geometry, launch helpers.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rmuscle.h"
+
+// Packed layer layout (private to the library).  Neuron n owns 3*H bf16 stored contiguously.  The chunk is cut
+// into NS = 8 column slices of Hs = H/8 columns; slice j holds
+//     [ Wg[n, j*Hs:(j+1)*Hs] | Wu[n, j*Hs:(j+1)*Hs] | Wd[j*Hs:(j+1)*Hs, n] ]
+// so that the CTA that owns column slice j of a cluster reads one contiguous 3*Hs*2-byte piece per neuron, and a
+// whole active neuron is one contiguous 6*H-byte read.
+constexpr int RM_NS = 8;
+
+struct rm_geom {
+    int L, H, I, Hs;                       // Hs = H / RM_NS
+    __host__ __device__ size_t neuron_elems() const { return (size_t)3 * H; }
+    // element offset of (neuron n, role, column k) inside a packed layer; role 0 gate, 1 up, 2 down
+    __host__ __device__ size_t off(int n, int role, int k) const {
+        int j = k / Hs, kk = k - j * Hs;
+        return (size_t)n * 3 * H + (size_t)j * 3 * Hs + (size_t)role * Hs + kk;
+    }
+};
+
+struct rm_ctx {
+    rm_model_desc desc;
+    rm_geom g;
+    int device;
+    int sm_count;
+    int* d_status;                         // device status word
+    int64_t launches;                      // host-side launch counter
+};
+
+#define RM_CUDA_TRY(expr)                                  \
+    do {                                                   \
+        cudaError_t _e = (expr);                           \
+        if (_e != cudaSuccess) return RM_ERR_CUDA;         \
+    } while (0)
+
+static inline bool rm_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+__device__ __forceinline__ void rm_set_status(int* status, int code) {
+    if (status) atomicCAS(status, 0, code);
+}
+
+__device__ __forceinline__ float rm_gelu_tanh(float g) {
+    // 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3)))
+    float inner = 0.7978845608028654f * (g + 0.044715f * g * g * g);
+    return 0.5f * g * (1.0f + tanhf(inner));
+}
+
+// ---- kernels implemented in the other translation units (host launchers)
+int rm_launch_pack(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, void* packed, float* colnorm,
+                   cudaStream_t s);
+int rm_launch_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out,
+                           int64_t stride, cudaStream_t s);
+
+// Portable path (CUDA cores): any H multiple of 64, any T, any I.
+struct rm_layer_args {
+    const __nv_bfloat16* packed;           // packed layer
+    const __nv_bfloat16* x;                // [B,T,H] bf16, or NULL when the layer normalises r_in itself
+    const float* r_in;                     // [B,T,H] fp32 residual (nullable => 0 when x is given)
+    float* r_out;                          // [B,T,H] fp32
+    const int32_t* idx;                    // [B, idx_stride] or NULL (dense)
+    const int32_t* count;                  // [B * count_stride] device counts (ignored when idx NULL)
+    int64_t idx_stride;                    // elements between episodes' lists
+    int64_t list_cap;                      // capacity of one list (a count above it is an error)
+    int64_t count_stride;                  // elements between episodes' counts
+    float* record;                         // [B, record_stride] or NULL
+    int64_t record_stride;
+    const float* record_scale;             // [I] or NULL
+    int B, T;
+};
+size_t rm_ref_workspace_bytes(const rm_ctx* ctx, int B, int T);
+int rm_launch_layer_ref(rm_ctx* ctx, const rm_layer_args& a, void* ws, cudaStream_t s);

@@ -16,6 +16,8 @@ in for them.
 from __future__ import annotations
 
 import math
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, field
 
 import numpy as np
@@ -61,15 +63,29 @@ def uniform(key: np.uint64, n: int, start: int = 0) -> np.ndarray:
     return (h >> _U64(11)).astype(np.float64) * (1.0 / 9007199254740992.0)
 
 
-def normal(key: np.uint64, n: int, start: int = 0, chunk: int = 1 << 22) -> np.ndarray:
-    """n standard normals as float32 (Box-Muller on the two 32-bit halves of one hash)."""
+def _normal_chunk(key: np.uint64, start: int, m: int) -> np.ndarray:
+    h = _hash_range(key, start, m)
+    u1 = ((h >> _U64(32)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
+    u2 = ((h & _U64(0xFFFFFFFF)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
+    return (np.sqrt(-2.0 * np.log(u1)) * np.cos((2.0 * math.pi) * u2)).astype(np.float32)
+
+
+def normal(key: np.uint64, n: int, start: int = 0, chunk: int = 1 << 20) -> np.ndarray:
+    """n standard normals as float32 (Box-Muller on the two 32-bit halves of one hash).  Element i depends only
+    on (key, start + i); large requests are cut into chunks and drawn by a thread pool."""
     out = np.empty(n, dtype=np.float32)
-    for s in range(0, n, chunk):
-        m = min(chunk, n - s)
-        h = _hash_range(key, start + s, m)
-        u1 = ((h >> _U64(32)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
-        u2 = ((h & _U64(0xFFFFFFFF)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
-        out[s:s + m] = (np.sqrt(-2.0 * np.log(u1)) * np.cos((2.0 * math.pi) * u2)).astype(np.float32)
+    spans = [(s, min(chunk, n - s)) for s in range(0, n, chunk)]
+    if len(spans) <= 1:
+        for s, m in spans:
+            out[s:s + m] = _normal_chunk(key, start + s, m)
+        return out
+
+    def work(span):
+        s, m = span
+        out[s:s + m] = _normal_chunk(key, start + s, m)
+
+    with ThreadPoolExecutor(max_workers=min(len(spans), os.cpu_count() or 1, 16)) as ex:
+        list(ex.map(work, spans))
     return out
 
 
@@ -132,12 +148,14 @@ def config2(seed: int = BASE_SEED, L: int = 18) -> Workload:
 
 
 def config3(density: float, B: int = 1, seed: int = BASE_SEED, L: int = 18) -> Workload:
-    return Workload(3, f"sweep-rho{density:g}-B{B}", L, 1024, 4096, 51, 0.02, 10, density, B=B, seed=seed)
+    # the sweep runs on the same model as config 1 (same weight streams)
+    return Workload(3, f"sweep-rho{density:g}-B{B}", L, 1024, 4096, 51, 0.02, 10, density, B=B, seed=seed,
+                    extra={"weights_config": 1})
 
 
 def config4(seed: int = BASE_SEED, L: int = 18) -> Workload:
     return Workload(4, "runs-vote-window4", L, 1024, 4096, 32, 0.02, 10, 0.15, seed=seed,
-                    extra={"window": 4, "min_votes": 3, "run_lo": 8, "run_hi": 64, "gap_lo": 8, "gap_hi": 400,
+                    extra={"weights_config": 1, "window": 4, "min_votes": 3, "run_lo": 8, "run_hi": 64, "gap_lo": 8, "gap_hi": 400,
                            "in_run_scale": 4.0})
 
 
@@ -153,7 +171,8 @@ def layer_weights(w: Workload, layer: int):
     """(W_gate [I,H], W_up [I,H], W_down [H,I]) as bf16 bit patterns, N(0, sigma^2) rounded to bf16."""
     out = []
     for role, shape in ((ROLE_WG, (w.I, w.H)), (ROLE_WU, (w.I, w.H)), (ROLE_WD, (w.H, w.I))):
-        v = normal(tensor_key(w.seed, w.config, layer, role), w.I * w.H) * np.float32(w.sigma)
+        v = normal(tensor_key(w.seed, w.extra.get("weights_config", w.config), layer, role), w.I * w.H)
+        v = v * np.float32(w.sigma)
         out.append(f32_to_bf16_bits(v).reshape(shape))
     return tuple(out)
 

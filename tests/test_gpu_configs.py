@@ -1,0 +1,247 @@
+"""The five workload configurations, GPU path against the oracle on the same seeded inputs.
+
+Protocol for masks that depend on computed activations: the GPU dense pass emits the activation records; the
+oracle's compaction of THOSE bytes must equal the GPU's lists bit-exactly; the oracle's own records must match the
+GPU's within the MLP tolerance; both sides then run the masked steps with the same lists.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_19104_b200 import workloads as wl
+from harness import Model, assert_close, dev, dev_bf16, lists_to_padded
+
+pytestmark = pytest.mark.gpu
+
+
+def f32_of(bits):
+    return wl.bf16_bits_to_f32(bits)
+
+
+def records_close(got, want):
+    # a record sums T magnitudes of h, so it inherits the per-element bound of the outputs
+    assert np.all(np.abs(got - want) <= 1e-2 * np.abs(want) + 2e-2)
+    assert np.linalg.norm(got - want) <= 5e-3 * np.linalg.norm(want)
+
+
+def gpu_dense_records(model, r0, B=1, scale=None):
+    """Dense step on the GPU; returns (r_out [B,T,H], records [B,L,I]) as numpy."""
+    import torch
+    w = model.w
+    rec = torch.zeros(B, w.L, w.I, dtype=torch.float32, device="cuda")
+    out = torch.empty(B, w.T, w.H, dtype=torch.float32, device="cuda")
+    model.ctx.rm_action_expert_step(model.packed, dev(r0), None, None, 0, out, records_out=rec,
+                                    record_scale=None if scale is None else dev(scale), B=B, T=w.T)
+    return out.cpu().numpy(), rec
+
+
+def gpu_topk_lists(lib, model, rec_list, k, n_lists, min_votes=1, scale=None, scale_per_list=False):
+    """rm_mask_compact on device-resident records; returns device idx/count and host copies."""
+    import torch
+    w = model.w
+    idx = torch.zeros(n_lists, w.I, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(n_lists, dtype=torch.int32, device="cuda")
+    model.ctx.rm_mask_compact(rec_list, lib.RM_SRC_SCORE_F32, lib.RM_REDUCE_TOPK, idx, cnt, w.I, n_lists=n_lists, k=k,
+                              min_votes=min_votes, scale=scale, scale_per_list=scale_per_list)
+    return idx, cnt, idx.cpu().numpy(), cnt.cpu().numpy()
+
+
+def gpu_sparse_step(model, r0, idx, cnt, B=1):
+    import torch
+    w = model.w
+    out = torch.empty(B, w.T, w.H, dtype=torch.float32, device="cuda")
+    model.ctx.rm_action_expert_step(model.packed, dev(r0), idx, cnt, w.I, out, B=B, T=w.T)
+    return out.cpu().numpy()
+
+
+def jaccard(a, b):
+    a, b = set(a.tolist()), set(b.tolist())
+    return len(a & b) / max(1, len(a | b))
+
+
+# ------------------------------------------------------------------------------------------------ config 0
+def test_config0_single_layer_bernoulli(lib):
+    import torch
+    w = wl.config0()
+    model = Model(lib, w)
+    x, r = wl.step_input(w, 0), wl.residual_input(w)
+    mask = wl.bernoulli_mask(w)
+    idx = torch.zeros(w.I, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    model.ctx.rm_mask_compact([dev(mask)], lib.RM_SRC_BOOL_U8, lib.RM_REDUCE_NONE, idx, cnt, w.I, n_lists=1)
+    want_idx = oracle.compact_bool(mask)
+    assert int(cnt.item()) == want_idx.size and np.array_equal(idx.cpu().numpy()[:want_idx.size], want_idx)
+    y = torch.empty(w.T, w.H, dtype=torch.float32, device="cuda")
+    model.ctx.rm_sparse_mlp(model.packed[0], dev_bf16(x), dev(r), idx, cnt, y)
+    rel = assert_close(y.cpu().numpy(), oracle.masked_mlp(x, model.Wg[0], model.Wu[0], model.Wd[0], r, want_idx),
+                       "config 0")
+    print(f"config0: K={want_idx.size} rel_l2={rel:.2e}")
+    assert model.ctx.rm_device_status() == 0
+    model.close()
+
+
+# ------------------------------------------------------------------------------------------------ configs 1, 3, 4
+@pytest.fixture(scope="module")
+def pi0(lib):
+    """The 18-layer H=1024 / I=4096 model shared by configs 1, 3 and 4, with the config-1 reference records."""
+    w = wl.config1()
+    model = Model(lib, w, B_max=8, with_colnorm=True)
+    r_ref = f32_of(wl.reference_input(w))[None]
+    out, rec = gpu_dense_records(model, r_ref)
+    want_out, want_rec = oracle.step(model.Wg, model.Wu, model.Wd, r_ref[0], return_records=True)
+    assert_close(out[0], want_out, "dense reference step")
+    records_close(rec.cpu().numpy()[0], want_rec)
+    yield model, rec, want_rec
+    model.close()
+
+
+def test_config1_stack_top25_reused_for_10_steps(lib, pi0):
+    model, rec, want_rec = pi0
+    w = model.w
+    K = w.K
+    assert K == 1024
+    idx, cnt, h_idx, h_cnt = gpu_topk_lists(lib, model, [rec], K, w.L)
+    rec_bytes = rec.cpu().numpy()[0]
+    jac = []
+    for l in range(w.L):
+        want = oracle.compact_scores(rec_bytes[l], oracle.RULE_TOPK, k=K)
+        assert h_cnt[l] == K and np.array_equal(h_idx[l, :K], want), f"layer {l}: list differs"
+        jac.append(jaccard(want, oracle.compact_scores(want_rec[l], oracle.RULE_TOPK, k=K)))
+    print(f"config1: top-k Jaccard GPU-record vs oracle-record lists: min {min(jac):.4f}")
+    rels = []
+    for s in range(w.steps):
+        r0 = f32_of(wl.step_input(w, s))
+        got = gpu_sparse_step(model, r0[None], idx, cnt)[0]
+        want = oracle.step(model.Wg, model.Wu, model.Wd, r0, h_idx, h_cnt)
+        rels.append(assert_close(got, want, f"config 1 step {s}"))
+    print(f"config1: rel_l2 per step max {max(rels):.2e}")
+    # Eq. 1 variant of the record: scale = ||W_down[:,n]||_2 computed by the pack kernel
+    cn = np.stack([c.cpu().numpy() for c in model.colnorm])
+    for l in (0, 7, 17):
+        assert np.allclose(cn[l], oracle.down_colnorm(model.Wd[l]), rtol=1e-5)
+    assert model.ctx.rm_device_status() == 0
+
+
+@pytest.mark.parametrize("density", [0.05, 0.10, 0.20, 0.40, 0.50, 1.0])
+def test_config3_density_sweep(lib, pi0, density):
+    model, rec, _ = pi0
+    w = wl.config3(density)
+    K = w.K
+    idx, cnt, h_idx, h_cnt = gpu_topk_lists(lib, model, [rec], K, w.L)
+    rec_bytes = rec.cpu().numpy()[0]
+    for l in range(w.L):
+        assert np.array_equal(h_idx[l, :h_cnt[l]], oracle.compact_scores(rec_bytes[l], oracle.RULE_TOPK, k=K))
+    r0 = f32_of(wl.step_input(wl.config1(), 3))
+    got = gpu_sparse_step(model, r0[None], idx, cnt)[0]
+    if density < 1.0:
+        want = oracle.step(model.Wg, model.Wu, model.Wd, r0, h_idx, h_cnt)
+        assert_close(got, want, f"config 3 rho={density}")
+    else:
+        # density 1.0 is checked against the oracle's separate dense loop, as a full list and as idx = NULL
+        want = oracle.step(model.Wg, model.Wu, model.Wd, r0)
+        assert_close(got, want, "config 3 rho=1.0 (full list)")
+        import torch
+        out = torch.empty(1, w.T, w.H, dtype=torch.float32, device="cuda")
+        model.ctx.rm_action_expert_step(model.packed, dev(r0[None]), None, None, 0, out, B=1, T=w.T)
+        assert_close(out.cpu().numpy()[0], want, "config 3 rho=1.0 (idx NULL)")
+
+
+def test_config3_batched_eight_episodes(lib, pi0):
+    model, _, _ = pi0
+    B = 8
+    w = wl.config3(0.25, B=B)
+    refs = np.stack([f32_of(wl.reference_input(w, episode=b)) for b in range(B)])
+    out, rec = gpu_dense_records(model, refs, B=B)
+    for b in (0, 5):                                               # two episodes of the dense pass in full
+        want_out, want_rec = oracle.step(model.Wg, model.Wu, model.Wd, refs[b], return_records=True)
+        assert_close(out[b], want_out, f"batched dense, episode {b}")
+        records_close(rec.cpu().numpy()[b], want_rec)
+    K = w.K
+    idx, cnt, h_idx, h_cnt = gpu_topk_lists(lib, model, [rec.view(B * w.L, w.I)], K, B * w.L)
+    rec_bytes = rec.cpu().numpy().reshape(B * w.L, w.I)
+    union = np.zeros((w.L, w.I), bool)
+    for i in range(B * w.L):
+        want = oracle.compact_scores(rec_bytes[i], oracle.RULE_TOPK, k=K)
+        assert h_cnt[i] == K and np.array_equal(h_idx[i, :K], want)
+        union[i % w.L, want] = True
+    print(f"config3 batched: mean union size per layer {union.sum(1).mean():.0f} of {w.I}")
+    steps = np.stack([f32_of(wl.step_input(w, 2, episode=b)) for b in range(B)])
+    got = gpu_sparse_step(model, steps, idx, cnt, B=B)
+    for b in range(B):
+        want = oracle.step(model.Wg, model.Wu, model.Wd, steps[b], h_idx[b * w.L:(b + 1) * w.L],
+                           h_cnt[b * w.L:(b + 1) * w.L])
+        assert_close(got[b], want, f"batched sparse, episode {b}")
+    assert model.ctx.rm_device_status() == 0
+
+
+def test_config4_run_structured_vote_window(lib, pi0):
+    import torch
+    model1, _, _ = pi0
+    w = wl.config4()
+    # same weights, T = 32: a second context on the same packed layers
+    ctx = lib.Context(w.L, w.H, w.I, T_max=w.T)
+
+    class View:
+        pass
+    model = View()
+    model.w, model.ctx, model.packed = w, ctx, model1.packed
+    Wg, Wu, Wd = model1.Wg, model1.Wu, model1.Wd
+    members, scales = zip(*[wl.run_structure(w, l) for l in range(w.L)])
+    scale = np.stack(scales)                                      # [L, I]: 4 inside a run, 1 elsewhere
+    n_rec = 7                                                      # three sliding windows of 4 over 7 records
+    recs = []
+    for i in range(n_rec):
+        r_ref = f32_of(wl.reference_input(w, record=i))[None]
+        out, rec = gpu_dense_records(model, r_ref, scale=scale)
+        recs.append(rec)
+        if i in (0, 4):
+            want_out, want_rec = oracle.step(Wg, Wu, Wd, r_ref[0], scale=scale, return_records=True)
+            assert_close(out[0], want_out, f"config 4 dense reference {i}")
+            records_close(rec.cpu().numpy()[0], want_rec)
+    K, votes = w.K, w.extra["min_votes"]
+    assert K == 615 and votes == 3
+    for start in (0, 1, 3):
+        window = recs[start:start + w.extra["window"]]
+        idx, cnt, h_idx, h_cnt = gpu_topk_lists(lib, model, window, K, w.L, min_votes=votes)
+        host = [r.cpu().numpy()[0] for r in window]
+        dens, runs = [], []
+        for l in range(w.L):
+            want = oracle.compact_scores([h[l] for h in host], oracle.RULE_TOPK, k=K, min_votes=votes)
+            assert h_cnt[l] == want.size and np.array_equal(h_idx[l, :want.size], want), f"window {start} layer {l}"
+            dens.append(want.size / w.I)
+            if want.size:
+                runs.append(want.size / (1 + np.count_nonzero(np.diff(want) != 1)))
+        print(f"config4 window {start}: density {np.mean(dens):.3f}, mean run length {np.mean(runs):.1f}")
+        for s in ((0, 4, 9) if start else range(w.steps)):
+            r0 = f32_of(wl.step_input(w, s))
+            got = gpu_sparse_step(model, r0[None], idx, cnt)[0]
+            assert_close(got, oracle.step(Wg, Wu, Wd, r0, h_idx, h_cnt), f"config 4 window {start} step {s}")
+    assert ctx.rm_device_status() == 0
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------------------------ config 2
+def test_config2_large_refresh_every_two_steps(lib):
+    # full H = 2048 / I = 16384 / T = 51 geometry; three layers keep the oracle's dense passes to seconds
+    w = wl.config2(L=3)
+    model = Model(lib, w)
+    K = w.K
+    assert K == 3277
+    idx = cnt = h_idx = h_cnt = None
+    for s in range(4):
+        r0 = f32_of(wl.step_input(w, s))
+        if s % w.extra["refresh_every"] == 0:
+            out, rec = gpu_dense_records(model, r0[None])
+            want_out, want_rec = oracle.step(model.Wg, model.Wu, model.Wd, r0, return_records=True)
+            assert_close(out[0], want_out, f"config 2 dense step {s}")
+            records_close(rec.cpu().numpy()[0], want_rec)
+            idx, cnt, h_idx, h_cnt = gpu_topk_lists(lib, model, [rec], K, w.L)
+            rec_bytes = rec.cpu().numpy()[0]
+            for l in range(w.L):
+                want = oracle.compact_scores(rec_bytes[l], oracle.RULE_TOPK, k=K)
+                assert h_cnt[l] == K and np.array_equal(h_idx[l, :K], want)
+        else:
+            got = gpu_sparse_step(model, r0[None], idx, cnt)[0]
+            assert_close(got, oracle.step(model.Wg, model.Wu, model.Wd, r0, h_idx, h_cnt), f"config 2 sparse step {s}")
+    assert model.ctx.rm_device_status() == 0
+    model.close()

@@ -1,0 +1,183 @@
+"""rm_pack_weights + rm_sparse_mlp + rm_action_expert_step against the oracle, element by element."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_19104_b200 import workloads as wl
+from harness import Model, assert_close, dev, dev_bf16, lists_to_padded
+
+pytestmark = pytest.mark.gpu
+
+
+def tiny(H=128, I=200, T=7, L=1, sigma=0.05, config=90, **kw):
+    return wl.Workload(config, "tiny", L, H, I, T, sigma, 1, 0.3, **kw)
+
+
+def run_layer(lib, model, x_bits, r, idx_list, dense=False, record=False, scale=None):
+    import torch
+    w = model.w
+    T = x_bits.shape[0]
+    y = torch.empty(T, w.H, dtype=torch.float32, device="cuda")
+    rec = torch.zeros(w.I, dtype=torch.float32, device="cuda") if record else None
+    idx = cnt = None
+    if not dense:
+        buf = np.zeros(max(w.I, 4), dtype=np.int32)
+        buf[:len(idx_list)] = idx_list
+        idx, cnt = dev(buf), dev(np.array([len(idx_list)], dtype=np.int32))
+    model.ctx.rm_sparse_mlp(model.packed[0], dev_bf16(x_bits), None if r is None else dev(r), idx, cnt, y,
+                            record_out=rec, record_scale=None if scale is None else dev(scale))
+    torch.cuda.synchronize()
+    return y.cpu().numpy(), (None if rec is None else rec.cpu().numpy())
+
+
+@pytest.mark.parametrize("H,I,T", [(64, 40, 1), (128, 200, 7), (256, 333, 51), (512, 1000, 70), (1024, 4096, 51),
+                                   (2048, 512, 32)])
+def test_single_layer_masked_and_dense(lib, H, I, T):
+    w = tiny(H=H, I=I, T=T, sigma=0.5 / np.sqrt(H))
+    model = Model(lib, w)
+    x = wl.step_input(w, 0)
+    r = wl.residual_input(w)
+    mask = wl.bernoulli_mask(w)
+    idx = np.flatnonzero(mask).astype(np.int32)
+    got, _ = run_layer(lib, model, x, r, idx)
+    assert_close(got, oracle.masked_mlp(x, model.Wg[0], model.Wu[0], model.Wd[0], r, idx), "masked")
+    # no residual
+    got, _ = run_layer(lib, model, x, None, idx)
+    assert_close(got, oracle.masked_mlp(x, model.Wg[0], model.Wu[0], model.Wd[0], None, idx), "masked, r=NULL")
+    # dense (idx NULL) with the activation record, and the full list
+    got, rec = run_layer(lib, model, x, r, None, dense=True, record=True)
+    want, want_rec = oracle.dense_mlp(x, model.Wg[0], model.Wu[0], model.Wd[0], r, return_record=True)
+    assert_close(got, want, "dense")
+    assert np.all(np.abs(rec - want_rec) <= 1e-2 * np.abs(want_rec) + 2e-2)
+    got, _ = run_layer(lib, model, x, r, np.arange(I, dtype=np.int32))
+    assert_close(got, want, "all-ones list")
+    assert model.ctx.rm_device_status() == 0
+    model.close()
+
+
+def test_empty_mask_returns_the_residual_exactly(lib):
+    w = tiny(H=256, I=300, T=9)
+    model = Model(lib, w)
+    x, r = wl.step_input(w, 0), wl.residual_input(w)
+    got, _ = run_layer(lib, model, x, r, np.zeros(0, np.int32))
+    assert got.tobytes() == r.tobytes()
+    got, _ = run_layer(lib, model, x, None, np.zeros(0, np.int32))
+    assert not got.any()
+    model.close()
+
+
+def test_exact_integer_case(lib):
+    # small integers and |g| >= 22: GeLU-tanh is exactly ReLU and every value is an integer below 2^24
+    rng = np.random.default_rng(5)
+    T, H, I = 6, 64, 96
+    x = rng.integers(1, 4, size=(T, H)).astype(np.float32)
+    x[:, 0] = 1.0
+    Wg = rng.integers(0, 3, size=(I, H)).astype(np.float32)
+    Wg[:, 1:] *= (rng.integers(0, 8, size=(I, H - 1)) == 0)                  # keep sum small
+    Wg[:, 0] = 512.0 * np.where(rng.integers(0, 2, size=I) == 0, -1.0, 1.0)
+    Wu = rng.integers(-2, 3, size=(I, H)).astype(np.float32) * (rng.integers(0, 4, size=(I, H)) == 0)
+    Wd = rng.integers(-3, 4, size=(H, I)).astype(np.float32)
+    r = rng.integers(-9, 10, size=(T, H)).astype(np.float32)
+    idx = np.flatnonzero(rng.integers(0, 2, size=I)).astype(np.int32)
+    import torch
+    ctx = lib.Context(1, H, I, T)
+    bits = wl.f32_to_bf16_bits
+    packed = ctx.rm_pack_weights(dev_bf16(bits(Wg)), dev_bf16(bits(Wu)), dev_bf16(bits(Wd)))
+    y = torch.empty(T, H, dtype=torch.float32, device="cuda")
+    buf = np.zeros(I, np.int32)
+    buf[:idx.size] = idx
+    ctx.rm_sparse_mlp(packed, dev_bf16(bits(x)), dev(r), dev(buf), dev(np.array([idx.size], np.int32)), y)
+    xi, gi, ui, di = (a.astype(np.int64) for a in (x, Wg, Wu, Wd))
+    g = xi @ gi.T
+    assert np.min(np.abs(g)) >= 10
+    want = r.astype(np.int64) + (np.maximum(g, 0) * (xi @ ui.T))[:, idx] @ di[:, idx].T
+    got = y.cpu().numpy()
+    # the tensor-core path rounds h to bf16; |h| here stays below 2^8 * small, so compare with a tight tolerance
+    assert np.max(np.abs(got - want)) <= 4e-3 * np.max(np.abs(want)) + 1e-3
+    ctx.close()
+
+
+def test_bad_index_is_reported_not_fatal(lib):
+    w = tiny(H=128, I=100, T=4)
+    model = Model(lib, w)
+    x, r = wl.step_input(w, 0), wl.residual_input(w)
+    idx = np.array([1, 5, 100, 7], dtype=np.int32)             # 100 is out of range
+    got, _ = run_layer(lib, model, x, r, idx)
+    assert model.ctx.rm_device_status() == lib.RM_ERR_INDEX
+    assert model.ctx.rm_device_status() == 0                      # cleared by the read
+    want = oracle.masked_mlp(x, model.Wg[0], model.Wu[0], model.Wd[0], r, np.array([1, 5, 7], np.int32))
+    assert_close(got, want, "bad index skipped")
+    model.close()
+
+
+def test_argument_errors(lib):
+    import torch
+    w = tiny(H=128, I=100, T=4)
+    model = Model(lib, w)
+    x = dev_bf16(wl.step_input(w, 0))
+    y = torch.empty(4, 128, dtype=torch.float32, device="cuda")
+    ctx = model.ctx
+    with pytest.raises(lib.RmError) as e:
+        ctx.rm_sparse_mlp(model.packed[0], x, None, None, None, y, T=5)
+    assert e.value.code == lib.RM_ERR_SHAPE
+    with pytest.raises(lib.RmError) as e:
+        ctx.rm_sparse_mlp(model.packed[0], x, None, None, None, y, ws=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == lib.RM_ERR_WORKSPACE
+    with pytest.raises(lib.RmError) as e:
+        ctx.rm_sparse_mlp(model.packed[0], x, None, torch.zeros(4, dtype=torch.int32, device="cuda"), None, y)
+    assert e.value.code == lib.RM_ERR_INVALID_ARG
+    with pytest.raises(lib.RmError) as e:
+        ctx.rm_sparse_mlp(model.packed[0], x.view(-1)[1:], None, None, None, y, T=3)
+    assert e.value.code == lib.RM_ERR_ALIGN
+    model.close()
+
+
+@pytest.mark.parametrize("H,I,T,L,B", [(128, 256, 5, 3, 1), (256, 512, 51, 4, 2), (512, 640, 33, 2, 3)])
+def test_step_masked_and_dense_small(lib, H, I, T, L, B):
+    import torch
+    w = tiny(H=H, I=I, T=T, L=L, sigma=1.0 / np.sqrt(H), B=B)
+    model = Model(lib, w, B_max=B)
+    r0 = np.stack([wl.bf16_bits_to_f32(wl.step_input(w, 0, episode=b)) for b in range(B)])
+    lists = [[np.flatnonzero(wl.bernoulli_mask(w, layer=l, episode=b)).astype(np.int32) for l in range(L)]
+             for b in range(B)]
+    stride = (I + 3) // 4 * 4
+    flat = [s for per_b in lists for s in per_b]
+    idx, cnt = lists_to_padded(flat, stride)
+    r_out = torch.empty(B, T, H, dtype=torch.float32, device="cuda")
+    model.ctx.rm_action_expert_step(model.packed, dev(r0), dev(idx), dev(cnt), stride, r_out, B=B, T=T)
+    got = r_out.cpu().numpy()
+    for b in range(B):
+        i_b, c_b = lists_to_padded(lists[b], stride)
+        want = oracle.step(model.Wg, model.Wu, model.Wd, r0[b], i_b, c_b)
+        assert_close(got[b], want, f"masked step, episode {b}")
+    # dense with records and a per-layer scale; in place
+    scale = (0.5 + wl.uniform(wl.tensor_key(1, 91, 0, 1), L * I)).astype(np.float32).reshape(L, I)
+    rec = torch.zeros(B, L, I, dtype=torch.float32, device="cuda")
+    r_io = dev(r0)
+    model.ctx.rm_action_expert_step(model.packed, r_io, None, None, 0, r_io, records_out=rec,
+                                    record_scale=dev(scale), B=B, T=T)
+    got, got_rec = r_io.cpu().numpy(), rec.cpu().numpy()
+    for b in range(B):
+        want, want_rec = oracle.step(model.Wg, model.Wu, model.Wd, r0[b], scale=scale, return_records=True)
+        assert_close(got[b], want, f"dense step, episode {b}")
+        assert np.all(np.abs(got_rec[b] - want_rec) <= 1e-2 * np.abs(want_rec) + 2e-2)
+    assert model.ctx.rm_device_status() == 0
+    model.close()
+
+
+def test_step_host_variant_matches_device_variant(lib):
+    import torch
+    w = tiny(H=256, I=512, T=17, L=3, sigma=1.0 / 16)
+    model = Model(lib, w)
+    r0 = wl.bf16_bits_to_f32(wl.step_input(w, 0))
+    lists = [np.flatnonzero(wl.bernoulli_mask(w, layer=l)).astype(np.int32) for l in range(w.L)]
+    idx, cnt = lists_to_padded(lists, w.I)
+    d_idx, d_cnt = dev(idx), dev(cnt)
+    r_out = torch.empty(w.T, w.H, dtype=torch.float32, device="cuda")
+    model.ctx.rm_action_expert_step(model.packed, dev(r0), d_idx, d_cnt, w.I, r_out, B=1, T=w.T)
+    h_in = torch.from_numpy(r0).pin_memory()
+    h_out = torch.empty(w.T, w.H, dtype=torch.float32).pin_memory()
+    model.ctx.rm_action_expert_step_host(model.packed, h_in, d_idx, d_cnt, w.I, h_out, B=1, T=w.T)
+    assert_close(h_out.numpy(), r_out.cpu().numpy(), "host variant")
+    assert_close(h_out.numpy(), oracle.step(model.Wg, model.Wu, model.Wd, r0, idx, cnt), "host variant vs oracle")
+    model.close()
