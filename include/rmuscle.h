@@ -138,6 +138,25 @@ int rm_device_status(rm_ctx* ctx, int* host_out, rm_stream_t stream);
 /* Number of kernels the library has launched through this context since creation (host counter). */
 int64_t rm_launch_count(const rm_ctx* ctx);
 
+/* Tuning knobs (host-side, take effect on later calls).  Names:
+ *   "path"                0 = choose per shape (default), 1 = portable CUDA-core kernels only, 2 = the tcgen05
+ *                         cluster kernel or RM_ERR_UNSUPPORTED
+ *   "pdl"                 1 = chain the layers of a step with programmatic dependent launch (default)
+ *   "neurons_per_cluster" active neurons a cluster should get before another cluster is used (default 64)
+ *   "count_hint"          expected active neurons per layer and episode; lets a launch use only as many clusters
+ *                         as that needs, so that the next layer's CTAs can become resident early (0 = unknown)
+ *   "max_clusters"        cap on the clusters per launch (0 = none)                                              */
+int rm_set_option(rm_ctx* ctx, const char* name, int value);
+
+/* Read-only facts: "fused_clusters" (co-resident clusters of the tcgen05 kernel, 0 when that path is
+ * unavailable for this geometry or device), "sm_count", "path". */
+int rm_get_info(const rm_ctx* ctx, const char* name, int* out);
+
+/* Profiling aid, available only in builds made with -DRM_PHASE_TIMING (RM_ERR_UNSUPPORTED otherwise): copies the
+ * per-CTA clock stamps the fused layer kernel took at its phase boundaries (host_out: n int64 values, 32 per CTA).
+ * Host-synchronous. */
+int rm_debug_phase_times(rm_ctx* ctx, long long* host_out, int n);
+
 const char* rm_status_string(int status);
 
 #ifdef __cplusplus

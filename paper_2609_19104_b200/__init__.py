@@ -22,7 +22,8 @@ RM_REDUCE_NONE, RM_REDUCE_THRESHOLD, RM_REDUCE_TOPK, RM_REDUCE_GROUP = 0, 1, 2, 
 
 EXPORTS = ["rm_create", "rm_destroy", "rm_packed_layer_bytes", "rm_workspace_bytes", "rm_pack_weights",
            "rm_mask_compact", "rm_sparse_mlp", "rm_action_expert_step", "rm_action_expert_step_host",
-           "rm_device_status", "rm_launch_count", "rm_status_string"]
+           "rm_device_status", "rm_launch_count", "rm_status_string", "rm_set_option", "rm_get_info",
+           "rm_debug_phase_times"]
 
 
 class RmError(RuntimeError):
@@ -70,6 +71,9 @@ def load_library() -> ctypes.CDLL:
     lib.rm_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
     lib.rm_launch_count.argtypes = [vp]
     lib.rm_launch_count.restype = i64
+    lib.rm_set_option.argtypes = [vp, ctypes.c_char_p, i32]
+    lib.rm_get_info.argtypes = [vp, ctypes.c_char_p, ctypes.POINTER(ctypes.c_int)]
+    lib.rm_debug_phase_times.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong), i32]
     lib.rm_status_string.argtypes = [i32]
     lib.rm_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -135,6 +139,21 @@ class Context:
         if self._ws is None or self._ws.numel() < need:
             self._ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
         return self._ws
+
+    def rm_set_option(self, name: str, value: int) -> None:
+        _check(self.lib.rm_set_option(self._h, name.encode(), int(value)), f"rm_set_option({name})")
+
+    def rm_get_info(self, name: str) -> int:
+        v = ctypes.c_int(0)
+        _check(self.lib.rm_get_info(self._h, name.encode(), ctypes.byref(v)), f"rm_get_info({name})")
+        return int(v.value)
+
+    def rm_debug_phase_times(self, n_ctas: int):
+        """Clock stamps [n_ctas, 32] of the last fused-layer launch (builds with -DRM_PHASE_TIMING only)."""
+        import numpy as np
+        buf = (ctypes.c_longlong * (n_ctas * 32))()
+        _check(self.lib.rm_debug_phase_times(self._h, buf, n_ctas * 32), "rm_debug_phase_times")
+        return np.frombuffer(buf, dtype=np.int64).reshape(n_ctas, 32).copy()
 
     def launch_count(self) -> int:
         return int(self.lib.rm_launch_count(self._h))

@@ -31,7 +31,8 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         tmp = LIB + f".tmp{os.getpid()}"
-        cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp, *sources()]
+        extra = os.environ.get("RM_EXTRA_NVCC_FLAGS", "").split()
+        cmd = [nvcc, *NVCC_FLAGS, *extra, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp, *sources()]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")

@@ -1,5 +1,6 @@
 // C-ABI entry points: argument validation and dispatch.  Every step of the path runs in the library's kernels.
 #include <new>
+#include <string>
 
 #include "rm_common.cuh"
 
@@ -11,6 +12,10 @@ inline bool all_aligned(std::initializer_list<const void*> ps) {
     for (const void* p : ps)
         if (p && !rm_aligned16(p)) return false;
     return true;
+}
+
+inline bool use_fused(const rm_ctx* ctx, int B, int T) {
+    return ctx->path != 1 && rm_fused_supported(ctx, B, T);
 }
 
 }  // namespace
@@ -41,6 +46,15 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
         return RM_ERR_CUDA;
     }
     c->sm_count = prop.multiProcessorCount;
+    c->path = 0;
+    c->use_pdl = 1;
+    c->npc_target = 64;
+    c->count_hint = 0;
+    c->max_clusters_override = 0;
+    c->fused_clusters = 0;
+    c->fused_blocks_per_sm = 0;
+    if (prop.major == 10) rm_fused_init(c);                 // failure leaves the portable path in charge
+    cudaGetLastError();
     *out = c;
     return RM_OK;
 }
@@ -58,9 +72,9 @@ size_t rm_packed_layer_bytes(const rm_ctx* ctx) {
 
 size_t rm_workspace_bytes(const rm_ctx* ctx, int B, int T) {
     if (!ctx || B < 1 || T < 1) return 0;
-    // layer scratch + two residual-stream buffers (ping-pong between layers, and the host variant's staging)
+    // three rotating residual-stream buffers, the host variant's staging buffer, then the portable path's scratch
     size_t r_bytes = align_up((size_t)B * T * ctx->g.H * sizeof(float), 256);
-    return rm_ref_workspace_bytes(ctx, B, T) + 2 * r_bytes;
+    return 4 * r_bytes + rm_ref_workspace_bytes(ctx, B, T);
 }
 
 int rm_pack_weights(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, void* packed_out,
@@ -120,21 +134,47 @@ int rm_sparse_mlp(rm_ctx* ctx, const void* packed_layer, const void* x, const fl
     a.record_scale = record_scale;
     a.B = 1;
     a.T = T;
-    return rm_launch_layer_ref(ctx, a, ws, static_cast<cudaStream_t>(stream));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t r_bytes = align_up((size_t)T * ctx->g.H * sizeof(float), 256);
+    if (use_fused(ctx, 1, T)) {
+        // y accumulates the CTAs' partial sums with atomics: start it from the residual (or zero)
+        if (y != residual) {
+            if (residual) RM_CUDA_TRY(cudaMemcpyAsync(y, residual, (size_t)T * ctx->g.H * sizeof(float),
+                                                      cudaMemcpyDeviceToDevice, s));
+            else RM_CUDA_TRY(cudaMemsetAsync(y, 0, (size_t)T * ctx->g.H * sizeof(float), s));
+        }
+        return rm_launch_layer_fused(ctx, a, nullptr, false, false, s);
+    }
+    if (ctx->path == 2) return RM_ERR_UNSUPPORTED;
+    return rm_launch_layer_ref(ctx, a, static_cast<char*>(ws) + 4 * r_bytes, s);
 }
 
 static int step_device(rm_ctx* ctx, const void* const* packed_layers, const float* r_in, const int32_t* idx,
                        const int32_t* count_dev, int64_t stride, float* r_out, float* records_out,
                        const float* record_scale, int B, int T, void* ws, cudaStream_t s) {
     const rm_geom& g = ctx->g;
-    char* layer_ws = static_cast<char*>(ws);
+    const size_t n_bytes = (size_t)B * T * g.H * sizeof(float);
+    const size_t r_bytes = align_up(n_bytes, 256);
+    char* layer_ws = static_cast<char*>(ws) + 4 * r_bytes;
+    const bool fused = use_fused(ctx, B, T);
+    if (!fused && ctx->path == 2) return RM_ERR_UNSUPPORTED;
+    float* rot[3] = {reinterpret_cast<float*>(static_cast<char*>(ws)),
+                     reinterpret_cast<float*>(static_cast<char*>(ws) + r_bytes),
+                     reinterpret_cast<float*>(static_cast<char*>(ws) + 2 * r_bytes)};
+    // Fused path: layer l reads rot[l%3] (the caller's r_in for l = 0), accumulates into rot[(l+1)%3] and clears
+    // rot[(l+2)%3] for the layer after next; the last layer accumulates straight into r_out when that is a
+    // different buffer from r_in.
+    const bool direct_out = fused && r_out != r_in;
+    if (fused) {
+        RM_CUDA_TRY(cudaMemsetAsync(g.L == 1 && direct_out ? r_out : rot[1], 0, n_bytes, s));
+        if (direct_out && g.L > 1) RM_CUDA_TRY(cudaMemsetAsync(r_out, 0, n_bytes, s));
+    }
     const float* cur = r_in;
     for (int l = 0; l < g.L; ++l) {
         rm_layer_args a{};
         a.packed = static_cast<const __nv_bfloat16*>(packed_layers[l]);
         a.x = nullptr;
         a.r_in = cur;
-        a.r_out = r_out;                                   // in place after the first layer
         a.idx = idx ? idx + (size_t)l * stride : nullptr;
         a.count = idx ? count_dev + l : nullptr;
         a.idx_stride = (int64_t)g.L * stride;
@@ -145,10 +185,23 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
         a.record_scale = record_scale ? record_scale + (size_t)l * g.I : nullptr;
         a.B = B;
         a.T = T;
-        int rc = rm_launch_layer_ref(ctx, a, layer_ws, s);
+        int rc;
+        if (fused) {
+            const bool last = l == g.L - 1;
+            a.r_out = (last && direct_out) ? r_out : rot[(l + 1) % 3];
+            // the buffer cleared here is the output of layer l+1 (unless that layer writes to r_out directly); it
+            // was the input of layer l-1, which has completed by the time this layer passes its dependency wait
+            float* zero = (l + 1 < g.L && !(l + 1 == g.L - 1 && direct_out)) ? rot[(l + 2) % 3] : nullptr;
+            rc = rm_launch_layer_fused(ctx, a, zero, true, ctx->use_pdl && l > 0, s);
+            cur = a.r_out;
+        } else {
+            a.r_out = r_out;                               // in place after the first layer
+            rc = rm_launch_layer_ref(ctx, a, layer_ws, s);
+            cur = r_out;
+        }
         if (rc != RM_OK) return rc;
-        cur = r_out;
     }
+    if (fused && !direct_out) RM_CUDA_TRY(cudaMemcpyAsync(r_out, cur, n_bytes, cudaMemcpyDeviceToDevice, s));
     return RM_OK;
 }
 
@@ -187,9 +240,8 @@ int rm_action_expert_step_host(rm_ctx* ctx, const void* const* packed_layers, co
     if (!ws || ws_bytes < rm_workspace_bytes(ctx, B, T)) return RM_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t n_bytes = (size_t)B * T * ctx->g.H * sizeof(float);
-    // the last residual-stream buffer of the workspace is the staging copy
-    float* stage = reinterpret_cast<float*>(static_cast<char*>(ws) + rm_workspace_bytes(ctx, B, T) -
-                                            align_up(n_bytes, 256));
+    // the fourth residual-stream buffer of the workspace is the staging copy
+    float* stage = reinterpret_cast<float*>(static_cast<char*>(ws) + 3 * align_up(n_bytes, 256));
     RM_CUDA_TRY(cudaMemcpyAsync(stage, r_in_host, n_bytes, cudaMemcpyHostToDevice, s));
     int rc = step_device(ctx, packed_layers, stage, idx, count_dev, stride, stage, nullptr, nullptr, B, T, ws, s);
     if (rc != RM_OK) return rc;
@@ -210,6 +262,45 @@ int rm_device_status(rm_ctx* ctx, int* host_out, rm_stream_t stream) {
 }
 
 int64_t rm_launch_count(const rm_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int rm_set_option(rm_ctx* ctx, const char* name, int value) {
+    if (!ctx || !name) return RM_ERR_INVALID_ARG;
+    const std::string n(name);
+    if (n == "path") {
+        if (value < 0 || value > 2) return RM_ERR_INVALID_ARG;
+        ctx->path = value;
+    } else if (n == "pdl") {
+        ctx->use_pdl = value != 0;
+    } else if (n == "neurons_per_cluster") {
+        if (value < 1) return RM_ERR_INVALID_ARG;
+        ctx->npc_target = value;
+    } else if (n == "count_hint") {
+        if (value < 0) return RM_ERR_INVALID_ARG;
+        ctx->count_hint = value;
+    } else if (n == "max_clusters") {
+        if (value < 0) return RM_ERR_INVALID_ARG;
+        ctx->max_clusters_override = value;
+    } else {
+        return RM_ERR_INVALID_ARG;
+    }
+    return RM_OK;
+}
+
+int rm_get_info(const rm_ctx* ctx, const char* name, int* out) {
+    if (!ctx || !name || !out) return RM_ERR_INVALID_ARG;
+    const std::string n(name);
+    if (n == "fused_clusters") *out = ctx->fused_clusters;
+    else if (n == "fused_blocks_per_sm") *out = ctx->fused_blocks_per_sm;
+    else if (n == "sm_count") *out = ctx->sm_count;
+    else if (n == "path") *out = ctx->path;
+    else return RM_ERR_INVALID_ARG;
+    return RM_OK;
+}
+
+int rm_debug_phase_times(rm_ctx* ctx, long long* host_out, int n) {
+    if (!ctx || !host_out || n < 0) return RM_ERR_INVALID_ARG;
+    return rm_fused_debug_stamps(host_out, n);
+}
 
 const char* rm_status_string(int status) {
     switch (status) {

@@ -30,6 +30,14 @@ struct rm_ctx {
     int sm_count;
     int* d_status;                         // device status word
     int64_t launches;                      // host-side launch counter
+    // tensor-core path (rm_mlp_sm100.cu)
+    int fused_clusters;                    // co-resident 8-CTA clusters of the fused layer kernel (0: unavailable)
+    int fused_blocks_per_sm;               // CTAs of that kernel one SM can hold
+    int path;                              // 0 auto, 1 portable kernels only, 2 fused kernel required
+    int use_pdl;                           // chain layers with programmatic dependent launch
+    int npc_target;                        // neurons per cluster aimed for when spreading a layer
+    int count_hint;                        // expected active neurons per layer and episode (0: unknown)
+    int max_clusters_override;             // > 0: cap on clusters per launch
 };
 
 #define RM_CUDA_TRY(expr)                                  \
@@ -73,4 +81,10 @@ struct rm_layer_args {
     int B, T;
 };
 size_t rm_ref_workspace_bytes(const rm_ctx* ctx, int B, int T);
+// Tensor-core path: H in {1024, 2048}, T <= 64 per episode, B <= 64.
+int rm_fused_init(rm_ctx* ctx);
+int rm_fused_debug_stamps(long long* host_out, int n);
+bool rm_fused_supported(const rm_ctx* ctx, int B, int T);
+int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& a, float* zero_buf, bool add_residual, bool pdl,
+                          cudaStream_t s);
 int rm_launch_layer_ref(rm_ctx* ctx, const rm_layer_args& a, void* ws, cudaStream_t s);
