@@ -30,6 +30,9 @@ from paper_2609_19104_b200 import workloads as wl  # noqa: E402
 METRIC = "masked_mlp_us_per_denoise_step"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one fused layer launch, from the ncu capture summarised in
+# profiles/fused_layer_config1.md
+TRAFFIC_BYTES_PER_LAUNCH = {"pi0-stack-top25": 6.78e6}
 
 
 def measured_hbm_peak():
@@ -170,6 +173,7 @@ def run_gpu(args, w: wl.Workload):
 
     B = w.B
     ctx = rm.Context(w.L, w.H, w.I, T_max=w.T, B_max=B)
+    ctx.rm_set_option("count_hint", w.K)          # the lists hold K neurons: launch one cluster per 64-neuron tile
     # weights: the workload's seeded draws (same on every rank: replicas of one model)
     packed = []
     for l in range(w.L):
@@ -282,7 +286,9 @@ def run_gpu(args, w: wl.Workload):
         peak, peak_kind = measured_hbm_peak()
         bytes_layer = wl.algorithmic_bytes_per_layer(w.H, w.T, int(round(K_mean))) * B
         bytes_step = bytes_layer * w.L
-        achieved = bytes_layer / (layer_us * 1e-6) / 1e9
+        launches_per_step = launches / args.steps                 # fused layer launches + mask compaction share
+        in_step_layer_us = us_per_step * B / w.L                  # average duration of a layer launch inside the step
+        achieved = bytes_layer / (in_step_layer_us * 1e-6) / 1e9
         io_bytes = B * w.T * w.H * 4
         cpu_us, cores, sample = time_oracle(w, steps=3, warmup=1) if world == 1 else (None, None, None)
         line = {
@@ -294,11 +300,11 @@ def run_gpu(args, w: wl.Workload):
                        "l2": "flushed before every timed step (512 MB fill, outside the timed interval)",
                        "multi_gpu": "replicas: each rank runs its own episodes, no collective on the data path"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_kind": f"{peak_kind} copy bandwidth",
-                         "kernel": "one layer of the masked MLP (rm_sparse_mlp launch sequence)",
-                         "bytes_per_launch": bytes_layer, "us_per_launch": layer_us,
-                         "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                         "step_effective_gbs": bytes_step / (us_per_step * B * 1e-6) / 1e9},
+                         "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name), "peak_kind": f"{peak_kind} copy bandwidth",
+                         "kernel": "fused_layer_kernel (one launch per layer, dependent-launch chained)",
+                         "bytes_per_launch": bytes_layer, "us_per_launch": in_step_layer_us,
+                         "us_per_launch_isolated_cold": layer_us, "launches_per_step": launches_per_step,
+                         "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
             "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes},
             "gpu_launches": int(launches),
             "clocks": clocks,

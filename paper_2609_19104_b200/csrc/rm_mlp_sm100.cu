@@ -1,20 +1,22 @@
 // Fused masked gated-MLP layer for sm_100a: one kernel per layer, thread-block clusters of 8 CTAs.
 //
-// Decomposition.  A cluster owns a contiguous range of the active neurons of a layer and walks it in tiles of 64
-// neurons.  CTA j of the cluster owns column slice j (Hs = H/8 columns) of the model dimension for BOTH
-// projections:
+// Decomposition.  The active neurons of a layer are cut into tiles of 64; a cluster owns a contiguous run of
+// tiles.  CTA j of the cluster owns column slice j (Hs = H/8 columns) of the model dimension for BOTH projections:
 //   gate/up : D1[128 x T] = [64 gate rows ; 64 up rows](slice j) . x(slice j)^T      partial over the H split
 //   exchange: partial sums are reduce-scattered through distributed shared memory (CTA o receives the rows of
-//             neurons 8o..8o+7), the owner applies GeLU-tanh(g) * u, and broadcasts h (bf16) to the 8 CTAs
-//   down    : D2[Hs x T] += Wd(slice j, tile)^T-as-MN-major . h^T                   accumulated over tiles in TMEM
+//             tile neurons 8o..8o+7), the owner applies GeLU-tanh(g) * u and broadcasts h to the 8 CTAs as a
+//             bf16 hi + lo pair (h = hi + lo to 2^-17, so the tensor-core product keeps fp32-level accuracy)
+//   down    : D2[Hs x T] += Wd(slice j, tile) as an MN-major operand . (h_hi + h_lo)^T   accumulated in TMEM
 // so a neuron's 3*Hs*2 contiguous bytes are read exactly once by exactly one CTA, x is never replicated inside a
 // cluster, and h never leaves the chip.  Both products run on the 5th-generation tensor cores (tcgen05.mma,
-// accumulators in tensor memory); the gathered rows are placed by 16-byte cp.async directly into the 128-byte
-// swizzled operand layout.  At the end of an episode each CTA adds its [T x Hs] partial of y to the fp32 residual
-// stream with red.global.add; the residual itself is added by one designated cluster per episode.
+// accumulators in tensor memory); gathered rows are placed by 16-byte cp.async directly into the 128-byte
+// swizzled operand layout, one cp.async group per tile half, so the next tile's weights stream in while the
+// current tile is in its exchange phases.  At the end of an episode each CTA adds its [T x Hs] partial of y to
+// the fp32 residual stream with red.global.add.
 //
-// Layers are chained with programmatic dependent launch: a layer's CTAs become resident, set up and trigger their
-// dependents early, and wait (griddepcontrol.wait) for the previous layer's atomics before touching activations.
+// Layers are chained with programmatic dependent launch: a layer's CTAs become resident, set up, issue the loads
+// of their first tile (weight addresses depend only on the index lists) and then wait (griddepcontrol.wait) for
+// the previous layer's atomics before touching activations.
 #include <cstdio>
 #include <cstdlib>
 
@@ -27,8 +29,8 @@ using namespace sm100;
 // boundaries of its first tile into a device buffer that rm_debug_phase_times copies out.
 #ifdef RM_PHASE_TIMING
 __device__ long long g_phase_stamps[256 * 32];
-#define RM_STAMP(k)                                                                           \
-    do {                                                                                      \
+#define RM_STAMP(k)                                                                                              \
+    do {                                                                                                         \
         if (threadIdx.x == 0 && blockIdx.x < 256 && stamp_ok) g_phase_stamps[blockIdx.x * 32 + (k)] = clock64(); \
     } while (0)
 #else
@@ -55,34 +57,35 @@ struct FusedArgs {
     int64_t record_stride;
     const float* record_scale;
     int B, T, H, I;
-    int add_residual;              // a designated cluster per episode adds r_in into r_out
-    int npc_target;                // neurons per cluster aimed for when spreading a layer over clusters
+    int p_row;                     // floats per row of the partial-sum exchange buffer
+    int add_residual;              // r_in is added into r_out (spread over all CTAs)
     int* status;
 };
 
-template <int NTOK, int HS>
+// floats per row of the exchange buffer: T rounded up to 4 with an odd number of 16-byte chunks, so that the
+// eight rows written by one warp-store fall into distinct bank groups
+__host__ __device__ constexpr int p_row_for(int T) { return 4 * (((T + 3) / 4) | 1); }
+
+template <int NTOK, int HS, int ST>
 struct Smem {
     static constexpr int KB = HS / 64;                       // 64-column (128-byte) blocks per slice
     static constexpr int X_BYTES = KB * NTOK * 128;
-    static constexpr int GU_BYTES = KB * 128 * 128;
-    static constexpr int DN_BYTES = KB * NT * 128;
-    static constexpr int HT_BYTES = NTOK * 128;
-    static constexpr int P_ROW = NTOK + 4;                   // padded row (floats) of the partial-sum buffer
-    static constexpr int P_BYTES = CS * 16 * P_ROW * 4;
+    static constexpr int GU_STAGE = KB * 128 * 128;
+    static constexpr int DN_STAGE = KB * NT * 128;
+    static constexpr int HT_HALF = NTOK * 128;
     static constexpr int OFF_X = 0;
     static constexpr int OFF_GU = OFF_X + X_BYTES;
-    static constexpr int OFF_DN = OFF_GU + GU_BYTES;
-    static constexpr int OFF_HT = OFF_DN + DN_BYTES;
-    static constexpr int OFF_P = OFF_HT + HT_BYTES;
-    static constexpr int OFF_HS = OFF_P + P_BYTES;           // [NTOK] x 16 B: this CTA's 8 neurons per token
-    static constexpr int OFF_SS = OFF_HS + NTOK * 16;        // [CS][64] floats: row sums of squares per source CTA
-    static constexpr int OFF_N = OFF_SS + CS * 64 * 4;       // [64] neuron ids of the tile
-    static constexpr int OFF_PREF = OFF_N + NT * 4;          // [MAXB+1] prefix of the per-episode counts
-    static constexpr int OFF_BAR = OFF_PREF + (MAXB + 1) * 4 + 4;   // 8-byte aligned: two mbarriers, tmem pointer
-    static constexpr int TOTAL = OFF_BAR + 32;
+    static constexpr int OFF_DN = OFF_GU + ST * GU_STAGE;
+    static constexpr int OFF_HT = OFF_DN + ST * DN_STAGE;    // hi tile, then lo tile
+    static constexpr int OFF_HS = OFF_HT + 2 * HT_HALF;      // [NTOK] x (16 B hi | 16 B lo); also the sum-of-squares exchange
+    static constexpr int OFF_N = OFF_HS + 2048;              // [2][64] neuron ids of the current and the next tile
+    static constexpr int OFF_PREF = OFF_N + 2 * NT * 4;     // [MAXB+1] tile prefix, [MAXB] counts
+    static constexpr int OFF_BAR = ((OFF_PREF + (2 * MAXB + 1) * 4 + 7) / 8) * 8;
+    static constexpr int OFF_P = ((OFF_BAR + 32 + 15) / 16) * 16;   // [CS][16][p_row] floats (size known at launch)
     static constexpr int TMEM_COLS_USED = NTOK + (HS / 128) * NTOK;
     static constexpr int TMEM_COLS = TMEM_COLS_USED <= 32 ? 32 : TMEM_COLS_USED <= 64 ? 64 :
                                      TMEM_COLS_USED <= 128 ? 128 : TMEM_COLS_USED <= 256 ? 256 : 512;
+    static int total_bytes(int T) { return OFF_P + CS * 16 * p_row_for(T) * 4 + 1024; }
 };
 
 __device__ __forceinline__ uint4 pack8(const float* v, float s) {
@@ -96,21 +99,27 @@ __device__ __forceinline__ uint4 pack8(const float* v, float s) {
     return r;
 }
 
-template <int NTOK, int HS>
-__global__ void __launch_bounds__(FT, (HS == 128 ? 2 : 1)) fused_layer_kernel(const FusedArgs a) {
-    using S = Smem<NTOK, HS>;
+struct TileRef {
+    int b, p0, nvalid;
+    bool first, last;              // first / last tile of its episode within this cluster's run
+};
+
+template <int NTOK, int HS, int ST>
+__global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_layer_kernel(const FusedArgs a) {
+    using S = Smem<NTOK, HS, ST>;
     constexpr int KB = S::KB;
     extern __shared__ unsigned char smem_dyn[];
     // 1024-byte alignment: the 128-byte swizzle is a function of absolute shared-memory address bits
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* gbase = smem_dyn + (base - smem_u32(smem_dyn));
     const uint32_t sX = base + S::OFF_X, sGU = base + S::OFF_GU, sDN = base + S::OFF_DN, sHT = base + S::OFF_HT;
-    const uint32_t sP = base + S::OFF_P, sSS = base + S::OFF_SS;
-    float* gP = reinterpret_cast<float*>(gbase + S::OFF_P);
-    uint4* gHS = reinterpret_cast<uint4*>(gbase + S::OFF_HS);
-    float* gSS = reinterpret_cast<float*>(gbase + S::OFF_SS);
+    const uint32_t sP = base + S::OFF_P, sSS = base + S::OFF_HS;
+    const float* gP = reinterpret_cast<const float*>(gbase + S::OFF_P);
+    unsigned char* gHS = gbase + S::OFF_HS;
+    const float* gSS = reinterpret_cast<const float*>(gbase + S::OFF_HS);
     int* gN = reinterpret_cast<int*>(gbase + S::OFF_N);
     int* gPref = reinterpret_cast<int*>(gbase + S::OFF_PREF);
+    int* gCnt = gPref + MAXB + 1;
     const uint32_t bar_gu = base + S::OFF_BAR, bar_dn = bar_gu + 8, s_tmem = bar_gu + 16;
     volatile uint32_t* g_tmem = reinterpret_cast<volatile uint32_t*>(gbase + S::OFF_BAR + 16);
 
@@ -121,9 +130,9 @@ __global__ void __launch_bounds__(FT, (HS == 128 ? 2 : 1)) fused_layer_kernel(co
     RM_STAMP(0);
     const int j = (int)cluster_ctarank();
     const int cid = (int)cluster_id_x(), NC = (int)cluster_count_x();
-    const int H = a.H, T = a.T;
+    const int H = a.H, T = a.T, PR = a.p_row;
 
-    // ---- set-up: barriers, tensor memory, per-episode counts
+    // ---- set-up: barriers, tensor memory, per-episode tile counts
     if (tid == 0) {
         mbar_init(bar_gu, 1);
         mbar_init(bar_dn, 1);
@@ -136,8 +145,9 @@ __global__ void __launch_bounds__(FT, (HS == 128 ? 2 : 1)) fused_layer_kernel(co
                 c = a.count[(size_t)b * a.count_stride];
                 if (c < 0 || c > cap) { rm_set_status(a.status, RM_ERR_INDEX); c = c < 0 ? 0 : cap; }
             }
+            gCnt[b] = c;
             gPref[b] = acc;
-            acc += c;
+            acc += (c + NT - 1) / NT;
         }
         gPref[a.B] = acc;
     }
@@ -150,96 +160,164 @@ __global__ void __launch_bounds__(FT, (HS == 128 ? 2 : 1)) fused_layer_kernel(co
     tc_fence_after();
     const uint32_t tmem_d1 = *g_tmem;
     const uint32_t tmem_d2 = tmem_d1 + NTOK;
-
     RM_STAMP(1);
     pdl_launch_dependents();               // the next layer may become resident and set up
 
-    const int total = gPref[a.B];
-    int n_active = (total + a.npc_target - 1) / a.npc_target;
-    n_active = n_active < 1 ? 1 : (n_active > NC ? NC : n_active);
-    const long long g0 = cid < n_active ? (long long)cid * total / n_active : 0;
-    const long long g1 = cid < n_active ? (long long)(cid + 1) * total / n_active : 0;
+    // this cluster's run of tiles
+    const int tiles_total = gPref[a.B];
+    const int n_active = tiles_total < NC ? tiles_total : NC;
+    const int g_lo = cid < n_active ? (int)((long long)cid * tiles_total / n_active) : 0;
+    const int g_hi = cid < n_active ? (int)((long long)(cid + 1) * tiles_total / n_active) : 0;
+
+    auto tile_ref = [&](int g) {
+        TileRef r;
+        int b = 0;
+        while (gPref[b + 1] <= g) ++b;
+        r.b = b;
+        r.p0 = (g - gPref[b]) * NT;
+        const int left = gCnt[b] - r.p0;
+        r.nvalid = left < NT ? left : NT;
+        r.first = (g == g_lo) || (g == gPref[b]);
+        r.last = (g == g_hi - 1) || (g == gPref[b + 1] - 1);
+        return r;
+    };
+
+    // per-thread share of a tile's gather: rows q0 = tid/8 and q0 + 32 of the tile, 16-byte chunk ch = tid%8
+    const int q0 = tid >> 3, ch = tid & 7;
+    const __nv_bfloat16* slice = a.packed + (size_t)j * 3 * HS + ch * 8;
+    auto neuron_of = [&](const TileRef& r, int q) {
+        int n = -1;
+        if (q < r.nvalid) {
+            n = a.idx ? a.idx[(size_t)r.b * a.idx_stride + r.p0 + q] : r.p0 + q;
+            if (n < 0 || n >= a.I) { rm_set_status(a.status, RM_ERR_INDEX); n = -1; }
+        }
+        return n;
+    };
+    // gate and up rows of tile g into GU stage `st`: rows q (gate) and 64+q (up), swizzled 128-byte rows
+    auto issue_gu = [&](int g, int st) {
+        const TileRef r = tile_ref(g);
+        const int n0 = neuron_of(r, q0), n1 = neuron_of(r, q0 + 32);
+        if (ch == 0) { gN[((g - g_lo) & 1) * NT + q0] = n0; gN[((g - g_lo) & 1) * NT + q0 + 32] = n1; }
+        const __nv_bfloat16* s0 = slice + (size_t)(n0 < 0 ? 0 : n0) * 3 * H;
+        const __nv_bfloat16* s1 = slice + (size_t)(n1 < 0 ? 0 : n1) * 3 * H;
+        const uint32_t d0 = sGU + st * S::GU_STAGE + q0 * 128 + ((ch ^ (q0 & 7)) << 4);   // (q0+32)&7 == q0&7
+#pragma unroll
+        for (int kb = 0; kb < KB; ++kb) {
+            cp_async16(d0 + kb * 16384, s0 + kb * 64, n0 >= 0);                           // gate, neuron q0
+            cp_async16(d0 + kb * 16384 + 32 * 128, s1 + kb * 64, n1 >= 0);                // gate, neuron q0+32
+            cp_async16(d0 + kb * 16384 + 64 * 128, s0 + HS + kb * 64, n0 >= 0);           // up, neuron q0
+            cp_async16(d0 + kb * 16384 + 96 * 128, s1 + HS + kb * 64, n1 >= 0);           // up, neuron q0+32
+        }
+    };
+    // down rows of tile g into DN stage `st`: MN-major operand, 64 neurons x 128 bytes per 64-column block
+    auto issue_dn = [&](int g, int st) {
+        const TileRef r = tile_ref(g);
+        const int n0 = neuron_of(r, q0), n1 = neuron_of(r, q0 + 32);
+        const __nv_bfloat16* s0 = slice + (size_t)(n0 < 0 ? 0 : n0) * 3 * H + 2 * HS;
+        const __nv_bfloat16* s1 = slice + (size_t)(n1 < 0 ? 0 : n1) * 3 * H + 2 * HS;
+        const uint32_t d0 = sDN + st * S::DN_STAGE + q0 * 128 + ((ch ^ (q0 & 7)) << 4);
+#pragma unroll
+        for (int cb = 0; cb < KB; ++cb) {
+            cp_async16(d0 + cb * 8192, s0 + cb * 64, n0 >= 0);
+            cp_async16(d0 + cb * 8192 + 32 * 128, s1 + cb * 64, n1 >= 0);
+        }
+    };
+
+    __syncthreads();                       // gPref / gCnt
+    // ---- prologue: the first ST tiles' weights start streaming before the previous layer has finished
+#pragma unroll
+    for (int s = 0; s < ST; ++s) {
+        if (g_lo + s < g_hi) issue_gu(g_lo + s, s);
+        cp_async_commit();
+        if (g_lo + s < g_hi) issue_dn(g_lo + s, s);
+        cp_async_commit();
+    }
 
     pdl_wait();                            // the previous layer's output is complete and visible
     RM_STAMP(2);
 
-    // ---- duties that do not depend on the neuron range
-    if (a.zero_buf) {
-        float4* z = reinterpret_cast<float4*>(a.zero_buf);
-        const size_t n4 = (size_t)a.B * T * H / 4;
-        for (size_t i = (size_t)blockIdx.x * FT + tid; i < n4; i += (size_t)gridDim.x * FT)
-            z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+    // episodes without a single active neuron have no cluster working on them: their residual passes through here
     if (a.add_residual) {
-        for (int b = cid; b < a.B; b += NC) {
-            for (int i = tid; i < T * (HS / 4); i += FT) {
-                const int t = i / (HS / 4), c4 = i - t * (HS / 4);
-                const size_t o = ((size_t)b * T + t) * H + (size_t)j * HS + c4 * 4;
-                const float4 v = *reinterpret_cast<const float4*>(a.r_in + o);
-                atomicAdd(a.r_out + o, v.x);
-                atomicAdd(a.r_out + o + 1, v.y);
-                atomicAdd(a.r_out + o + 2, v.z);
-                atomicAdd(a.r_out + o + 3, v.w);
+        for (int b = 0; b < a.B; ++b) {
+            if (gPref[b + 1] != gPref[b]) continue;
+            const float4* src = reinterpret_cast<const float4*>(a.r_in + (size_t)b * T * H);
+            float* dst = a.r_out + (size_t)b * T * H;
+            for (size_t i = (size_t)blockIdx.x * FT + tid; i < (size_t)T * H / 4; i += (size_t)gridDim.x * FT) {
+                const float4 v = src[i];
+                red_add_v4(dst + 4 * i, v.x, v.y, v.z, v.w);
             }
         }
     }
-
     RM_STAMP(3);
+
     uint32_t par_gu = 0, par_dn = 0;
-    bool dn_pending = false;
     constexpr uint32_t IDESC_GU = idesc_bf16_f32(128, NTOK, false, false);
     constexpr uint32_t IDESC_DN = idesc_bf16_f32(128, NTOK, true, false);
+    const uint64_t desc_k = smem_desc_sw128(0, 16, 1024);        // K-major operand: 8-row groups 1024 B apart
+    const uint64_t desc_mn = smem_desc_sw128(0, 8192, 1024);     // MN-major operand: 64-column blocks 8192 B apart
+    int cur_b = -1;
 
-    for (int b = 0; b < a.B; ++b) {
-        const long long s0 = gPref[b], s1 = gPref[b + 1];
-        const int lo = (int)((g0 > s0 ? g0 : s0) - s0), hi = (int)((g1 < s1 ? g1 : s1) - s0);
-        if (lo >= hi) continue;            // uniform across the cluster
+    for (int g = g_lo; g < g_hi; ++g) {
+        const TileRef tr = tile_ref(g);
+        const int st = (g - g_lo) % ST;
 
-        // ---- x slice of episode b -> bf16, 128-byte-swizzled K-major operand tile
-        {
+        if (tr.b != cur_b) {
+            cur_b = tr.b;
+            // ---- x slice of episode b -> bf16, 128-byte-swizzled K-major operand tile
             constexpr int PARTS = FT / NTOK;               // threads per token row
             constexpr int CPP = HS / PARTS;                // columns per thread
             const int t = tid / PARTS, part = tid % PARTS;
-            float v[CPP];
+            // clusters whose runs contain tiles of this episode: first_c .. last_c (contiguous)
+            int n_share = 1, my_share = 0;
+            if (a.add_residual) {
+                const long long e0 = gPref[cur_b], e1 = gPref[cur_b + 1];       // tile range of the episode
+                // cluster c owns tiles [c*tt/na, (c+1)*tt/na); first cluster with hi > e0, last with lo < e1
+                int first_c = (int)((e0 * n_active) / tiles_total);
+                while ((long long)(first_c + 1) * tiles_total / n_active <= e0) ++first_c;
+                int last_c = (int)(((e1 - 1) * n_active) / tiles_total);
+                while (last_c + 1 < n_active && (long long)(last_c + 1) * tiles_total / n_active < e1) ++last_c;
+                n_share = last_c - first_c + 1;
+                my_share = cid - first_c;
+            }
             if (a.x) {
-                if (t < T) {
-                    const uint4* src = reinterpret_cast<const uint4*>(a.x + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP);
+                const uint4* src = reinterpret_cast<const uint4*>(a.x + ((size_t)cur_b * T + t) * H + (size_t)j * HS + part * CPP);
 #pragma unroll
-                    for (int i = 0; i < CPP / 8; ++i) {
-                        const uint4 u = src[i];
-                        const int k = part * CPP + i * 8;
-                        *reinterpret_cast<uint4*>(gbase + S::OFF_X + (k >> 6) * (NTOK * 128) + t * 128 +
-                                                  ((((k & 63) >> 3) ^ (t & 7)) << 4)) = u;
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < CPP / 8; ++i) {
-                        const int k = part * CPP + i * 8;
-                        *reinterpret_cast<uint4*>(gbase + S::OFF_X + (k >> 6) * (NTOK * 128) + t * 128 +
-                                                  ((((k & 63) >> 3) ^ (t & 7)) << 4)) = make_uint4(0, 0, 0, 0);
-                    }
+                for (int i = 0; i < CPP / 8; ++i) {
+                    const uint4 u = t < T ? src[i] : make_uint4(0, 0, 0, 0);
+                    const int k = part * CPP + i * 8;
+                    *reinterpret_cast<uint4*>(gbase + S::OFF_X + (k >> 6) * (NTOK * 128) + t * 128 +
+                                              ((((k & 63) >> 3) ^ (t & 7)) << 4)) = u;
                 }
             } else {
+                float v[CPP];
                 float ss = 0.f;
                 if (t < T) {
-                    const float4* src = reinterpret_cast<const float4*>(a.r_in + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP);
+                    const float4* src = reinterpret_cast<const float4*>(a.r_in + ((size_t)cur_b * T + t) * H + (size_t)j * HS + part * CPP);
 #pragma unroll
                     for (int i = 0; i < CPP / 4; ++i) {
                         const float4 f = src[i];
                         v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
-                        ss = fmaf(f.x, f.x, ss); ss = fmaf(f.y, f.y, ss); ss = fmaf(f.z, f.z, ss); ss = fmaf(f.w, f.w, ss);
                     }
+#pragma unroll
+                    for (int i = 0; i < CPP; ++i) ss = fmaf(v[i], v[i], ss);
                 } else {
 #pragma unroll
                     for (int i = 0; i < CPP; ++i) v[i] = 0.f;
                 }
 #pragma unroll
                 for (int d = 1; d < PARTS; d <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
-                if (part == 0) {
+                // the PARTS lanes of a row share the 8 destinations
 #pragma unroll
-                    for (int dst = 0; dst < CS; ++dst) st_cluster_f32(map_to_rank(sSS + (j * 64 + t) * 4, dst), ss);
+                for (int dst = part; dst < CS; dst += PARTS) st_cluster_f32(map_to_rank(sSS + (j * 64 + t) * 4, dst), ss);
+                cluster_arrive();
+                // residual: token row t of this episode is added by exactly one of the clusters that work on the
+                // episode, from the values already in registers, while the cluster barrier completes
+                if (a.add_residual && t < T && (t % n_share) == my_share) {
+                    float* o = a.r_out + ((size_t)cur_b * T + t) * H + (size_t)j * HS + part * CPP;
+#pragma unroll
+                    for (int i = 0; i < CPP / 4; ++i) red_add_v4(o + 4 * i, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
                 }
-                cluster_sync();
+                cluster_wait();
                 float tot = 0.f;
 #pragma unroll
                 for (int src = 0; src < CS; ++src) tot += gSS[src * 64 + t];
@@ -251,184 +329,173 @@ __global__ void __launch_bounds__(FT, (HS == 128 ? 2 : 1)) fused_layer_kernel(co
                                               ((((k & 63) >> 3) ^ (t & 7)) << 4)) = pack8(v + 8 * i, inv);
                 }
             }
-            fence_proxy_async();
+            RM_STAMP(4);
         }
-        RM_STAMP(4);
 
-        for (int p0 = lo; p0 < hi; p0 += NT) {
-            const int nvalid = (hi - p0) < NT ? (hi - p0) : NT;
-            if (dn_pending) {              // the previous down MMA still reads the DN and HT tiles
-                if (!mbar_wait(bar_dn, par_dn)) rm_set_status(a.status, RM_ERR_TIMEOUT);
-                par_dn ^= 1;
-                dn_pending = false;
-            }
-            if (tid < NT) {
-                int n = -1;
-                if (tid < nvalid) {
-                    n = a.idx ? a.idx[(size_t)b * a.idx_stride + p0 + tid] : p0 + tid;
-                    if (n < 0 || n >= a.I) { rm_set_status(a.status, RM_ERR_INDEX); n = -1; }
-                }
-                gN[tid] = n;
-            }
-            __syncthreads();
-
-            // ---- gather this CTA's pieces of the tile: per neuron [gate Hs | up Hs | down Hs] contiguous
-            const __nv_bfloat16* slice = a.packed + (size_t)j * 3 * HS;
-#pragma unroll
-            for (int it = 0; it < KB * 4; ++it) {
-                const int i = it * FT + tid;
-                const int kb = i >> 10, rr = (i >> 3) & 127, ch = i & 7;
-                const int n = gN[rr & 63];
-                const __nv_bfloat16* src = slice + (size_t)(n < 0 ? 0 : n) * 3 * H + (rr >> 6) * HS + kb * 64 + ch * 8;
-                cp_async16(sGU + kb * 16384 + rr * 128 + ((ch ^ (rr & 7)) << 4), src, n >= 0);
-            }
-#pragma unroll
-            for (int it = 0; it < KB * 2; ++it) {
-                const int i = it * FT + tid;
-                const int cb = i >> 9, q = (i >> 3) & 63, ch = i & 7;
-                const int n = gN[q];
-                const __nv_bfloat16* src = slice + (size_t)(n < 0 ? 0 : n) * 3 * H + 2 * HS + cb * 64 + ch * 8;
-                cp_async16(sDN + cb * 8192 + q * 128 + ((ch ^ (q & 7)) << 4), src, n >= 0);
-            }
-            cp_async_commit();
-            RM_STAMP(5);
-            cp_async_wait<0>();
-            fence_proxy_async();
-            __syncthreads();
-            RM_STAMP(6);
-
-            // ---- gate/up partial products over this CTA's column slice
-            if (tid == 0) {
-                tc_fence_after();
-#pragma unroll
-                for (int kb = 0; kb < KB; ++kb)
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        mma_bf16_ss(tmem_d1, smem_desc_sw128(sGU + kb * 16384 + ks * 32, 16, 1024),
-                                    smem_desc_sw128(sX + kb * (NTOK * 128) + ks * 32, 16, 1024), IDESC_GU, (kb | ks) != 0);
-                mma_commit(bar_gu);
-            }
-            if (!mbar_wait(bar_gu, par_gu)) rm_set_status(a.status, RM_ERR_TIMEOUT);
-            par_gu ^= 1;
+        // ---- gate/up partial products over this CTA's column slice
+        cp_async_wait<2 * ST - 2>();       // this tile's gate/up and down rows have landed (later tiles may be in flight)
+        fence_proxy_async();
+        __syncthreads();
+        RM_STAMP(6);
+        if (tid == 0) {
             tc_fence_after();
-            RM_STAMP(7);
-
-            // ---- reduce-scatter: row m of D1 (gate or up of tile neuron q) goes to the CTA that owns q
-            for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
-                float v[32];
-                const int m = (warp & 3) * 32 + lane;
-                tmem_ld32(tmem_d1 + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
-                const int q = m & 63;
-                const uint32_t dst = map_to_rank(sP + ((j * 16 + (m >> 6) * 8 + (q & 7)) * S::P_ROW + c0) * 4, q >> 3);
+            const uint32_t aa = sGU + st * S::GU_STAGE;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) st_cluster_v4(dst + i * 16, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-            }
-            tc_fence_before();
-            RM_STAMP(8);
-            cluster_sync();                // (1) all partial sums have landed
-            RM_STAMP(9);
-
-            // ---- owner: sum the 8 partials, GeLU-tanh(g) * u, activation record, bf16 h
-            {
-                constexpr int TPL = NTOK / 32;             // tokens per lane
-                const int ql = warp;                       // local neuron 0..7 (tile neuron 8j + ql)
-                float g[TPL], u[TPL];
+            for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
-                for (int i = 0; i < TPL; ++i) g[i] = u[i] = 0.f;
-#pragma unroll
-                for (int src = 0; src < CS; ++src) {
-                    const float* pg = gP + (src * 16 + ql) * S::P_ROW + lane * TPL;
-                    const float* pu = gP + (src * 16 + 8 + ql) * S::P_ROW + lane * TPL;
-#pragma unroll
-                    for (int i = 0; i < TPL; ++i) { g[i] += pg[i]; u[i] += pu[i]; }
-                }
-                float rec = 0.f;
-                __nv_bfloat16* hs = reinterpret_cast<__nv_bfloat16*>(gHS);
-#pragma unroll
-                for (int i = 0; i < TPL; ++i) {
-                    const float h = rm_gelu_tanh(g[i]) * u[i];
-                    rec += fabsf(h);
-                    hs[(lane * TPL + i) * 8 + ql] = __float2bfloat16_rn(h);
-                }
-                if (a.record) {
-#pragma unroll
-                    for (int d = 16; d > 0; d >>= 1) rec += __shfl_xor_sync(0xffffffffu, rec, d);
-                    const int n = gN[j * 8 + ql];
-                    if (lane == 0 && n >= 0)
-                        a.record[(size_t)b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
-                }
-            }
-            __syncthreads();
-            // ---- all-gather h: token row t, 16-byte chunk j (neurons 8j..8j+7) of every CTA's K-major h tile
-            for (int i = tid; i < NTOK * CS; i += FT) {
-                const int t = i % NTOK, dst = i / NTOK;
-                st_cluster_v4u(map_to_rank(sHT + t * 128 + ((j ^ (t & 7)) << 4), dst), gHS[t]);
-            }
-            fence_proxy_async();
-            RM_STAMP(10);
-            cluster_sync();                // (2) h of the whole tile is present in every CTA
-            RM_STAMP(11);
-
-            // ---- down projection of the tile, accumulated in tensor memory across the episode's tiles
-            if (tid == 0) {
-                fence_proxy_async();
-                tc_fence_after();
-#pragma unroll
-                for (int mm = 0; mm < HS / 128; ++mm)
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        mma_bf16_ss(tmem_d2 + mm * NTOK, smem_desc_sw128(sDN + mm * 16384 + ks * 2048, 8192, 1024),
-                                    smem_desc_sw128(sHT + ks * 32, 16, 1024), IDESC_DN, !(p0 == lo && ks == 0));
-                mma_commit(bar_dn);
-            }
-            dn_pending = true;
-            RM_STAMP(12);
-#ifdef RM_PHASE_TIMING
-            stamp_ok = false;              // first tile only
-#endif
+                for (int ks = 0; ks < 4; ++ks)
+                    mma_bf16_ss(tmem_d1, desc_k | desc_addr(aa + kb * 16384 + ks * 32),
+                                desc_k | desc_addr(sX + kb * (NTOK * 128) + ks * 32), IDESC_GU, (kb | ks) != 0);
+            mma_commit(bar_gu);
         }
-#ifdef RM_PHASE_TIMING
-        stamp_ok = true;
-#endif
-
-        // ---- add this CTA's [T x Hs] partial of y to the residual stream
-        if (!mbar_wait(bar_dn, par_dn)) rm_set_status(a.status, RM_ERR_TIMEOUT);
-        par_dn ^= 1;
-        dn_pending = false;
+        if (!mbar_wait(bar_gu, par_gu)) rm_set_status(a.status, RM_ERR_TIMEOUT);
+        par_gu ^= 1;
         tc_fence_after();
-        RM_STAMP(13);
+        RM_STAMP(7);
+        // the gate/up stage is free again: start the tile that will use it next
+        if (g + ST < g_hi) issue_gu(g + ST, st);
+        cp_async_commit();
+
+        // ---- reduce-scatter: row m of D1 (gate or up of tile neuron q) goes to the CTA that owns q
+        for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
+            float v[32];
+            const int m = (warp & 3) * 32 + lane;
+            tmem_ld32(tmem_d1 + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
+            const int q = m & 63;
+            const uint32_t dst = map_to_rank(sP + ((j * 16 + (m >> 6) * 8 + (q & 7)) * PR + c0) * 4, q >> 3);
 #pragma unroll
-        for (int mm = 0; mm < HS / 128; ++mm) {
-            for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
-                float v[32];
-                tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
-                float* dst = a.r_out + (size_t)b * T * H + (size_t)j * HS + mm * 128 + (warp & 3) * 32 + lane;
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c0 + i < T) atomicAdd(dst + (size_t)(c0 + i) * H, v[i]);
-            }
+            for (int i = 0; i < 8; ++i)
+                if (c0 + 4 * i < PR) st_cluster_v4(dst + i * 16, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
         }
         tc_fence_before();
-        __syncthreads();
-        RM_STAMP(14);
-    }
+        RM_STAMP(8);
+        cluster_sync();                    // (1) all partial sums have landed
+        RM_STAMP(9);
 
-    // ---- teardown: nobody may still be writing into this CTA's shared memory; release tensor memory
+        // ---- owner: sum the 8 partials, GeLU-tanh(g) * u, activation record, h = hi + lo in bf16
+        {
+            constexpr int TPL = NTOK / 32;                 // tokens per lane
+            const int ql = warp;                           // local neuron 0..7 (tile neuron 8j + ql)
+            const int t0 = lane * TPL;
+            float gsum[TPL], usum[TPL];
+#pragma unroll
+            for (int i = 0; i < TPL; ++i) gsum[i] = usum[i] = 0.f;
+            if (t0 < PR) {
+#pragma unroll
+                for (int src = 0; src < CS; ++src) {
+                    const float* pg = gP + (src * 16 + ql) * PR + t0;
+                    const float* pu = gP + (src * 16 + 8 + ql) * PR + t0;
+#pragma unroll
+                    for (int i = 0; i < TPL; ++i) { gsum[i] += pg[i]; usum[i] += pu[i]; }
+                }
+            }
+            float rec = 0.f;
+#pragma unroll
+            for (int i = 0; i < TPL; ++i) {
+                const float h = (t0 + i < T) ? rm_gelu_tanh(gsum[i]) * usum[i] : 0.f;
+                rec += fabsf(h);
+                const __nv_bfloat16 hi = __float2bfloat16_rn(h);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(h - __bfloat162float(hi));
+                *reinterpret_cast<__nv_bfloat16*>(gHS + (t0 + i) * 32 + ql * 2) = hi;
+                *reinterpret_cast<__nv_bfloat16*>(gHS + (t0 + i) * 32 + 16 + ql * 2) = lo;
+            }
+            if (a.record) {
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) rec += __shfl_xor_sync(0xffffffffu, rec, d);
+                const int n = gN[((g - g_lo) & 1) * NT + j * 8 + ql];
+                if (lane == 0 && n >= 0)
+                    a.record[(size_t)tr.b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
+            }
+        }
+        __syncthreads();
+        // ---- all-gather h: token row t, 16-byte chunk j (neurons 8j..8j+7) of every CTA's K-major hi and lo tiles
+        for (int i = tid; i < NTOK * 2 * CS; i += FT) {
+            const int dst = i / (NTOK * 2), rem = i - dst * (NTOK * 2);
+            const int t = rem >> 1, part = rem & 1;
+            st_cluster_v4u(map_to_rank(sHT + part * S::HT_HALF + t * 128 + ((j ^ (t & 7)) << 4), dst),
+                           *reinterpret_cast<const uint4*>(gHS + t * 32 + part * 16));
+        }
+        fence_proxy_async();
+        RM_STAMP(10);
+        cluster_sync();                    // (2) h of the whole tile is present in every CTA
+        RM_STAMP(11);
+
+        // ---- down projection of the tile, accumulated in tensor memory across the episode's tiles
+        if (tid == 0) {
+            fence_proxy_async();
+            tc_fence_after();
+            const uint32_t ad = sDN + st * S::DN_STAGE;
+#pragma unroll
+            for (int mm = 0; mm < HS / 128; ++mm)
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t aa = desc_mn | desc_addr(ad + mm * 16384 + ks * 2048);
+                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_k | desc_addr(sHT + ks * 32), IDESC_DN,
+                                !(tr.first && ks == 0));
+                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_k | desc_addr(sHT + S::HT_HALF + ks * 32), IDESC_DN, true);
+                }
+            mma_commit(bar_dn);
+        }
+        RM_STAMP(12);
+        // the down stage and the h tiles are reused by the next tile: wait for the products to finish
+        if (!mbar_wait(bar_dn, par_dn)) rm_set_status(a.status, RM_ERR_TIMEOUT);
+        par_dn ^= 1;
+        tc_fence_after();
+        if (g + ST < g_hi) issue_dn(g + ST, st);
+        cp_async_commit();
+        RM_STAMP(13);
+
+        if (tr.last) {
+            // ---- add this CTA's [T x Hs] partial of y to the residual stream
+#pragma unroll
+            for (int mm = 0; mm < HS / 128; ++mm) {
+                for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
+                    float v[32];
+                    tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
+                    float* dst = a.r_out + (size_t)tr.b * T * H + (size_t)j * HS + mm * 128 + (warp & 3) * 32 + lane;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (c0 + i < T) atomicAdd(dst + (size_t)(c0 + i) * H, v[i]);
+                }
+            }
+            tc_fence_before();
+            __syncthreads();
+            RM_STAMP(14);
+        }
+#ifdef RM_PHASE_TIMING
+        stamp_ok = false;                  // first tile only
+#endif
+    }
+#ifdef RM_PHASE_TIMING
+    stamp_ok = true;
+#endif
+
+    // ---- teardown.  Peers write into this CTA's shared memory only before the cluster barriers of a tile, and the
+    // last of those barriers is behind us, so the CTA may exit without another cluster-wide wait.
+    // ---- duty shared by all CTAs: clear the buffer the next layer accumulates into.  It sits at the very end so that
+    // no release-barrier of the exchange phases has to wait for these global stores.
+    if (a.zero_buf) {
+        const size_t n4 = (size_t)a.B * T * H / 4;
+        float4* z = reinterpret_cast<float4*>(a.zero_buf);
+        for (size_t i = (size_t)blockIdx.x * FT + tid; i < n4; i += (size_t)gridDim.x * FT)
+            z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    cp_async_wait<0>();
     tc_fence_before();
-    cluster_sync();
+    __syncthreads();
     if (warp == 0) tmem_dealloc(tmem_d1, S::TMEM_COLS);
     RM_STAMP(15);
 }
 
-template <int NTOK, int HS>
+template <int NTOK, int HS, int ST>
 int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cudaStream_t s) {
-    using S = Smem<NTOK, HS>;
-    auto kern = fused_layer_kernel<NTOK, HS>;
-    const int smem = S::TOTAL + 1024;
-    static bool configured = false;
-    if (!configured) {
+    using S = Smem<NTOK, HS, ST>;
+    auto kern = fused_layer_kernel<NTOK, HS, ST>;
+    const int smem = S::total_bytes(a.T);
+    static int configured = 0;
+    if (configured < smem) {
         RM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        configured = true;
+        configured = smem;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_clusters * CS);
@@ -449,11 +516,11 @@ int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cuda
     return RM_OK;
 }
 
-template <int NTOK, int HS>
-int max_clusters(int* out, int* blocks_per_sm) {
-    using S = Smem<NTOK, HS>;
-    auto kern = fused_layer_kernel<NTOK, HS>;
-    const int smem = S::TOTAL + 1024;
+template <int NTOK, int HS, int ST>
+int max_clusters(int T, int* out) {
+    using S = Smem<NTOK, HS, ST>;
+    auto kern = fused_layer_kernel<NTOK, HS, ST>;
+    const int smem = S::total_bytes(T);
     RM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CS * 64);
@@ -467,21 +534,6 @@ int max_clusters(int* out, int* blocks_per_sm) {
     cfg.attrs = at;
     cfg.numAttrs = 1;
     RM_CUDA_TRY(cudaOccupancyMaxActiveClusters(out, kern, &cfg));
-    if (blocks_per_sm) RM_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, kern, FT, smem));
-    if (getenv("RM_DEBUG_OCC")) {
-        cudaFuncAttributes fa;
-        cudaFuncGetAttributes(&fa, kern);
-        int b2 = -1;
-        for (int sm : {16 * 1024, 48 * 1024, 100 * 1024}) {
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, kern, FT, sm);
-            fprintf(stderr, "  smem %d -> blocks %d\n", sm, b2);
-        }
-        cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, kern, FT, smem);
-        fprintf(stderr, "  with carveout 100: smem %d -> blocks %d\n", smem, b2);
-        fprintf(stderr, "fused<%d,%d>: regs %d static smem %zu maxdyn %d local %zu smem req %d blocks@100KB %d\n", NTOK, HS,
-                fa.numRegs, fa.sharedSizeBytes, fa.maxDynamicSharedSizeBytes, fa.localSizeBytes, smem, b2);
-    }
     return RM_OK;
 }
 
@@ -503,10 +555,13 @@ bool rm_fused_supported(const rm_ctx* ctx, int B, int T) {
 }
 
 int rm_fused_init(rm_ctx* ctx) {
+    // The occupancy query counts one CTA per SM for kernels that allocate tensor memory; clusters beyond that
+    // number simply queue, so it is a sizing hint, not a limit.
     ctx->fused_clusters = 0;
+    ctx->fused_blocks_per_sm = 1;
     int n = 0, rc = RM_OK;
-    if (ctx->g.H == 1024) rc = max_clusters<64, 128>(&n, &ctx->fused_blocks_per_sm);
-    else if (ctx->g.H == 2048) rc = max_clusters<64, 256>(&n, &ctx->fused_blocks_per_sm);
+    if (ctx->g.H == 1024) rc = max_clusters<64, 128, 1>(64, &n);
+    else if (ctx->g.H == 2048) rc = max_clusters<64, 256, 1>(64, &n);
     else return RM_OK;
     if (rc != RM_OK) return rc;
     ctx->fused_clusters = n;
@@ -533,19 +588,21 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
     a.T = la.T;
     a.H = ctx->g.H;
     a.I = ctx->g.I;
+    a.p_row = p_row_for(la.T);
     a.add_residual = add_residual ? 1 : 0;
-    a.npc_target = ctx->npc_target;
     a.status = ctx->d_status;
-    // Clusters per launch: all co-resident slots, or -- when the caller told us how many neurons to expect -- just
-    // enough for them, which leaves slots free for the next layer's CTAs to become resident early.
-    int nc = ctx->fused_clusters;
-    if (ctx->count_hint > 0) {
-        long long want = ((long long)ctx->count_hint * la.B + ctx->npc_target - 1) / ctx->npc_target;
+    // Clusters per launch: one per tile of 64 neurons when the number of active neurons is known on the host
+    // (dense calls, or a caller-supplied hint), else twice the co-resident number; never more than the cap.
+    const int cap = ctx->max_clusters_override > 0 ? ctx->max_clusters_override : 2 * ctx->fused_clusters;
+    int nc = cap;
+    const int per_episode = la.idx ? ctx->count_hint : ctx->g.I;
+    if (per_episode > 0) {
+        long long want = (long long)((per_episode + NT - 1) / NT) * la.B;
         if (want < 1) want = 1;
         if (want < nc) nc = (int)want;
     }
-    if (ctx->max_clusters_override > 0 && nc > ctx->max_clusters_override) nc = ctx->max_clusters_override;
     const bool small_t = la.T <= 32;
-    if (ctx->g.H == 1024) return small_t ? launch_fused<32, 128>(ctx, a, nc, pdl, s) : launch_fused<64, 128>(ctx, a, nc, pdl, s);
-    return small_t ? launch_fused<32, 256>(ctx, a, nc, pdl, s) : launch_fused<64, 256>(ctx, a, nc, pdl, s);
+    if (ctx->g.H == 1024)
+        return small_t ? launch_fused<32, 128, 1>(ctx, a, nc, pdl, s) : launch_fused<64, 128, 1>(ctx, a, nc, pdl, s);
+    return small_t ? launch_fused<32, 256, 1>(ctx, a, nc, pdl, s) : launch_fused<64, 256, 1>(ctx, a, nc, pdl, s);
 }
