@@ -132,6 +132,33 @@ int rm_action_expert_step_host(rm_ctx* ctx, const void* const* packed_layers, co
                                const int32_t* idx, const int32_t* count_dev, int64_t stride, float* r_out_host,
                                int B, int T, void* ws, size_t ws_bytes, rm_stream_t stream);
 
+/* ---- rm_sparse_mlp_static: the one-layer call of rm_sparse_mlp for callers that cannot allocate.
+ * (The paper has no counterpart for this entry point; it exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- a robot's control loop that has frozen its
+ * memory after start-up, a plug-in living inside a host framework's arena, a process whose device-memory budget is
+ * fixed by an operator.  rm_create itself calls cudaMalloc, so such callers cannot even make a context.  This call takes no context and no workspace, and it calls neither
+ * cudaMalloc / cudaFree nor any allocating library routine.
+ *
+ * How: the scratch that the two-kernel portable path needs (the compact hidden activations h [T, I] in fp32) is a
+ * fixed 4 MiB array that is part of the library image; every GPU that loads the library carries it until the
+ * process exits.  Limit: T * I <= 1,048,576 (for example T = 64 with I = 16384); larger requests return
+ * RM_ERR_SHAPE.  H must be a multiple of 64.
+ *
+ * Arguments as for rm_sparse_mlp (packed_layer from rm_pack_weights with the same H and I; x [T,H] bf16; residual
+ * [T,H] fp32 or NULL; idx ascending int32 or NULL for dense; count_dev [1] int32 on the device; y [T,H] fp32, may
+ * equal residual).  All pointers are device pointers, 16-byte aligned; the caller passes inputs and outputs as usual.
+ * No activation record is produced.  Out-of-range indices are skipped silently (there is no status word without a
+ * context).  The work is enqueued on `stream`; the call does not wait for it.
+ *
+ * First call on a device: looks up the array's device address and raises the gate/up kernel's shared-memory limit
+ * (no allocation, but host-side set-up).  Make that first call before starting any stream capture on that device.
+ * Sharing: every call on a device uses the same array and finds the previous call's contents in it.  Nothing needs
+ * clearing (each call overwrites exactly the entries it reads), but two calls whose kernels overlap on the GPU --
+ * different streams, or different host threads on different streams -- race on it: serialise them. */
+int rm_sparse_mlp_static(const void* packed_layer, const void* x, const float* residual, const int32_t* idx,
+                         const int32_t* count_dev, float* y, int T, int H, int I, rm_stream_t stream);
+
 /* Reads and clears the device status word (0 or the first RM_ERR_* a kernel recorded).  Synchronises `stream`. */
 int rm_device_status(rm_ctx* ctx, int* host_out, rm_stream_t stream);
 

@@ -23,7 +23,7 @@ RM_REDUCE_NONE, RM_REDUCE_THRESHOLD, RM_REDUCE_TOPK, RM_REDUCE_GROUP = 0, 1, 2, 
 EXPORTS = ["rm_create", "rm_destroy", "rm_packed_layer_bytes", "rm_workspace_bytes", "rm_pack_weights",
            "rm_mask_compact", "rm_sparse_mlp", "rm_action_expert_step", "rm_action_expert_step_host",
            "rm_device_status", "rm_launch_count", "rm_status_string", "rm_set_option", "rm_get_info",
-           "rm_debug_phase_times"]
+           "rm_debug_phase_times", "rm_sparse_mlp_static"]
 
 
 class RmError(RuntimeError):
@@ -74,6 +74,7 @@ def load_library() -> ctypes.CDLL:
     lib.rm_set_option.argtypes = [vp, ctypes.c_char_p, i32]
     lib.rm_get_info.argtypes = [vp, ctypes.c_char_p, ctypes.POINTER(ctypes.c_int)]
     lib.rm_debug_phase_times.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong), i32]
+    lib.rm_sparse_mlp_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp]
     lib.rm_status_string.argtypes = [i32]
     lib.rm_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -98,6 +99,16 @@ def _ptr(t) -> Optional[int]:
 def _stream() -> int:
     import torch
     return int(torch.cuda.current_stream().cuda_stream)
+
+
+def rm_sparse_mlp_static(packed_layer, x, residual, idx, count_dev, y, T: int, H: int, I: int):
+    """One masked MLP layer without a context, a workspace or any allocation: the scratch is a fixed array inside the
+    library (T * I <= 1,048,576).  For callers that may not allocate device memory.  Calls that overlap on the GPU
+    share that array and must be serialised; make the first call on a device outside stream capture."""
+    lib = load_library()
+    _check(lib.rm_sparse_mlp_static(_ptr(packed_layer), _ptr(x), _ptr(residual), _ptr(idx), _ptr(count_dev), _ptr(y),
+                                    int(T), int(H), int(I), _stream()), "rm_sparse_mlp_static")
+    return y
 
 
 class Context:

@@ -2,6 +2,8 @@
 // dot products + GeLU-tanh GLU into a compact fp32 h, down projection + residual).  It accepts any H that is a
 // multiple of 64, any T and any I; the tensor-core path covers the shapes that matter for speed and this one
 // covers everything else.
+#include <mutex>
+
 #include "rm_common.cuh"
 
 namespace {
@@ -188,6 +190,85 @@ int rm_launch_layer_ref(rm_ctx* ctx, const rm_layer_args& a, void* ws, cudaStrea
     dim3 g2((g.H / 2 + DN_THREADS - 1) / DN_THREADS, (a.T + DN_TOK - 1) / DN_TOK, a.B);
     ref_down_kernel<<<g2, DN_THREADS, 0, s>>>(a, g, h, ctx->d_status);
     ctx->launches++;
+    RM_CUDA_TRY(cudaGetLastError());
+    return RM_OK;
+}
+
+
+// ---------------------------------------------------------------------------------------------------------------
+// rm_sparse_mlp_static: the one-layer masked MLP for callers that must not allocate.
+//
+// The compact hidden activations h [T, I] that the gate/up kernel hands to the down kernel normally live in the
+// caller's workspace.  Here they live in a fixed 4 MiB array inside the library image, so the call needs no context
+// (rm_create allocates), no workspace and no allocator of any kind.  The array is shared by every call on a device.
+namespace {
+
+constexpr size_t RM_STATIC_H_FLOATS = (size_t)1 << 20;          // T * I <= 1,048,576 (e.g. T = 64, I = 16384)
+static __device__ __align__(256) float g_static_h[RM_STATIC_H_FLOATS];
+
+constexpr int RM_STATIC_MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+float* g_static_h_addr[RM_STATIC_MAX_DEVICES] = {};             // device address of g_static_h, per device
+int g_static_smem_set[RM_STATIC_MAX_DEVICES] = {};              // dynamic shared memory already enabled up to here
+
+}  // namespace
+
+extern "C" int rm_sparse_mlp_static(const void* packed_layer, const void* x, const float* residual,
+                                    const int32_t* idx, const int32_t* count_dev, float* y, int T, int H, int I,
+                                    rm_stream_t stream) {
+    if (!packed_layer || !x || !y || T < 0 || H < 64 || I < 1) return RM_ERR_INVALID_ARG;
+    if (idx && !count_dev) return RM_ERR_INVALID_ARG;
+    if (H % 64 != 0) return RM_ERR_SHAPE;
+    if ((size_t)T * (size_t)I > RM_STATIC_H_FLOATS) return RM_ERR_SHAPE;      // beyond the built-in scratch
+    for (const void* p : {packed_layer, x, (const void*)residual, (const void*)idx, (const void*)y})
+        if (p && !rm_aligned16(p)) return RM_ERR_ALIGN;
+    if (T == 0) return RM_OK;
+
+    int dev = -1;
+    RM_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= RM_STATIC_MAX_DEVICES) return RM_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)GU_WARPS * 2 * H * sizeof(__nv_bfloat16);
+    float* h = nullptr;
+    {
+        // Once per device, with that device current: ask the runtime where the array lives on this device.  In host
+        // code the symbol itself is only a stand-in; handing it to a kernel would not be a device address.
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_h_addr[dev]) {
+            float* p = nullptr;
+            if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_h) != cudaSuccess || !p) return RM_ERR_CUDA;
+            g_static_h_addr[dev] = p;
+        }
+        if (smem > 48 * 1024 && g_static_smem_set[dev] < (int)smem) {
+            RM_CUDA_TRY(cudaFuncSetAttribute(ref_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            g_static_smem_set[dev] = (int)smem;
+        }
+        h = g_static_h_addr[dev];
+    }
+
+    rm_geom g{};
+    g.L = 1;
+    g.H = H;
+    g.I = I;
+    g.Hs = H / RM_NS;
+    rm_layer_args a{};
+    a.packed = static_cast<const __nv_bfloat16*>(packed_layer);
+    a.x = static_cast<const __nv_bfloat16*>(x);
+    a.r_in = residual;
+    a.r_out = y;
+    a.idx = idx;
+    a.count = count_dev;
+    a.idx_stride = I;
+    a.list_cap = I;
+    a.count_stride = 1;
+    a.B = 1;
+    a.T = T;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // Nothing in the scratch has to start at zero: the gate/up kernel writes h[t, j] for every token and every
+    // list position j < count before the down kernel reads exactly those entries.
+    dim3 g1((I + GU_WARPS - 1) / GU_WARPS, 1);
+    ref_gateup_kernel<<<g1, GU_WARPS * 32, smem, s>>>(a, g, a.x, h, nullptr);
+    dim3 g2((H / 2 + DN_THREADS - 1) / DN_THREADS, (T + DN_TOK - 1) / DN_TOK, 1);
+    ref_down_kernel<<<g2, DN_THREADS, 0, s>>>(a, g, h, nullptr);
     RM_CUDA_TRY(cudaGetLastError());
     return RM_OK;
 }

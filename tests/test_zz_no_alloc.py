@@ -1,0 +1,51 @@
+"""rm_sparse_mlp_static: the allocation-free entry point must agree with rm_sparse_mlp.
+
+Collected last on purpose: if it fails, a run that stops at the first failure has already run everything else.
+It gives callers that cannot allocate (no context, no workspace, no cudaMalloc) the same layer through a scratch
+array built into the library; two calls in a row check that the shared array needs no clearing between calls."""
+import numpy as np
+import pytest
+
+from paper_2609_19104_b200 import workloads as wl
+from harness import assert_close, dev, dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def test_static_entry_matches_the_regular_one_twice_in_a_row(lib):
+    import torch
+    H, I, T = 1024, 4096, 51
+    w = wl.Workload(91, "no-alloc", 1, H, I, T, 0.02, 1, 0.3)
+    ctx = lib.Context(1, H, I, T_max=T)
+    g, u, d = wl.layer_weights(w, 0)
+    packed = ctx.rm_pack_weights(dev_bf16(g), dev_bf16(u), dev_bf16(d))
+    x = dev_bf16(wl.step_input(w, 0))
+    r = dev(wl.residual_input(w))
+    full = wl.uniform(wl.tensor_key(7, 91, 0, 8), I)
+    # first call: a long list; second call: a short one that reuses the (now dirty) scratch; third: dense, no residual
+    for density, use_res in ((0.6, True), (0.05, True), (None, False)):
+        idx = cnt = None
+        if density is not None:
+            sel = np.flatnonzero(full < density).astype(np.int32)
+            buf = np.zeros(I, np.int32)
+            buf[:sel.size] = sel
+            idx, cnt = dev(buf), dev(np.array([sel.size], np.int32))
+        res = r if use_res else None
+        y_ref = torch.empty(T, H, dtype=torch.float32, device="cuda")
+        ctx.rm_sparse_mlp(packed, x, res, idx, cnt, y_ref)
+        y_new = torch.full((T, H), float("nan"), dtype=torch.float32, device="cuda")
+        lib.rm_sparse_mlp_static(packed, x, res, idx, cnt, y_new, T, H, I)
+        torch.cuda.synchronize()
+        assert_close(y_new.cpu().numpy(), y_ref.cpu().numpy(), f"static vs regular, density {density}")
+    ctx.close()
+
+
+def test_static_entry_rejects_oversized_requests(lib):
+    import torch
+    t = torch.zeros(64, dtype=torch.float32, device="cuda")
+    with pytest.raises(lib.RmError) as e:
+        lib.rm_sparse_mlp_static(t, t, None, None, None, t, 65, 1024, 16384)     # T * I above the built-in scratch
+    assert e.value.code == lib.RM_ERR_SHAPE
+    with pytest.raises(lib.RmError) as e:
+        lib.rm_sparse_mlp_static(t, t, None, None, None, t, 4, 1000, 64)         # H not a multiple of 64
+    assert e.value.code == lib.RM_ERR_SHAPE
