@@ -176,10 +176,18 @@ def run_gpu(args, w: wl.Workload):
     ctx.rm_set_option("count_hint", w.K)          # the lists hold K neurons: launch one cluster per 64-neuron tile
     # weights: the workload's seeded draws (same on every rank: replicas of one model)
     packed = []
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed)
     for l in range(w.L):
-        g, u, d = wl.layer_weights(w, l)
-        to = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
-        packed.append(ctx.rm_pack_weights(to(g), to(u), to(d)))
+        if args.device_weights:
+            # same distribution drawn on the device (seeded torch generator): for the large workloads, where the
+            # host-side counter-based draws of 1.8 G weights would take minutes
+            mk = lambda shape: (torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32) * w.sigma).to(torch.bfloat16)
+            packed.append(ctx.rm_pack_weights(mk((w.I, w.H)), mk((w.I, w.H)), mk((w.H, w.I))))
+        else:
+            g, u, d = wl.layer_weights(w, l)
+            to = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+            packed.append(ctx.rm_pack_weights(to(g), to(u), to(d)))
     torch.cuda.synchronize()
 
     # every rank runs its own episodes (replicas; no data-path collective)
@@ -290,7 +298,8 @@ def run_gpu(args, w: wl.Workload):
         in_step_layer_us = us_per_step * B / w.L                  # average duration of a layer launch inside the step
         achieved = bytes_layer / (in_step_layer_us * 1e-6) / 1e9
         io_bytes = B * w.T * w.H * 4
-        cpu_us, cores, sample = time_oracle(w, steps=3, warmup=1) if world == 1 else (None, None, None)
+        cpu_us, cores, sample = (time_oracle(w, steps=3, warmup=1) if world == 1 and not args.no_cpu_baseline
+                                 else (None, None, None))
         line = {
             "metric": METRIC, "value": us_per_step, "unit": "us", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": False,
@@ -323,6 +332,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config1")
+    ap.add_argument("--device-weights", action="store_true",
+                    help="draw the weights on the device with a seeded torch generator instead of the host generator")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = pick_workload(args.workload)

@@ -51,6 +51,7 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->npc_target = 64;
     c->count_hint = 0;
     c->max_clusters_override = 0;
+    c->variant_override = 0;
     c->fused_clusters = 0;
     c->fused_blocks_per_sm = 0;
     if (prop.major == 10) rm_fused_init(c);                 // failure leaves the portable path in charge
@@ -277,6 +278,9 @@ int rm_set_option(rm_ctx* ctx, const char* name, int value) {
     } else if (n == "count_hint") {
         if (value < 0) return RM_ERR_INVALID_ARG;
         ctx->count_hint = value;
+    } else if (n == "variant") {
+        if (value < 0 || value > 2) return RM_ERR_INVALID_ARG;
+        ctx->variant_override = value;
     } else if (n == "max_clusters") {
         if (value < 0) return RM_ERR_INVALID_ARG;
         ctx->max_clusters_override = value;
@@ -298,7 +302,7 @@ int rm_get_info(const rm_ctx* ctx, const char* name, int* out) {
 }
 
 int rm_debug_phase_times(rm_ctx* ctx, long long* host_out, int n) {
-    if (!ctx || !host_out || n < 0) return RM_ERR_INVALID_ARG;
+    if (!ctx || !host_out) return RM_ERR_INVALID_ARG;
     return rm_fused_debug_stamps(host_out, n);
 }
 

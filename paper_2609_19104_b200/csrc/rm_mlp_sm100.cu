@@ -33,8 +33,21 @@ __device__ long long g_phase_stamps[256 * 32];
     do {                                                                                                         \
         if (threadIdx.x == 0 && blockIdx.x < 256 && stamp_ok) g_phase_stamps[blockIdx.x * 32 + (k)] = clock64(); \
     } while (0)
+__device__ __forceinline__ long long rm_globaltimer() {
+    long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// wall-clock (ns) stamps per launch: slot = launch sequence number taken from a device counter
+__device__ long long g_wall_stamps[64 * 256 * 4];
+__device__ int g_wall_seq;
+#define RM_WALL(k)                                                                                          \
+    do {                                                                                                    \
+        if (threadIdx.x == 0 && blockIdx.x < 256) g_wall_stamps[((wall_seq & 63) * 256 + blockIdx.x) * 4 + (k)] = rm_globaltimer(); \
+    } while (0)
 #else
 #define RM_STAMP(k) do { } while (0)
+#define RM_WALL(k) do { } while (0)
 #endif
 
 namespace {
@@ -60,32 +73,35 @@ struct FusedArgs {
     int p_row;                     // floats per row of the partial-sum exchange buffer
     int add_residual;              // r_in is added into r_out (spread over all CTAs)
     int* status;
+    int wall_seq;                  // launch sequence number (phase-timing builds only)
 };
 
 // floats per row of the exchange buffer: T rounded up to 4 with an odd number of 16-byte chunks, so that the
 // eight rows written by one warp-store fall into distinct bank groups
 __host__ __device__ constexpr int p_row_for(int T) { return 4 * (((T + 3) / 4) | 1); }
 
-template <int NTOK, int HS, int ST>
+template <int NTOK, int HS, int ST, bool DS>
 struct Smem {
     static constexpr int KB = HS / 64;                       // 64-column (128-byte) blocks per slice
     static constexpr int X_BYTES = KB * NTOK * 128;
     static constexpr int GU_STAGE = KB * 128 * 128;
     static constexpr int DN_STAGE = KB * NT * 128;
-    static constexpr int HT_HALF = NTOK * 128;
+    static constexpr int HT_HALF = NT * 128;                 // 8 atoms of [8 neurons x 64 tokens] bf16
     static constexpr int OFF_X = 0;
     static constexpr int OFF_GU = OFF_X + X_BYTES;
     static constexpr int OFF_DN = OFF_GU + ST * GU_STAGE;
     static constexpr int OFF_HT = OFF_DN + ST * DN_STAGE;    // hi tile, then lo tile
-    static constexpr int OFF_HS = OFF_HT + 2 * HT_HALF;      // [NTOK] x (16 B hi | 16 B lo); also the sum-of-squares exchange
-    static constexpr int OFF_N = OFF_HS + 2048;              // [2][64] neuron ids of the current and the next tile
+    static constexpr int OFF_HS = OFF_HT + 2 * HT_HALF;      // this CTA's h atom (1 KB hi, 1 KB lo)
+    static constexpr int OFF_SS = OFF_HS + 2048;             // [CS][64] floats: row sums of squares per source CTA
+    static constexpr int OFF_N = OFF_SS + CS * 64 * 4;       // [2][64] neuron ids of the current and the next tile
     static constexpr int OFF_PREF = OFF_N + 2 * NT * 4;     // [MAXB+1] tile prefix, [MAXB] counts
     static constexpr int OFF_BAR = ((OFF_PREF + (2 * MAXB + 1) * 4 + 7) / 8) * 8;
-    static constexpr int OFF_P = ((OFF_BAR + 32 + 15) / 16) * 16;   // [CS][16][p_row] floats (size known at launch)
+    static constexpr int OFF_P = ((OFF_BAR + 64 + 15) / 16) * 16;   // [CS][16][p_row] floats (size known at launch)
     static constexpr int TMEM_COLS_USED = NTOK + (HS / 128) * NTOK;
     static constexpr int TMEM_COLS = TMEM_COLS_USED <= 32 ? 32 : TMEM_COLS_USED <= 64 ? 64 :
                                      TMEM_COLS_USED <= 128 ? 128 : TMEM_COLS_USED <= 256 ? 256 : 512;
-    static int total_bytes(int T) { return OFF_P + CS * 16 * p_row_for(T) * 4 + 1024; }
+    // the exchange buffer, and (DS) a staging buffer of the same size for the outgoing partial sums
+    static int total_bytes(int T) { return OFF_P + (DS ? 2 : 1) * CS * 16 * p_row_for(T) * 4 + 1024; }
 };
 
 __device__ __forceinline__ uint4 pack8(const float* v, float s) {
@@ -104,30 +120,36 @@ struct TileRef {
     bool first, last;              // first / last tile of its episode within this cluster's run
 };
 
-template <int NTOK, int HS, int ST>
-__global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_layer_kernel(const FusedArgs a) {
-    using S = Smem<NTOK, HS, ST>;
+template <int NTOK, int HS, int ST, bool DS>
+__global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 && !DS ? 2 : 1)) fused_layer_kernel(const FusedArgs a) {
+    using S = Smem<NTOK, HS, ST, DS>;
     constexpr int KB = S::KB;
     extern __shared__ unsigned char smem_dyn[];
     // 1024-byte alignment: the 128-byte swizzle is a function of absolute shared-memory address bits
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* gbase = smem_dyn + (base - smem_u32(smem_dyn));
     const uint32_t sX = base + S::OFF_X, sGU = base + S::OFF_GU, sDN = base + S::OFF_DN, sHT = base + S::OFF_HT;
-    const uint32_t sP = base + S::OFF_P, sSS = base + S::OFF_HS;
+    const uint32_t sP = base + S::OFF_P, sSS = base + S::OFF_SS;
     const float* gP = reinterpret_cast<const float*>(gbase + S::OFF_P);
     unsigned char* gHS = gbase + S::OFF_HS;
-    const float* gSS = reinterpret_cast<const float*>(gbase + S::OFF_HS);
+    const float* gSS = reinterpret_cast<const float*>(gbase + S::OFF_SS);
     int* gN = reinterpret_cast<int*>(gbase + S::OFF_N);
     int* gPref = reinterpret_cast<int*>(gbase + S::OFF_PREF);
     int* gCnt = gPref + MAXB + 1;
-    const uint32_t bar_gu = base + S::OFF_BAR, bar_dn = bar_gu + 8, s_tmem = bar_gu + 16;
-    volatile uint32_t* g_tmem = reinterpret_cast<volatile uint32_t*>(gbase + S::OFF_BAR + 16);
+    // mbarriers: MMA completion (gate/up, down) and arrival of the three exchanges (partial sums, h, sums of squares)
+    const uint32_t bar_gu = base + S::OFF_BAR, bar_dn = bar_gu + 8, bar_p = bar_gu + 16, bar_h = bar_gu + 24;
+    const uint32_t bar_s = bar_gu + 32, s_tmem = bar_gu + 40;
+    volatile uint32_t* g_tmem = reinterpret_cast<volatile uint32_t*>(gbase + S::OFF_BAR + 40);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef RM_PHASE_TIMING
     bool stamp_ok = true;
 #endif
     RM_STAMP(0);
+#ifdef RM_PHASE_TIMING
+    const int wall_seq = a.wall_seq;
+#endif
+    RM_WALL(0);
     const int j = (int)cluster_ctarank();
     const int cid = (int)cluster_id_x(), NC = (int)cluster_count_x();
     const int H = a.H, T = a.T, PR = a.p_row;
@@ -136,6 +158,9 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
     if (tid == 0) {
         mbar_init(bar_gu, 1);
         mbar_init(bar_dn, 1);
+        mbar_init(bar_p, 1);
+        mbar_init(bar_h, 1);
+        mbar_init(bar_s, 1);
         fence_mbar_init();
         int acc = 0;
         const int cap = (int)(a.list_cap < (int64_t)a.I ? a.list_cap : (int64_t)a.I);
@@ -233,8 +258,10 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
         cp_async_commit();
     }
 
+    RM_WALL(1);
     pdl_wait();                            // the previous layer's output is complete and visible
     RM_STAMP(2);
+    RM_WALL(2);
 
     // episodes without a single active neuron have no cluster working on them: their residual passes through here
     if (a.add_residual) {
@@ -250,9 +277,9 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
     }
     RM_STAMP(3);
 
-    uint32_t par_gu = 0, par_dn = 0;
+    uint32_t par_gu = 0, par_dn = 0, par_p = 0, par_h = 0, par_s = 0;
     constexpr uint32_t IDESC_GU = idesc_bf16_f32(128, NTOK, false, false);
-    constexpr uint32_t IDESC_DN = idesc_bf16_f32(128, NTOK, true, false);
+    constexpr uint32_t IDESC_DN = idesc_bf16_f32(128, NTOK, true, true);
     const uint64_t desc_k = smem_desc_sw128(0, 16, 1024);        // K-major operand: 8-row groups 1024 B apart
     const uint64_t desc_mn = smem_desc_sw128(0, 8192, 1024);     // MN-major operand: 64-column blocks 8192 B apart
     int cur_b = -1;
@@ -307,17 +334,19 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
 #pragma unroll
                 for (int d = 1; d < PARTS; d <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
                 // the PARTS lanes of a row share the 8 destinations
+                if (tid == 0) mbar_arrive_expect_tx(bar_s, CS * NTOK * 4);
 #pragma unroll
-                for (int dst = part; dst < CS; dst += PARTS) st_cluster_f32(map_to_rank(sSS + (j * 64 + t) * 4, dst), ss);
-                cluster_arrive();
+                for (int dst = part; dst < CS; dst += PARTS)
+                    st_async_f32(map_to_rank(sSS + (j * 64 + t) * 4, dst), ss, map_to_rank(bar_s, dst));
                 // residual: token row t of this episode is added by exactly one of the clusters that work on the
-                // episode, from the values already in registers, while the cluster barrier completes
+                // episode, from the values already in registers, while the exchange is in flight
                 if (a.add_residual && t < T && (t % n_share) == my_share) {
                     float* o = a.r_out + ((size_t)cur_b * T + t) * H + (size_t)j * HS + part * CPP;
 #pragma unroll
                     for (int i = 0; i < CPP / 4; ++i) red_add_v4(o + 4 * i, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
                 }
-                cluster_wait();
+                if (!mbar_wait(bar_s, par_s)) rm_set_status(a.status, RM_ERR_TIMEOUT);
+                par_s ^= 1;
                 float tot = 0.f;
 #pragma unroll
                 for (int src = 0; src < CS; ++src) tot += gSS[src * 64 + t];
@@ -333,6 +362,10 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
         }
 
         // ---- gate/up partial products over this CTA's column slice
+        if (tid == 0) {                    // bytes the two exchanges of this tile will deliver into this CTA
+            mbar_arrive_expect_tx(bar_p, CS * 16 * PR * 4);
+            mbar_arrive_expect_tx(bar_h, CS * 2048);
+        }
         cp_async_wait<2 * ST - 2>();       // this tile's gate/up and down rows have landed (later tiles may be in flight)
         fence_proxy_async();
         __syncthreads();
@@ -356,20 +389,48 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
         if (g + ST < g_hi) issue_gu(g + ST, st);
         cp_async_commit();
 
-        // ---- reduce-scatter: row m of D1 (gate or up of tile neuron q) goes to the CTA that owns q
-        for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
-            float v[32];
-            const int m = (warp & 3) * 32 + lane;
-            tmem_ld32(tmem_d1 + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
-            const int q = m & 63;
-            const uint32_t dst = map_to_rank(sP + ((j * 16 + (m >> 6) * 8 + (q & 7)) * PR + c0) * 4, q >> 3);
+        // ---- reduce-scatter: row m of D1 (gate or up of tile neuron q) goes to the CTA that owns q.  When a staging
+        // area is free (a dedicated one, or this tile's gate/up stage when no further tile will refill it) the rows
+        // are laid out per destination in local shared memory and moved by 8 bulk copies; otherwise every thread
+        // sends its row with asynchronous 16-byte stores.
+        const bool stage_in_gu = !(g + ST < g_hi) && CS * 16 * PR * 4 <= S::GU_STAGE;
+        if (DS || stage_in_gu) {
+            unsigned char* stg = DS ? gbase + S::OFF_P + CS * 16 * PR * 4 : gbase + S::OFF_GU + st * S::GU_STAGE;
+            for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
+                float v[32];
+                const int m = (warp & 3) * 32 + lane;
+                tmem_ld32(tmem_d1 + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
+                const int q = m & 63;
+                float* row = reinterpret_cast<float*>(stg) + (((q >> 3) * 16 + (m >> 6) * 8 + (q & 7)) * PR + c0);
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (c0 + 4 * i < PR) st_cluster_v4(dst + i * 16, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                for (int i = 0; i < 8; ++i)
+                    if (c0 + 4 * i < PR)
+                        *reinterpret_cast<float4*>(row + 4 * i) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+            tc_fence_before();
+            fence_proxy_async();
+            __syncthreads();
+            if (tid < CS)
+                bulk_copy_to_peer(map_to_rank(sP + (j * 16 * PR) * 4, tid), smem_u32(stg) + tid * 16 * PR * 4,
+                                  16 * PR * 4, map_to_rank(bar_p, tid));
+        } else {
+            for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
+                float v[32];
+                const int m = (warp & 3) * 32 + lane;
+                tmem_ld32(tmem_d1 + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
+                const int q = m & 63;
+                const uint32_t dst = map_to_rank(sP + ((j * 16 + (m >> 6) * 8 + (q & 7)) * PR + c0) * 4, q >> 3);
+                const uint32_t rbar = map_to_rank(bar_p, q >> 3);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (c0 + 4 * i < PR) st_async_v4(dst + i * 16, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3], rbar);
+            }
         }
         tc_fence_before();
         RM_STAMP(8);
-        cluster_sync();                    // (1) all partial sums have landed
+        // (1) every source's partial sums for this CTA's 8 neurons have arrived
+        if (!mbar_wait(bar_p, par_p)) rm_set_status(a.status, RM_ERR_TIMEOUT);
+        par_p ^= 1;
         RM_STAMP(9);
 
         // ---- owner: sum the 8 partials, GeLU-tanh(g) * u, activation record, h = hi + lo in bf16
@@ -390,14 +451,27 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
                 }
             }
             float rec = 0.f;
+            float hv[TPL];
 #pragma unroll
             for (int i = 0; i < TPL; ++i) {
-                const float h = (t0 + i < T) ? rm_gelu_tanh(gsum[i]) * usum[i] : 0.f;
-                rec += fabsf(h);
-                const __nv_bfloat16 hi = __float2bfloat16_rn(h);
-                const __nv_bfloat16 lo = __float2bfloat16_rn(h - __bfloat162float(hi));
-                *reinterpret_cast<__nv_bfloat16*>(gHS + (t0 + i) * 32 + ql * 2) = hi;
-                *reinterpret_cast<__nv_bfloat16*>(gHS + (t0 + i) * 32 + 16 + ql * 2) = lo;
+                hv[i] = (t0 + i < T) ? rm_gelu_tanh(gsum[i]) * usum[i] : 0.f;
+                rec += fabsf(hv[i]);
+            }
+            // this CTA's atom of the h operand: row = local neuron, 128 bytes = 64 tokens, 16-byte chunks swizzled
+            // by the row; hi at offset 0, lo (h - hi) at offset 1024
+            {
+                unsigned char* rowp = gHS + ql * 128 + ((((t0 >> 3) ^ ql) & 7) << 4) + (t0 & 7) * 2;
+                if (TPL == 2) {
+                    const __nv_bfloat162 hi = __floats2bfloat162_rn(hv[0], hv[TPL - 1]);
+                    const float2 hf = __bfloat1622float2(hi);
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(hv[0] - hf.x, hv[TPL - 1] - hf.y);
+                    *reinterpret_cast<__nv_bfloat162*>(rowp) = hi;
+                    *reinterpret_cast<__nv_bfloat162*>(rowp + 1024) = lo;
+                } else {
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(hv[0]);
+                    *reinterpret_cast<__nv_bfloat16*>(rowp) = hi;
+                    *reinterpret_cast<__nv_bfloat16*>(rowp + 1024) = __float2bfloat16_rn(hv[0] - __bfloat162float(hi));
+                }
             }
             if (a.record) {
 #pragma unroll
@@ -407,17 +481,18 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
                     a.record[(size_t)tr.b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
             }
         }
-        __syncthreads();
-        // ---- all-gather h: token row t, 16-byte chunk j (neurons 8j..8j+7) of every CTA's K-major hi and lo tiles
-        for (int i = tid; i < NTOK * 2 * CS; i += FT) {
-            const int dst = i / (NTOK * 2), rem = i - dst * (NTOK * 2);
-            const int t = rem >> 1, part = rem & 1;
-            st_cluster_v4u(map_to_rank(sHT + part * S::HT_HALF + t * 128 + ((j ^ (t & 7)) << 4), dst),
-                           *reinterpret_cast<const uint4*>(gHS + t * 32 + part * 16));
-        }
         fence_proxy_async();
+        __syncthreads();
+        // ---- all-gather h: this CTA's atom becomes atom j of the MN-major hi and lo operand tiles of every CTA
+        if (tid < 2 * CS) {
+            const int dst = tid >> 1, part = tid & 1;
+            bulk_copy_to_peer(map_to_rank(sHT + part * S::HT_HALF + j * 1024, dst), smem_u32(gHS) + part * 1024, 1024,
+                              map_to_rank(bar_h, dst));
+        }
         RM_STAMP(10);
-        cluster_sync();                    // (2) h of the whole tile is present in every CTA
+        // (2) h of the whole tile (all 8 owners' chunks) has arrived in this CTA
+        if (!mbar_wait(bar_h, par_h)) rm_set_status(a.status, RM_ERR_TIMEOUT);
+        par_h ^= 1;
         RM_STAMP(11);
 
         // ---- down projection of the tile, accumulated in tensor memory across the episode's tiles
@@ -430,9 +505,9 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
                     const uint64_t aa = desc_mn | desc_addr(ad + mm * 16384 + ks * 2048);
-                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_k | desc_addr(sHT + ks * 32), IDESC_DN,
+                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(sHT + ks * 2048), IDESC_DN,
                                 !(tr.first && ks == 0));
-                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_k | desc_addr(sHT + S::HT_HALF + ks * 32), IDESC_DN, true);
+                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(sHT + S::HT_HALF + ks * 2048), IDESC_DN, true);
                 }
             mma_commit(bar_dn);
         }
@@ -470,8 +545,8 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
     stamp_ok = true;
 #endif
 
-    // ---- teardown.  Peers write into this CTA's shared memory only before the cluster barriers of a tile, and the
-    // last of those barriers is behind us, so the CTA may exit without another cluster-wide wait.
+    // ---- teardown.  Everything peers send into this CTA's shared memory is counted on barriers this CTA has waited
+    // for, so nothing is in flight towards it any more and it may exit without a cluster-wide wait.
     // ---- duty shared by all CTAs: clear the buffer the next layer accumulates into.  It sits at the very end so that
     // no release-barrier of the exchange phases has to wait for these global stores.
     if (a.zero_buf) {
@@ -485,12 +560,13 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 ? 2 : 1)) fused_laye
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem_d1, S::TMEM_COLS);
     RM_STAMP(15);
+    RM_WALL(3);
 }
 
-template <int NTOK, int HS, int ST>
+template <int NTOK, int HS, int ST, bool DS>
 int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cudaStream_t s) {
-    using S = Smem<NTOK, HS, ST>;
-    auto kern = fused_layer_kernel<NTOK, HS, ST>;
+    using S = Smem<NTOK, HS, ST, DS>;
+    auto kern = fused_layer_kernel<NTOK, HS, ST, DS>;
     const int smem = S::total_bytes(a.T);
     static int configured = 0;
     if (configured < smem) {
@@ -516,10 +592,10 @@ int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cuda
     return RM_OK;
 }
 
-template <int NTOK, int HS, int ST>
+template <int NTOK, int HS, int ST, bool DS>
 int max_clusters(int T, int* out) {
-    using S = Smem<NTOK, HS, ST>;
-    auto kern = fused_layer_kernel<NTOK, HS, ST>;
+    using S = Smem<NTOK, HS, ST, DS>;
+    auto kern = fused_layer_kernel<NTOK, HS, ST, DS>;
     const int smem = S::total_bytes(T);
     RM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     cudaLaunchConfig_t cfg = {};
@@ -541,6 +617,11 @@ int max_clusters(int T, int* out) {
 
 int rm_fused_debug_stamps(long long* host_out, int n) {
 #ifdef RM_PHASE_TIMING
+    if (n < 0) {                           // negative n: the wall-clock stamps, -n values
+        n = -n;
+        if (n > 64 * 256 * 4) n = 64 * 256 * 4;
+        return cudaMemcpyFromSymbol(host_out, g_wall_stamps, sizeof(long long) * n) == cudaSuccess ? RM_OK : RM_ERR_CUDA;
+    }
     if (n > 256 * 32) n = 256 * 32;
     return cudaMemcpyFromSymbol(host_out, g_phase_stamps, sizeof(long long) * n) == cudaSuccess ? RM_OK : RM_ERR_CUDA;
 #else
@@ -560,8 +641,8 @@ int rm_fused_init(rm_ctx* ctx) {
     ctx->fused_clusters = 0;
     ctx->fused_blocks_per_sm = 1;
     int n = 0, rc = RM_OK;
-    if (ctx->g.H == 1024) rc = max_clusters<64, 128, 1>(64, &n);
-    else if (ctx->g.H == 2048) rc = max_clusters<64, 256, 1>(64, &n);
+    if (ctx->g.H == 1024) rc = max_clusters<64, 128, 1, false>(64, &n);
+    else if (ctx->g.H == 2048) rc = max_clusters<64, 256, 1, true>(64, &n);
     else return RM_OK;
     if (rc != RM_OK) return rc;
     ctx->fused_clusters = n;
@@ -591,6 +672,7 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
     a.p_row = p_row_for(la.T);
     a.add_residual = add_residual ? 1 : 0;
     a.status = ctx->d_status;
+    a.wall_seq = (int)(ctx->launches & 63);
     // Clusters per launch: one per tile of 64 neurons when the number of active neurons is known on the host
     // (dense calls, or a caller-supplied hint), else twice the co-resident number; never more than the cap.
     const int cap = ctx->max_clusters_override > 0 ? ctx->max_clusters_override : 2 * ctx->fused_clusters;
@@ -601,8 +683,16 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
         if (want < 1) want = 1;
         if (want < nc) nc = (int)want;
     }
+    // Variant: at H = 1024 the lean kernel (112 KB, two CTAs per SM so that consecutive layers overlap) serves launches
+    // where a cluster gets a single tile; when clusters walk several tiles, the variant with a dedicated staging
+    // buffer for the outgoing partial sums keeps the exchange on the copy engine for every tile.
+    long long tiles = per_episode > 0 ? (long long)((per_episode + NT - 1) / NT) * la.B : 0;
+    const bool multi = ctx->variant_override ? ctx->variant_override == 2 : (tiles == 0 || tiles > nc);
     const bool small_t = la.T <= 32;
-    if (ctx->g.H == 1024)
-        return small_t ? launch_fused<32, 128, 1>(ctx, a, nc, pdl, s) : launch_fused<64, 128, 1>(ctx, a, nc, pdl, s);
-    return small_t ? launch_fused<32, 256, 1>(ctx, a, nc, pdl, s) : launch_fused<64, 256, 1>(ctx, a, nc, pdl, s);
+    if (ctx->g.H == 1024) {
+        if (multi)
+            return small_t ? launch_fused<32, 128, 1, true>(ctx, a, nc, pdl, s) : launch_fused<64, 128, 1, true>(ctx, a, nc, pdl, s);
+        return small_t ? launch_fused<32, 128, 1, false>(ctx, a, nc, pdl, s) : launch_fused<64, 128, 1, false>(ctx, a, nc, pdl, s);
+    }
+    return small_t ? launch_fused<32, 256, 1, true>(ctx, a, nc, pdl, s) : launch_fused<64, 256, 1, true>(ctx, a, nc, pdl, s);
 }
