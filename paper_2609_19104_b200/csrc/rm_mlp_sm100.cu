@@ -80,28 +80,29 @@ struct FusedArgs {
 // eight rows written by one warp-store fall into distinct bank groups
 __host__ __device__ constexpr int p_row_for(int T) { return 4 * (((T + 3) / 4) | 1); }
 
-template <int NTOK, int HS, int ST, bool DS>
+template <int NTOK, int HS, bool PIPE>
 struct Smem {
     static constexpr int KB = HS / 64;                       // 64-column (128-byte) blocks per slice
+    static constexpr int NB = PIPE ? 2 : 1;                  // buffers of the exchange state (tiles in flight)
+    static constexpr bool STAGED = PIPE && HS == 128;        // dedicated staging area for the outgoing partial sums
     static constexpr int X_BYTES = KB * NTOK * 128;
     static constexpr int GU_STAGE = KB * 128 * 128;
     static constexpr int DN_STAGE = KB * NT * 128;
     static constexpr int HT_HALF = NT * 128;                 // 8 atoms of [8 neurons x 64 tokens] bf16
     static constexpr int OFF_X = 0;
     static constexpr int OFF_GU = OFF_X + X_BYTES;
-    static constexpr int OFF_DN = OFF_GU + ST * GU_STAGE;
-    static constexpr int OFF_HT = OFF_DN + ST * DN_STAGE;    // hi tile, then lo tile
-    static constexpr int OFF_HS = OFF_HT + 2 * HT_HALF;      // this CTA's h atom (1 KB hi, 1 KB lo)
-    static constexpr int OFF_SS = OFF_HS + 2048;             // [CS][64] floats: row sums of squares per source CTA
-    static constexpr int OFF_N = OFF_SS + CS * 64 * 4;       // [2][64] neuron ids of the current and the next tile
-    static constexpr int OFF_PREF = OFF_N + 2 * NT * 4;     // [MAXB+1] tile prefix, [MAXB] counts
+    static constexpr int OFF_DN = OFF_GU + GU_STAGE;
+    static constexpr int OFF_HT = OFF_DN + DN_STAGE;         // per buffer: hi tile, then lo tile
+    static constexpr int OFF_HS = OFF_HT + NB * 2 * HT_HALF; // per buffer: this CTA's h atom (1 KB hi, 1 KB lo)
+    static constexpr int OFF_SS = OFF_HS + NB * 2048;        // [CS][64] floats: row sums of squares per source CTA
+    static constexpr int OFF_N = OFF_SS + CS * 64 * 4;       // [2][64] neuron ids of two consecutive tiles
+    static constexpr int OFF_PREF = OFF_N + 2 * NT * 4;      // [MAXB+1] tile prefix, [MAXB] counts
     static constexpr int OFF_BAR = ((OFF_PREF + (2 * MAXB + 1) * 4 + 7) / 8) * 8;
-    static constexpr int OFF_P = ((OFF_BAR + 64 + 15) / 16) * 16;   // [CS][16][p_row] floats (size known at launch)
-    static constexpr int TMEM_COLS_USED = NTOK + (HS / 128) * NTOK;
+    static constexpr int OFF_P = ((OFF_BAR + 96 + 15) / 16) * 16;   // NB x [CS][16][p_row] floats (+ staging), sized at launch
+    static constexpr int TMEM_COLS_USED = NB * NTOK + (HS / 128) * NTOK;
     static constexpr int TMEM_COLS = TMEM_COLS_USED <= 32 ? 32 : TMEM_COLS_USED <= 64 ? 64 :
                                      TMEM_COLS_USED <= 128 ? 128 : TMEM_COLS_USED <= 256 ? 256 : 512;
-    // the exchange buffer, and (DS) a staging buffer of the same size for the outgoing partial sums
-    static int total_bytes(int T) { return OFF_P + (DS ? 2 : 1) * CS * 16 * p_row_for(T) * 4 + 1024; }
+    static int total_bytes(int T) { return OFF_P + (NB + (STAGED ? 1 : 0)) * CS * 16 * p_row_for(T) * 4 + 1024; }
 };
 
 __device__ __forceinline__ uint4 pack8(const float* v, float s) {
@@ -120,9 +121,10 @@ struct TileRef {
     bool first, last;              // first / last tile of its episode within this cluster's run
 };
 
-template <int NTOK, int HS, int ST, bool DS>
-__global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 && !DS ? 2 : 1)) fused_layer_kernel(const FusedArgs a) {
-    using S = Smem<NTOK, HS, ST, DS>;
+template <int NTOK, int HS, bool PIPE>
+__global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_kernel(const FusedArgs a) {
+    using S = Smem<NTOK, HS, PIPE>;
+    constexpr int NB = S::NB;
     constexpr int KB = S::KB;
     extern __shared__ unsigned char smem_dyn[];
     // 1024-byte alignment: the 128-byte swizzle is a function of absolute shared-memory address bits
@@ -130,16 +132,18 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 && !DS ? 2 : 1)) fus
     unsigned char* gbase = smem_dyn + (base - smem_u32(smem_dyn));
     const uint32_t sX = base + S::OFF_X, sGU = base + S::OFF_GU, sDN = base + S::OFF_DN, sHT = base + S::OFF_HT;
     const uint32_t sP = base + S::OFF_P, sSS = base + S::OFF_SS;
-    const float* gP = reinterpret_cast<const float*>(gbase + S::OFF_P);
-    unsigned char* gHS = gbase + S::OFF_HS;
     const float* gSS = reinterpret_cast<const float*>(gbase + S::OFF_SS);
     int* gN = reinterpret_cast<int*>(gbase + S::OFF_N);
     int* gPref = reinterpret_cast<int*>(gbase + S::OFF_PREF);
     int* gCnt = gPref + MAXB + 1;
-    // mbarriers: MMA completion (gate/up, down) and arrival of the three exchanges (partial sums, h, sums of squares)
-    const uint32_t bar_gu = base + S::OFF_BAR, bar_dn = bar_gu + 8, bar_p = bar_gu + 16, bar_h = bar_gu + 24;
-    const uint32_t bar_s = bar_gu + 32, s_tmem = bar_gu + 40;
-    volatile uint32_t* g_tmem = reinterpret_cast<volatile uint32_t*>(gbase + S::OFF_BAR + 40);
+    // mbarriers: MMA completion (gate/up per buffer, down) and arrival of the exchanges (partial sums and h per
+    // buffer, sums of squares)
+    const uint32_t bar0 = base + S::OFF_BAR;
+    const uint32_t bar_dn = bar0 + 48, bar_s = bar0 + 56, s_tmem = bar0 + 64;
+    auto bar_gu = [&](int pb) { return bar0 + 8 * pb; };
+    auto bar_p = [&](int pb) { return bar0 + 16 + 8 * pb; };
+    auto bar_h = [&](int pb) { return bar0 + 32 + 8 * pb; };
+    volatile uint32_t* g_tmem = reinterpret_cast<volatile uint32_t*>(gbase + S::OFF_BAR + 64);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef RM_PHASE_TIMING
@@ -156,10 +160,8 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 && !DS ? 2 : 1)) fus
 
     // ---- set-up: barriers, tensor memory, per-episode tile counts
     if (tid == 0) {
-        mbar_init(bar_gu, 1);
+        for (int pb = 0; pb < 2; ++pb) { mbar_init(bar_gu(pb), 1); mbar_init(bar_p(pb), 1); mbar_init(bar_h(pb), 1); }
         mbar_init(bar_dn, 1);
-        mbar_init(bar_p, 1);
-        mbar_init(bar_h, 1);
         mbar_init(bar_s, 1);
         fence_mbar_init();
         int acc = 0;
@@ -184,7 +186,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 && !DS ? 2 : 1)) fus
     cluster_sync();                        // peers' shared memory and barriers are live from here on
     tc_fence_after();
     const uint32_t tmem_d1 = *g_tmem;
-    const uint32_t tmem_d2 = tmem_d1 + NTOK;
+    const uint32_t tmem_d2 = tmem_d1 + NB * NTOK;
     RM_STAMP(1);
     pdl_launch_dependents();               // the next layer may become resident and set up
 
@@ -219,13 +221,13 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 && !DS ? 2 : 1)) fus
         return n;
     };
     // gate and up rows of tile g into GU stage `st`: rows q (gate) and 64+q (up), swizzled 128-byte rows
-    auto issue_gu = [&](int g, int st) {
+    auto issue_gu = [&](int g) {
         const TileRef r = tile_ref(g);
         const int n0 = neuron_of(r, q0), n1 = neuron_of(r, q0 + 32);
         if (ch == 0) { gN[((g - g_lo) & 1) * NT + q0] = n0; gN[((g - g_lo) & 1) * NT + q0 + 32] = n1; }
         const __nv_bfloat16* s0 = slice + (size_t)(n0 < 0 ? 0 : n0) * 3 * H;
         const __nv_bfloat16* s1 = slice + (size_t)(n1 < 0 ? 0 : n1) * 3 * H;
-        const uint32_t d0 = sGU + st * S::GU_STAGE + q0 * 128 + ((ch ^ (q0 & 7)) << 4);   // (q0+32)&7 == q0&7
+        const uint32_t d0 = sGU + q0 * 128 + ((ch ^ (q0 & 7)) << 4);   // (q0+32)&7 == q0&7
 #pragma unroll
         for (int kb = 0; kb < KB; ++kb) {
             cp_async16(d0 + kb * 16384, s0 + kb * 64, n0 >= 0);                           // gate, neuron q0
@@ -235,12 +237,12 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 && !DS ? 2 : 1)) fus
         }
     };
     // down rows of tile g into DN stage `st`: MN-major operand, 64 neurons x 128 bytes per 64-column block
-    auto issue_dn = [&](int g, int st) {
+    auto issue_dn = [&](int g) {
         const TileRef r = tile_ref(g);
         const int n0 = neuron_of(r, q0), n1 = neuron_of(r, q0 + 32);
         const __nv_bfloat16* s0 = slice + (size_t)(n0 < 0 ? 0 : n0) * 3 * H + 2 * HS;
         const __nv_bfloat16* s1 = slice + (size_t)(n1 < 0 ? 0 : n1) * 3 * H + 2 * HS;
-        const uint32_t d0 = sDN + st * S::DN_STAGE + q0 * 128 + ((ch ^ (q0 & 7)) << 4);
+        const uint32_t d0 = sDN + q0 * 128 + ((ch ^ (q0 & 7)) << 4);
 #pragma unroll
         for (int cb = 0; cb < KB; ++cb) {
             cp_async16(d0 + cb * 8192, s0 + cb * 64, n0 >= 0);
@@ -249,14 +251,11 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 && !DS ? 2 : 1)) fus
     };
 
     __syncthreads();                       // gPref / gCnt
-    // ---- prologue: the first ST tiles' weights start streaming before the previous layer has finished
-#pragma unroll
-    for (int s = 0; s < ST; ++s) {
-        if (g_lo + s < g_hi) issue_gu(g_lo + s, s);
-        cp_async_commit();
-        if (g_lo + s < g_hi) issue_dn(g_lo + s, s);
-        cp_async_commit();
-    }
+    // ---- prologue: the first tile's weights start streaming before the previous layer has finished
+    if (g_lo < g_hi) issue_gu(g_lo);
+    cp_async_commit();
+    if (g_lo < g_hi) issue_dn(g_lo);
+    cp_async_commit();
 
     RM_WALL(1);
     pdl_wait();                            // the previous layer's output is complete and visible
@@ -277,269 +276,351 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 && !DS ? 2 : 1)) fus
     }
     RM_STAMP(3);
 
-    uint32_t par_gu = 0, par_dn = 0, par_p = 0, par_h = 0, par_s = 0;
+    uint32_t par_dn = 0, par_s = 0;
     constexpr uint32_t IDESC_GU = idesc_bf16_f32(128, NTOK, false, false);
     constexpr uint32_t IDESC_DN = idesc_bf16_f32(128, NTOK, true, true);
     const uint64_t desc_k = smem_desc_sw128(0, 16, 1024);        // K-major operand: 8-row groups 1024 B apart
-    const uint64_t desc_mn = smem_desc_sw128(0, 8192, 1024);     // MN-major operand: 64-column blocks 8192 B apart
+    const uint64_t desc_mn = smem_desc_sw128(0, 8192, 1024);     // MN-major operand: 64-element blocks 8192 B apart
+    const int n_tiles = g_hi - g_lo;
+    const int p_bytes = CS * 16 * PR * 4;                        // one exchange buffer
     int cur_b = -1;
+    // buffer and barrier phase of local tile i (every second tile reuses a buffer when two are in flight)
+    auto buf_of = [&](int i) { return PIPE ? (i & 1) : 0; };
+    auto phase_of = [&](int i) { return (uint32_t)(PIPE ? ((i >> 1) & 1) : (i & 1)); };
+    auto wait_bar = [&](uint32_t bar, uint32_t parity) {
+        if (!mbar_wait(bar, parity)) rm_set_status(a.status, RM_ERR_TIMEOUT);
+    };
 
-    for (int g = g_lo; g < g_hi; ++g) {
-        const TileRef tr = tile_ref(g);
-        const int st = (g - g_lo) % ST;
-
-        if (tr.b != cur_b) {
-            cur_b = tr.b;
-            // ---- x slice of episode b -> bf16, 128-byte-swizzled K-major operand tile
-            constexpr int PARTS = FT / NTOK;               // threads per token row
-            constexpr int CPP = HS / PARTS;                // columns per thread
-            const int t = tid / PARTS, part = tid % PARTS;
-            // clusters whose runs contain tiles of this episode: first_c .. last_c (contiguous)
-            int n_share = 1, my_share = 0;
-            if (a.add_residual) {
-                const long long e0 = gPref[cur_b], e1 = gPref[cur_b + 1];       // tile range of the episode
-                // cluster c owns tiles [c*tt/na, (c+1)*tt/na); first cluster with hi > e0, last with lo < e1
-                int first_c = (int)((e0 * n_active) / tiles_total);
-                while ((long long)(first_c + 1) * tiles_total / n_active <= e0) ++first_c;
-                int last_c = (int)(((e1 - 1) * n_active) / tiles_total);
-                while (last_c + 1 < n_active && (long long)(last_c + 1) * tiles_total / n_active < e1) ++last_c;
-                n_share = last_c - first_c + 1;
-                my_share = cid - first_c;
-            }
-            if (a.x) {
-                const uint4* src = reinterpret_cast<const uint4*>(a.x + ((size_t)cur_b * T + t) * H + (size_t)j * HS + part * CPP);
+    // ---- phase: x slice of episode b -> bf16, 128-byte-swizzled K-major operand tile (cluster-collective)
+    auto xprep = [&](int b) {
+        cur_b = b;
+        constexpr int PARTS = FT / NTOK;                   // threads per token row
+        constexpr int CPP = HS / PARTS;                    // columns per thread
+        const int t = tid / PARTS, part = tid % PARTS;
+        // clusters whose runs contain tiles of this episode: first_c .. last_c (contiguous)
+        int n_share = 1, my_share = 0;
+        if (a.add_residual) {
+            const long long e0 = gPref[b], e1 = gPref[b + 1];                  // tile range of the episode
+            // cluster c owns tiles [c*tt/na, (c+1)*tt/na); first cluster with hi > e0, last with lo < e1
+            int first_c = (int)((e0 * n_active) / tiles_total);
+            while ((long long)(first_c + 1) * tiles_total / n_active <= e0) ++first_c;
+            int last_c = (int)(((e1 - 1) * n_active) / tiles_total);
+            while (last_c + 1 < n_active && (long long)(last_c + 1) * tiles_total / n_active < e1) ++last_c;
+            n_share = last_c - first_c + 1;
+            my_share = cid - first_c;
+        }
+        if (a.x) {
+            const uint4* src = reinterpret_cast<const uint4*>(a.x + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP);
 #pragma unroll
-                for (int i = 0; i < CPP / 8; ++i) {
-                    const uint4 u = t < T ? src[i] : make_uint4(0, 0, 0, 0);
-                    const int k = part * CPP + i * 8;
-                    *reinterpret_cast<uint4*>(gbase + S::OFF_X + (k >> 6) * (NTOK * 128) + t * 128 +
-                                              ((((k & 63) >> 3) ^ (t & 7)) << 4)) = u;
+            for (int i = 0; i < CPP / 8; ++i) {
+                const uint4 u = t < T ? src[i] : make_uint4(0, 0, 0, 0);
+                const int k = part * CPP + i * 8;
+                *reinterpret_cast<uint4*>(gbase + S::OFF_X + (k >> 6) * (NTOK * 128) + t * 128 +
+                                          ((((k & 63) >> 3) ^ (t & 7)) << 4)) = u;
+            }
+        } else {
+            float v[CPP];
+            float ss = 0.f;
+            if (t < T) {
+                const float4* src = reinterpret_cast<const float4*>(a.r_in + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP);
+#pragma unroll
+                for (int i = 0; i < CPP / 4; ++i) {
+                    const float4 f = src[i];
+                    v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
                 }
+#pragma unroll
+                for (int i = 0; i < CPP; ++i) ss = fmaf(v[i], v[i], ss);
             } else {
-                float v[CPP];
-                float ss = 0.f;
-                if (t < T) {
-                    const float4* src = reinterpret_cast<const float4*>(a.r_in + ((size_t)cur_b * T + t) * H + (size_t)j * HS + part * CPP);
 #pragma unroll
-                    for (int i = 0; i < CPP / 4; ++i) {
-                        const float4 f = src[i];
-                        v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
-                    }
-#pragma unroll
-                    for (int i = 0; i < CPP; ++i) ss = fmaf(v[i], v[i], ss);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < CPP; ++i) v[i] = 0.f;
-                }
-#pragma unroll
-                for (int d = 1; d < PARTS; d <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
-                // the PARTS lanes of a row share the 8 destinations
-                if (tid == 0) mbar_arrive_expect_tx(bar_s, CS * NTOK * 4);
-#pragma unroll
-                for (int dst = part; dst < CS; dst += PARTS)
-                    st_async_f32(map_to_rank(sSS + (j * 64 + t) * 4, dst), ss, map_to_rank(bar_s, dst));
-                // residual: token row t of this episode is added by exactly one of the clusters that work on the
-                // episode, from the values already in registers, while the exchange is in flight
-                if (a.add_residual && t < T && (t % n_share) == my_share) {
-                    float* o = a.r_out + ((size_t)cur_b * T + t) * H + (size_t)j * HS + part * CPP;
-#pragma unroll
-                    for (int i = 0; i < CPP / 4; ++i) red_add_v4(o + 4 * i, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                }
-                if (!mbar_wait(bar_s, par_s)) rm_set_status(a.status, RM_ERR_TIMEOUT);
-                par_s ^= 1;
-                float tot = 0.f;
-#pragma unroll
-                for (int src = 0; src < CS; ++src) tot += gSS[src * 64 + t];
-                const float inv = 1.0f / sqrtf(tot / (float)H + 1e-6f);
-#pragma unroll
-                for (int i = 0; i < CPP / 8; ++i) {
-                    const int k = part * CPP + i * 8;
-                    *reinterpret_cast<uint4*>(gbase + S::OFF_X + (k >> 6) * (NTOK * 128) + t * 128 +
-                                              ((((k & 63) >> 3) ^ (t & 7)) << 4)) = pack8(v + 8 * i, inv);
-                }
+                for (int i = 0; i < CPP; ++i) v[i] = 0.f;
             }
-            RM_STAMP(4);
+#pragma unroll
+            for (int d = 1; d < PARTS; d <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+            // all-gather of the row sums of squares: the PARTS lanes of a row share the 8 destinations
+            if (tid == 0) mbar_arrive_expect_tx(bar_s, CS * NTOK * 4);
+#pragma unroll
+            for (int dst = part; dst < CS; dst += PARTS)
+                st_async_f32(map_to_rank(sSS + (j * 64 + t) * 4, dst), ss, map_to_rank(bar_s, dst));
+            // residual: token row t of this episode is added by exactly one of the clusters that work on the
+            // episode, from the values already in registers, while the exchange is in flight
+            if (a.add_residual && t < T && (t % n_share) == my_share) {
+                float* o = a.r_out + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP;
+#pragma unroll
+                for (int i = 0; i < CPP / 4; ++i) red_add_v4(o + 4 * i, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+            wait_bar(bar_s, par_s);
+            par_s ^= 1;
+            float tot = 0.f;
+#pragma unroll
+            for (int src = 0; src < CS; ++src) tot += gSS[src * 64 + t];
+            const float inv = 1.0f / sqrtf(tot / (float)H + 1e-6f);
+#pragma unroll
+            for (int i = 0; i < CPP / 8; ++i) {
+                const int k = part * CPP + i * 8;
+                *reinterpret_cast<uint4*>(gbase + S::OFF_X + (k >> 6) * (NTOK * 128) + t * 128 +
+                                          ((((k & 63) >> 3) ^ (t & 7)) << 4)) = pack8(v + 8 * i, inv);
+            }
         }
+        RM_STAMP(4);
+    };
 
-        // ---- gate/up partial products over this CTA's column slice
-        if (tid == 0) {                    // bytes the two exchanges of this tile will deliver into this CTA
-            mbar_arrive_expect_tx(bar_p, CS * 16 * PR * 4);
-            mbar_arrive_expect_tx(bar_h, CS * 2048);
+    // ---- phase: open local tile i (announce the bytes its two exchanges deliver here; new episode -> new x)
+    auto open_tile = [&](int i) {
+        if (tid == 0) {
+            mbar_arrive_expect_tx(bar_p(buf_of(i)), p_bytes);
+            mbar_arrive_expect_tx(bar_h(buf_of(i)), CS * 2048);
         }
-        cp_async_wait<2 * ST - 2>();       // this tile's gate/up and down rows have landed (later tiles may be in flight)
-        fence_proxy_async();
-        __syncthreads();
-        RM_STAMP(6);
+        const TileRef tr = tile_ref(g_lo + i);
+        if (tr.b != cur_b) xprep(tr.b);
+    };
+
+    // ---- phase: gate/up partial products of tile i over this CTA's column slice (operands are in shared memory
+    // and a CTA-wide barrier has made them visible)
+    auto mma_gu = [&](int i) {
         if (tid == 0) {
             tc_fence_after();
-            const uint32_t aa = sGU + st * S::GU_STAGE;
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                    mma_bf16_ss(tmem_d1, desc_k | desc_addr(aa + kb * 16384 + ks * 32),
+                    mma_bf16_ss(tmem_d1 + buf_of(i) * NTOK, desc_k | desc_addr(sGU + kb * 16384 + ks * 32),
                                 desc_k | desc_addr(sX + kb * (NTOK * 128) + ks * 32), IDESC_GU, (kb | ks) != 0);
-            mma_commit(bar_gu);
+            mma_commit(bar_gu(buf_of(i)));
         }
-        if (!mbar_wait(bar_gu, par_gu)) rm_set_status(a.status, RM_ERR_TIMEOUT);
-        par_gu ^= 1;
-        tc_fence_after();
-        RM_STAMP(7);
-        // the gate/up stage is free again: start the tile that will use it next
-        if (g + ST < g_hi) issue_gu(g + ST, st);
-        cp_async_commit();
+    };
 
-        // ---- reduce-scatter: row m of D1 (gate or up of tile neuron q) goes to the CTA that owns q.  When a staging
-        // area is free (a dedicated one, or this tile's gate/up stage when no further tile will refill it) the rows
-        // are laid out per destination in local shared memory and moved by 8 bulk copies; otherwise every thread
-        // sends its row with asynchronous 16-byte stores.
-        const bool stage_in_gu = !(g + ST < g_hi) && CS * 16 * PR * 4 <= S::GU_STAGE;
-        if (DS || stage_in_gu) {
-            unsigned char* stg = DS ? gbase + S::OFF_P + CS * 16 * PR * 4 : gbase + S::OFF_GU + st * S::GU_STAGE;
+    // ---- phase: reduce-scatter of tile i.  Row m of D1 (gate or up of tile neuron q) goes to the CTA that owns q.
+    // When a staging area is free (the dedicated one, or the gate/up stage when no further tile will refill it) the
+    // rows are laid out per destination in local shared memory and moved by 8 bulk copies; otherwise every thread
+    // sends its row with asynchronous 16-byte stores.  `refill` says whether the gate/up stage is being refilled.
+    auto scatter = [&](int i, bool refill) {
+        const int pb = buf_of(i);
+        const uint32_t d1 = tmem_d1 + pb * NTOK;
+        const bool stage_in_gu = !refill && p_bytes <= S::GU_STAGE;
+        if (S::STAGED || stage_in_gu) {
+            unsigned char* stg = S::STAGED ? gbase + S::OFF_P + NB * p_bytes : gbase + S::OFF_GU;
             for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
                 float v[32];
                 const int m = (warp & 3) * 32 + lane;
-                tmem_ld32(tmem_d1 + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
+                tmem_ld32(d1 + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
                 const int q = m & 63;
                 float* row = reinterpret_cast<float*>(stg) + (((q >> 3) * 16 + (m >> 6) * 8 + (q & 7)) * PR + c0);
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (c0 + 4 * i < PR)
-                        *reinterpret_cast<float4*>(row + 4 * i) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                for (int k = 0; k < 8; ++k)
+                    if (c0 + 4 * k < PR)
+                        *reinterpret_cast<float4*>(row + 4 * k) = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
             }
             tc_fence_before();
             fence_proxy_async();
             __syncthreads();
             if (tid < CS)
-                bulk_copy_to_peer(map_to_rank(sP + (j * 16 * PR) * 4, tid), smem_u32(stg) + tid * 16 * PR * 4,
-                                  16 * PR * 4, map_to_rank(bar_p, tid));
+                bulk_copy_to_peer(map_to_rank(sP + pb * p_bytes + (j * 16 * PR) * 4, tid), smem_u32(stg) + tid * 16 * PR * 4,
+                                  16 * PR * 4, map_to_rank(bar_p(pb), tid));
         } else {
             for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
                 float v[32];
                 const int m = (warp & 3) * 32 + lane;
-                tmem_ld32(tmem_d1 + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
+                tmem_ld32(d1 + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
                 const int q = m & 63;
-                const uint32_t dst = map_to_rank(sP + ((j * 16 + (m >> 6) * 8 + (q & 7)) * PR + c0) * 4, q >> 3);
-                const uint32_t rbar = map_to_rank(bar_p, q >> 3);
+                const uint32_t dst = map_to_rank(sP + pb * p_bytes + ((j * 16 + (m >> 6) * 8 + (q & 7)) * PR + c0) * 4, q >> 3);
+                const uint32_t rbar = map_to_rank(bar_p(pb), q >> 3);
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (c0 + 4 * i < PR) st_async_v4(dst + i * 16, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3], rbar);
+                for (int k = 0; k < 8; ++k)
+                    if (c0 + 4 * k < PR) st_async_v4(dst + k * 16, v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3], rbar);
+            }
+            tc_fence_before();
+        }
+        RM_STAMP(8);
+    };
+
+    // ---- phase: owner work of tile i -- sum the 8 partials, GeLU-tanh(g) * u, activation record, h = hi + lo in
+    // bf16 as this CTA's atom of the MN-major h operand, then all-gather the atom into every CTA (bulk copies)
+    auto reduce_bcast = [&](int i, const TileRef& tr) {
+        const int pb = buf_of(i);
+        constexpr int TPL = NTOK / 32;                     // tokens per lane
+        const int ql = warp;                               // local neuron 0..7 (tile neuron 8j + ql)
+        const int t0 = lane * TPL;
+        const float* gP = reinterpret_cast<const float*>(gbase + S::OFF_P + pb * p_bytes);
+        unsigned char* gHS = gbase + S::OFF_HS + pb * 2048;
+        float gsum[TPL], usum[TPL];
+#pragma unroll
+        for (int k = 0; k < TPL; ++k) gsum[k] = usum[k] = 0.f;
+        if (t0 < PR) {
+#pragma unroll
+            for (int src = 0; src < CS; ++src) {
+                const float* pg = gP + (src * 16 + ql) * PR + t0;
+                const float* pu = gP + (src * 16 + 8 + ql) * PR + t0;
+#pragma unroll
+                for (int k = 0; k < TPL; ++k) { gsum[k] += pg[k]; usum[k] += pu[k]; }
             }
         }
-        tc_fence_before();
-        RM_STAMP(8);
-        // (1) every source's partial sums for this CTA's 8 neurons have arrived
-        if (!mbar_wait(bar_p, par_p)) rm_set_status(a.status, RM_ERR_TIMEOUT);
-        par_p ^= 1;
-        RM_STAMP(9);
-
-        // ---- owner: sum the 8 partials, GeLU-tanh(g) * u, activation record, h = hi + lo in bf16
+        float rec = 0.f;
+        float hv[TPL];
+#pragma unroll
+        for (int k = 0; k < TPL; ++k) {
+            hv[k] = (t0 + k < T) ? rm_gelu_tanh(gsum[k]) * usum[k] : 0.f;
+            rec += fabsf(hv[k]);
+        }
+        // row = local neuron, 128 bytes = 64 tokens, 16-byte chunks swizzled by the row; hi at 0, lo at 1024
         {
-            constexpr int TPL = NTOK / 32;                 // tokens per lane
-            const int ql = warp;                           // local neuron 0..7 (tile neuron 8j + ql)
-            const int t0 = lane * TPL;
-            float gsum[TPL], usum[TPL];
-#pragma unroll
-            for (int i = 0; i < TPL; ++i) gsum[i] = usum[i] = 0.f;
-            if (t0 < PR) {
-#pragma unroll
-                for (int src = 0; src < CS; ++src) {
-                    const float* pg = gP + (src * 16 + ql) * PR + t0;
-                    const float* pu = gP + (src * 16 + 8 + ql) * PR + t0;
-#pragma unroll
-                    for (int i = 0; i < TPL; ++i) { gsum[i] += pg[i]; usum[i] += pu[i]; }
-                }
+            unsigned char* rowp = gHS + ql * 128 + ((((t0 >> 3) ^ ql) & 7) << 4) + (t0 & 7) * 2;
+            if (TPL == 2) {
+                const __nv_bfloat162 hi = __floats2bfloat162_rn(hv[0], hv[TPL - 1]);
+                const float2 hf = __bfloat1622float2(hi);
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(hv[0] - hf.x, hv[TPL - 1] - hf.y);
+                *reinterpret_cast<__nv_bfloat162*>(rowp) = hi;
+                *reinterpret_cast<__nv_bfloat162*>(rowp + 1024) = lo;
+            } else {
+                const __nv_bfloat16 hi = __float2bfloat16_rn(hv[0]);
+                *reinterpret_cast<__nv_bfloat16*>(rowp) = hi;
+                *reinterpret_cast<__nv_bfloat16*>(rowp + 1024) = __float2bfloat16_rn(hv[0] - __bfloat162float(hi));
             }
-            float rec = 0.f;
-            float hv[TPL];
+        }
+        if (a.record) {
 #pragma unroll
-            for (int i = 0; i < TPL; ++i) {
-                hv[i] = (t0 + i < T) ? rm_gelu_tanh(gsum[i]) * usum[i] : 0.f;
-                rec += fabsf(hv[i]);
-            }
-            // this CTA's atom of the h operand: row = local neuron, 128 bytes = 64 tokens, 16-byte chunks swizzled
-            // by the row; hi at offset 0, lo (h - hi) at offset 1024
-            {
-                unsigned char* rowp = gHS + ql * 128 + ((((t0 >> 3) ^ ql) & 7) << 4) + (t0 & 7) * 2;
-                if (TPL == 2) {
-                    const __nv_bfloat162 hi = __floats2bfloat162_rn(hv[0], hv[TPL - 1]);
-                    const float2 hf = __bfloat1622float2(hi);
-                    const __nv_bfloat162 lo = __floats2bfloat162_rn(hv[0] - hf.x, hv[TPL - 1] - hf.y);
-                    *reinterpret_cast<__nv_bfloat162*>(rowp) = hi;
-                    *reinterpret_cast<__nv_bfloat162*>(rowp + 1024) = lo;
-                } else {
-                    const __nv_bfloat16 hi = __float2bfloat16_rn(hv[0]);
-                    *reinterpret_cast<__nv_bfloat16*>(rowp) = hi;
-                    *reinterpret_cast<__nv_bfloat16*>(rowp + 1024) = __float2bfloat16_rn(hv[0] - __bfloat162float(hi));
-                }
-            }
-            if (a.record) {
-#pragma unroll
-                for (int d = 16; d > 0; d >>= 1) rec += __shfl_xor_sync(0xffffffffu, rec, d);
-                const int n = gN[((g - g_lo) & 1) * NT + j * 8 + ql];
-                if (lane == 0 && n >= 0)
-                    a.record[(size_t)tr.b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
-            }
+            for (int d = 16; d > 0; d >>= 1) rec += __shfl_xor_sync(0xffffffffu, rec, d);
+            const int n = gN[(i & 1) * NT + j * 8 + ql];
+            if (lane == 0 && n >= 0)
+                a.record[(size_t)tr.b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
         }
         fence_proxy_async();
         __syncthreads();
-        // ---- all-gather h: this CTA's atom becomes atom j of the MN-major hi and lo operand tiles of every CTA
         if (tid < 2 * CS) {
             const int dst = tid >> 1, part = tid & 1;
-            bulk_copy_to_peer(map_to_rank(sHT + part * S::HT_HALF + j * 1024, dst), smem_u32(gHS) + part * 1024, 1024,
-                              map_to_rank(bar_h, dst));
+            bulk_copy_to_peer(map_to_rank(sHT + pb * 2 * S::HT_HALF + part * S::HT_HALF + j * 1024, dst),
+                              smem_u32(gHS) + part * 1024, 1024, map_to_rank(bar_h(pb), dst));
         }
         RM_STAMP(10);
-        // (2) h of the whole tile (all 8 owners' chunks) has arrived in this CTA
-        if (!mbar_wait(bar_h, par_h)) rm_set_status(a.status, RM_ERR_TIMEOUT);
-        par_h ^= 1;
-        RM_STAMP(11);
+    };
 
-        // ---- down projection of the tile, accumulated in tensor memory across the episode's tiles
+    // ---- phase: down projection of tile i, accumulated in tensor memory across the episode's tiles
+    auto mma_dn = [&](int i, const TileRef& tr) {
         if (tid == 0) {
             fence_proxy_async();
             tc_fence_after();
-            const uint32_t ad = sDN + st * S::DN_STAGE;
+            const uint32_t ht = sHT + buf_of(i) * 2 * S::HT_HALF;
 #pragma unroll
             for (int mm = 0; mm < HS / 128; ++mm)
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t aa = desc_mn | desc_addr(ad + mm * 16384 + ks * 2048);
-                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(sHT + ks * 2048), IDESC_DN,
+                    const uint64_t aa = desc_mn | desc_addr(sDN + mm * 16384 + ks * 2048);
+                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + ks * 2048), IDESC_DN,
                                 !(tr.first && ks == 0));
-                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(sHT + S::HT_HALF + ks * 2048), IDESC_DN, true);
+                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + S::HT_HALF + ks * 2048), IDESC_DN, true);
                 }
             mma_commit(bar_dn);
         }
         RM_STAMP(12);
-        // the down stage and the h tiles are reused by the next tile: wait for the products to finish
-        if (!mbar_wait(bar_dn, par_dn)) rm_set_status(a.status, RM_ERR_TIMEOUT);
-        par_dn ^= 1;
-        tc_fence_after();
-        if (g + ST < g_hi) issue_dn(g + ST, st);
-        cp_async_commit();
-        RM_STAMP(13);
+    };
 
-        if (tr.last) {
-            // ---- add this CTA's [T x Hs] partial of y to the residual stream
+    // ---- phase: add this CTA's [T x Hs] partial of y to the residual stream
+    auto flush = [&](const TileRef& tr) {
 #pragma unroll
-            for (int mm = 0; mm < HS / 128; ++mm) {
-                for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
-                    float v[32];
-                    tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
-                    float* dst = a.r_out + (size_t)tr.b * T * H + (size_t)j * HS + mm * 128 + (warp & 3) * 32 + lane;
+        for (int mm = 0; mm < HS / 128; ++mm) {
+            for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
+                float v[32];
+                tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
+                float* dst = a.r_out + (size_t)tr.b * T * H + (size_t)j * HS + mm * 128 + (warp & 3) * 32 + lane;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (c0 + i < T) atomicAdd(dst + (size_t)(c0 + i) * H, v[i]);
-                }
+                for (int k = 0; k < 32; ++k)
+                    if (c0 + k < T) atomicAdd(dst + (size_t)(c0 + k) * H, v[k]);
             }
-            tc_fence_before();
-            __syncthreads();
-            RM_STAMP(14);
         }
+        tc_fence_before();
+        __syncthreads();
+        RM_STAMP(14);
+    };
+
+    if (!PIPE) {
+        // ---- one tile at a time: open, gate/up, scatter, owner work, down.  Loads of the next tile are issued as
+        // soon as the stage they go to is free, so they travel during the exchanges.
+        for (int i = 0; i < n_tiles; ++i) {
+            const TileRef tr = tile_ref(g_lo + i);
+            open_tile(i);
+            cp_async_wait<0>();            // this tile's gate/up and down rows have landed
+            fence_proxy_async();
+            __syncthreads();
+            RM_STAMP(6);
+            mma_gu(i);
+            wait_bar(bar_gu(0), phase_of(i));
+            tc_fence_after();
+            RM_STAMP(7);
+            const bool refill = i + 1 < n_tiles;
+            if (refill) issue_gu(g_lo + i + 1);
+            cp_async_commit();
+            scatter(i, refill);
+            wait_bar(bar_p(0), phase_of(i));           // every source's partial sums for this CTA's neurons are here
+            RM_STAMP(9);
+            reduce_bcast(i, tr);
+            wait_bar(bar_h(0), phase_of(i));           // h of the whole tile (all 8 owners' atoms) is here
+            RM_STAMP(11);
+            mma_dn(i, tr);
+            wait_bar(bar_dn, par_dn);                  // the down stage and the h tiles may be reused
+            par_dn ^= 1;
+            tc_fence_after();
+            if (refill) issue_dn(g_lo + i + 1);
+            cp_async_commit();
+            RM_STAMP(13);
+            if (tr.last) flush(tr);
 #ifdef RM_PHASE_TIMING
-        stamp_ok = false;                  // first tile only
+            stamp_ok = false;              // first tile only
 #endif
+        }
+    } else if (n_tiles > 0) {
+        // ---- two tiles in flight: the gate/up product and the scatter of tile i+1 are issued before the owner work
+        // and the down projection of tile i, so each exchange travels while the other tile's work runs.
+        open_tile(0);
+        cp_async_wait<0>();
+        fence_proxy_async();
+        __syncthreads();
+        RM_STAMP(6);
+        mma_gu(0);
+        wait_bar(bar_gu(0), 0);
+        tc_fence_after();
+        RM_STAMP(7);
+        if (1 < n_tiles) issue_gu(g_lo + 1);
+        cp_async_commit();
+        scatter(0, 1 < n_tiles);
+        for (int i = 0; i < n_tiles; ++i) {
+            const TileRef tr = tile_ref(g_lo + i);
+            const bool more = i + 1 < n_tiles;
+            if (more) {
+                open_tile(i + 1);
+                if (i == 0) cp_async_wait<0>(); else cp_async_wait<1>();      // gate/up rows of tile i+1 have landed
+                fence_proxy_async();
+                __syncthreads();
+                mma_gu(i + 1);
+            }
+            wait_bar(bar_p(buf_of(i)), phase_of(i));
+            RM_STAMP(9);
+            reduce_bcast(i, tr);
+            if (more) {
+                wait_bar(bar_gu(buf_of(i + 1)), phase_of(i + 1));
+                tc_fence_after();
+                const bool refill = i + 2 < n_tiles;
+                if (refill) issue_gu(g_lo + i + 2);
+                cp_async_commit();
+                scatter(i + 1, refill);
+            } else {
+                cp_async_commit();
+            }
+            wait_bar(bar_h(buf_of(i)), phase_of(i));
+            RM_STAMP(11);
+            cp_async_wait<1>();            // down rows of tile i have landed
+            fence_proxy_async();
+            __syncthreads();
+            mma_dn(i, tr);
+            wait_bar(bar_dn, par_dn);
+            par_dn ^= 1;
+            tc_fence_after();
+            if (more) issue_dn(g_lo + i + 1);
+            cp_async_commit();
+            RM_STAMP(13);
+            if (tr.last) flush(tr);
+#ifdef RM_PHASE_TIMING
+            stamp_ok = false;
+#endif
+        }
     }
 #ifdef RM_PHASE_TIMING
     stamp_ok = true;
@@ -563,10 +644,10 @@ __global__ void __launch_bounds__(FT, (HS == 128 && ST == 1 && !DS ? 2 : 1)) fus
     RM_WALL(3);
 }
 
-template <int NTOK, int HS, int ST, bool DS>
+template <int NTOK, int HS, bool PIPE>
 int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cudaStream_t s) {
-    using S = Smem<NTOK, HS, ST, DS>;
-    auto kern = fused_layer_kernel<NTOK, HS, ST, DS>;
+    using S = Smem<NTOK, HS, PIPE>;
+    auto kern = fused_layer_kernel<NTOK, HS, PIPE>;
     const int smem = S::total_bytes(a.T);
     static int configured = 0;
     if (configured < smem) {
@@ -592,10 +673,10 @@ int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cuda
     return RM_OK;
 }
 
-template <int NTOK, int HS, int ST, bool DS>
+template <int NTOK, int HS, bool PIPE>
 int max_clusters(int T, int* out) {
-    using S = Smem<NTOK, HS, ST, DS>;
-    auto kern = fused_layer_kernel<NTOK, HS, ST, DS>;
+    using S = Smem<NTOK, HS, PIPE>;
+    auto kern = fused_layer_kernel<NTOK, HS, PIPE>;
     const int smem = S::total_bytes(T);
     RM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     cudaLaunchConfig_t cfg = {};
@@ -641,8 +722,8 @@ int rm_fused_init(rm_ctx* ctx) {
     ctx->fused_clusters = 0;
     ctx->fused_blocks_per_sm = 1;
     int n = 0, rc = RM_OK;
-    if (ctx->g.H == 1024) rc = max_clusters<64, 128, 1, false>(64, &n);
-    else if (ctx->g.H == 2048) rc = max_clusters<64, 256, 1, true>(64, &n);
+    if (ctx->g.H == 1024) rc = max_clusters<64, 128, false>(64, &n);
+    else if (ctx->g.H == 2048) rc = max_clusters<64, 256, false>(64, &n);
     else return RM_OK;
     if (rc != RM_OK) return rc;
     ctx->fused_clusters = n;
@@ -683,16 +764,20 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
         if (want < 1) want = 1;
         if (want < nc) nc = (int)want;
     }
-    // Variant: at H = 1024 the lean kernel (112 KB, two CTAs per SM so that consecutive layers overlap) serves launches
-    // where a cluster gets a single tile; when clusters walk several tiles, the variant with a dedicated staging
-    // buffer for the outgoing partial sums keeps the exchange on the copy engine for every tile.
+    // Variant: the lean kernel (H = 1024 only: 112 KB, two CTAs per SM so that consecutive layers overlap) serves
+    // launches where a cluster gets a single tile; when clusters walk several tiles, the pipelined variant keeps two
+    // tiles in flight per cluster (double-buffered exchange state, one CTA per SM).
     long long tiles = per_episode > 0 ? (long long)((per_episode + NT - 1) / NT) * la.B : 0;
-    const bool multi = ctx->variant_override ? ctx->variant_override == 2 : (tiles == 0 || tiles > nc);
+    const bool pipe = ctx->variant_override ? ctx->variant_override == 2 : (tiles == 0 || tiles > nc);
     const bool small_t = la.T <= 32;
     if (ctx->g.H == 1024) {
-        if (multi)
-            return small_t ? launch_fused<32, 128, 1, true>(ctx, a, nc, pdl, s) : launch_fused<64, 128, 1, true>(ctx, a, nc, pdl, s);
-        return small_t ? launch_fused<32, 128, 1, false>(ctx, a, nc, pdl, s) : launch_fused<64, 128, 1, false>(ctx, a, nc, pdl, s);
+        if (pipe)
+            return small_t ? launch_fused<32, 128, true>(ctx, a, nc, pdl, s) : launch_fused<64, 128, true>(ctx, a, nc, pdl, s);
+        return small_t ? launch_fused<32, 128, false>(ctx, a, nc, pdl, s) : launch_fused<64, 128, false>(ctx, a, nc, pdl, s);
     }
-    return small_t ? launch_fused<32, 256, 1, true>(ctx, a, nc, pdl, s) : launch_fused<64, 256, 1, true>(ctx, a, nc, pdl, s);
+    // H = 2048: the pipelined variant when its buffers fit the 227 KB of an SM (they do up to T = 60), else serial
+    const bool fits = Smem<64, 256, true>::total_bytes(la.T) <= 232448;
+    if (small_t)
+        return pipe ? launch_fused<32, 256, true>(ctx, a, nc, pdl, s) : launch_fused<32, 256, false>(ctx, a, nc, pdl, s);
+    return (pipe && fits) ? launch_fused<64, 256, true>(ctx, a, nc, pdl, s) : launch_fused<64, 256, false>(ctx, a, nc, pdl, s);
 }
