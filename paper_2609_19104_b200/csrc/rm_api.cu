@@ -279,7 +279,7 @@ int rm_set_option(rm_ctx* ctx, const char* name, int value) {
         if (value < 0) return RM_ERR_INVALID_ARG;
         ctx->count_hint = value;
     } else if (n == "variant") {
-        if (value < 0 || value > 2) return RM_ERR_INVALID_ARG;
+        if (value < 0 || value > 3) return RM_ERR_INVALID_ARG;
         ctx->variant_override = value;
     } else if (n == "max_clusters") {
         if (value < 0) return RM_ERR_INVALID_ARG;

@@ -644,6 +644,501 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     RM_WALL(3);
 }
 
+// ===============================================================================================================
+// Warp-specialised variant for launches in which a cluster walks many tiles (large K, dense passes, batches).
+// The same decomposition and exchanges as above, but the phases of consecutive tiles run concurrently on different
+// warps, connected by mbarriers:
+//   warps 0-3  scatter : wait for the gate/up product of tile i, read it from tensor memory, send the partial sums
+//                        to their owners; at the end of an episode, add the down accumulator to the residual stream
+//   warps 4-7  owner   : wait for the 8 partial sums of tile i, GeLU-tanh(g)*u, record, h atom, all-gather
+//   warp  8    mma     : one thread issues gate/up(i) as soon as its rows have landed and down(i-1) as soon as h(i-1)
+//                        is complete in this CTA
+//   warps 9-10 loader  : one neuron per thread; cp.async gathers of the next tile as soon as a stage is free, also
+//                        across the dependency wait on the previous layer
+// Exchange state (D1 in tensor memory, partial-sum buffer, h tiles, h atom, staging) is double-buffered by tile
+// parity.  An episode change drains the pipeline (CTA-wide barrier), prepares the new x slice and restarts.
+constexpr int WT = 352;            // threads per CTA of the warp-specialised kernel
+
+template <int NTOK, int HS>
+struct SmemWS {
+    static constexpr int KB = HS / 64;
+    static constexpr bool STAGED = HS == 128;                // room for staging buffers only at H = 1024
+    static constexpr int X_BYTES = KB * NTOK * 128;
+    static constexpr int GU_STAGE = KB * 128 * 128;
+    static constexpr int DN_STAGE = KB * NT * 128;
+    static constexpr int HT_HALF = NT * 128;
+    static constexpr int OFF_X = 0;
+    static constexpr int OFF_GU = OFF_X + X_BYTES;
+    static constexpr int OFF_DN = OFF_GU + GU_STAGE;
+    static constexpr int OFF_HT = OFF_DN + DN_STAGE;         // [2 buffers][hi, lo]
+    static constexpr int OFF_HS = OFF_HT + 4 * HT_HALF;      // [2 buffers] h atom (1 KB hi, 1 KB lo)
+    static constexpr int OFF_SS = OFF_HS + 2 * 2048;
+    static constexpr int OFF_N = OFF_SS + CS * 64 * 4;
+    static constexpr int OFF_PREF = OFF_N + 4 * NT * 4;     // neuron ids of four consecutive tiles (the loader runs ahead)
+    static constexpr int OFF_BAR = ((OFF_PREF + (2 * MAXB + 1) * 4 + 7) / 8) * 8;
+    static constexpr int OFF_P = ((OFF_BAR + 160 + 15) / 16) * 16;  // [2][CS][16][p_row] (+ [2] staging), sized at launch
+    static constexpr int TMEM_COLS = 256;                    // D1 x 2 (NTOK each) + D2 (HS/128 x NTOK) <= 256
+    static int total_bytes(int T) { return OFF_P + (STAGED ? 4 : 2) * CS * 16 * p_row_for(T) * 4 + 1024; }
+};
+
+template <int NTOK, int HS>
+__global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a) {
+    using S = SmemWS<NTOK, HS>;
+    constexpr int KB = S::KB;
+    extern __shared__ unsigned char smem_dyn[];
+    const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    unsigned char* gbase = smem_dyn + (base - smem_u32(smem_dyn));
+    const uint32_t sX = base + S::OFF_X, sGU = base + S::OFF_GU, sDN = base + S::OFF_DN, sHT = base + S::OFF_HT;
+    const uint32_t sP = base + S::OFF_P, sSS = base + S::OFF_SS;
+    const float* gSS = reinterpret_cast<const float*>(gbase + S::OFF_SS);
+    int* gN = reinterpret_cast<int*>(gbase + S::OFF_N);
+    int* gPref = reinterpret_cast<int*>(gbase + S::OFF_PREF);
+    int* gCnt = gPref + MAXB + 1;
+    const uint32_t bar0 = base + S::OFF_BAR;
+    auto bar_gu = [&](int pb) { return bar0 + 8 * pb; };           // gate/up product of a tile is complete
+    auto bar_p = [&](int pb) { return bar0 + 16 + 8 * pb; };       // all partial sums for this owner have arrived
+    auto bar_h = [&](int pb) { return bar0 + 32 + 8 * pb; };       // all h atoms have arrived
+    auto d1_free = [&](int pb) { return bar0 + 48 + 8 * pb; };     // the scatter warps have read D1[pb]
+    const uint32_t bar_dn = bar0 + 64, bar_s = bar0 + 72, gu_full = bar0 + 80, dn_full = bar0 + 88;
+    const uint32_t s_tmem = bar0 + 96;
+    volatile uint32_t* g_tmem = reinterpret_cast<volatile uint32_t*>(gbase + S::OFF_BAR + 96);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int j = (int)cluster_ctarank();
+    const int cid = (int)cluster_id_x(), NC = (int)cluster_count_x();
+    const int H = a.H, T = a.T, PR = a.p_row;
+    const int p_bytes = CS * 16 * PR * 4;
+
+    if (tid == 0) {
+        for (int pb = 0; pb < 2; ++pb) {
+            mbar_init(bar_gu(pb), 1); mbar_init(bar_p(pb), 1); mbar_init(bar_h(pb), 1); mbar_init(d1_free(pb), 4);
+        }
+        mbar_init(bar_dn, 1);
+        mbar_init(bar_s, 1);
+        mbar_init(gu_full, 32);
+        mbar_init(dn_full, 32);
+        fence_mbar_init();
+        int acc = 0;
+        const int cap = (int)(a.list_cap < (int64_t)a.I ? a.list_cap : (int64_t)a.I);
+        for (int b = 0; b < a.B; ++b) {
+            int c = a.I;
+            if (a.idx) {
+                c = a.count[(size_t)b * a.count_stride];
+                if (c < 0 || c > cap) { rm_set_status(a.status, RM_ERR_INDEX); c = c < 0 ? 0 : cap; }
+            }
+            gCnt[b] = c;
+            gPref[b] = acc;
+            acc += (c + NT - 1) / NT;
+        }
+        gPref[a.B] = acc;
+    }
+    if (warp == 8) tmem_alloc(s_tmem, S::TMEM_COLS);
+    tc_fence_before();
+    cluster_sync();
+    tc_fence_after();
+    const uint32_t tmem_d1 = *g_tmem;
+    const uint32_t tmem_d2 = tmem_d1 + 2 * NTOK;
+    pdl_launch_dependents();
+
+    const int tiles_total = gPref[a.B];
+    const int n_active = tiles_total < NC ? tiles_total : NC;
+    const int g_lo = cid < n_active ? (int)((long long)cid * tiles_total / n_active) : 0;
+    const int g_hi = cid < n_active ? (int)((long long)(cid + 1) * tiles_total / n_active) : 0;
+
+    auto tile_ref = [&](int g) {
+        TileRef r;
+        int b = 0;
+        while (gPref[b + 1] <= g) ++b;
+        r.b = b;
+        r.p0 = (g - gPref[b]) * NT;
+        const int left = gCnt[b] - r.p0;
+        r.nvalid = left < NT ? left : NT;
+        r.first = (g == g_lo) || (g == gPref[b]);
+        r.last = (g == g_hi - 1) || (g == gPref[b + 1] - 1);
+        return r;
+    };
+    auto wait_bar = [&](uint32_t bar, uint32_t parity) {
+        if (!mbar_wait(bar, parity)) rm_set_status(a.status, RM_ERR_TIMEOUT);
+    };
+
+    // loaders: lane l owns tile neurons l and l + 32; `it` is the cluster-local tile sequence number.  Warp 9 gathers
+    // the gate and up rows, warp 10 the down rows, so neither waits for the other's stage.
+    auto tile_neuron = [&](const TileRef& r, int q, bool report) {
+        int n = -1;
+        if (q < r.nvalid) {
+            n = a.idx ? a.idx[(size_t)r.b * a.idx_stride + r.p0 + q] : r.p0 + q;
+            if (n < 0 || n >= a.I) { if (report) rm_set_status(a.status, RM_ERR_INDEX); n = -1; }
+        }
+        return n;
+    };
+    auto load_gu = [&](int g, int it) {
+        const TileRef r = tile_ref(g);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int q = lane + 32 * half;
+            const int n = tile_neuron(r, q, true);
+            gN[(it & 3) * NT + q] = n;
+            const __nv_bfloat16* src = a.packed + (size_t)(n < 0 ? 0 : n) * 3 * H + (size_t)j * 3 * HS;
+            const uint32_t d0 = sGU + q * 128;
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t off = kb * 16384 + ((c ^ (q & 7)) << 4);
+                    cp_async16(d0 + off, src + kb * 64 + c * 8, n >= 0);                      // gate row
+                    cp_async16(d0 + off + 64 * 128, src + HS + kb * 64 + c * 8, n >= 0);      // up row
+                }
+        }
+        __threadfence_block();             // the neuron ids are read by the owner warps much later
+        cp_async_arrive_noinc(gu_full);
+    };
+    auto load_dn = [&](int g) {
+        const TileRef r = tile_ref(g);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int q = lane + 32 * half;
+            const int n = tile_neuron(r, q, false);
+            const __nv_bfloat16* src = a.packed + (size_t)(n < 0 ? 0 : n) * 3 * H + (size_t)j * 3 * HS + 2 * HS;
+            const uint32_t d0 = sDN + q * 128;
+#pragma unroll
+            for (int cb = 0; cb < KB; ++cb)
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    cp_async16(d0 + cb * 8192 + ((c ^ (q & 7)) << 4), src + cb * 64 + c * 8, n >= 0);
+        }
+        cp_async_arrive_noinc(dn_full);
+    };
+
+    __syncthreads();                       // gPref / gCnt
+
+    constexpr uint32_t IDESC_GU = idesc_bf16_f32(128, NTOK, false, false);
+    constexpr uint32_t IDESC_DN = idesc_bf16_f32(128, NTOK, true, true);
+    const uint64_t desc_k = smem_desc_sw128(0, 16, 1024);
+    const uint64_t desc_mn = smem_desc_sw128(0, 8192, 1024);
+    const int n_tiles = g_hi - g_lo;
+    uint32_t par_s = 0;
+    bool waited_prev = false;              // griddepcontrol.wait has been executed by this thread
+
+    // ---- segments: maximal runs of this cluster's tiles within one episode
+    int it0 = 0;                            // cluster-local sequence number of the segment's first tile
+    while (it0 < n_tiles) {
+        const TileRef tr0 = tile_ref(g_lo + it0);
+        const int b = tr0.b;
+        int seg = 1;
+        while (it0 + seg < n_tiles && tile_ref(g_lo + it0 + seg).b == b) ++seg;
+
+        if (warp >= 9) {
+            // loader warps: the segment's first tile goes out before anything else (stages are free after a drain)
+            if (warp == 9) load_gu(g_lo + it0, it0); else load_dn(g_lo + it0);
+        } else if (warp < 8) {
+            // scatter and owner warps: x slice of episode b (256-thread mapping)
+            if (!waited_prev) { pdl_wait(); waited_prev = true; }
+            constexpr int PARTS = 256 / NTOK;
+            constexpr int CPP = HS / PARTS;
+            const int t = tid / PARTS, part = tid % PARTS;
+            int n_share = 1, my_share = 0;
+            if (a.add_residual) {
+                const long long e0 = gPref[b], e1 = gPref[b + 1];
+                int first_c = (int)((e0 * n_active) / tiles_total);
+                while ((long long)(first_c + 1) * tiles_total / n_active <= e0) ++first_c;
+                int last_c = (int)(((e1 - 1) * n_active) / tiles_total);
+                while (last_c + 1 < n_active && (long long)(last_c + 1) * tiles_total / n_active < e1) ++last_c;
+                n_share = last_c - first_c + 1;
+                my_share = cid - first_c;
+            }
+            if (a.x) {
+                const uint4* src = reinterpret_cast<const uint4*>(a.x + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP);
+#pragma unroll
+                for (int i = 0; i < CPP / 8; ++i) {
+                    const uint4 u = t < T ? src[i] : make_uint4(0, 0, 0, 0);
+                    const int k = part * CPP + i * 8;
+                    *reinterpret_cast<uint4*>(gbase + S::OFF_X + (k >> 6) * (NTOK * 128) + t * 128 +
+                                              ((((k & 63) >> 3) ^ (t & 7)) << 4)) = u;
+                }
+            } else {
+                float v[CPP];
+                float ss = 0.f;
+                if (t < T) {
+                    const float4* src = reinterpret_cast<const float4*>(a.r_in + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP);
+#pragma unroll
+                    for (int i = 0; i < CPP / 4; ++i) {
+                        const float4 f = src[i];
+                        v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+                    }
+#pragma unroll
+                    for (int i = 0; i < CPP; ++i) ss = fmaf(v[i], v[i], ss);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < CPP; ++i) v[i] = 0.f;
+                }
+#pragma unroll
+                for (int d = 1; d < PARTS; d <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+                if (tid == 0) mbar_arrive_expect_tx(bar_s, CS * NTOK * 4);
+#pragma unroll
+                for (int dst = part; dst < CS; dst += PARTS)
+                    st_async_f32(map_to_rank(sSS + (j * 64 + t) * 4, dst), ss, map_to_rank(bar_s, dst));
+                if (a.add_residual && t < T && (t % n_share) == my_share) {
+                    float* o = a.r_out + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP;
+#pragma unroll
+                    for (int i = 0; i < CPP / 4; ++i) red_add_v4(o + 4 * i, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                }
+                wait_bar(bar_s, par_s);
+                float tot = 0.f;
+#pragma unroll
+                for (int src = 0; src < CS; ++src) tot += gSS[src * 64 + t];
+                const float inv = 1.0f / sqrtf(tot / (float)H + 1e-6f);
+#pragma unroll
+                for (int i = 0; i < CPP / 8; ++i) {
+                    const int k = part * CPP + i * 8;
+                    *reinterpret_cast<uint4*>(gbase + S::OFF_X + (k >> 6) * (NTOK * 128) + t * 128 +
+                                              ((((k & 63) >> 3) ^ (t & 7)) << 4)) = pack8(v + 8 * i, inv);
+                }
+            }
+            fence_proxy_async();
+        }
+        if (!a.x) par_s ^= 1;
+        __syncthreads();                   // x is in place for the mma warp
+
+        if (warp < 4) {
+            // ================= scatter warps
+            for (int k = 0; k < seg; ++k) {
+                const int it = it0 + k, pb = it & 1;
+                wait_bar(bar_gu(pb), (it >> 1) & 1);
+                tc_fence_after();
+                const uint32_t d1 = tmem_d1 + pb * NTOK;
+                const bool last_of_all = it == n_tiles - 1;
+                const bool stage_in_gu = !S::STAGED && last_of_all && p_bytes <= S::GU_STAGE;
+                if (S::STAGED || stage_in_gu) {
+                    unsigned char* stg = S::STAGED ? gbase + S::OFF_P + (2 + pb) * p_bytes : gbase + S::OFF_GU;
+                    for (int c0 = 0; c0 < NTOK; c0 += 32) {
+                        float v[32];
+                        const int m = warp * 32 + lane;
+                        tmem_ld32(d1 + ((uint32_t)(warp * 32) << 16) + c0, v);
+                        const int q = m & 63;
+                        float* row = reinterpret_cast<float*>(stg) + (((q >> 3) * 16 + (m >> 6) * 8 + (q & 7)) * PR + c0);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            if (c0 + 4 * e < PR)
+                                *reinterpret_cast<float4*>(row + 4 * e) = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(d1_free(pb));
+                    fence_proxy_async();
+                    named_barrier(2, 128);
+                    if (tid < CS)
+                        bulk_copy_to_peer(map_to_rank(sP + pb * p_bytes + (j * 16 * PR) * 4, tid),
+                                          smem_u32(stg) + tid * 16 * PR * 4, 16 * PR * 4, map_to_rank(bar_p(pb), tid));
+                } else {
+                    for (int c0 = 0; c0 < NTOK; c0 += 32) {
+                        float v[32];
+                        const int m = warp * 32 + lane;
+                        tmem_ld32(d1 + ((uint32_t)(warp * 32) << 16) + c0, v);
+                        const int q = m & 63;
+                        const uint32_t dst = map_to_rank(sP + pb * p_bytes + ((j * 16 + (m >> 6) * 8 + (q & 7)) * PR + c0) * 4, q >> 3);
+                        const uint32_t rbar = map_to_rank(bar_p(pb), q >> 3);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            if (c0 + 4 * e < PR) st_async_v4(dst + e * 16, v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3], rbar);
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(d1_free(pb));
+                }
+                // follow every phase of the down barrier (a parity wait can only tell the current phase from the
+                // previous one); down(it-1) is issued right after gate/up(it), so this does not hold the warps back
+                if (k >= 1) wait_bar(bar_dn, (it - 1) & 1);
+            }
+            // end of the episode's run: add this CTA's [T x Hs] partial of y to the residual stream
+            {
+                const int it = it0 + seg - 1;
+                wait_bar(bar_dn, it & 1);
+                tc_fence_after();
+#pragma unroll
+                for (int mm = 0; mm < HS / 128; ++mm) {
+                    for (int c0 = 0; c0 < NTOK; c0 += 32) {
+                        float v[32];
+                        tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)(warp * 32) << 16) + c0, v);
+                        float* dst = a.r_out + (size_t)b * T * H + (size_t)j * HS + mm * 128 + warp * 32 + lane;
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (c0 + e < T) atomicAdd(dst + (size_t)(c0 + e) * H, v[e]);
+                    }
+                }
+                tc_fence_before();
+            }
+        } else if (warp < 8) {
+            // ================= owner warps: warp ow handles local neurons ow and ow + 4
+            const int ow = warp - 4, ot = tid - 128;
+            constexpr int TPL = NTOK / 32;
+            const int t0 = lane * TPL;
+            for (int k = 0; k < seg; ++k) {
+                const int it = it0 + k, pb = it & 1;
+                if (ot == 0) mbar_arrive_expect_tx(bar_p(pb), p_bytes);
+                wait_bar(bar_p(pb), (it >> 1) & 1);
+                const float* gP = reinterpret_cast<const float*>(gbase + S::OFF_P + pb * p_bytes);
+                unsigned char* gHS = gbase + S::OFF_HS + pb * 2048;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int ql = ow + 4 * half;
+                    float gsum[TPL], usum[TPL];
+#pragma unroll
+                    for (int e = 0; e < TPL; ++e) gsum[e] = usum[e] = 0.f;
+                    if (t0 < PR) {
+#pragma unroll
+                        for (int src = 0; src < CS; ++src) {
+                            const float* pg = gP + (src * 16 + ql) * PR + t0;
+                            const float* pu = gP + (src * 16 + 8 + ql) * PR + t0;
+#pragma unroll
+                            for (int e = 0; e < TPL; ++e) { gsum[e] += pg[e]; usum[e] += pu[e]; }
+                        }
+                    }
+                    float rec = 0.f;
+                    float hv[TPL];
+#pragma unroll
+                    for (int e = 0; e < TPL; ++e) {
+                        hv[e] = (t0 + e < T) ? rm_gelu_tanh(gsum[e]) * usum[e] : 0.f;
+                        rec += fabsf(hv[e]);
+                    }
+                    unsigned char* rowp = gHS + ql * 128 + ((((t0 >> 3) ^ ql) & 7) << 4) + (t0 & 7) * 2;
+                    if (TPL == 2) {
+                        const __nv_bfloat162 hi = __floats2bfloat162_rn(hv[0], hv[TPL - 1]);
+                        const float2 hf = __bfloat1622float2(hi);
+                        *reinterpret_cast<__nv_bfloat162*>(rowp) = hi;
+                        *reinterpret_cast<__nv_bfloat162*>(rowp + 1024) = __floats2bfloat162_rn(hv[0] - hf.x, hv[TPL - 1] - hf.y);
+                    } else {
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(hv[0]);
+                        *reinterpret_cast<__nv_bfloat16*>(rowp) = hi;
+                        *reinterpret_cast<__nv_bfloat16*>(rowp + 1024) = __float2bfloat16_rn(hv[0] - __bfloat162float(hi));
+                    }
+                    if (a.record) {
+#pragma unroll
+                        for (int d = 16; d > 0; d >>= 1) rec += __shfl_xor_sync(0xffffffffu, rec, d);
+                        const int n = gN[(it & 3) * NT + j * 8 + ql];
+                        if (lane == 0 && n >= 0)
+                            a.record[(size_t)b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
+                    }
+                }
+                fence_proxy_async();
+                named_barrier(1, 128);
+                if (ot < 2 * CS) {
+                    const int dst = ot >> 1, part = ot & 1;
+                    bulk_copy_to_peer(map_to_rank(sHT + pb * 2 * S::HT_HALF + part * S::HT_HALF + j * 1024, dst),
+                                      smem_u32(gHS) + part * 1024, 1024, map_to_rank(bar_h(pb), dst));
+                }
+            }
+        } else if (warp == 8) {
+            // ================= mma warp (one thread)
+            if (lane == 0) {
+                auto do_dn = [&](int it) {
+                    const int pb = it & 1;
+                    wait_bar(bar_h(pb), (it >> 1) & 1);
+                    wait_bar(dn_full, it & 1);
+                    fence_proxy_async();
+                    tc_fence_after();
+                    const uint32_t ht = sHT + pb * 2 * S::HT_HALF;
+                    const bool first = it == it0;
+#pragma unroll
+                    for (int mm = 0; mm < HS / 128; ++mm)
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t aa = desc_mn | desc_addr(sDN + mm * 16384 + ks * 2048);
+                            mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + ks * 2048), IDESC_DN, !(first && ks == 0));
+                            mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + S::HT_HALF + ks * 2048), IDESC_DN, true);
+                        }
+                    mma_commit(bar_dn);
+                };
+                for (int k = 0; k < seg; ++k) {
+                    const int it = it0 + k, pb = it & 1;
+                    mbar_arrive_expect_tx(bar_h(pb), CS * 2048);
+                    wait_bar(gu_full, it & 1);
+                    if (it >= 2) wait_bar(d1_free(pb), ((it - 2) >> 1) & 1);
+                    fence_proxy_async();
+                    tc_fence_after();
+#pragma unroll
+                    for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            mma_bf16_ss(tmem_d1 + pb * NTOK, desc_k | desc_addr(sGU + kb * 16384 + ks * 32),
+                                        desc_k | desc_addr(sX + kb * (NTOK * 128) + ks * 32), IDESC_GU, (kb | ks) != 0);
+                    mma_commit(bar_gu(pb));
+                    if (k >= 1) do_dn(it - 1);
+                }
+                do_dn(it0 + seg - 1);
+            }
+        } else {
+            // ================= loader warps: tiles after the segment's first
+            for (int k = 1; k < seg; ++k) {
+                const int it = it0 + k;
+                if (warp == 9) {
+                    wait_bar(bar_gu((it - 1) & 1), ((it - 1) >> 1) & 1);     // gate/up stage is free
+                    load_gu(g_lo + it, it);
+                } else {
+                    wait_bar(bar_dn, (it - 1) & 1);                           // down stage is free
+                    load_dn(g_lo + it);
+                }
+            }
+        }
+        __syncthreads();                   // drain: every role is done with this episode's run
+        it0 += seg;
+    }
+
+    // ---- duties: residual of episodes without active neurons, and the buffer a later layer accumulates into
+    if (warp < 8) {
+        if (!waited_prev) { pdl_wait(); waited_prev = true; }
+        if (a.add_residual) {
+            for (int b = 0; b < a.B; ++b) {
+                if (gPref[b + 1] != gPref[b]) continue;
+                const float4* src = reinterpret_cast<const float4*>(a.r_in + (size_t)b * T * H);
+                float* dst = a.r_out + (size_t)b * T * H;
+                for (size_t i = (size_t)blockIdx.x * 256 + tid; i < (size_t)T * H / 4; i += (size_t)gridDim.x * 256) {
+                    const float4 v = src[i];
+                    red_add_v4(dst + 4 * i, v.x, v.y, v.z, v.w);
+                }
+            }
+        }
+        if (a.zero_buf) {
+            const size_t n4 = (size_t)a.B * T * H / 4;
+            float4* z = reinterpret_cast<float4*>(a.zero_buf);
+            for (size_t i = (size_t)blockIdx.x * 256 + tid; i < n4; i += (size_t)gridDim.x * 256)
+                z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
+    cp_async_wait<0>();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) tmem_dealloc(tmem_d1, S::TMEM_COLS);
+}
+
+template <int NTOK, int HS>
+int launch_fused_ws(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cudaStream_t s) {
+    using S = SmemWS<NTOK, HS>;
+    auto kern = fused_layer_ws_kernel<NTOK, HS>;
+    const int smem = S::total_bytes(a.T);
+    static int configured = 0;
+    if (configured < smem) {
+        RM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        configured = smem;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_clusters * CS);
+    cfg.blockDim = dim3(WT);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = CS;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 2 : 1;
+    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, a));
+    ctx->launches++;
+    return RM_OK;
+}
+
 template <int NTOK, int HS, bool PIPE>
 int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cudaStream_t s) {
     using S = Smem<NTOK, HS, PIPE>;
@@ -764,18 +1259,30 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
         if (want < 1) want = 1;
         if (want < nc) nc = (int)want;
     }
-    // Variant: the lean kernel (H = 1024 only: 112 KB, two CTAs per SM so that consecutive layers overlap) serves
-    // launches where a cluster gets a single tile; when clusters walk several tiles, the pipelined variant keeps two
-    // tiles in flight per cluster (double-buffered exchange state, one CTA per SM).
+    // Variant.  Launches in which a cluster gets a single tile run the lean kernel (H = 1024: 112 KB, two CTAs per
+    // SM so that consecutive layers overlap).  When clusters walk several tiles, the warp-specialised kernel runs the
+    // phases of consecutive tiles concurrently (one CTA per SM, so no more clusters than are co-resident).
     long long tiles = per_episode > 0 ? (long long)((per_episode + NT - 1) / NT) * la.B : 0;
-    const bool pipe = ctx->variant_override ? ctx->variant_override == 2 : (tiles == 0 || tiles > nc);
+    int variant = ctx->variant_override;
+    if (variant == 0) variant = (tiles == 0 || tiles > nc) ? 3 : 1;
     const bool small_t = la.T <= 32;
+    if (variant == 3) {
+        const int fits_t = ctx->g.H == 1024 ? SmemWS<64, 128>::total_bytes(la.T) : SmemWS<64, 256>::total_bytes(la.T);
+        if (fits_t > 232448) variant = 2;
+    }
+    if (variant == 3) {
+        if (nc > ctx->fused_clusters) nc = ctx->fused_clusters;
+        if (ctx->g.H == 1024)
+            return small_t ? launch_fused_ws<32, 128>(ctx, a, nc, pdl, s) : launch_fused_ws<64, 128>(ctx, a, nc, pdl, s);
+        return small_t ? launch_fused_ws<32, 256>(ctx, a, nc, pdl, s) : launch_fused_ws<64, 256>(ctx, a, nc, pdl, s);
+    }
+    const bool pipe = variant == 2;
     if (ctx->g.H == 1024) {
         if (pipe)
             return small_t ? launch_fused<32, 128, true>(ctx, a, nc, pdl, s) : launch_fused<64, 128, true>(ctx, a, nc, pdl, s);
         return small_t ? launch_fused<32, 128, false>(ctx, a, nc, pdl, s) : launch_fused<64, 128, false>(ctx, a, nc, pdl, s);
     }
-    // H = 2048: the pipelined variant when its buffers fit the 227 KB of an SM (they do up to T = 60), else serial
+    // H = 2048: the two-tile variant when its buffers fit the 227 KB of an SM (they do up to T = 60), else serial
     const bool fits = Smem<64, 256, true>::total_bytes(la.T) <= 232448;
     if (small_t)
         return pipe ? launch_fused<32, 256, true>(ctx, a, nc, pdl, s) : launch_fused<32, 256, false>(ctx, a, nc, pdl, s);

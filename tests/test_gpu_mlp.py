@@ -181,3 +181,41 @@ def test_step_host_variant_matches_device_variant(lib):
     assert_close(h_out.numpy(), r_out.cpu().numpy(), "host variant")
     assert_close(h_out.numpy(), oracle.step(model.Wg, model.Wu, model.Wd, r0, idx, cnt), "host variant vs oracle")
     model.close()
+
+
+@pytest.mark.parametrize("variant", [1, 2, 3])
+@pytest.mark.parametrize("H,I,T,B", [(1024, 2048, 51, 2), (1024, 1024, 32, 1), (2048, 1024, 51, 1)])
+def test_every_tensor_core_variant_and_the_portable_path_agree_with_the_oracle(lib, variant, H, I, T, B):
+    """The lean, two-tiles-in-flight and warp-specialised kernels (and the CUDA-core path) on the same step."""
+    import torch
+    L = 2
+    w = tiny(H=H, I=I, T=T, L=L, sigma=1.0 / np.sqrt(H), B=B, config=92)
+    model = Model(lib, w, B_max=B)
+    assert model.ctx.rm_get_info("fused_clusters") > 0
+    r0 = np.stack([wl.bf16_bits_to_f32(wl.step_input(w, 0, episode=b)) for b in range(B)])
+    # episode 0 gets long lists (several tiles per cluster), the last episode's first layer is empty
+    lists = [[np.flatnonzero(wl.uniform(wl.tensor_key(3, 92, l, 8, b), I) < (0.9 if b == 0 else 0.2)).astype(np.int32)
+              for l in range(L)] for b in range(B)]
+    lists[B - 1][0] = np.zeros(0, np.int32)
+    stride = I
+    idx, cnt = lists_to_padded([s for per_b in lists for s in per_b], stride)
+    outs = {}
+    for path, var in ((1, 0), (2, variant)):
+        model.ctx.rm_set_option("path", path)
+        model.ctx.rm_set_option("variant", var)
+        r_out = torch.empty(B, T, H, dtype=torch.float32, device="cuda")
+        model.ctx.rm_action_expert_step(model.packed, dev(r0), dev(idx), dev(cnt), stride, r_out, B=B, T=T)
+        rec = torch.zeros(B, L, I, dtype=torch.float32, device="cuda")
+        d_out = torch.empty(B, T, H, dtype=torch.float32, device="cuda")
+        model.ctx.rm_action_expert_step(model.packed, dev(r0), None, None, 0, d_out, records_out=rec, B=B, T=T)
+        outs[path] = (r_out.cpu().numpy(), d_out.cpu().numpy(), rec.cpu().numpy())
+    for b in range(B):
+        i_b, c_b = lists_to_padded(lists[b], stride)
+        want = oracle.step(model.Wg, model.Wu, model.Wd, r0[b], i_b, c_b)
+        want_d, want_rec = oracle.step(model.Wg, model.Wu, model.Wd, r0[b], return_records=True)
+        for path in (1, 2):
+            assert_close(outs[path][0][b], want, f"masked step, path {path} variant {variant}, episode {b}")
+            assert_close(outs[path][1][b], want_d, f"dense step, path {path} variant {variant}, episode {b}")
+            assert np.all(np.abs(outs[path][2][b] - want_rec) <= 1e-2 * np.abs(want_rec) + 2e-2)
+    assert model.ctx.rm_device_status() == 0
+    model.close()
