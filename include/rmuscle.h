@@ -173,6 +173,8 @@ int64_t rm_launch_count(const rm_ctx* ctx);
  *   "count_hint"          expected active neurons per layer and episode; lets a launch use only as many clusters
  *                         as that needs, so that the next layer's CTAs can become resident early (0 = unknown)
  *   "max_clusters"        cap on the clusters per launch (0 = none)
+ *   "l2_prefetch"         warp-specialised kernel: number of tiles ahead for which the weights are pulled into L2
+ *                         (0 = off, the default)
  *   "variant"             tcgen05 kernel variant: 0 = choose per launch, 1 = lean (one tile at a time, two CTAs per
  *                         SM at H = 1024), 2 = two tiles in flight per cluster, 3 = warp-specialised (the phases
  *                         of consecutive tiles run concurrently; for clusters that walk many tiles)              */

@@ -52,6 +52,7 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->count_hint = 0;
     c->max_clusters_override = 0;
     c->variant_override = 0;
+    c->l2_prefetch = 0;
     c->fused_clusters = 0;
     c->fused_blocks_per_sm = 0;
     if (prop.major == 10) rm_fused_init(c);                 // failure leaves the portable path in charge
@@ -281,6 +282,9 @@ int rm_set_option(rm_ctx* ctx, const char* name, int value) {
     } else if (n == "variant") {
         if (value < 0 || value > 3) return RM_ERR_INVALID_ARG;
         ctx->variant_override = value;
+    } else if (n == "l2_prefetch") {
+        if (value < 0 || value > 16) return RM_ERR_INVALID_ARG;
+        ctx->l2_prefetch = value;
     } else if (n == "max_clusters") {
         if (value < 0) return RM_ERR_INVALID_ARG;
         ctx->max_clusters_override = value;

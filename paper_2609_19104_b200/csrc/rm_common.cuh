@@ -38,6 +38,7 @@ struct rm_ctx {
     int npc_target;                        // neurons per cluster aimed for when spreading a layer
     int count_hint;                        // expected active neurons per layer and episode (0: unknown)
     int max_clusters_override;             // > 0: cap on clusters per launch
+    int l2_prefetch;                       // L2 prefetch distance (tiles) of the warp-specialised kernel
     int variant_override;                  // 0 auto, 1 lean kernel, 2 kernel with a dedicated staging buffer
 };
 

@@ -45,9 +45,16 @@ __device__ int g_wall_seq;
     do {                                                                                                    \
         if (threadIdx.x == 0 && blockIdx.x < 256) g_wall_stamps[((wall_seq & 63) * 256 + blockIdx.x) * 4 + (k)] = rm_globaltimer(); \
     } while (0)
+// warp-specialised kernel: globaltimer per (CTA < 16, tile < 16, event < 8), written by each role's first thread
+__device__ long long g_ws_stamps[16 * 16 * 16];
+#define RM_WS(tile, ev)                                                                                   \
+    do {                                                                                                  \
+        if (blockIdx.x < 16 && (tile) < 16) g_ws_stamps[(blockIdx.x * 16 + (tile)) * 16 + (ev)] = rm_globaltimer(); \
+    } while (0)
 #else
 #define RM_STAMP(k) do { } while (0)
 #define RM_WALL(k) do { } while (0)
+#define RM_WS(tile, ev) do { } while (0)
 #endif
 
 namespace {
@@ -74,6 +81,7 @@ struct FusedArgs {
     int add_residual;              // r_in is added into r_out (spread over all CTAs)
     int* status;
     int wall_seq;                  // launch sequence number (phase-timing builds only)
+    int l2_prefetch;               // tiles of L2 prefetch distance in the warp-specialised kernel (0: off)
 };
 
 // floats per row of the exchange buffer: T rounded up to 4 with an odd number of 16-byte chunks, so that the
@@ -651,13 +659,13 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
 //   warps 0-3  scatter : wait for the gate/up product of tile i, read it from tensor memory, send the partial sums
 //                        to their owners; at the end of an episode, add the down accumulator to the residual stream
 //   warps 4-7  owner   : wait for the 8 partial sums of tile i, GeLU-tanh(g)*u, record, h atom, all-gather
-//   warp  8    mma     : one thread issues gate/up(i) as soon as its rows have landed and down(i-1) as soon as h(i-1)
-//                        is complete in this CTA
-//   warps 9-10 loader  : one neuron per thread; cp.async gathers of the next tile as soon as a stage is free, also
-//                        across the dependency wait on the previous layer
+//   warp  8    mma     : one thread issues the gate/up products of tile i, one K half at a time as the rows land
+//   warps 9-10 loader  : cp.async gathers of the next tile's gate/up rows (warp 9) and down rows (warp 10) as soon
+//                        as the stage (half) they go to is free
+//   warp  11   mma     : one thread issues the down product of tile i as soon as h(i) is complete in this CTA
 // Exchange state (D1 in tensor memory, partial-sum buffer, h tiles, h atom, staging) is double-buffered by tile
 // parity.  An episode change drains the pipeline (CTA-wide barrier), prepares the new x slice and restarts.
-constexpr int WT = 352;            // threads per CTA of the warp-specialised kernel
+constexpr int WT = 384;            // threads per CTA of the warp-specialised kernel (12 warps)
 
 template <int NTOK, int HS>
 struct SmemWS {
@@ -674,9 +682,10 @@ struct SmemWS {
     static constexpr int OFF_HS = OFF_HT + 4 * HT_HALF;      // [2 buffers] h atom (1 KB hi, 1 KB lo)
     static constexpr int OFF_SS = OFF_HS + 2 * 2048;
     static constexpr int OFF_N = OFF_SS + CS * 64 * 4;
-    static constexpr int OFF_PREF = OFF_N + 4 * NT * 4;     // neuron ids of four consecutive tiles (the loader runs ahead)
+    static constexpr int OFF_PREF = OFF_N + 8 * NT * 4;     // neuron ids of eight consecutive tiles: the loader may run up
+                                                            // to six tiles ahead of the owner warps that read them
     static constexpr int OFF_BAR = ((OFF_PREF + (2 * MAXB + 1) * 4 + 7) / 8) * 8;
-    static constexpr int OFF_P = ((OFF_BAR + 160 + 15) / 16) * 16;  // [2][CS][16][p_row] (+ [2] staging), sized at launch
+    static constexpr int OFF_P = ((OFF_BAR + 224 + 15) / 16) * 16;  // [2][CS][16][p_row] (+ [2] staging), sized at launch
     static constexpr int TMEM_COLS = 256;                    // D1 x 2 (NTOK each) + D2 (HS/128 x NTOK) <= 256
     static int total_bytes(int T) { return OFF_P + (STAGED ? 4 : 2) * CS * 16 * p_row_for(T) * 4 + 1024; }
 };
@@ -699,9 +708,16 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
     auto bar_p = [&](int pb) { return bar0 + 16 + 8 * pb; };       // all partial sums for this owner have arrived
     auto bar_h = [&](int pb) { return bar0 + 32 + 8 * pb; };       // all h atoms have arrived
     auto d1_free = [&](int pb) { return bar0 + 48 + 8 * pb; };     // the scatter warps have read D1[pb]
-    const uint32_t bar_dn = bar0 + 64, bar_s = bar0 + 72, gu_full = bar0 + 80, dn_full = bar0 + 88;
-    const uint32_t s_tmem = bar0 + 96;
-    volatile uint32_t* g_tmem = reinterpret_cast<volatile uint32_t*>(gbase + S::OFF_BAR + 96);
+    const uint32_t bar_dn = bar0 + 64, bar_s = bar0 + 72;
+    // the down stage is filled and consumed in two halves too (tile neurons 0..31 and 32..63)
+    auto dnh_full = [&](int h) { return bar0 + 128 + 8 * h; };
+    auto dnh_free = [&](int h) { return bar0 + 144 + 8 * h; };
+    // the gate/up stage is filled and consumed in two halves of the K range, so that loading one half overlaps
+    // the products of the other
+    auto guh_full = [&](int h) { return bar0 + 88 + 8 * h; };      // the rows of one K half have landed
+    auto guh_free = [&](int h) { return bar0 + 104 + 8 * h; };     // the products over one K half are complete
+    const uint32_t s_tmem = bar0 + 120;
+    volatile uint32_t* g_tmem = reinterpret_cast<volatile uint32_t*>(gbase + S::OFF_BAR + 120);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int j = (int)cluster_ctarank();
@@ -715,8 +731,8 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
         }
         mbar_init(bar_dn, 1);
         mbar_init(bar_s, 1);
-        mbar_init(gu_full, 32);
-        mbar_init(dn_full, 32);
+        for (int h = 0; h < 2; ++h) { mbar_init(guh_full(h), 32); mbar_init(guh_free(h), 1); }
+        for (int h = 0; h < 2; ++h) { mbar_init(dnh_full(h), 32); mbar_init(dnh_free(h), 1); }
         fence_mbar_init();
         int acc = 0;
         const int cap = (int)(a.list_cap < (int64_t)a.I ? a.list_cap : (int64_t)a.I);
@@ -761,52 +777,84 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
         if (!mbar_wait(bar, parity)) rm_set_status(a.status, RM_ERR_TIMEOUT);
     };
 
-    // loaders: lane l owns tile neurons l and l + 32; `it` is the cluster-local tile sequence number.  Warp 9 gathers
-    // the gate and up rows, warp 10 the down rows, so neither waits for the other's stage.
-    auto tile_neuron = [&](const TileRef& r, int q, bool report) {
-        int n = -1;
-        if (q < r.nvalid) {
-            n = a.idx ? a.idx[(size_t)r.b * a.idx_stride + r.p0 + q] : r.p0 + q;
-            if (n < 0 || n >= a.I) { if (report) rm_set_status(a.status, RM_ERR_INDEX); n = -1; }
-        }
-        return n;
-    };
-    auto load_gu = [&](int g, int it) {
+    // loaders: one warp gathers the gate and up rows (warp 9), one the down rows (warp 10), so neither waits for the
+    // other's stage.  Lane l = (r, c): per instruction the warp covers 4 tile neurons x one 128-byte row segment
+    // (8 lanes x 16 bytes, coalesced); the 16 groups of 4 neurons are walked in turn.  `it` is the cluster-local
+    // tile sequence number.
+    const int lr = lane >> 3, lc = lane & 7;
+    // the 16 neuron ids this lane needs for a tile.  The raw loads are issued one tile ahead of their use (under a
+    // saturated memory system a dependent 4-byte read costs microseconds); range checks happen at use time.
+    auto fetch_ids = [&](int g, int (&nn)[16]) {
         const TileRef r = tile_ref(g);
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int q = lane + 32 * half;
-            const int n = tile_neuron(r, q, true);
-            gN[(it & 3) * NT + q] = n;
-            const __nv_bfloat16* src = a.packed + (size_t)(n < 0 ? 0 : n) * 3 * H + (size_t)j * 3 * HS;
-            const uint32_t d0 = sGU + q * 128;
+        for (int grp = 0; grp < 16; ++grp) {
+            const int q = grp * 4 + lr;
+            nn[grp] = a.idx ? (q < r.nvalid ? __ldg(a.idx + (size_t)r.b * a.idx_stride + r.p0 + q) : -1)
+                            : (q < r.nvalid ? r.p0 + q : -1);
+        }
+    };
+    auto check_ids = [&](int g, int (&nn)[16], bool report) {
+        const TileRef r = tile_ref(g);
+        bool bad = false;
 #pragma unroll
-            for (int kb = 0; kb < KB; ++kb)
+        for (int grp = 0; grp < 16; ++grp) {
+            const int q = grp * 4 + lr;
+            if (q < r.nvalid && (nn[grp] < 0 || nn[grp] >= a.I)) { bad = true; nn[grp] = -1; }
+        }
+        if (bad && report) rm_set_status(a.status, RM_ERR_INDEX);
+    };
+    // gate/up: the ids are checked and published before the stage is known to be free; the gathers go out after
+    auto publish_gu = [&](int g, int it, int (&nn)[16]) {
+        check_ids(g, nn, lc == 0);
+        if (lc == 0) {
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint32_t off = kb * 16384 + ((c ^ (q & 7)) << 4);
-                    cp_async16(d0 + off, src + kb * 64 + c * 8, n >= 0);                      // gate row
-                    cp_async16(d0 + off + 64 * 128, src + HS + kb * 64 + c * 8, n >= 0);      // up row
-                }
+            for (int grp = 0; grp < 16; ++grp) gN[(it & 7) * NT + grp * 4 + lr] = nn[grp];
         }
         __threadfence_block();             // the neuron ids are read by the owner warps much later
-        cp_async_arrive_noinc(gu_full);
     };
-    auto load_dn = [&](int g) {
+    constexpr int KH = KB / 2;                             // 64-column blocks per K half (1 at H = 1024, 2 at H = 2048)
+    auto issue_gu_half = [&](int it, int h, const int (&nn)[16]) {
+        if (lane == 0 && h == 0) RM_WS(it, 0);
+#pragma unroll
+        for (int grp = 0; grp < 16; ++grp) {
+            const int q = grp * 4 + lr, n = nn[grp];
+            const __nv_bfloat16* src = a.packed + (size_t)(n < 0 ? 0 : n) * 3 * H + (size_t)j * 3 * HS + lc * 8;
+            const uint32_t d0 = sGU + q * 128 + ((lc ^ (q & 7)) << 4);
+#pragma unroll
+            for (int kk = 0; kk < KH; ++kk) {
+                const int kb = h * KH + kk;
+                cp_async16(d0 + kb * 16384, src + kb * 64, n >= 0);                       // gate row
+                cp_async16(d0 + kb * 16384 + 64 * 128, src + HS + kb * 64, n >= 0);       // up row
+            }
+        }
+        cp_async_arrive_noinc(guh_full(h));
+    };
+    // L2 prefetch of this CTA's pieces (3*Hs*2 contiguous bytes per neuron) of a tile that is still several tiles
+    // away: the later gathers into shared memory then find their lines in the 126 MB L2, so the amount of weight data
+    // in flight from HBM is no longer bounded by the shared-memory stages.  Two neurons per lane.
+    auto prefetch_tile = [&](int g) {
         const TileRef r = tile_ref(g);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             const int q = lane + 32 * half;
-            const int n = tile_neuron(r, q, false);
-            const __nv_bfloat16* src = a.packed + (size_t)(n < 0 ? 0 : n) * 3 * H + (size_t)j * 3 * HS + 2 * HS;
-            const uint32_t d0 = sDN + q * 128;
-#pragma unroll
-            for (int cb = 0; cb < KB; ++cb)
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    cp_async16(d0 + cb * 8192 + ((c ^ (q & 7)) << 4), src + cb * 64 + c * 8, n >= 0);
+            if (q < r.nvalid) {
+                const int n = a.idx ? __ldg(a.idx + (size_t)r.b * a.idx_stride + r.p0 + q) : r.p0 + q;
+                if (n >= 0 && n < a.I) prefetch_l2(a.packed + (size_t)n * 3 * H + (size_t)j * 3 * HS, 3 * HS * 2);
+            }
         }
-        cp_async_arrive_noinc(dn_full);
+    };
+    const int PD = a.l2_prefetch;                          // prefetch distance in tiles
+    auto issue_dn_half = [&](int h, const int (&nn)[16]) {
+#pragma unroll
+        for (int g8 = 0; g8 < 8; ++g8) {
+            const int grp = h * 8 + g8;
+            const int q = grp * 4 + lr, n = nn[grp];
+            const __nv_bfloat16* src = a.packed + (size_t)(n < 0 ? 0 : n) * 3 * H + (size_t)j * 3 * HS + 2 * HS + lc * 8;
+            const uint32_t d0 = sDN + q * 128 + ((lc ^ (q & 7)) << 4);
+#pragma unroll
+            for (int cb = 0; cb < KB; ++cb) cp_async16(d0 + cb * 8192, src + cb * 64, n >= 0);
+        }
+        cp_async_arrive_noinc(dnh_full(h));
     };
 
     __syncthreads();                       // gPref / gCnt
@@ -827,9 +875,17 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
         int seg = 1;
         while (it0 + seg < n_tiles && tile_ref(g_lo + it0 + seg).b == b) ++seg;
 
-        if (warp >= 9) {
+        if (warp == 9 || warp == 10) {
             // loader warps: the segment's first tile goes out before anything else (stages are free after a drain)
-            if (warp == 9) load_gu(g_lo + it0, it0); else load_dn(g_lo + it0);
+            int nn[16];
+            fetch_ids(g_lo + it0, nn);
+            if (warp == 9) { publish_gu(g_lo + it0, it0, nn); issue_gu_half(it0, 0, nn); issue_gu_half(it0, 1, nn); }
+            else {
+                check_ids(g_lo + it0, nn, false);
+                issue_dn_half(0, nn);
+                issue_dn_half(1, nn);
+                for (int d = 1; d <= PD && d < seg; ++d) prefetch_tile(g_lo + it0 + d);
+            }
         } else if (warp < 8) {
             // scatter and owner warps: x slice of episode b (256-thread mapping)
             if (!waited_prev) { pdl_wait(); waited_prev = true; }
@@ -905,6 +961,11 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 const int it = it0 + k, pb = it & 1;
                 wait_bar(bar_gu(pb), (it >> 1) & 1);
                 tc_fence_after();
+                if (tid == 0) RM_WS(it, 2);
+                // down(it-2) has finished reading the h tiles of this parity, and (through the chain h(it-2) <- every
+                // owner's reduction) the owners are done with the exchange buffer of this parity: only now may this
+                // tile's partial sums go out, because they let the owners refill both
+                if (k >= 2) wait_bar(bar_dn, (it - 2) & 1);
                 const uint32_t d1 = tmem_d1 + pb * NTOK;
                 const bool last_of_all = it == n_tiles - 1;
                 const bool stage_in_gu = !S::STAGED && last_of_all && p_bytes <= S::GU_STAGE;
@@ -945,10 +1006,11 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                     __syncwarp();
                     if (lane == 0) mbar_arrive(d1_free(pb));
                 }
-                // follow every phase of the down barrier (a parity wait can only tell the current phase from the
-                // previous one); down(it-1) is issued right after gate/up(it), so this does not hold the warps back
-                if (k >= 1) wait_bar(bar_dn, (it - 1) & 1);
+                if (tid == 0) RM_WS(it, 3);
             }
+            // follow the remaining phases of the down barrier in order (a parity wait can only tell the current phase
+            // from the previous one)
+            if (seg >= 2) wait_bar(bar_dn, (it0 + seg - 2) & 1);
             // end of the episode's run: add this CTA's [T x Hs] partial of y to the residual stream
             {
                 const int it = it0 + seg - 1;
@@ -968,56 +1030,71 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 tc_fence_before();
             }
         } else if (warp < 8) {
-            // ================= owner warps: warp ow handles local neurons ow and ow + 4
+            // ================= owner warps: warp ow handles local neurons ow and ow + 4, one per half-warp; a lane
+            // owns TPL consecutive tokens of its neuron
             const int ow = warp - 4, ot = tid - 128;
-            constexpr int TPL = NTOK / 32;
-            const int t0 = lane * TPL;
+            constexpr int TPL = NTOK / 16;                 // 4 tokens per lane at NTOK = 64, 2 at NTOK = 32
+            const int ql = ow + 4 * (lane >> 4);
+            const int t0 = (lane & 15) * TPL;
             for (int k = 0; k < seg; ++k) {
                 const int it = it0 + k, pb = it & 1;
                 if (ot == 0) mbar_arrive_expect_tx(bar_p(pb), p_bytes);
                 wait_bar(bar_p(pb), (it >> 1) & 1);
+                if (ot == 0) RM_WS(it, 4);
                 const float* gP = reinterpret_cast<const float*>(gbase + S::OFF_P + pb * p_bytes);
                 unsigned char* gHS = gbase + S::OFF_HS + pb * 2048;
+                float gsum[TPL], usum[TPL];
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const int ql = ow + 4 * half;
-                    float gsum[TPL], usum[TPL];
+                for (int e = 0; e < TPL; ++e) gsum[e] = usum[e] = 0.f;
+                if (t0 < PR) {
 #pragma unroll
-                    for (int e = 0; e < TPL; ++e) gsum[e] = usum[e] = 0.f;
-                    if (t0 < PR) {
-#pragma unroll
-                        for (int src = 0; src < CS; ++src) {
-                            const float* pg = gP + (src * 16 + ql) * PR + t0;
-                            const float* pu = gP + (src * 16 + 8 + ql) * PR + t0;
-#pragma unroll
-                            for (int e = 0; e < TPL; ++e) { gsum[e] += pg[e]; usum[e] += pu[e]; }
+                    for (int src = 0; src < CS; ++src) {
+                        const float* pg = gP + (src * 16 + ql) * PR + t0;
+                        const float* pu = gP + (src * 16 + 8 + ql) * PR + t0;
+                        if (TPL == 4) {
+                            const float4 g4 = *reinterpret_cast<const float4*>(pg), u4 = *reinterpret_cast<const float4*>(pu);
+                            gsum[0] += g4.x; gsum[1] += g4.y; gsum[2] += g4.z; gsum[TPL - 1] += g4.w;
+                            usum[0] += u4.x; usum[1] += u4.y; usum[2] += u4.z; usum[TPL - 1] += u4.w;
+                        } else {
+                            const float2 g2 = *reinterpret_cast<const float2*>(pg), u2 = *reinterpret_cast<const float2*>(pu);
+                            gsum[0] += g2.x; gsum[TPL - 1] += g2.y;
+                            usum[0] += u2.x; usum[TPL - 1] += u2.y;
                         }
                     }
-                    float rec = 0.f;
-                    float hv[TPL];
+                }
+                float rec = 0.f;
+                float hv[TPL];
 #pragma unroll
-                    for (int e = 0; e < TPL; ++e) {
-                        hv[e] = (t0 + e < T) ? rm_gelu_tanh(gsum[e]) * usum[e] : 0.f;
-                        rec += fabsf(hv[e]);
-                    }
-                    unsigned char* rowp = gHS + ql * 128 + ((((t0 >> 3) ^ ql) & 7) << 4) + (t0 & 7) * 2;
-                    if (TPL == 2) {
-                        const __nv_bfloat162 hi = __floats2bfloat162_rn(hv[0], hv[TPL - 1]);
-                        const float2 hf = __bfloat1622float2(hi);
-                        *reinterpret_cast<__nv_bfloat162*>(rowp) = hi;
-                        *reinterpret_cast<__nv_bfloat162*>(rowp + 1024) = __floats2bfloat162_rn(hv[0] - hf.x, hv[TPL - 1] - hf.y);
+                for (int e = 0; e < TPL; ++e) {
+                    hv[e] = (t0 + e < T) ? rm_gelu_tanh(gsum[e]) * usum[e] : 0.f;
+                    rec += fabsf(hv[e]);
+                }
+                // TPL consecutive tokens of one neuron row: one 8-byte (or 4-byte) store each for hi and lo
+                unsigned char* rowp = gHS + ql * 128 + ((((t0 >> 3) ^ ql) & 7) << 4) + (t0 & 7) * 2;
+                {
+                    const __nv_bfloat162 hi0 = __floats2bfloat162_rn(hv[0], hv[1]);
+                    const float2 f0 = __bfloat1622float2(hi0);
+                    const __nv_bfloat162 lo0 = __floats2bfloat162_rn(hv[0] - f0.x, hv[1] - f0.y);
+                    if (TPL == 4) {
+                        const __nv_bfloat162 hi1 = __floats2bfloat162_rn(hv[2], hv[TPL - 1]);
+                        const float2 f1 = __bfloat1622float2(hi1);
+                        const __nv_bfloat162 lo1 = __floats2bfloat162_rn(hv[2] - f1.x, hv[TPL - 1] - f1.y);
+                        uint2 hw, lw;
+                        hw.x = *reinterpret_cast<const uint32_t*>(&hi0); hw.y = *reinterpret_cast<const uint32_t*>(&hi1);
+                        lw.x = *reinterpret_cast<const uint32_t*>(&lo0); lw.y = *reinterpret_cast<const uint32_t*>(&lo1);
+                        *reinterpret_cast<uint2*>(rowp) = hw;
+                        *reinterpret_cast<uint2*>(rowp + 1024) = lw;
                     } else {
-                        const __nv_bfloat16 hi = __float2bfloat16_rn(hv[0]);
-                        *reinterpret_cast<__nv_bfloat16*>(rowp) = hi;
-                        *reinterpret_cast<__nv_bfloat16*>(rowp + 1024) = __float2bfloat16_rn(hv[0] - __bfloat162float(hi));
+                        *reinterpret_cast<__nv_bfloat162*>(rowp) = hi0;
+                        *reinterpret_cast<__nv_bfloat162*>(rowp + 1024) = lo0;
                     }
-                    if (a.record) {
+                }
+                if (a.record) {
 #pragma unroll
-                        for (int d = 16; d > 0; d >>= 1) rec += __shfl_xor_sync(0xffffffffu, rec, d);
-                        const int n = gN[(it & 3) * NT + j * 8 + ql];
-                        if (lane == 0 && n >= 0)
-                            a.record[(size_t)b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
-                    }
+                    for (int d = 8; d > 0; d >>= 1) rec += __shfl_xor_sync(0xffffffffu, rec, d);
+                    const int n = gN[(it & 7) * NT + j * 8 + ql];
+                    if ((lane & 15) == 0 && n >= 0)
+                        a.record[(size_t)b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
                 }
                 fence_proxy_async();
                 named_barrier(1, 128);
@@ -1026,56 +1103,91 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                     bulk_copy_to_peer(map_to_rank(sHT + pb * 2 * S::HT_HALF + part * S::HT_HALF + j * 1024, dst),
                                       smem_u32(gHS) + part * 1024, 1024, map_to_rank(bar_h(pb), dst));
                 }
+                if (ot == 0) RM_WS(it, 5);
             }
         } else if (warp == 8) {
-            // ================= mma warp (one thread)
+            // ================= gate/up issuer (one thread)
             if (lane == 0) {
-                auto do_dn = [&](int it) {
-                    const int pb = it & 1;
-                    wait_bar(bar_h(pb), (it >> 1) & 1);
-                    wait_bar(dn_full, it & 1);
-                    fence_proxy_async();
-                    tc_fence_after();
-                    const uint32_t ht = sHT + pb * 2 * S::HT_HALF;
-                    const bool first = it == it0;
+                for (int k = 0; k < seg; ++k) {
+                    const int it = it0 + k, pb = it & 1;
+                    if (it >= 2) wait_bar(d1_free(pb), ((it - 2) >> 1) & 1);      // the scatter warps have read D1[pb]
 #pragma unroll
-                    for (int mm = 0; mm < HS / 128; ++mm)
+                    for (int h = 0; h < 2; ++h) {
+                        wait_bar(guh_full(h), it & 1);
+                        if (h == 0) RM_WS(it, 1);
+                        fence_proxy_async();
+                        tc_fence_after();
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks) {
-                            const uint64_t aa = desc_mn | desc_addr(sDN + mm * 16384 + ks * 2048);
-                            mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + ks * 2048), IDESC_DN, !(first && ks == 0));
-                            mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + S::HT_HALF + ks * 2048), IDESC_DN, true);
-                        }
-                    mma_commit(bar_dn);
-                };
+                        for (int kk = 0; kk < KH; ++kk)
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks) {
+                                const int kb = h * KH + kk;
+                                mma_bf16_ss(tmem_d1 + pb * NTOK, desc_k | desc_addr(sGU + kb * 16384 + ks * 32),
+                                            desc_k | desc_addr(sX + kb * (NTOK * 128) + ks * 32), IDESC_GU, (kb | ks) != 0);
+                            }
+                        mma_commit(guh_free(h));
+                    }
+                    mma_commit(bar_gu(pb));
+                }
+            }
+        } else if (warp == 11) {
+            // ================= down issuer (one thread)
+            if (lane == 0) {
                 for (int k = 0; k < seg; ++k) {
                     const int it = it0 + k, pb = it & 1;
                     mbar_arrive_expect_tx(bar_h(pb), CS * 2048);
-                    wait_bar(gu_full, it & 1);
-                    if (it >= 2) wait_bar(d1_free(pb), ((it - 2) >> 1) & 1);
-                    fence_proxy_async();
-                    tc_fence_after();
+                    wait_bar(bar_h(pb), (it >> 1) & 1);
+                    RM_WS(it, 6);
+                    const uint32_t ht = sHT + pb * 2 * S::HT_HALF;
 #pragma unroll
-                    for (int kb = 0; kb < KB; ++kb)
+                    for (int h = 0; h < 2; ++h) {
+                        wait_bar(dnh_full(h), it & 1);
+                        RM_WS(it, 8 + 2 * h);
+                        fence_proxy_async();
+                        tc_fence_after();
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            mma_bf16_ss(tmem_d1 + pb * NTOK, desc_k | desc_addr(sGU + kb * 16384 + ks * 32),
-                                        desc_k | desc_addr(sX + kb * (NTOK * 128) + ks * 32), IDESC_GU, (kb | ks) != 0);
-                    mma_commit(bar_gu(pb));
-                    if (k >= 1) do_dn(it - 1);
+                        for (int mm = 0; mm < HS / 128; ++mm)
+#pragma unroll
+                            for (int k2 = 0; k2 < 2; ++k2) {
+                                const int ks = h * 2 + k2;
+                                const uint64_t aa = desc_mn | desc_addr(sDN + mm * 16384 + ks * 2048);
+                                mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + ks * 2048), IDESC_DN, !(k == 0 && ks == 0));
+                                mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + S::HT_HALF + ks * 2048), IDESC_DN, true);
+                            }
+                        mma_commit(dnh_free(h));
+                        if (h == 0) RM_WS(it, 9);
+                    }
+                    mma_commit(bar_dn);
+                    RM_WS(it, 7);
                 }
-                do_dn(it0 + seg - 1);
             }
         } else {
             // ================= loader warps: tiles after the segment's first
+            int nxt[16];
+            if (seg > 1) fetch_ids(g_lo + it0 + 1, nxt);
             for (int k = 1; k < seg; ++k) {
                 const int it = it0 + k;
+                int nn[16];
+#pragma unroll
+                for (int grp = 0; grp < 16; ++grp) nn[grp] = nxt[grp];
+                if (k + 1 < seg) fetch_ids(g_lo + it + 1, nxt);              // in flight while this tile is handled
                 if (warp == 9) {
-                    wait_bar(bar_gu((it - 1) & 1), ((it - 1) >> 1) & 1);     // gate/up stage is free
-                    load_gu(g_lo + it, it);
+                    publish_gu(g_lo + it, it, nn);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        wait_bar(guh_free(h), (it - 1) & 1);                  // the previous tile is done with this half
+                        issue_gu_half(it, h, nn);
+                    }
                 } else {
-                    wait_bar(bar_dn, (it - 1) & 1);                           // down stage is free
-                    load_dn(g_lo + it);
+                    if (k + PD < seg) prefetch_tile(g_lo + it + PD);
+                    check_ids(g_lo + it, nn, false);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        wait_bar(dnh_free(h), (it - 1) & 1);                  // the previous tile is done with this half
+                        if (lane == 0) RM_WS(it, 11 + 2 * h);
+                        issue_dn_half(h, nn);
+                        if (lane == 0 && h == 0) RM_WS(it, 12);
+                    }
                 }
             }
         }
@@ -1193,6 +1305,8 @@ int max_clusters(int T, int* out) {
 
 int rm_fused_debug_stamps(long long* host_out, int n) {
 #ifdef RM_PHASE_TIMING
+    if (n == -(16 * 16 * 16))
+        return cudaMemcpyFromSymbol(host_out, g_ws_stamps, sizeof(long long) * 16 * 16 * 16) == cudaSuccess ? RM_OK : RM_ERR_CUDA;
     if (n < 0) {                           // negative n: the wall-clock stamps, -n values
         n = -n;
         if (n > 64 * 256 * 4) n = 64 * 256 * 4;
@@ -1249,6 +1363,7 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
     a.add_residual = add_residual ? 1 : 0;
     a.status = ctx->d_status;
     a.wall_seq = (int)(ctx->launches & 63);
+    a.l2_prefetch = ctx->l2_prefetch;
     // Clusters per launch: one per tile of 64 neurons when the number of active neurons is known on the host
     // (dense calls, or a caller-supplied hint), else twice the co-resident number; never more than the cap.
     const int cap = ctx->max_clusters_override > 0 ? ctx->max_clusters_override : 2 * ctx->fused_clusters;

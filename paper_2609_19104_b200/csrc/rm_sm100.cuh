@@ -86,6 +86,10 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool v
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// ask the copy engine to bring `bytes` (multiple of 16, 16-byte aligned) of global memory into L2
+__device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
 // arrive on an mbarrier (of this CTA) once all cp.async operations this thread has issued so far have landed; the
 // arrival is one of the barrier's expected count (no increment)
 __device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
@@ -100,6 +104,8 @@ __device__ __forceinline__ void named_barrier(int id, int count) {
 }
 // make generic-proxy writes to shared memory visible to the async proxy (tcgen05.mma reads operands through it)
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// the same for this CTA's shared memory only (cheaper; enough when the reader is this CTA's own copy engine or MMA)
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
