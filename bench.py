@@ -247,6 +247,11 @@ def run_gpu(args, w: wl.Workload):
         dist.barrier()
     torch.cuda.synchronize()
     launches = ctx.launch_count() - launches0
+    status = ctx.rm_device_status()
+    if status != 0:
+        log = [ctx.rm_get_info(f"status_log:{i}") for i in range(ctx.rm_get_info("status_log_count"))]
+        raise RuntimeError(f"device status {status} ({rm.status_string(status)}) after the timed steps; waits that gave "
+                           f"up (source line, CTA): {[(d >> 12, d & 0xfff) for d in log]}: the timing is void")
     step_ms = [a.elapsed_time(b) for a, b in events]
     total_ms = float(sum(step_ms))
 

@@ -181,7 +181,12 @@ int64_t rm_launch_count(const rm_ctx* ctx);
 int rm_set_option(rm_ctx* ctx, const char* name, int value);
 
 /* Read-only facts: "fused_clusters" (co-resident clusters of the tcgen05 kernel, 0 when that path is
- * unavailable for this geometry or device), "sm_count", "path". */
+ * unavailable for this geometry or device), "fused_blocks_per_sm", "sm_count", "path", and "status_detail": for
+ * the last non-zero status that rm_device_status returned, where the kernel gave up (a bounded wait that ran out:
+ * source line of the wait << 12 | CTA index & 0xfff); 0 when that status carried no detail.
+ * "last_cuda_error" (ctx may be NULL) is the cudaError_t of the last runtime call that made an entry point return
+ * RM_ERR_CUDA.  "status_log_count" and "status_log:<i>" give the detail words of up to 60 errors of that launch in the order in
+ * which they were recorded. */
 int rm_get_info(const rm_ctx* ctx, const char* name, int* out);
 
 /* Profiling aid, available only in builds made with -DRM_PHASE_TIMING (RM_ERR_UNSUPPORTED otherwise): copies the

@@ -29,7 +29,12 @@ EXPORTS = ["rm_create", "rm_destroy", "rm_packed_layer_bytes", "rm_workspace_byt
 class RmError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
-        super().__init__(f"{where}: {status_string(code)} ({code})")
+        extra = ""
+        if code == -5 and _lib is not None:                # RM_ERR_CUDA: add the runtime's own error code
+            v = ctypes.c_int(0)
+            if _lib.rm_get_info(None, b"last_cuda_error", ctypes.byref(v)) == 0:
+                extra = f" [cudaError_t {v.value}]"
+        super().__init__(f"{where}: {status_string(code)} ({code}){extra}")
 
 
 class rm_model_desc(ctypes.Structure):

@@ -1,8 +1,12 @@
 // C-ABI entry points: argument validation and dispatch.  Every step of the path runs in the library's kernels.
 #include <new>
+#include <cstring>
+#include <cstdlib>
 #include <string>
 
 #include "rm_common.cuh"
+
+int rm_last_cuda_error = 0;
 
 namespace {
 
@@ -37,6 +41,7 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->g.I = desc->I;
     c->g.Hs = desc->H / RM_NS;
     c->launches = 0;
+    c->status_detail = 0;
     c->d_status = nullptr;
     cudaDeviceProp prop;
     if (cudaGetDevice(&c->device) != cudaSuccess || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess ||
@@ -255,11 +260,13 @@ int rm_action_expert_step_host(rm_ctx* ctx, const void* const* packed_layers, co
 int rm_device_status(rm_ctx* ctx, int* host_out, rm_stream_t stream) {
     if (!ctx || !host_out) return RM_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int v = 0;
-    RM_CUDA_TRY(cudaMemcpyAsync(&v, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, s));
-    RM_CUDA_TRY(cudaMemsetAsync(ctx->d_status, 0, sizeof(int), s));
+    int v[64] = {0};
+    RM_CUDA_TRY(cudaMemcpyAsync(v, ctx->d_status, sizeof(v), cudaMemcpyDeviceToHost, s));
+    RM_CUDA_TRY(cudaMemsetAsync(ctx->d_status, 0, sizeof(v), s));
     RM_CUDA_TRY(cudaStreamSynchronize(s));
-    *host_out = v;
+    *host_out = v[0];
+    ctx->status_detail = v[0] ? v[1] : 0;
+    std::memcpy(ctx->status_log, v, sizeof(v));
     return RM_OK;
 }
 
@@ -295,12 +302,21 @@ int rm_set_option(rm_ctx* ctx, const char* name, int value) {
 }
 
 int rm_get_info(const rm_ctx* ctx, const char* name, int* out) {
-    if (!ctx || !name || !out) return RM_ERR_INVALID_ARG;
+    if (!name || !out) return RM_ERR_INVALID_ARG;
     const std::string n(name);
+    if (n == "last_cuda_error") { *out = rm_last_cuda_error; return RM_OK; }   // process-wide: needs no context
+    if (!ctx) return RM_ERR_INVALID_ARG;
     if (n == "fused_clusters") *out = ctx->fused_clusters;
     else if (n == "fused_blocks_per_sm") *out = ctx->fused_blocks_per_sm;
     else if (n == "sm_count") *out = ctx->sm_count;
     else if (n == "path") *out = ctx->path;
+    else if (n == "status_detail") *out = ctx->status_detail;
+    else if (n == "status_log_count") *out = ctx->status_log[2] < RM_STATUS_LOG ? ctx->status_log[2] : RM_STATUS_LOG;
+    else if (n.rfind("status_log:", 0) == 0) {
+        const int i = std::atoi(n.c_str() + 11);
+        if (i < 0 || i >= RM_STATUS_LOG) return RM_ERR_INVALID_ARG;
+        *out = ctx->status_log[4 + i];
+    }
     else return RM_ERR_INVALID_ARG;
     return RM_OK;
 }

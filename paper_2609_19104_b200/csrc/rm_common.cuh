@@ -28,7 +28,9 @@ struct rm_ctx {
     rm_geom g;
     int device;
     int sm_count;
-    int* d_status;                         // device status word
+    int* d_status;                         // device status word, then the detail word of the first error
+    int status_detail;                     // detail word seen by the last rm_device_status call
+    int status_log[64];                    // the whole status block of that call
     int64_t launches;                      // host-side launch counter
     // tensor-core path (rm_mlp_sm100.cu)
     int fused_clusters;                    // co-resident 8-CTA clusters of the fused layer kernel (0: unavailable)
@@ -42,16 +44,25 @@ struct rm_ctx {
     int variant_override;                  // 0 auto, 1 lean kernel, 2 kernel with a dedicated staging buffer
 };
 
+extern int rm_last_cuda_error;            // cudaError_t of the last failed runtime call (diagnostics; "last_cuda_error")
 #define RM_CUDA_TRY(expr)                                  \
     do {                                                   \
         cudaError_t _e = (expr);                           \
-        if (_e != cudaSuccess) return RM_ERR_CUDA;         \
+        if (_e != cudaSuccess) { rm_last_cuda_error = (int)_e; return RM_ERR_CUDA; } \
     } while (0)
 
 static inline bool rm_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 __device__ __forceinline__ void rm_set_status(int* status, int code) {
     if (status) atomicCAS(status, 0, code);
+}
+constexpr int RM_STATUS_LOG = 60;        // detail words kept per status read (the status block is 64 ints)
+// The first error of a launch also leaves a detail word (where a wait gave up) next to the status word.
+__device__ __forceinline__ void rm_set_status_at(int* status, int code, int detail) {
+    if (!status) return;
+    if (atomicCAS(status, 0, code) == 0) status[1] = detail;
+    const int slot = atomicAdd(status + 2, 1);             // every error of the launch, in arrival order, while room
+    if (slot < RM_STATUS_LOG) status[4 + slot] = detail;
 }
 
 __device__ __forceinline__ float rm_gelu_tanh(float g) {

@@ -88,6 +88,9 @@ struct FusedArgs {
 // eight rows written by one warp-store fall into distinct bank groups
 __host__ __device__ constexpr int p_row_for(int T) { return 4 * (((T + 3) / 4) | 1); }
 
+// A wait that ran out of polls records the source line of the wait and the CTA (readable as "status_detail").
+#define wait_bar(bar, parity) wait_bar_at((bar), (parity), __LINE__)
+
 template <int NTOK, int HS, bool PIPE>
 struct Smem {
     static constexpr int KB = HS / 64;                       // 64-column (128-byte) blocks per slice
@@ -295,8 +298,8 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     // buffer and barrier phase of local tile i (every second tile reuses a buffer when two are in flight)
     auto buf_of = [&](int i) { return PIPE ? (i & 1) : 0; };
     auto phase_of = [&](int i) { return (uint32_t)(PIPE ? ((i >> 1) & 1) : (i & 1)); };
-    auto wait_bar = [&](uint32_t bar, uint32_t parity) {
-        if (!mbar_wait(bar, parity)) rm_set_status(a.status, RM_ERR_TIMEOUT);
+    auto wait_bar_at = [&](uint32_t bar, uint32_t parity, int line) {
+        if (!mbar_wait(bar, parity)) rm_set_status_at(a.status, RM_ERR_TIMEOUT, (line << 12) | (int)(blockIdx.x & 0xfffu));
     };
 
     // ---- phase: x slice of episode b -> bf16, 128-byte-swizzled K-major operand tile (cluster-collective)
@@ -708,7 +711,12 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
     auto bar_p = [&](int pb) { return bar0 + 16 + 8 * pb; };       // all partial sums for this owner have arrived
     auto bar_h = [&](int pb) { return bar0 + 32 + 8 * pb; };       // all h atoms have arrived
     auto d1_free = [&](int pb) { return bar0 + 48 + 8 * pb; };     // the scatter warps have read D1[pb]
-    const uint32_t bar_dn = bar0 + 64, bar_s = bar0 + 72;
+    // down product of a tile is complete.  One barrier per tile parity: a scatter warp waits for down(it - 2) only when
+    // it is about to send tile it, and by then down(it - 1) may be complete as well; on a single barrier that wait
+    // would then see the parity of the phase two ahead and never return.  With two, the next phase of the barrier it
+    // waits on (down(it)) cannot complete before the warp itself has sent tile it.
+    auto bar_dn = [&](int pb) { return bar0 + 64 + 16 * pb; };
+    const uint32_t bar_s = bar0 + 72;
     // the down stage is filled and consumed in two halves too (tile neurons 0..31 and 32..63)
     auto dnh_full = [&](int h) { return bar0 + 128 + 8 * h; };
     auto dnh_free = [&](int h) { return bar0 + 144 + 8 * h; };
@@ -729,7 +737,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
         for (int pb = 0; pb < 2; ++pb) {
             mbar_init(bar_gu(pb), 1); mbar_init(bar_p(pb), 1); mbar_init(bar_h(pb), 1); mbar_init(d1_free(pb), 4);
         }
-        mbar_init(bar_dn, 1);
+        mbar_init(bar_dn(0), 1); mbar_init(bar_dn(1), 1);
         mbar_init(bar_s, 1);
         for (int h = 0; h < 2; ++h) { mbar_init(guh_full(h), 32); mbar_init(guh_free(h), 1); }
         for (int h = 0; h < 2; ++h) { mbar_init(dnh_full(h), 32); mbar_init(dnh_free(h), 1); }
@@ -773,8 +781,8 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
         r.last = (g == g_hi - 1) || (g == gPref[b + 1] - 1);
         return r;
     };
-    auto wait_bar = [&](uint32_t bar, uint32_t parity) {
-        if (!mbar_wait(bar, parity)) rm_set_status(a.status, RM_ERR_TIMEOUT);
+    auto wait_bar_at = [&](uint32_t bar, uint32_t parity, int line) {
+        if (!mbar_wait(bar, parity)) rm_set_status_at(a.status, RM_ERR_TIMEOUT, (line << 12) | (int)(blockIdx.x & 0xfffu));
     };
 
     // loaders: one warp gathers the gate and up rows (warp 9), one the down rows (warp 10), so neither waits for the
@@ -965,7 +973,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 // down(it-2) has finished reading the h tiles of this parity, and (through the chain h(it-2) <- every
                 // owner's reduction) the owners are done with the exchange buffer of this parity: only now may this
                 // tile's partial sums go out, because they let the owners refill both
-                if (k >= 2) wait_bar(bar_dn, (it - 2) & 1);
+                if (k >= 2) wait_bar(bar_dn(pb), ((it - 2) >> 1) & 1);
                 const uint32_t d1 = tmem_d1 + pb * NTOK;
                 const bool last_of_all = it == n_tiles - 1;
                 const bool stage_in_gu = !S::STAGED && last_of_all && p_bytes <= S::GU_STAGE;
@@ -1010,11 +1018,11 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
             }
             // follow the remaining phases of the down barrier in order (a parity wait can only tell the current phase
             // from the previous one)
-            if (seg >= 2) wait_bar(bar_dn, (it0 + seg - 2) & 1);
+            if (seg >= 2) wait_bar(bar_dn((it0 + seg - 2) & 1), ((it0 + seg - 2) >> 1) & 1);
             // end of the episode's run: add this CTA's [T x Hs] partial of y to the residual stream
             {
                 const int it = it0 + seg - 1;
-                wait_bar(bar_dn, it & 1);
+                wait_bar(bar_dn(it & 1), (it >> 1) & 1);
                 tc_fence_after();
 #pragma unroll
                 for (int mm = 0; mm < HS / 128; ++mm) {
@@ -1157,7 +1165,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                         mma_commit(dnh_free(h));
                         if (h == 0) RM_WS(it, 9);
                     }
-                    mma_commit(bar_dn);
+                    mma_commit(bar_dn(pb));
                     RM_WS(it, 7);
                 }
             }

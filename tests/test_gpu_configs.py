@@ -244,4 +244,16 @@ def test_config2_large_refresh_every_two_steps(lib):
             got = gpu_sparse_step(model, r0[None], idx, cnt)[0]
             assert_close(got, oracle.step(model.Wg, model.Wu, model.Wd, r0, h_idx, h_cnt), f"config 2 sparse step {s}")
     assert model.ctx.rm_device_status() == 0
+    # The same sparse step behind a write larger than L2, as the benchmark runs it: with every weight row coming from
+    # HBM the loads, not the exchange chain, set the pace of a cluster, which is the order of events in which a
+    # pipeline hand-off that relies on timing would stall (a stall shows as a non-zero status and a slow step).
+    import torch
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    r0 = f32_of(wl.step_input(w, 1))
+    want = oracle.step(model.Wg, model.Wu, model.Wd, r0, h_idx, h_cnt)
+    for rep in range(6):
+        flush.fill_(rep)
+        got = gpu_sparse_step(model, r0[None], idx, cnt)[0]
+        assert model.ctx.rm_device_status() == 0, f"cold-cache repetition {rep}"
+        assert_close(got, want, f"config 2 cold-cache sparse step, repetition {rep}")
     model.close()
