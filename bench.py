@@ -174,6 +174,10 @@ def run_gpu(args, w: wl.Workload):
     B = w.B
     ctx = rm.Context(w.L, w.H, w.I, T_max=w.T, B_max=B)
     ctx.rm_set_option("count_hint", w.K)          # the lists hold K neurons: launch one cluster per 64-neuron tile
+    if args.variant:
+        ctx.rm_set_option("variant", args.variant)
+    if args.max_clusters:
+        ctx.rm_set_option("max_clusters", args.max_clusters)
     # weights: the workload's seeded draws (same on every rank: replicas of one model)
     packed = []
     gen = torch.Generator(device="cuda")
@@ -340,6 +344,9 @@ def main():
     ap.add_argument("--device-weights", action="store_true",
                     help="draw the weights on the device with a seeded torch generator instead of the host generator")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--variant", type=int, default=0,
+                    help="kernel variant override (library option \"variant\": 0 = chosen per launch)")
+    ap.add_argument("--max-clusters", type=int, default=0, help="library option \"max_clusters\" (0 = default)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = pick_workload(args.workload)

@@ -298,8 +298,12 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     // buffer and barrier phase of local tile i (every second tile reuses a buffer when two are in flight)
     auto buf_of = [&](int i) { return PIPE ? (i & 1) : 0; };
     auto phase_of = [&](int i) { return (uint32_t)(PIPE ? ((i >> 1) & 1) : (i & 1)); };
+    bool gave_up = false;
     auto wait_bar_at = [&](uint32_t bar, uint32_t parity, int line) {
-        if (!mbar_wait(bar, parity)) rm_set_status_at(a.status, RM_ERR_TIMEOUT, (line << 12) | (int)(blockIdx.x & 0xfffu));
+        if (!mbar_wait(bar, parity)) {
+            rm_set_status_at(a.status, RM_ERR_TIMEOUT, (line << 12) | (int)(blockIdx.x & 0xfffu));
+            gave_up = true;
+        }
     };
 
     // ---- phase: x slice of episode b -> bf16, 128-byte-swizzled K-major operand tile (cluster-collective)
@@ -376,9 +380,16 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     };
 
     // ---- phase: open local tile i (announce the bytes its two exchanges deliver here; new episode -> new x)
+    // Bytes of partial sums a tile delivers to each owner.  The bulk-copy route moves whole padded rows; the
+    // per-thread stores send only the columns that exist in tensor memory (the row pad can exceed the token tile).
+    const int p_cols = PR < NTOK ? PR : NTOK;
+    auto p_tx_bytes = [&](int i) {
+        const bool bulk = S::STAGED || (!(i + 1 < n_tiles) && p_bytes <= S::GU_STAGE);
+        return bulk ? p_bytes : CS * 16 * p_cols * 4;
+    };
     auto open_tile = [&](int i) {
         if (tid == 0) {
-            mbar_arrive_expect_tx(bar_p(buf_of(i)), p_bytes);
+            mbar_arrive_expect_tx(bar_p(buf_of(i)), p_tx_bytes(i));
             mbar_arrive_expect_tx(bar_h(buf_of(i)), CS * 2048);
         }
         const TileRef tr = tile_ref(g_lo + i);
@@ -649,7 +660,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     }
     cp_async_wait<0>();
     tc_fence_before();
-    __syncthreads();
+    if (__syncthreads_or(gave_up)) linger_after_timeout();
     if (warp == 0) tmem_dealloc(tmem_d1, S::TMEM_COLS);
     RM_STAMP(15);
     RM_WALL(3);
@@ -781,8 +792,12 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
         r.last = (g == g_hi - 1) || (g == gPref[b + 1] - 1);
         return r;
     };
+    bool gave_up = false;
     auto wait_bar_at = [&](uint32_t bar, uint32_t parity, int line) {
-        if (!mbar_wait(bar, parity)) rm_set_status_at(a.status, RM_ERR_TIMEOUT, (line << 12) | (int)(blockIdx.x & 0xfffu));
+        if (!mbar_wait(bar, parity)) {
+            rm_set_status_at(a.status, RM_ERR_TIMEOUT, (line << 12) | (int)(blockIdx.x & 0xfffu));
+            gave_up = true;
+        }
     };
 
     // loaders: one warp gathers the gate and up rows (warp 9), one the down rows (warp 10), so neither waits for the
@@ -1046,7 +1061,12 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
             const int t0 = (lane & 15) * TPL;
             for (int k = 0; k < seg; ++k) {
                 const int it = it0 + k, pb = it & 1;
-                if (ot == 0) mbar_arrive_expect_tx(bar_p(pb), p_bytes);
+                if (ot == 0) {
+                    // the bulk-copy route moves whole padded rows, the per-thread stores only the columns that exist
+                    // in tensor memory (the row pad can exceed the token tile)
+                    const bool bulk = S::STAGED || (it == n_tiles - 1 && p_bytes <= S::GU_STAGE);
+                    mbar_arrive_expect_tx(bar_p(pb), bulk ? p_bytes : CS * 16 * (PR < NTOK ? PR : NTOK) * 4);
+                }
                 wait_bar(bar_p(pb), (it >> 1) & 1);
                 if (ot == 0) RM_WS(it, 4);
                 const float* gP = reinterpret_cast<const float*>(gbase + S::OFF_P + pb * p_bytes);
@@ -1226,7 +1246,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
     }
     cp_async_wait<0>();
     tc_fence_before();
-    __syncthreads();
+    if (__syncthreads_or(gave_up)) linger_after_timeout();
     if (warp == 8) tmem_dealloc(tmem_d1, S::TMEM_COLS);
 }
 
@@ -1372,29 +1392,38 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
     a.status = ctx->d_status;
     a.wall_seq = (int)(ctx->launches & 63);
     a.l2_prefetch = ctx->l2_prefetch;
-    // Clusters per launch: one per tile of 64 neurons when the number of active neurons is known on the host
-    // (dense calls, or a caller-supplied hint), else twice the co-resident number; never more than the cap.
-    const int cap = ctx->max_clusters_override > 0 ? ctx->max_clusters_override : 2 * ctx->fused_clusters;
-    int nc = cap;
+    // Tiles of 64 neurons in this launch, when the host knows the number of active neurons (dense calls, or the
+    // caller's hint); 0 = unknown.
     const int per_episode = la.idx ? ctx->count_hint : ctx->g.I;
-    if (per_episode > 0) {
-        long long want = (long long)((per_episode + NT - 1) / NT) * la.B;
-        if (want < 1) want = 1;
-        if (want < nc) nc = (int)want;
-    }
-    // Variant.  Launches in which a cluster gets a single tile run the lean kernel (H = 1024: 112 KB, two CTAs per
-    // SM so that consecutive layers overlap).  When clusters walk several tiles, the warp-specialised kernel runs the
-    // phases of consecutive tiles concurrently (one CTA per SM, so no more clusters than are co-resident).
-    long long tiles = per_episode > 0 ? (long long)((per_episode + NT - 1) / NT) * la.B : 0;
+    const long long tiles = per_episode > 0 ? (long long)((per_episode + NT - 1) / NT) * la.B : 0;
+    // Variant.  H = 1024: the lean kernel for every launch (112 KB and 107 registers: two CTAs per SM, so a cluster's
+    // exchange waits are covered by its SM-mate and consecutive layers overlap); measured, 33 of its clusters are
+    // co-resident, two more than twice the number the occupancy query reports for one CTA per SM.  H = 2048 (one CTA
+    // per SM either way): the lean kernel while every cluster gets a single tile, else the warp-specialised kernel,
+    // which runs the phases of consecutive tiles concurrently.
+    // (an SM has 228 KB of shared memory, of which every resident CTA also takes 1 KB of system space)
+    const int lean_bytes = la.T <= 32 ? Smem<32, 128, false>::total_bytes(la.T) : Smem<64, 128, false>::total_bytes(la.T);
+    const bool two_per_sm = ctx->g.H == 1024 && 2 * (lean_bytes + 1024) <= 228 * 1024;
+    int cap = two_per_sm ? 2 * ctx->fused_clusters + 2 : ctx->fused_clusters;
+    if (ctx->max_clusters_override > 0) cap = ctx->max_clusters_override;
     int variant = ctx->variant_override;
-    if (variant == 0) variant = (tiles == 0 || tiles > nc) ? 3 : 1;
-    const bool small_t = la.T <= 32;
+    if (variant == 0) variant = (ctx->g.H == 1024 || (tiles > 0 && tiles <= cap)) ? 1 : 3;
     if (variant == 3) {
         const int fits_t = ctx->g.H == 1024 ? SmemWS<64, 128>::total_bytes(la.T) : SmemWS<64, 256>::total_bytes(la.T);
         if (fits_t > 232448) variant = 2;
+        else if (ctx->max_clusters_override <= 0 || cap > ctx->fused_clusters) cap = ctx->fused_clusters;
     }
+    if (variant == 2 && ctx->max_clusters_override <= 0) cap = ctx->fused_clusters;      // one CTA per SM
+    // Clusters: no more than the cap, and when the tile count is known, the fewest that keep the longest run of
+    // tiles per cluster as short as the cap allows (40 tiles under a cap of 32: 20 clusters of 2, not 32 of 1 or 2).
+    // (The warp-specialised kernel streams, and is faster with every co-resident cluster pulling on the memory.)
+    int nc = cap;
+    if (tiles > 0) {
+        const long long run = (tiles + cap - 1) / cap;
+        nc = variant == 3 ? (int)(tiles < cap ? tiles : cap) : (int)((tiles + run - 1) / run);
+    }
+    const bool small_t = la.T <= 32;
     if (variant == 3) {
-        if (nc > ctx->fused_clusters) nc = ctx->fused_clusters;
         if (ctx->g.H == 1024)
             return small_t ? launch_fused_ws<32, 128>(ctx, a, nc, pdl, s) : launch_fused_ws<64, 128>(ctx, a, nc, pdl, s);
         return small_t ? launch_fused_ws<32, 256>(ctx, a, nc, pdl, s) : launch_fused_ws<64, 256>(ctx, a, nc, pdl, s);

@@ -135,6 +135,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
     return false;
 }
 
+// After a wait has given up, peers may still be sending into this CTA's shared memory (messages it stopped waiting
+// for).  A CTA must not leave the cluster under them, so the error path idles for longer than a peer's own bounded
+// waits can last before it tears down.  Bounded; reached only with an error status already recorded.
+__device__ __forceinline__ void linger_after_timeout() {
+    for (uint32_t i = 0; i < (1u << 21); ++i) __nanosleep(256);
+}
+
 // ---------------------------------------------------------------- tensor memory
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_result, uint32_t ncols) {      // one full warp
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols) : "memory");

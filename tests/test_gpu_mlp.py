@@ -184,7 +184,8 @@ def test_step_host_variant_matches_device_variant(lib):
 
 
 @pytest.mark.parametrize("variant", [1, 2, 3])
-@pytest.mark.parametrize("H,I,T,B", [(1024, 2048, 51, 2), (1024, 1024, 32, 1), (2048, 1024, 51, 1)])
+@pytest.mark.parametrize("H,I,T,B", [(1024, 2048, 51, 2), (1024, 1024, 32, 1), (2048, 1024, 51, 1),
+                                     (2048, 1024, 32, 1), (1024, 1024, 64, 1), (2048, 1024, 64, 1)])
 def test_every_tensor_core_variant_and_the_portable_path_agree_with_the_oracle(lib, variant, H, I, T, B):
     """The lean, two-tiles-in-flight and warp-specialised kernels (and the CUDA-core path) on the same step."""
     import torch
@@ -199,10 +200,13 @@ def test_every_tensor_core_variant_and_the_portable_path_agree_with_the_oracle(l
     lists[B - 1][0] = np.zeros(0, np.int32)
     stride = I
     idx, cnt = lists_to_padded([s for per_b in lists for s in per_b], stride)
+    # every variant runs twice: with the default number of clusters (mostly one tile per cluster) and with three
+    # clusters, so that each cluster walks many tiles and every hand-off between consecutive tiles is exercised
     outs = {}
-    for path, var in ((1, 0), (2, variant)):
-        model.ctx.rm_set_option("path", path)
+    for path, var, max_clusters in ((1, 0, 0), (2, variant, 0), (3, variant, 3)):
+        model.ctx.rm_set_option("path", min(path, 2))
         model.ctx.rm_set_option("variant", var)
+        model.ctx.rm_set_option("max_clusters", max_clusters)
         r_out = torch.empty(B, T, H, dtype=torch.float32, device="cuda")
         model.ctx.rm_action_expert_step(model.packed, dev(r0), dev(idx), dev(cnt), stride, r_out, B=B, T=T)
         rec = torch.zeros(B, L, I, dtype=torch.float32, device="cuda")
@@ -213,7 +217,7 @@ def test_every_tensor_core_variant_and_the_portable_path_agree_with_the_oracle(l
         i_b, c_b = lists_to_padded(lists[b], stride)
         want = oracle.step(model.Wg, model.Wu, model.Wd, r0[b], i_b, c_b)
         want_d, want_rec = oracle.step(model.Wg, model.Wu, model.Wd, r0[b], return_records=True)
-        for path in (1, 2):
+        for path in (1, 2, 3):
             assert_close(outs[path][0][b], want, f"masked step, path {path} variant {variant}, episode {b}")
             assert_close(outs[path][1][b], want_d, f"dense step, path {path} variant {variant}, episode {b}")
             assert np.all(np.abs(outs[path][2][b] - want_rec) <= 1e-2 * np.abs(want_rec) + 2e-2)
