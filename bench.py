@@ -31,8 +31,8 @@ METRIC = "masked_mlp_us_per_denoise_step"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused layer launch, from the ncu capture summarised in
-# profiles/fused_layer_config1.md
-TRAFFIC_BYTES_PER_LAUNCH = {"pi0-stack-top25": 6.78e6}
+# profiles/fused_layer_kernel_config1.md
+TRAFFIC_BYTES_PER_LAUNCH = {"pi0-stack-top25": 6.797e6}
 
 
 def measured_hbm_peak():
@@ -319,7 +319,8 @@ def run_gpu(args, w: wl.Workload):
                        "multi_gpu": "replicas: each rank runs its own episodes, no collective on the data path"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name), "peak_kind": f"{peak_kind} copy bandwidth",
-                         "kernel": "fused_layer_kernel (one launch per layer, dependent-launch chained)",
+                         "kernel": ("fused_layer_kernel<64,128,false>" if w.H == 1024 else "fused_layer_ws_kernel<64,256>")
+                                   + " (one launch per layer, dependent-launch chained)",
                          "bytes_per_launch": bytes_layer, "us_per_launch": in_step_layer_us,
                          "us_per_launch_isolated_cold": layer_us, "launches_per_step": launches_per_step,
                          "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
