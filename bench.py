@@ -142,8 +142,7 @@ def time_oracle(w: wl.Workload, steps: int, warmup: int, sample_layers: int = 3)
 
 
 def run_reference(args, w: wl.Workload):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if rank_env()[1] != 0:                 # under a multi-rank launch rank 0 alone runs and prints
         return
     us, cores, sample = time_oracle(w, args.steps, args.warmup)
     line = {
@@ -158,15 +157,41 @@ def run_reference(args, w: wl.Workload):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------------------------------------ ranks
+# The path has no exchange step: N GPUs run N replicas of the model, each on its own episodes.  The only things the
+# ranks share are the barrier around the timed region and the maximum of their device times.
+def rank_env():
+    return (int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def episodes_of_rank(rank: int, B: int):
+    """Episode numbers (seeds of the synthetic inputs) rank `rank` works on: disjoint across ranks."""
+    return list(range(rank * B, (rank + 1) * B))
+
+
+def max_over_ranks(values, world: int, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank defines the job's time)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def job_us_per_step(total_ms: float, steps: int, world: int, B: int) -> float:
+    """Whole-job metric: every rank ran `steps` steps of B episodes in `total_ms` (max over ranks)."""
+    return total_ms * 1e3 / (steps * world * B)
+
+
 # ------------------------------------------------------------------------------------------------ GPU arm
 def run_gpu(args, w: wl.Workload):
     import torch
     import torch.distributed as dist
     import paper_2609_19104_b200 as rm
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = rank_env()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -195,7 +220,7 @@ def run_gpu(args, w: wl.Workload):
     torch.cuda.synchronize()
 
     # every rank runs its own episodes (replicas; no data-path collective)
-    ep0 = rank * B
+    ep0 = episodes_of_rank(rank, B)[0]
     f32 = lambda bits: torch.from_numpy(wl.bf16_bits_to_f32(bits))
     refs = torch.stack([f32(wl.reference_input(w, episode=ep0 + b)) for b in range(B)]).cuda()
     step_inputs = [torch.stack([f32(wl.step_input(w, s, episode=ep0 + b)) for b in range(B)]) for s in range(w.steps)]
@@ -291,15 +316,11 @@ def run_gpu(args, w: wl.Workload):
     layer_us = float(np.mean([a.elapsed_time(b) for a, b in layer_ms])) * 1e3
     clocks = sampler.stop() if rank == 0 else None
 
-    t = torch.tensor([total_ms, e2e_total_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_total_ms = float(t[0].item()), float(t[1].item())
+    total_ms, e2e_total_ms = max_over_ranks([total_ms, e2e_total_ms], world, device="cuda")
 
     if rank == 0:
-        units = args.steps * world * B                      # denoising steps of one episode, whole job
-        us_per_step = total_ms * 1e3 / units
-        e2e_us = e2e_total_ms * 1e3 / units
+        us_per_step = job_us_per_step(total_ms, args.steps, world, B)   # per denoising step of one episode, whole job
+        e2e_us = job_us_per_step(e2e_total_ms, args.steps, world, B)
         peak, peak_kind = measured_hbm_peak()
         bytes_layer = wl.algorithmic_bytes_per_layer(w.H, w.T, int(round(K_mean))) * B
         bytes_step = bytes_layer * w.L
