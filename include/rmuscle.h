@@ -132,6 +132,28 @@ int rm_action_expert_step_host(rm_ctx* ctx, const void* const* packed_layers, co
                                const int32_t* idx, const int32_t* count_dev, int64_t stride, float* r_out_host,
                                int B, int T, void* ws, size_t ws_bytes, rm_stream_t stream);
 
+/* ---- rm_action_expert_step_ex: the same stack with the anchor-relative local update of the Action Cache (Sec. 4.1
+ * "Anchors with Mask Recomputation", Eq. 4) and the output gate that follows it ("the output follows the normal
+ * adaptive gate and residual addition").  Per layer l and episode:
+ *   RM_ANCHOR_WRITE  (the group's anchor step; normally dense, idx = NULL):
+ *       y_a = sum_{n in S} h_n Wd[:,n]   (S = every neuron when idx is NULL),   r_{l+1} = r_l + gate * y_a,
+ *       and the call retains y_a in y_anchor and h_n[t] (n in S) in h_anchor.
+ *   RM_ANCHOR_UPDATE (a non-anchor step with mask M = the list):
+ *       y_hat = y_a + sum_{n in M} (h_n - h_a,n) Wd[:,n],                         r_{l+1} = r_l + gate * y_hat,
+ *       with y_a, h_a read from y_anchor / h_anchor: neurons outside M keep the anchor step's contribution.
+ *   RM_ANCHOR_NONE: rm_action_expert_step with the gate applied (zero-fill form).
+ *   y_anchor [L,B,T,H] fp32 (pre-gate, pre-residual).   h_anchor [L,B,I,h_stride] fp32, neuron-major: the T
+ *   activations of a neuron are contiguous, so a step may use any mask without an index map (the paper keeps
+ *   h_a^M compact for one fixed mask); h_stride >= T and a multiple of 4.   out_gate [L,B,H] fp32 or NULL (= 1).
+ *   With zero anchors (y_anchor = 0, h_anchor = 0) RM_ANCHOR_UPDATE equals the zero-fill form.
+ *   In RM_ANCHOR_WRITE the call clears y_anchor itself.  Everything else as for rm_action_expert_step. */
+enum { RM_ANCHOR_NONE = 0, RM_ANCHOR_WRITE = 1, RM_ANCHOR_UPDATE = 2 };
+int rm_action_expert_step_ex(rm_ctx* ctx, const void* const* packed_layers, const float* r_in, const int32_t* idx,
+                             const int32_t* count_dev, int64_t stride, float* r_out, float* records_out,
+                             const float* record_scale, int B, int T, int anchor_mode, float* y_anchor,
+                             float* h_anchor, int64_t h_stride, const float* out_gate, void* ws, size_t ws_bytes,
+                             rm_stream_t stream);
+
 /* ---- rm_sparse_mlp_static: the one-layer call of rm_sparse_mlp for callers that cannot allocate.
  * (The paper has no counterpart for this entry point; it exists for integration reasons only.)
  *

@@ -118,20 +118,52 @@ def dense_mlp(x, Wg, Wu, Wd, r, scale=None, return_h: bool = False, return_recor
     return out[0] if len(out) == 1 else tuple(out)
 
 
-def anchor_mlp(x, Wg, Wu, Wd, r, idx, y_anchor, h_anchor):
-    """Eq. 4 followed by the residual add: out = r + y_anchor + (h^M - h_anchor^M) W_down[:,M]."""
+def anchor_mlp(x, Wg, Wu, Wd, r, idx, y_anchor, h_anchor, gate=None):
+    """Eq. 4, then gate and residual: out = r + gate * (y_anchor + (h^M - h_anchor^M) W_down[:,M])."""
     x, Wg, Wu, Wd = _u16(x), _u16(Wg), _u16(Wu), _u16(Wd)
     T, H = x.shape
     I = Wg.shape[0]
     idx = _i32(idx)
     K = int(idx.shape[0])
-    r, y_anchor, h_anchor = _f32(r), _f32(y_anchor), _f32(h_anchor)
+    r, y_anchor, h_anchor, gate = _f32(r), _f32(y_anchor), _f32(h_anchor), _f32(gate)
     if h_anchor is not None:
         assert h_anchor.shape == (T, K)
+    if gate is not None:
+        assert gate.shape == (H,)
     out = np.empty((T, H), dtype=np.float32)
     _load().orc_anchor_mlp(_p(x), _p(Wg), _p(Wu), _p(Wd), _p(r), _p(idx), ctypes.c_int(K), ctypes.c_int(T),
-                           ctypes.c_int(H), ctypes.c_int(I), _p(y_anchor), _p(h_anchor), _p(out))
+                           ctypes.c_int(H), ctypes.c_int(I), _p(y_anchor), _p(h_anchor), _p(gate), _p(out))
     return out
+
+
+def anchor_step_write(Wg_layers, Wu_layers, Wd_layers, r_in, gate=None, scale=None):
+    """The dense anchor step of a group (Sec. 4.1 "Anchors with Mask Recomputation"): every layer runs the dense
+    FFN on x_l = bf16(RMSNorm(r_l)), retains its output y_a (before gate and residual) and its activations h_a, and
+    continues with r_{l+1} = r_l + gate_l * y_a.  Returns r_L, y_anchor [L,T,H], h_anchor [L,T,I], records [L,I]."""
+    L = len(Wg_layers)
+    r = np.ascontiguousarray(r_in, dtype=np.float32)
+    ys, hs, recs = [], [], []
+    for l in range(L):
+        x = rmsnorm_bf16(r)
+        y, h, rec = dense_mlp(x, Wg_layers[l], Wu_layers[l], Wd_layers[l], None, scale=None if scale is None else scale[l],
+                              return_h=True, return_record=True)
+        g = 1.0 if gate is None else np.asarray(gate[l], dtype=np.float64)[None, :]
+        r = (r.astype(np.float64) + g * y.astype(np.float64)).astype(np.float32)
+        ys.append(y), hs.append(h), recs.append(rec)
+    return r, np.stack(ys), np.stack(hs), np.stack(recs)
+
+
+def anchor_step_update(Wg_layers, Wu_layers, Wd_layers, r_in, idx, count, y_anchor, h_anchor, gate=None):
+    """A non-anchor step: every layer applies Eq. 4 on its mask M_l = idx[l, :count[l]] against the retained anchor
+    state, then gate and residual."""
+    L = len(Wg_layers)
+    r = np.ascontiguousarray(r_in, dtype=np.float32)
+    for l in range(L):
+        x = rmsnorm_bf16(r)
+        M = np.ascontiguousarray(idx[l, :int(count[l])], dtype=np.int32)
+        r = anchor_mlp(x, Wg_layers[l], Wu_layers[l], Wd_layers[l], r, M, y_anchor[l],
+                       np.ascontiguousarray(h_anchor[l][:, M]), None if gate is None else gate[l])
+    return r
 
 
 def rmsnorm_bf16(r):

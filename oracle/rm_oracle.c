@@ -125,11 +125,13 @@ void orc_dense_mlp(const uint16_t* x, const uint16_t* Wg, const uint16_t* Wu, co
 }
 
 /* Anchor-relative local update (Eq. 4): y_hat = y_anchor + (h_t^M - h_anchor^M) W_down[:,M], followed by the
- * residual addition out = r + y_hat.  y_anchor [T,H] is the anchor step's pre-residual FFN output, h_anchor
- * [T,K] its activations on the mask.  With y_anchor = 0 and h_anchor = 0 this is the zero-fill form. */
+ * output gate and the residual addition (Sec. 4.1: "the output follows the normal adaptive gate and residual
+ * addition"): out = r + gate * y_hat, gate [H] per output channel, NULL = 1.  y_anchor [T,H] is the anchor step's
+ * FFN output before gate and residual, h_anchor [T,K] its activations on the mask.  With y_anchor = 0 and
+ * h_anchor = 0 this is the zero-fill form. */
 void orc_anchor_mlp(const uint16_t* x, const uint16_t* Wg, const uint16_t* Wu, const uint16_t* Wd,
                     const float* r, const int32_t* idx, int K, int T, int H, int I,
-                    const float* y_anchor, const float* h_anchor, float* out) {
+                    const float* y_anchor, const float* h_anchor, const float* gate, float* out) {
     float* d = (float*)malloc(sizeof(float) * (size_t)(T > 0 ? T : 1) * (size_t)(K > 0 ? K : 1));
 #pragma omp parallel for schedule(static)
     for (int j = 0; j < K; ++j) {
@@ -146,9 +148,9 @@ void orc_anchor_mlp(const uint16_t* x, const uint16_t* Wg, const uint16_t* Wu, c
             double acc = 0.0;
             for (int j = 0; j < K; ++j)
                 acc += (double)d[(size_t)t * K + j] * (double)bf16_to_f32(Wd[(size_t)c * I + (size_t)idx[j]]);
-            double base = (r ? (double)r[(size_t)t * H + c] : 0.0) +
-                          (y_anchor ? (double)y_anchor[(size_t)t * H + c] : 0.0);
-            out[(size_t)t * H + c] = (float)(base + acc);
+            double y_hat = (y_anchor ? (double)y_anchor[(size_t)t * H + c] : 0.0) + acc;
+            double base = r ? (double)r[(size_t)t * H + c] : 0.0;
+            out[(size_t)t * H + c] = (float)(base + (gate ? (double)gate[c] : 1.0) * y_hat);
         }
     }
     free(d);

@@ -19,9 +19,11 @@ RM_ERR_CUDA, RM_ERR_INDEX, RM_ERR_TIMEOUT, RM_ERR_UNSUPPORTED = -5, -6, -7, -8
 RM_ACT_GELU_TANH = 0
 RM_SRC_BOOL_U8, RM_SRC_SCORE_F32 = 0, 1
 RM_REDUCE_NONE, RM_REDUCE_THRESHOLD, RM_REDUCE_TOPK, RM_REDUCE_GROUP = 0, 1, 2, 3
+RM_ANCHOR_NONE, RM_ANCHOR_WRITE, RM_ANCHOR_UPDATE = 0, 1, 2
 
 EXPORTS = ["rm_create", "rm_destroy", "rm_packed_layer_bytes", "rm_workspace_bytes", "rm_pack_weights",
            "rm_mask_compact", "rm_sparse_mlp", "rm_action_expert_step", "rm_action_expert_step_host",
+           "rm_action_expert_step_ex",
            "rm_device_status", "rm_launch_count", "rm_status_string", "rm_set_option", "rm_get_info",
            "rm_debug_phase_times", "rm_sparse_mlp_static"]
 
@@ -73,6 +75,8 @@ def load_library() -> ctypes.CDLL:
     lib.rm_sparse_mlp.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
     lib.rm_action_expert_step.argtypes = [vp, ctypes.POINTER(vp), vp, vp, vp, i64, vp, vp, vp, i32, i32, vp, sz, vp]
     lib.rm_action_expert_step_host.argtypes = [vp, ctypes.POINTER(vp), vp, vp, vp, i64, vp, i32, i32, vp, sz, vp]
+    lib.rm_action_expert_step_ex.argtypes = [vp, ctypes.POINTER(vp), vp, vp, vp, i64, vp, vp, vp, i32, i32, i32, vp, vp,
+                                             i64, vp, vp, sz, vp]
     lib.rm_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
     lib.rm_launch_count.argtypes = [vp]
     lib.rm_launch_count.restype = i64
@@ -214,6 +218,20 @@ class Context:
                                               _ptr(count_dev), int(stride), _ptr(r_out), _ptr(records_out),
                                               _ptr(record_scale), B, T, _ptr(ws), int(ws.numel()), _stream()),
                "rm_action_expert_step")
+        return r_out
+
+    def rm_action_expert_step_ex(self, packed_layers, r_in, idx, count_dev, stride: int, r_out, anchor_mode: int,
+                                 y_anchor, h_anchor, h_stride: int, out_gate=None, records_out=None,
+                                 record_scale=None, B: int = 1, T: Optional[int] = None, ws=None):
+        """The step with the anchor-relative update (Eq. 4): y_anchor [L,B,T,H], h_anchor [L,B,I,h_stride] fp32."""
+        T = int(r_in.shape[-2]) if T is None else T
+        ws = self.workspace(max(B, 1), max(T, 1)) if ws is None else ws
+        _check(self.lib.rm_action_expert_step_ex(self._h, self._layer_ptrs(packed_layers), _ptr(r_in), _ptr(idx),
+                                                 _ptr(count_dev), int(stride), _ptr(r_out), _ptr(records_out),
+                                                 _ptr(record_scale), B, T, int(anchor_mode), _ptr(y_anchor),
+                                                 _ptr(h_anchor), int(h_stride), _ptr(out_gate), _ptr(ws),
+                                                 int(ws.numel()), _stream()),
+               "rm_action_expert_step_ex")
         return r_out
 
     def rm_action_expert_step_host(self, packed_layers, r_in_host, idx, count_dev, stride: int, r_out_host,

@@ -156,9 +156,20 @@ int rm_sparse_mlp(rm_ctx* ctx, const void* packed_layer, const void* x, const fl
     return rm_launch_layer_ref(ctx, a, static_cast<char*>(ws) + 4 * r_bytes, s);
 }
 
+namespace {
+struct AnchorIO {                      // whole-stack anchor state (Eq. 4); mode RM_ANCHOR_NONE and NULLs for none
+    int mode = RM_ANCHOR_NONE;
+    float* y = nullptr;                // [L,B,T,H]
+    float* h = nullptr;                // [L,B,I,h_stride]
+    int64_t h_stride = 0;
+    const float* gate = nullptr;       // [L,B,H]
+};
+}  // namespace
+
 static int step_device(rm_ctx* ctx, const void* const* packed_layers, const float* r_in, const int32_t* idx,
                        const int32_t* count_dev, int64_t stride, float* r_out, float* records_out,
-                       const float* record_scale, int B, int T, void* ws, cudaStream_t s) {
+                       const float* record_scale, int B, int T, void* ws, cudaStream_t s,
+                       const AnchorIO& an = AnchorIO()) {
     const rm_geom& g = ctx->g;
     const size_t n_bytes = (size_t)B * T * g.H * sizeof(float);
     const size_t r_bytes = align_up(n_bytes, 256);
@@ -176,6 +187,9 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
         RM_CUDA_TRY(cudaMemsetAsync(g.L == 1 && direct_out ? r_out : rot[1], 0, n_bytes, s));
         if (direct_out && g.L > 1) RM_CUDA_TRY(cudaMemsetAsync(r_out, 0, n_bytes, s));
     }
+    // the anchor step's outputs are accumulated by the CTAs' atomics: start them from zero
+    if (fused && an.mode == RM_ANCHOR_WRITE)
+        RM_CUDA_TRY(cudaMemsetAsync(an.y, 0, (size_t)g.L * n_bytes, s));
     const float* cur = r_in;
     for (int l = 0; l < g.L; ++l) {
         rm_layer_args a{};
@@ -192,6 +206,11 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
         a.record_scale = record_scale ? record_scale + (size_t)l * g.I : nullptr;
         a.B = B;
         a.T = T;
+        a.anchor_mode = an.mode;
+        a.y_anchor = an.y ? an.y + (size_t)l * B * T * g.H : nullptr;
+        a.h_anchor = an.h ? an.h + (size_t)l * B * g.I * an.h_stride : nullptr;
+        a.h_stride = an.h_stride;
+        a.gate = an.gate ? an.gate + (size_t)l * B * g.H : nullptr;
         int rc;
         if (fused) {
             const bool last = l == g.L - 1;
@@ -229,6 +248,40 @@ int rm_action_expert_step(rm_ctx* ctx, const void* const* packed_layers, const f
     if (!ws || ws_bytes < rm_workspace_bytes(ctx, B, T)) return RM_ERR_WORKSPACE;
     return step_device(ctx, packed_layers, r_in, idx, count_dev, stride, r_out, records_out, record_scale, B, T, ws,
                        static_cast<cudaStream_t>(stream));
+}
+
+int rm_action_expert_step_ex(rm_ctx* ctx, const void* const* packed_layers, const float* r_in, const int32_t* idx,
+                             const int32_t* count_dev, int64_t stride, float* r_out, float* records_out,
+                             const float* record_scale, int B, int T, int anchor_mode, float* y_anchor,
+                             float* h_anchor, int64_t h_stride, const float* out_gate, void* ws, size_t ws_bytes,
+                             rm_stream_t stream) {
+    if (!ctx || !packed_layers || !r_in || !r_out || B < 0 || T < 0) return RM_ERR_INVALID_ARG;
+    if (idx && (!count_dev || stride < 1)) return RM_ERR_INVALID_ARG;
+    if (idx && records_out) return RM_ERR_INVALID_ARG;
+    if (anchor_mode != RM_ANCHOR_NONE && anchor_mode != RM_ANCHOR_WRITE && anchor_mode != RM_ANCHOR_UPDATE)
+        return RM_ERR_INVALID_ARG;
+    if (anchor_mode != RM_ANCHOR_NONE) {
+        if (!y_anchor || !h_anchor || h_stride < T) return RM_ERR_INVALID_ARG;
+        if (h_stride % 4 != 0) return RM_ERR_ALIGN;
+        // the anchor state is read (or accumulated) while the outputs are written: no overlap with them
+        if (y_anchor == r_out || y_anchor == r_in) return RM_ERR_INVALID_ARG;
+    }
+    if (B > ctx->desc.B_max || T > ctx->desc.T_max) return RM_ERR_SHAPE;
+    for (int l = 0; l < ctx->g.L; ++l) {
+        if (!packed_layers[l]) return RM_ERR_INVALID_ARG;
+        if (!rm_aligned16(packed_layers[l])) return RM_ERR_ALIGN;
+    }
+    if (!all_aligned({r_in, idx, r_out, records_out, record_scale, ws, y_anchor, h_anchor, out_gate}))
+        return RM_ERR_ALIGN;
+    if (idx && (stride % 4) != 0) return RM_ERR_ALIGN;
+    if (B == 0 || T == 0) return RM_OK;
+    if (!ws || ws_bytes < rm_workspace_bytes(ctx, B, T)) return RM_ERR_WORKSPACE;
+    AnchorIO an;
+    an.mode = anchor_mode;
+    if (anchor_mode != RM_ANCHOR_NONE) { an.y = y_anchor; an.h = h_anchor; an.h_stride = h_stride; }
+    an.gate = out_gate;
+    return step_device(ctx, packed_layers, r_in, idx, count_dev, stride, r_out, records_out, record_scale, B, T, ws,
+                       static_cast<cudaStream_t>(stream), an);
 }
 
 int rm_action_expert_step_host(rm_ctx* ctx, const void* const* packed_layers, const float* r_in_host,

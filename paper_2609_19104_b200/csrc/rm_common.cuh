@@ -92,6 +92,12 @@ struct rm_layer_args {
     int64_t record_stride;
     const float* record_scale;             // [I] or NULL
     int B, T;
+    // anchor-relative update (Eq. 4); all NULL / RM_ANCHOR_NONE for the zero-fill form
+    int anchor_mode;                       // RM_ANCHOR_*
+    float* y_anchor;                       // [B,T,H] fp32: FFN output of the anchor step before gate and residual
+    float* h_anchor;                       // [B,I,h_stride] fp32: the anchor step's hidden activations, neuron-major
+    int64_t h_stride;                      // floats between neurons (>= T, multiple of 4)
+    const float* gate;                     // [B,H] fp32 output gate, or NULL (= 1)
 };
 size_t rm_ref_workspace_bytes(const rm_ctx* ctx, int B, int T);
 // Tensor-core path: H in {1024, 2048}, T <= 64 per episode, B <= 64.

@@ -94,7 +94,15 @@ __global__ void __launch_bounds__(GU_WARPS * 32) ref_gateup_kernel(rm_layer_args
         }
         float hv = bad ? 0.0f : rm_gelu_tanh(ag) * au;
         rec += fabsf(hv);
-        if (lane == 0) h[((size_t)b * a.T + t) * g.I + j] = hv;
+        if (lane == 0) {
+            // Eq. 4: the anchor step retains h, a later step contributes its difference from the anchor's h
+            if (a.anchor_mode != RM_ANCHOR_NONE && !bad) {
+                float* ha = a.h_anchor + ((size_t)b * g.I + n) * a.h_stride + t;
+                if (a.anchor_mode == RM_ANCHOR_WRITE) *ha = hv;
+                else hv -= *ha;
+            }
+            h[((size_t)b * a.T + t) * g.I + j] = hv;
+        }
     }
     if (a.record && lane == 0 && !bad)
         a.record[(size_t)b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
@@ -154,7 +162,16 @@ __global__ void __launch_bounds__(DN_THREADS) ref_down_kernel(rm_layer_args a, r
         if (t >= a.T) break;
         size_t o = ((size_t)b * a.T + t) * g.H + c;
         float2 base = a.r_in ? *reinterpret_cast<const float2*>(a.r_in + o) : make_float2(0.0f, 0.0f);
-        *reinterpret_cast<float2*>(a.r_out + o) = make_float2(base.x + acc[tt][0], base.y + acc[tt][1]);
+        float2 y = make_float2(acc[tt][0], acc[tt][1]);
+        if (a.anchor_mode == RM_ANCHOR_WRITE) {
+            *reinterpret_cast<float2*>(a.y_anchor + o) = y;
+        } else if (a.anchor_mode == RM_ANCHOR_UPDATE) {
+            const float2 ya = *reinterpret_cast<const float2*>(a.y_anchor + o);
+            y.x += ya.x;
+            y.y += ya.y;
+        }
+        const float2 gt = a.gate ? *reinterpret_cast<const float2*>(a.gate + (size_t)b * g.H + c) : make_float2(1.0f, 1.0f);
+        *reinterpret_cast<float2*>(a.r_out + o) = make_float2(base.x + gt.x * y.x, base.y + gt.y * y.y);
     }
 }
 

@@ -82,7 +82,25 @@ struct FusedArgs {
     int* status;
     int wall_seq;                  // launch sequence number (phase-timing builds only)
     int l2_prefetch;               // tiles of L2 prefetch distance in the warp-specialised kernel (0: off)
+    // anchor-relative update (Eq. 4): see rm_layer_args
+    int anchor_mode;
+    float* y_anchor;
+    float* h_anchor;
+    int64_t h_stride;
+    const float* gate;
 };
+
+// r_out[0..3] += r[0..3] (+ gate * y_anchor in an update step, Eq. 4): the residual part of a layer's output
+__device__ __forceinline__ void add_residual4(const FusedArgs& a, float* o, size_t off_bt_h, int col, int b,
+                                              float r0, float r1, float r2, float r3) {
+    if (a.anchor_mode == RM_ANCHOR_UPDATE) {
+        const float4 ya = *reinterpret_cast<const float4*>(a.y_anchor + off_bt_h + col);
+        float4 g = make_float4(1.f, 1.f, 1.f, 1.f);
+        if (a.gate) g = *reinterpret_cast<const float4*>(a.gate + (size_t)b * a.H + col);
+        r0 = fmaf(g.x, ya.x, r0); r1 = fmaf(g.y, ya.y, r1); r2 = fmaf(g.z, ya.z, r2); r3 = fmaf(g.w, ya.w, r3);
+    }
+    red_add_v4(o, r0, r1, r2, r3);
+}
 
 // floats per row of the exchange buffer: T rounded up to 4 with an odd number of 16-byte chunks, so that the
 // eight rows written by one warp-store fall into distinct bank groups
@@ -281,7 +299,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             float* dst = a.r_out + (size_t)b * T * H;
             for (size_t i = (size_t)blockIdx.x * FT + tid; i < (size_t)T * H / 4; i += (size_t)gridDim.x * FT) {
                 const float4 v = src[i];
-                red_add_v4(dst + 4 * i, v.x, v.y, v.z, v.w);
+                add_residual4(a, dst + 4 * i, (size_t)b * T * H + (4 * i / H) * H, (int)(4 * i % H), b, v.x, v.y, v.z, v.w);
             }
         }
     }
@@ -359,9 +377,11 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             // residual: token row t of this episode is added by exactly one of the clusters that work on the
             // episode, from the values already in registers, while the exchange is in flight
             if (a.add_residual && t < T && (t % n_share) == my_share) {
-                float* o = a.r_out + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP;
+                const size_t row = ((size_t)b * T + t) * H;
+                const int col = j * HS + part * CPP;
 #pragma unroll
-                for (int i = 0; i < CPP / 4; ++i) red_add_v4(o + 4 * i, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                for (int i = 0; i < CPP / 4; ++i)
+                    add_residual4(a, a.r_out + row + col + 4 * i, row, col + 4 * i, b, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
             }
             wait_bar(bar_s, par_s);
             par_s ^= 1;
@@ -457,9 +477,25 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
 
     // ---- phase: owner work of tile i -- sum the 8 partials, GeLU-tanh(g) * u, activation record, h = hi + lo in
     // bf16 as this CTA's atom of the MN-major h operand, then all-gather the atom into every CTA (bulk copies)
-    auto reduce_bcast = [&](int i, const TileRef& tr) {
+    constexpr int TPL = NTOK / 32;                         // owner work: tokens per lane
+    // Eq. 4 update steps: the anchor's h for this lane's tokens of its neuron of tile i.  Requested as soon as the
+    // tile's neuron ids are in shared memory, long before the partial sums arrive.
+    auto anchor_prefetch = [&](int i, const TileRef& tr, float (&ha_pre)[TPL]) {
+#pragma unroll
+        for (int k = 0; k < TPL; ++k) ha_pre[k] = 0.f;
+        if (a.anchor_mode != RM_ANCHOR_UPDATE) return;
+        const int n = gN[(i & 1) * NT + j * 8 + warp];
+        const int t0 = lane * TPL;
+        if (n >= 0 && t0 < T) {
+            const float* hap = a.h_anchor + ((size_t)tr.b * a.I + n) * a.h_stride + t0;
+            if (TPL == 2) { const float2 f = *reinterpret_cast<const float2*>(hap); ha_pre[0] = f.x; ha_pre[TPL - 1] = f.y; }
+            else ha_pre[0] = *hap;
+#pragma unroll
+            for (int k = 0; k < TPL; ++k) if (t0 + k >= T) ha_pre[k] = 0.f;
+        }
+    };
+    auto reduce_bcast = [&](int i, const TileRef& tr, const float (&ha_pre)[TPL]) {
         const int pb = buf_of(i);
-        constexpr int TPL = NTOK / 32;                     // tokens per lane
         const int ql = warp;                               // local neuron 0..7 (tile neuron 8j + ql)
         const int t0 = lane * TPL;
         const float* gP = reinterpret_cast<const float*>(gbase + S::OFF_P + pb * p_bytes);
@@ -482,6 +518,20 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
         for (int k = 0; k < TPL; ++k) {
             hv[k] = (t0 + k < T) ? rm_gelu_tanh(gsum[k]) * usum[k] : 0.f;
             rec += fabsf(hv[k]);
+        }
+        // Eq. 4: the anchor step retains h; a later step sends its difference from the anchor's h down the projection
+        if (a.anchor_mode != RM_ANCHOR_NONE) {
+            const int n = gN[(i & 1) * NT + j * 8 + ql];
+            if (n >= 0 && t0 < T) {
+                float* hap = a.h_anchor + ((size_t)tr.b * a.I + n) * a.h_stride + t0;
+                if (a.anchor_mode == RM_ANCHOR_WRITE) {
+                    if (TPL == 2) *reinterpret_cast<float2*>(hap) = make_float2(hv[0], hv[TPL - 1]);
+                    else *hap = hv[0];
+                } else {
+#pragma unroll
+                    for (int k = 0; k < TPL; ++k) hv[k] -= ha_pre[k];
+                }
+            }
         }
         // row = local neuron, 128 bytes = 64 tokens, 16-byte chunks swizzled by the row; hi at 0, lo at 1024
         {
@@ -542,10 +592,17 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
                 float v[32];
                 tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
-                float* dst = a.r_out + (size_t)tr.b * T * H + (size_t)j * HS + mm * 128 + (warp & 3) * 32 + lane;
+                const size_t off = (size_t)tr.b * T * H + (size_t)j * HS + mm * 128 + (warp & 3) * 32 + lane;
+                float* dst = a.r_out + off;
+                const float gc = a.gate ? a.gate[(size_t)tr.b * H + j * HS + mm * 128 + (warp & 3) * 32 + lane] : 1.f;
+                if (a.anchor_mode == RM_ANCHOR_WRITE) {    // the anchor step also retains its ungated FFN output
+#pragma unroll
+                    for (int k = 0; k < 32; ++k)
+                        if (c0 + k < T) atomicAdd(a.y_anchor + off + (size_t)(c0 + k) * H, v[k]);
+                }
 #pragma unroll
                 for (int k = 0; k < 32; ++k)
-                    if (c0 + k < T) atomicAdd(dst + (size_t)(c0 + k) * H, v[k]);
+                    if (c0 + k < T) atomicAdd(dst + (size_t)(c0 + k) * H, gc * v[k]);
             }
         }
         tc_fence_before();
@@ -563,6 +620,8 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             fence_proxy_async();
             __syncthreads();
             RM_STAMP(6);
+            float ha_pre[TPL];
+            anchor_prefetch(i, tr, ha_pre);
             mma_gu(i);
             wait_bar(bar_gu(0), phase_of(i));
             tc_fence_after();
@@ -573,7 +632,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             scatter(i, refill);
             wait_bar(bar_p(0), phase_of(i));           // every source's partial sums for this CTA's neurons are here
             RM_STAMP(9);
-            reduce_bcast(i, tr);
+            reduce_bcast(i, tr, ha_pre);
             wait_bar(bar_h(0), phase_of(i));           // h of the whole tile (all 8 owners' atoms) is here
             RM_STAMP(11);
             mma_dn(i, tr);
@@ -613,9 +672,11 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
                 __syncthreads();
                 mma_gu(i + 1);
             }
+            float ha_pre[TPL];
+            anchor_prefetch(i, tr, ha_pre);
             wait_bar(bar_p(buf_of(i)), phase_of(i));
             RM_STAMP(9);
-            reduce_bcast(i, tr);
+            reduce_bcast(i, tr, ha_pre);
             if (more) {
                 wait_bar(bar_gu(buf_of(i + 1)), phase_of(i + 1));
                 tc_fence_after();
@@ -957,9 +1018,11 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 for (int dst = part; dst < CS; dst += PARTS)
                     st_async_f32(map_to_rank(sSS + (j * 64 + t) * 4, dst), ss, map_to_rank(bar_s, dst));
                 if (a.add_residual && t < T && (t % n_share) == my_share) {
-                    float* o = a.r_out + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP;
+                    const size_t row = ((size_t)b * T + t) * H;
+                    const int col = j * HS + part * CPP;
 #pragma unroll
-                    for (int i = 0; i < CPP / 4; ++i) red_add_v4(o + 4 * i, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    for (int i = 0; i < CPP / 4; ++i)
+                        add_residual4(a, a.r_out + row + col + 4 * i, row, col + 4 * i, b, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
                 }
                 wait_bar(bar_s, par_s);
                 float tot = 0.f;
@@ -1044,10 +1107,17 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                     for (int c0 = 0; c0 < NTOK; c0 += 32) {
                         float v[32];
                         tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)(warp * 32) << 16) + c0, v);
-                        float* dst = a.r_out + (size_t)b * T * H + (size_t)j * HS + mm * 128 + warp * 32 + lane;
+                        const size_t off = (size_t)b * T * H + (size_t)j * HS + mm * 128 + warp * 32 + lane;
+                        float* dst = a.r_out + off;
+                        const float gc = a.gate ? a.gate[(size_t)b * H + j * HS + mm * 128 + warp * 32 + lane] : 1.f;
+                        if (a.anchor_mode == RM_ANCHOR_WRITE) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (c0 + e < T) atomicAdd(a.y_anchor + off + (size_t)(c0 + e) * H, v[e]);
+                        }
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
-                            if (c0 + e < T) atomicAdd(dst + (size_t)(c0 + e) * H, v[e]);
+                            if (c0 + e < T) atomicAdd(dst + (size_t)(c0 + e) * H, gc * v[e]);
                     }
                 }
                 tc_fence_before();
@@ -1069,6 +1139,25 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 }
                 wait_bar(bar_p(pb), (it >> 1) & 1);
                 if (ot == 0) RM_WS(it, 4);
+                // Eq. 4: the anchor's h for this lane's tokens (the tile's neuron ids are known to be published only
+                // now: the partial sums that just arrived were computed from rows gathered by those ids)
+                float ha_pre[TPL];
+#pragma unroll
+                for (int e = 0; e < TPL; ++e) ha_pre[e] = 0.f;
+                const int n_own = a.anchor_mode != RM_ANCHOR_NONE ? gN[(it & 7) * NT + j * 8 + ql] : -1;
+                float* hap = (n_own >= 0 && t0 < T) ? a.h_anchor + ((size_t)b * a.I + n_own) * a.h_stride + t0 : nullptr;
+                if (a.anchor_mode == RM_ANCHOR_UPDATE && hap) {
+                    if (TPL == 4) {
+                        const float4 f = *reinterpret_cast<const float4*>(hap);
+                        ha_pre[0] = f.x; ha_pre[1] = f.y; ha_pre[2] = f.z; ha_pre[TPL - 1] = f.w;
+                    } else {
+                        const float2 f = *reinterpret_cast<const float2*>(hap);
+                        ha_pre[0] = f.x; ha_pre[TPL - 1] = f.y;
+                    }
+#pragma unroll
+                    for (int e = 0; e < TPL; ++e) if (t0 + e >= T) ha_pre[e] = 0.f;
+                }
+
                 const float* gP = reinterpret_cast<const float*>(gbase + S::OFF_P + pb * p_bytes);
                 unsigned char* gHS = gbase + S::OFF_HS + pb * 2048;
                 float gsum[TPL], usum[TPL];
@@ -1096,6 +1185,15 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 for (int e = 0; e < TPL; ++e) {
                     hv[e] = (t0 + e < T) ? rm_gelu_tanh(gsum[e]) * usum[e] : 0.f;
                     rec += fabsf(hv[e]);
+                }
+                if (hap) {
+                    if (a.anchor_mode == RM_ANCHOR_WRITE) {
+                        if (TPL == 4) *reinterpret_cast<float4*>(hap) = make_float4(hv[0], hv[1], hv[2], hv[TPL - 1]);
+                        else *reinterpret_cast<float2*>(hap) = make_float2(hv[0], hv[TPL - 1]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < TPL; ++e) hv[e] -= ha_pre[e];
+                    }
                 }
                 // TPL consecutive tokens of one neuron row: one 8-byte (or 4-byte) store each for hi and lo
                 unsigned char* rowp = gHS + ql * 128 + ((((t0 >> 3) ^ ql) & 7) << 4) + (t0 & 7) * 2;
@@ -1233,7 +1331,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 float* dst = a.r_out + (size_t)b * T * H;
                 for (size_t i = (size_t)blockIdx.x * 256 + tid; i < (size_t)T * H / 4; i += (size_t)gridDim.x * 256) {
                     const float4 v = src[i];
-                    red_add_v4(dst + 4 * i, v.x, v.y, v.z, v.w);
+                    add_residual4(a, dst + 4 * i, (size_t)b * T * H + (4 * i / H) * H, (int)(4 * i % H), b, v.x, v.y, v.z, v.w);
                 }
             }
         }
@@ -1392,6 +1490,11 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
     a.status = ctx->d_status;
     a.wall_seq = (int)(ctx->launches & 63);
     a.l2_prefetch = ctx->l2_prefetch;
+    a.anchor_mode = la.anchor_mode;
+    a.y_anchor = la.y_anchor;
+    a.h_anchor = la.h_anchor;
+    a.h_stride = la.h_stride;
+    a.gate = la.gate;
     // Tiles of 64 neurons in this launch, when the host knows the number of active neurons (dense calls, or the
     // caller's hint); 0 = unknown.
     const int per_episode = la.idx ? ctx->count_hint : ctx->g.I;

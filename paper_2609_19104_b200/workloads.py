@@ -32,7 +32,7 @@ _M2 = _U64(0x94D049BB133111EB)
 # tensor roles (part of the tensor id)
 ROLE_WG, ROLE_WU, ROLE_WD = 1, 2, 3
 ROLE_X0, ROLE_REF_NOISE, ROLE_STEP_DIR, ROLE_RESIDUAL = 4, 5, 6, 7
-ROLE_BOOL_MASK, ROLE_RUNS = 8, 9
+ROLE_BOOL_MASK, ROLE_RUNS, ROLE_GATE = 8, 9, 10
 
 
 def _mix(z: np.ndarray) -> np.ndarray:
@@ -159,6 +159,13 @@ def config4(seed: int = BASE_SEED, L: int = 18) -> Workload:
                            "in_run_scale": 4.0})
 
 
+def config5(seed: int = BASE_SEED, L: int = 18) -> Workload:
+    # the anchor schedule of the Action Cache on the config-1 model: 10 denoising steps in two groups of five, the
+    # first step of a group is the dense anchor, the other four update the group's shared mask (top-k = 2048 of 4096)
+    return Workload(5, "pi0-anchor-groups-top50", L, 1024, 4096, 51, 0.02, 10, 0.50, seed=seed,
+                    extra={"weights_config": 1, "group": 5})
+
+
 def scaled(w: Workload, **kw) -> Workload:
     """A smaller (or otherwise altered) copy of a workload for tests; same recipe, same seed stream."""
     d = dict(config=w.config, name=w.name + "-scaled", L=w.L, H=w.H, I=w.I, T=w.T, sigma=w.sigma, steps=w.steps,
@@ -196,6 +203,21 @@ def reference_input(w: Workload, record: int = 0, episode: int = 0, cosine: floa
     x0 = base_input(w, episode)
     e = normal(tensor_key(w.seed, w.config, 0, ROLE_REF_NOISE, episode * 64 + record), w.T * w.H).reshape(w.T, w.H)
     return f32_to_bf16_bits(np.float32(cosine) * x0 + np.float32(math.sqrt(1.0 - cosine * cosine)) * e)
+
+
+def reference_step_input(w: Workload, s: int, episode: int = 0, cosine: float = 0.95) -> np.ndarray:
+    """Step s of a 'similar earlier execution' as bf16 bits [T,H]: cosine * X_s + sqrt(1-cosine^2) * E_s, X_s the
+    episode's own step input (before rounding the mixture)."""
+    xs = bf16_bits_to_f32(step_input(w, s, episode))
+    e = normal(tensor_key(w.seed, w.config, 0, ROLE_REF_NOISE, episode * 64 + 32 + s), w.T * w.H).reshape(w.T, w.H)
+    return f32_to_bf16_bits(np.float32(cosine) * xs + np.float32(math.sqrt(1.0 - cosine * cosine)) * e)
+
+
+def output_gate(w: Workload, s: int = 0, episode: int = 0) -> np.ndarray:
+    """Per-layer, per-channel output gate [L,H] fp32 of denoising step s: 1 + 0.25 * standard normal (the adaptive
+    gate depends on the step's time conditioning, so every step draws its own)."""
+    g = normal(tensor_key(w.seed, w.config, s, ROLE_GATE, episode), w.L * w.H).reshape(w.L, w.H)
+    return (np.float32(1.0) + np.float32(0.25) * g).astype(np.float32)
 
 
 def residual_input(w: Workload, episode: int = 0) -> np.ndarray:

@@ -257,3 +257,59 @@ def test_config2_large_refresh_every_two_steps(lib):
         assert model.ctx.rm_device_status() == 0, f"cold-cache repetition {rep}"
         assert_close(got, want, f"config 2 cold-cache sparse step, repetition {rep}")
     model.close()
+
+
+# ------------------------------------------------------------------------------------------------ config 5
+def test_config5_anchor_groups_of_five_steps(lib, pi0):
+    """The Action Cache schedule (Sec. 4.1): steps 0 and 5 are dense anchors that retain y_a and h_a, steps 1-4 and
+    6-9 apply Eq. 4 on their group's shared mask, every step passes through its own output gate.  The group masks
+    come from a similar earlier execution (Sec. 5): per-step top-K, union within the group, ranked by summed
+    contribution, top K kept -- built on the GPU from the GPU's records and checked against the oracle's
+    construction on the same bytes."""
+    import torch
+    model, _, _ = pi0
+    w = wl.config5()
+    L, T, H, I, K, G = w.L, w.T, w.H, w.I, w.K, w.extra["group"]
+    assert (K, G, w.steps) == (2048, 5, 10)
+    ctx = model.ctx
+    # reference execution: ten dense steps, one record per step and layer
+    recs = []
+    for s in range(w.steps):
+        _, rec = gpu_dense_records(model, f32_of(wl.reference_step_input(w, s))[None])
+        recs.append(rec.view(L, I))
+    groups = []
+    for g in range(w.steps // G):
+        idx = torch.zeros(L, I, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros(L, dtype=torch.int32, device="cuda")
+        members = recs[g * G:(g + 1) * G]
+        ctx.rm_mask_compact(members, lib.RM_SRC_SCORE_F32, lib.RM_REDUCE_GROUP, idx, cnt, I, n_lists=L, k=K)
+        h_idx, h_cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        host = [m.cpu().numpy() for m in members]
+        for l in range(L):
+            want = oracle.compact_group([m[l] for m in host], K)
+            assert h_cnt[l] == K and np.array_equal(h_idx[l, :K], want), f"group {g} layer {l}: mask differs"
+        groups.append((idx, cnt, h_idx, h_cnt))
+    # the current execution
+    h_stride = 52
+    y_an = torch.zeros(L, 1, T, H, dtype=torch.float32, device="cuda")
+    h_an = torch.zeros(L, 1, I, h_stride, dtype=torch.float32, device="cuda")
+    out = torch.empty(1, T, H, dtype=torch.float32, device="cuda")
+    state = None
+    rels = []
+    for s in range(w.steps):
+        r0 = f32_of(wl.step_input(w, s))
+        gate = wl.output_gate(w, s)                                   # [L,H]
+        d_gate = dev(gate[:, None, :])
+        if s % G == 0:
+            ctx.rm_action_expert_step_ex(model.packed, dev(r0[None]), None, None, 0, out, lib.RM_ANCHOR_WRITE, y_an, h_an,
+                                         h_stride, out_gate=d_gate, B=1, T=T)
+            want, y_a, h_a, _ = oracle.anchor_step_write(model.Wg, model.Wu, model.Wd, r0, gate)
+            state = (y_a, h_a)
+        else:
+            idx, cnt, h_idx, h_cnt = groups[s // G]
+            ctx.rm_action_expert_step_ex(model.packed, dev(r0[None]), idx, cnt, I, out, lib.RM_ANCHOR_UPDATE, y_an, h_an,
+                                         h_stride, out_gate=d_gate, B=1, T=T)
+            want = oracle.anchor_step_update(model.Wg, model.Wu, model.Wd, r0, h_idx, h_cnt, state[0], state[1], gate)
+        rels.append(assert_close(out.cpu().numpy()[0], want, f"config 5 step {s}"))
+    print(f"config5: rel_l2 per step max {max(rels):.2e}")
+    assert ctx.rm_device_status() == 0

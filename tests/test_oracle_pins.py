@@ -366,6 +366,73 @@ def test_eq4_special_cases():
     assert np.max(np.abs(out - want)) <= 1e-5 * np.max(np.abs(want))
 
 
+def test_eq4_output_gate():
+    """out = r + gate * y_hat: no gate == unit gate, zero gate returns r, and the gated increment is the ungated
+    increment scaled per channel (a brute-force y_hat from library matmuls pins the placement of the gate: it
+    multiplies the anchor output and the delta, not the residual)."""
+    x, Wg, Wu, Wd, r = small_problem(23)
+    xa = bf(wl.bf16_bits_to_f32(x) * 0.8 + 0.2 * wl.normal(wl.tensor_key(23, 99, 1, 1), x.size).reshape(x.shape))
+    H = x.shape[1]
+    idx = np.array([0, 3, 4, 17, 40], dtype=np.int32)
+    y_a, h_a = oracle.dense_mlp(xa, Wg, Wu, Wd, None, return_h=True)
+    gate = (0.5 + wl.uniform(wl.tensor_key(23, 99, 2, 2), H) * 1.5).astype(np.float32)
+    plain = oracle.anchor_mlp(x, Wg, Wu, Wd, r, idx, y_a, h_a[:, idx])
+    assert np.array_equal(oracle.anchor_mlp(x, Wg, Wu, Wd, r, idx, y_a, h_a[:, idx], np.ones(H, np.float32)), plain)
+    assert np.array_equal(oracle.anchor_mlp(x, Wg, Wu, Wd, r, idx, y_a, h_a[:, idx], np.zeros(H, np.float32)), r)
+    gated = oracle.anchor_mlp(x, Wg, Wu, Wd, r, idx, y_a, h_a[:, idx], gate)
+    _, h_t = oracle.dense_mlp(x, Wg, Wu, Wd, None, return_h=True)
+    Wd_f = wl.bf16_bits_to_f32(Wd).astype(np.float64)
+    y_hat = y_a.astype(np.float64) + (h_t[:, idx].astype(np.float64) - h_a[:, idx]) @ Wd_f[:, idx].T
+    want = r + gate[None, :].astype(np.float64) * y_hat
+    assert np.max(np.abs(gated - want)) <= 1e-5 * np.max(np.abs(want))
+    # a gate on the residual instead (a plausible slip) would differ visibly
+    assert np.max(np.abs(gated - gate[None, :] * (r + y_hat))) > 1e-2
+
+
+def test_anchor_steps_over_a_stack():
+    """Write then update through L layers: an update on the anchor's own input reproduces the anchor step bit for
+    bit whatever the masks; with every neuron in the mask the update equals the dense step of the new input; with
+    zero anchors and no gate it is the zero-fill masked step."""
+    L, T, H, I = 3, 5, 32, 64
+    W = [small_problem(50 + l, T=T, H=H, I=I, sigma=0.2)[1:4] for l in range(L)]
+    Wg, Wu, Wd = zip(*W)
+    r_a = wl.normal(wl.tensor_key(50, 99, 0, 7), T * H).reshape(T, H)
+    r_t = (r_a + 0.3 * wl.normal(wl.tensor_key(50, 99, 0, 8), T * H).reshape(T, H)).astype(np.float32)
+    gate = (0.5 + wl.uniform(wl.tensor_key(50, 99, 0, 9), L * H).reshape(L, H)).astype(np.float32)
+    idx = np.zeros((L, I), np.int32)
+    cnt = np.zeros(L, np.int32)
+    for l in range(L):
+        sel = np.flatnonzero(wl.uniform(wl.tensor_key(50, 99, l, 10), I) < 0.4).astype(np.int32)
+        idx[l, :sel.size] = sel
+        cnt[l] = sel.size
+    out_a, y_a, h_a, rec = oracle.anchor_step_write(Wg, Wu, Wd, r_a, gate)
+    assert y_a.shape == (L, T, H) and h_a.shape == (L, T, I) and rec.shape == (L, I)
+    assert np.allclose(rec, np.abs(h_a).sum(axis=1), rtol=1e-6, atol=1e-6)
+    # unit gate: the anchor step is the plain dense step
+    out_plain, _, _, _ = oracle.anchor_step_write(Wg, Wu, Wd, r_a, None)
+    assert np.allclose(out_plain, oracle.step(Wg, Wu, Wd, r_a), rtol=1e-6, atol=1e-6)
+    # same input: nothing changes
+    assert np.array_equal(oracle.anchor_step_update(Wg, Wu, Wd, r_a, idx, cnt, y_a, h_a, gate), out_a)
+    # every neuron selected: the dense gated step of the new input
+    full = np.tile(np.arange(I, dtype=np.int32), (L, 1))
+    got = oracle.anchor_step_update(Wg, Wu, Wd, r_t, full, np.full(L, I, np.int32), y_a, h_a, gate)
+    want, _, _, _ = oracle.anchor_step_write(Wg, Wu, Wd, r_t, gate)
+    assert np.max(np.abs(got - want)) <= 2e-5 * np.max(np.abs(want))
+    # zero anchors, no gate: zero-fill
+    got = oracle.anchor_step_update(Wg, Wu, Wd, r_t, idx, cnt, np.zeros_like(y_a), np.zeros_like(h_a))
+    want = oracle.step(Wg, Wu, Wd, r_t, idx, cnt)
+    assert np.max(np.abs(got - want)) <= 2e-6 * np.max(np.abs(want))
+    # a partial mask really keeps the anchor's contribution of the other neurons: layer 0 by hand
+    x0 = oracle.rmsnorm_bf16(r_t)
+    _, h_t = oracle.dense_mlp(x0, Wg[0], Wu[0], Wd[0], None, return_h=True)
+    hm = h_a[0].astype(np.float64).copy()
+    M = idx[0, :cnt[0]]
+    hm[:, M] = h_t[:, M]
+    want0 = r_t + gate[0][None, :].astype(np.float64) * (hm @ wl.bf16_bits_to_f32(Wd[0]).astype(np.float64).T)
+    one = oracle.anchor_step_update(Wg[:1], Wu[:1], Wd[:1], r_t, idx[:1], cnt[:1], y_a[:1], h_a[:1], gate[:1])
+    assert np.max(np.abs(one - want0)) <= 1e-5 * np.max(np.abs(want0))
+
+
 def test_step_is_the_composition_of_layers():
     L, T, H, I = 3, 4, 32, 64
     W = [small_problem(20 + l, T=T, H=H, I=I, sigma=0.2)[1:4] for l in range(L)]
