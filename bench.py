@@ -51,6 +51,8 @@ def pick_workload(name: str) -> wl.Workload:
         return wl.config2()
     if name == "config4":
         return wl.config4()
+    if name == "config5":
+        return wl.config5()
     if name.startswith("config3"):
         parts = name.split(":")
         rho = float(parts[1]) if len(parts) > 1 else 0.25
@@ -234,15 +236,53 @@ def run_gpu(args, w: wl.Workload):
     n_lists = B * w.L
     rec_flat = records.view(n_lists, w.I)
 
-    # reference pass (dense, emits the activation records), then the masks
-    ctx.rm_action_expert_step(packed, refs, None, None, 0, r_out, records_out=records, B=B, T=w.T)
+    anchored = "group" in w.extra                 # the anchor schedule of Eq. 4 (dense anchor, then masked updates)
+    if not anchored:
+        # reference pass (dense, emits the activation records), then the masks
+        ctx.rm_action_expert_step(packed, refs, None, None, 0, r_out, records_out=records, B=B, T=w.T)
 
-    def compact():
-        ctx.rm_mask_compact([rec_flat], rm.RM_SRC_SCORE_F32, rm.RM_REDUCE_TOPK, idx, cnt, w.I, n_lists=n_lists, k=w.K)
+        def compact():
+            ctx.rm_mask_compact([rec_flat], rm.RM_SRC_SCORE_F32, rm.RM_REDUCE_TOPK, idx, cnt, w.I, n_lists=n_lists, k=w.K)
+    else:
+        # reference execution of all steps (one record per step), group masks by the group reduce (Sec. 5), anchor
+        # state buffers and one output gate per step
+        G = w.extra["group"]
+        n_groups = w.steps // G
+        step_recs = []
+        for s in range(w.steps):
+            ref_s = torch.stack([f32(wl.reference_step_input(w, s, episode=ep0 + b)) for b in range(B)]).cuda()
+            rec_s = torch.zeros(B, w.L, w.I, dtype=torch.float32, device="cuda")
+            ctx.rm_action_expert_step(packed, ref_s, None, None, 0, r_out, records_out=rec_s, B=B, T=w.T)
+            step_recs.append(rec_s.view(n_lists, w.I))
+        g_idx = [torch.zeros(n_lists, w.I, dtype=torch.int32, device="cuda") for _ in range(n_groups)]
+        g_cnt = [torch.zeros(n_lists, dtype=torch.int32, device="cuda") for _ in range(n_groups)]
+        idx, cnt = g_idx[0], g_cnt[0]
+        h_stride = (w.T + 3) // 4 * 4
+        y_an = torch.zeros(w.L, B, w.T, w.H, dtype=torch.float32, device="cuda")
+        h_an = torch.zeros(w.L, B, w.I, h_stride, dtype=torch.float32, device="cuda")
+        gates = [torch.stack([torch.from_numpy(wl.output_gate(w, s, episode=ep0 + b)) for b in range(B)], dim=1)
+                 .contiguous().cuda() for s in range(w.steps)]                      # [L,B,H] per step
+
+        def compact():
+            for g in range(n_groups):
+                ctx.rm_mask_compact(step_recs[g * G:(g + 1) * G], rm.RM_SRC_SCORE_F32, rm.RM_REDUCE_GROUP, g_idx[g],
+                                    g_cnt[g], w.I, n_lists=n_lists, k=w.K)
 
     compact()
     torch.cuda.synchronize()
     K_mean = float(cnt.float().mean().item())
+
+    def run_step(s, r_in):
+        """One denoising step of the workload on device-resident input."""
+        ss = s % w.steps
+        if not anchored:
+            ctx.rm_action_expert_step(packed, r_in, idx, cnt, w.I, r_out, B=B, T=w.T)
+        elif ss % G == 0:
+            ctx.rm_action_expert_step_ex(packed, r_in, None, None, 0, r_out, rm.RM_ANCHOR_WRITE, y_an, h_an, h_stride,
+                                         out_gate=gates[ss], B=B, T=w.T)
+        else:
+            ctx.rm_action_expert_step_ex(packed, r_in, g_idx[ss // G], g_cnt[ss // G], w.I, r_out, rm.RM_ANCHOR_UPDATE,
+                                         y_an, h_an, h_stride, out_gate=gates[ss], B=B, T=w.T)
 
     flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
@@ -253,7 +293,7 @@ def run_gpu(args, w: wl.Workload):
             timed_events[0].record(stream)
         if s % w.steps == 0:
             compact()
-        ctx.rm_action_expert_step(packed, dev_inputs[s % w.steps], idx, cnt, w.I, r_out, B=B, T=w.T)
+        run_step(s, dev_inputs[s % w.steps])
         if timed_events is not None:
             timed_events[1].record(stream)
 
@@ -284,13 +324,21 @@ def run_gpu(args, w: wl.Workload):
     step_ms = [a.elapsed_time(b) for a, b in events]
     total_ms = float(sum(step_ms))
 
+    e2e_in = torch.empty(B, w.T, w.H, dtype=torch.float32, device="cuda")
     # end to end through the host-buffer entry point (H2D of the step input, step, D2H of the result, sync)
     e2e_times = []
     for s in range(args.warmup + args.steps):
         flush.fill_(s & 0xFF)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        ctx.rm_action_expert_step_host(packed, pinned_in[s % w.steps], idx, cnt, w.I, pinned_out, B=B, T=w.T)
+        if not anchored:
+            ctx.rm_action_expert_step_host(packed, pinned_in[s % w.steps], idx, cnt, w.I, pinned_out, B=B, T=w.T)
+        else:
+            # the anchored step has no host-buffer entry point: the same three stages through the binding
+            e2e_in.copy_(pinned_in[s % w.steps], non_blocking=True)
+            run_step(s, e2e_in)
+            pinned_out.copy_(r_out, non_blocking=True)
+            torch.cuda.synchronize()
         dt = time.perf_counter() - t0
         if s >= args.warmup:
             e2e_times.append(dt)
@@ -322,20 +370,28 @@ def run_gpu(args, w: wl.Workload):
         us_per_step = job_us_per_step(total_ms, args.steps, world, B)   # per denoising step of one episode, whole job
         e2e_us = job_us_per_step(e2e_total_ms, args.steps, world, B)
         peak, peak_kind = measured_hbm_peak()
-        bytes_layer = wl.algorithmic_bytes_per_layer(w.H, w.T, int(round(K_mean))) * B
+        if anchored:
+            # average layer launch of the schedule: one dense anchor and G-1 masked updates per group
+            bytes_layer = (wl.algorithmic_bytes_per_anchor_layer(w.H, w.T, w.I) +
+                           (G - 1) * wl.algorithmic_bytes_per_update_layer(w.H, w.T, int(round(K_mean)))) // G * B
+        else:
+            bytes_layer = wl.algorithmic_bytes_per_layer(w.H, w.T, int(round(K_mean))) * B
         bytes_step = bytes_layer * w.L
         launches_per_step = launches / args.steps                 # fused layer launches + mask compaction share
         in_step_layer_us = us_per_step * B / w.L                  # average duration of a layer launch inside the step
         achieved = bytes_layer / (in_step_layer_us * 1e-6) / 1e9
         io_bytes = B * w.T * w.H * 4
-        cpu_us, cores, sample = (time_oracle(w, steps=3, warmup=1) if world == 1 and not args.no_cpu_baseline
+        cpu_us, cores, sample = (time_oracle(w, steps=3, warmup=1) if world == 1 and not args.no_cpu_baseline and not anchored
                                  else (None, None, None))
         line = {
             "metric": METRIC, "value": us_per_step, "unit": "us", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (fp32 accumulate)", "data": "synthetic",
             "config": {"workload": w.name, "L": w.L, "H": w.H, "I": w.I, "T": w.T, "B": B,
-                       "K_per_layer": K_mean, "mask": "top-k of dense reference records, rebuilt every 10 steps",
+                       "K_per_layer": K_mean,
+                       "mask": ("group masks (union of per-step top-k, ranked by summed score) of a reference execution, "
+                                "rebuilt every 10 steps; schedule: dense anchor step, then 4 update steps (Eq. 4), gated"
+                                if anchored else "top-k of dense reference records, rebuilt every 10 steps"),
                        "l2": "flushed before every timed step (512 MB fill, outside the timed interval)",
                        "multi_gpu": "replicas: each rank runs its own episodes, no collective on the data path"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

@@ -265,5 +265,17 @@ def algorithmic_bytes_per_layer(H: int, T: int, K: int) -> int:
     return K * 3 * H * 2 + T * H * 2 + 2 * T * H * 4 + 4 * K
 
 
+def algorithmic_bytes_per_anchor_layer(H: int, T: int, I: int) -> int:
+    """Dense anchor layer (Eq. 4 bookkeeping): every weight, x, residual in/out, plus the retained state it writes:
+    h_a [I,T] and y_a [T,H] in fp32, and the gate [H]."""
+    return I * 3 * H * 2 + T * H * 2 + 2 * T * H * 4 + I * T * 4 + T * H * 4 + H * 4
+
+
+def algorithmic_bytes_per_update_layer(H: int, T: int, K: int) -> int:
+    """Masked update layer (Eq. 4): the masked layer's bytes plus the anchor state it reads: h_a on the mask
+    [K,T] and y_a [T,H] in fp32, and the gate [H]."""
+    return algorithmic_bytes_per_layer(H, T, K) + K * T * 4 + T * H * 4 + H * 4
+
+
 def algorithmic_flops_per_layer(H: int, T: int, K: int) -> int:
     return 2 * T * K * 3 * H
