@@ -241,8 +241,17 @@ def run_gpu(args, w: wl.Workload):
         # reference pass (dense, emits the activation records), then the masks
         ctx.rm_action_expert_step(packed, refs, None, None, 0, r_out, records_out=records, B=B, T=w.T)
 
+        compact_layers = None
+        if args.gather_once:
+            if B != 1:
+                raise SystemExit("--gather-once: compact layers are shared by the batch, so B must be 1")
+            compact_layers = [torch.empty(ctx.packed_layer_bytes(), dtype=torch.uint8, device="cuda") for _ in range(w.L)]
+
         def compact():
             ctx.rm_mask_compact([rec_flat], rm.RM_SRC_SCORE_F32, rm.RM_REDUCE_TOPK, idx, cnt, w.I, n_lists=n_lists, k=w.K)
+            if compact_layers is not None:
+                for l in range(w.L):
+                    ctx.rm_gather_weights(packed[l], idx[l], cnt[l:l + 1], w.I, compact_layers[l])
     else:
         # reference execution of all steps (one record per step), group masks by the group reduce (Sec. 5), anchor
         # state buffers and one output gate per step
@@ -276,7 +285,10 @@ def run_gpu(args, w: wl.Workload):
         """One denoising step of the workload on device-resident input."""
         ss = s % w.steps
         if not anchored:
-            ctx.rm_action_expert_step(packed, r_in, idx, cnt, w.I, r_out, B=B, T=w.T)
+            if compact_layers is not None:
+                ctx.rm_action_expert_step(compact_layers, r_in, None, cnt, 0, r_out, B=B, T=w.T)
+            else:
+                ctx.rm_action_expert_step(packed, r_in, idx, cnt, w.I, r_out, B=B, T=w.T)
         elif ss % G == 0:
             ctx.rm_action_expert_step_ex(packed, r_in, None, None, 0, r_out, rm.RM_ANCHOR_WRITE, y_an, h_an, h_stride,
                                          out_gate=gates[ss], B=B, T=w.T)
@@ -391,7 +403,8 @@ def run_gpu(args, w: wl.Workload):
                        "K_per_layer": K_mean,
                        "mask": ("group masks (union of per-step top-k, ranked by summed score) of a reference execution, "
                                 "rebuilt every 10 steps; schedule: dense anchor step, then 4 update steps (Eq. 4), gated"
-                                if anchored else "top-k of dense reference records, rebuilt every 10 steps"),
+                                if anchored else "top-k of dense reference records, rebuilt every 10 steps"
+                                + (", rows copied to compact layers at every rebuild (gather-once)" if args.gather_once else "")),
                        "l2": "flushed before every timed step (512 MB fill, outside the timed interval)",
                        "multi_gpu": "replicas: each rank runs its own episodes, no collective on the data path"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -422,6 +435,9 @@ def main():
     ap.add_argument("--device-weights", action="store_true",
                     help="draw the weights on the device with a seeded torch generator instead of the host generator")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--gather-once", action="store_true",
+                    help="the paper's preparation of the weights: copy the masked rows into compact layers when the "
+                         "masks are rebuilt (inside the timed region), then run the steps on the compact layers")
     ap.add_argument("--variant", type=int, default=0,
                     help="kernel variant override (library option \"variant\": 0 = chosen per launch)")
     ap.add_argument("--max-clusters", type=int, default=0, help="library option \"max_clusters\" (0 = default)")

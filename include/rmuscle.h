@@ -100,12 +100,24 @@ typedef struct {
 int rm_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out, int64_t stride,
                     rm_stream_t stream);
 
+/* ---- rm_gather_weights: the paper's own preparation of the selected weights (Sec. 4.1: "Selected weights are
+ * prepared in shared compact buffers and reused across each group's steps"; Sec. 5 "Overlapping Retrieval and Weight
+ * Gathering"), as a comparison variant to gathering inside the products.  Copies the packed rows of the listed
+ * neurons to the front of compact_out: compact row p = packed row idx[p] for p < count.  compact_out holds at least
+ * min(list_cap, I) rows of 3*H bf16 (rm_packed_layer_bytes is always enough) and is itself a packed layer: pass it to
+ * rm_sparse_mlp / rm_action_expert_step with idx = NULL and the same count_dev ("the leading count neurons"), and the
+ * result is the masked layer over the listed neurons.  Activation records and anchor activations of such a call are
+ * indexed by compact position.  Call it on a side stream to overlap it with other work; ordering is the caller's. */
+int rm_gather_weights(rm_ctx* ctx, const void* packed_layer, const int32_t* idx, const int32_t* count_dev,
+                      int64_t list_cap, void* compact_out, rm_stream_t stream);
+
 /* ---- rm_sparse_mlp: one layer, zero-fill form of the masked evaluation (Sec. 4.1: "compute only the selected
  * neurons' hidden activations and update the output using their down-projection weights"):
  *     y[t,:] = residual[t,:] + sum_{n in S} gelu_tanh(<x_t, Wg_n>) * <x_t, Wu_n> * Wd[:,n]
  *   packed_layer: output of rm_pack_weights.   x [T,H] bf16.   residual [T,H] fp32, nullable (=> 0).
- *   idx [>= count] int32 ascending, nullable => every neuron (dense);  count_dev [1] int32 on the device
- *   (ignored when idx is NULL).   y [T,H] fp32; may equal residual (in place).
+ *   idx [>= count] int32 ascending, nullable => every neuron (dense);  count_dev [1] int32 on the device.
+ *   idx NULL with count_dev given: the leading count neurons of the layer (a compact layer from rm_gather_weights).
+ *   y [T,H] fp32; may equal residual (in place).
  *   record_out (nullable) [I] fp32: dense mode only; receives A[n] = sum_t |h[t,n]| (* record_scale[n] when
  *   record_scale is given) -- the activation part of Eq. 1, or Eq. 1 itself with record_scale = down_colnorm.
  *   ws / ws_bytes: scratch of at least rm_workspace_bytes(ctx, 1, T). */
@@ -118,7 +130,8 @@ int rm_sparse_mlp(rm_ctx* ctx, const void* packed_layer, const void* x, const fl
  *     r_0 = r_in;  x_l = bf16(r_l / sqrt(mean_k r_l[t,k]^2 + 1e-6));  r_{l+1} = r_l + MLP_l(x_l; S_l);  r_out = r_L
  *   The residual stream stays fp32.  Attention, conditioning and the adaptive gate are not part of this path.
  *   packed_layers: HOST array of L device pointers.   r_in, r_out [B,T,H] fp32 (r_out may equal r_in).
- *   idx [B,L,stride] int32, nullable => dense;  count_dev [B,L] int32 (device).
+ *   idx [B,L,stride] int32, nullable => dense;  count_dev [B,L] int32 (device); idx NULL with count_dev given:
+ *   layer l of episode b uses the leading count_dev[b,l] neurons of packed_layers[l] (compact layers).
  *   records_out (nullable, dense only) [B,L,I] fp32;  record_scale (nullable) [L,I] fp32. */
 int rm_action_expert_step(rm_ctx* ctx, const void* const* packed_layers, const float* r_in, const int32_t* idx,
                           const int32_t* count_dev, int64_t stride, float* r_out, float* records_out,

@@ -23,7 +23,7 @@ RM_ANCHOR_NONE, RM_ANCHOR_WRITE, RM_ANCHOR_UPDATE = 0, 1, 2
 
 EXPORTS = ["rm_create", "rm_destroy", "rm_packed_layer_bytes", "rm_workspace_bytes", "rm_pack_weights",
            "rm_mask_compact", "rm_sparse_mlp", "rm_action_expert_step", "rm_action_expert_step_host",
-           "rm_action_expert_step_ex",
+           "rm_action_expert_step_ex", "rm_gather_weights",
            "rm_device_status", "rm_launch_count", "rm_status_string", "rm_set_option", "rm_get_info",
            "rm_debug_phase_times", "rm_sparse_mlp_static"]
 
@@ -75,6 +75,7 @@ def load_library() -> ctypes.CDLL:
     lib.rm_sparse_mlp.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
     lib.rm_action_expert_step.argtypes = [vp, ctypes.POINTER(vp), vp, vp, vp, i64, vp, vp, vp, i32, i32, vp, sz, vp]
     lib.rm_action_expert_step_host.argtypes = [vp, ctypes.POINTER(vp), vp, vp, vp, i64, vp, i32, i32, vp, sz, vp]
+    lib.rm_gather_weights.argtypes = [vp, vp, vp, vp, i64, vp, vp]
     lib.rm_action_expert_step_ex.argtypes = [vp, ctypes.POINTER(vp), vp, vp, vp, i64, vp, vp, vp, i32, i32, i32, vp, vp,
                                              i64, vp, vp, sz, vp]
     lib.rm_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
@@ -197,6 +198,15 @@ class Context:
                           int(n_lists), self.I)
         _check(self.lib.rm_mask_compact(self._h, ctypes.byref(src), _ptr(idx_out), _ptr(count_out), int(stride),
                                         _stream()), "rm_mask_compact")
+
+    def rm_gather_weights(self, packed_layer, idx, count_dev, list_cap: int, compact_out=None):
+        """Compact copy of the listed neurons' packed rows (a packed layer whose leading `count` neurons are the list)."""
+        import torch
+        if compact_out is None:
+            compact_out = torch.empty(self.packed_layer_bytes(), dtype=torch.uint8, device="cuda")
+        _check(self.lib.rm_gather_weights(self._h, _ptr(packed_layer), _ptr(idx), _ptr(count_dev), int(list_cap),
+                                          _ptr(compact_out), _stream()), "rm_gather_weights")
+        return compact_out
 
     def rm_sparse_mlp(self, packed_layer, x, residual, idx, count_dev, y, record_out=None, record_scale=None,
                       T: Optional[int] = None, ws=None):

@@ -91,6 +91,15 @@ int rm_pack_weights(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd,
     return rm_launch_pack(ctx, Wg, Wu, Wd, packed_out, down_colnorm, static_cast<cudaStream_t>(stream));
 }
 
+int rm_gather_weights(rm_ctx* ctx, const void* packed_layer, const int32_t* idx, const int32_t* count_dev,
+                      int64_t list_cap, void* compact_out, rm_stream_t stream) {
+    if (!ctx || !packed_layer || !idx || !count_dev || !compact_out || list_cap < 0) return RM_ERR_INVALID_ARG;
+    if (!all_aligned({packed_layer, idx, compact_out})) return RM_ERR_ALIGN;
+    if (compact_out == packed_layer) return RM_ERR_INVALID_ARG;
+    return rm_launch_gather_rows(ctx, packed_layer, idx, count_dev, list_cap, compact_out,
+                                 static_cast<cudaStream_t>(stream));
+}
+
 int rm_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out, int64_t stride,
                     rm_stream_t stream) {
     if (!ctx || !src || !idx_out || !count_out || !src->records) return RM_ERR_INVALID_ARG;
@@ -197,9 +206,9 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
         a.x = nullptr;
         a.r_in = cur;
         a.idx = idx ? idx + (size_t)l * stride : nullptr;
-        a.count = idx ? count_dev + l : nullptr;
+        a.count = count_dev ? count_dev + l : nullptr;
         a.idx_stride = (int64_t)g.L * stride;
-        a.list_cap = stride;
+        a.list_cap = idx ? stride : g.I;
         a.count_stride = g.L;
         a.record = records_out ? records_out + (size_t)l * g.I : nullptr;
         a.record_stride = (int64_t)g.L * g.I;

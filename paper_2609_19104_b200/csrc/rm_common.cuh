@@ -74,6 +74,8 @@ __device__ __forceinline__ float rm_gelu_tanh(float g) {
 // ---- kernels implemented in the other translation units (host launchers)
 int rm_launch_pack(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, void* packed, float* colnorm,
                    cudaStream_t s);
+int rm_launch_gather_rows(rm_ctx* ctx, const void* packed, const int32_t* idx, const int32_t* count, int64_t cap,
+                          void* out, cudaStream_t s);
 int rm_launch_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out,
                            int64_t stride, cudaStream_t s);
 

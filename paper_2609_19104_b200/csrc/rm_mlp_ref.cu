@@ -14,7 +14,7 @@ constexpr int DN_TOK = 8;          // tokens per CTA in the down kernel
 constexpr int DN_CHUNK = 64;       // neurons staged per iteration
 
 __device__ __forceinline__ int clamp_count(const rm_layer_args& a, int b, const rm_geom& g, int* status) {
-    if (!a.idx) return g.I;
+    if (!a.count) return g.I;          // a count without a list: the leading `count` neurons (compact layer)
     int c = a.count[(size_t)b * a.count_stride];
     int cap = (int)(a.list_cap < (int64_t)g.I ? a.list_cap : (int64_t)g.I);
     if (c < 0 || c > cap) {
@@ -200,7 +200,7 @@ int rm_launch_layer_ref(rm_ctx* ctx, const rm_layer_args& a, void* ws, cudaStrea
     size_t smem = (size_t)GU_WARPS * 2 * g.H * sizeof(__nv_bfloat16);
     if (smem > 48 * 1024)
         RM_CUDA_TRY(cudaFuncSetAttribute(ref_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int kcap = a.idx ? (int)(a.list_cap < (int64_t)g.I ? a.list_cap : (int64_t)g.I) : g.I;
+    int kcap = a.count ? (int)(a.list_cap < (int64_t)g.I ? a.list_cap : (int64_t)g.I) : g.I;
     dim3 g1((kcap + GU_WARPS - 1) / GU_WARPS, a.B);
     ref_gateup_kernel<<<g1, GU_WARPS * 32, smem, s>>>(a, g, x, h, ctx->d_status);
     ctx->launches++;
@@ -273,7 +273,7 @@ extern "C" int rm_sparse_mlp_static(const void* packed_layer, const void* x, con
     a.r_in = residual;
     a.r_out = y;
     a.idx = idx;
-    a.count = count_dev;
+    a.count = idx ? count_dev : nullptr;
     a.idx_stride = I;
     a.list_cap = I;
     a.count_stride = 1;

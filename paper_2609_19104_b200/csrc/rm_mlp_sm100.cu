@@ -197,7 +197,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
         const int cap = (int)(a.list_cap < (int64_t)a.I ? a.list_cap : (int64_t)a.I);
         for (int b = 0; b < a.B; ++b) {
             int c = a.I;                   // dense: every neuron
-            if (a.idx) {
+            if (a.count) {                 // a list, or (no list) the leading `count` neurons of a compact layer
                 c = a.count[(size_t)b * a.count_stride];
                 if (c < 0 || c > cap) { rm_set_status(a.status, RM_ERR_INDEX); c = c < 0 ? 0 : cap; }
             }
@@ -818,7 +818,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
         const int cap = (int)(a.list_cap < (int64_t)a.I ? a.list_cap : (int64_t)a.I);
         for (int b = 0; b < a.B; ++b) {
             int c = a.I;
-            if (a.idx) {
+            if (a.count) {                 // a list, or (no list) the leading `count` neurons of a compact layer
                 c = a.count[(size_t)b * a.count_stride];
                 if (c < 0 || c > cap) { rm_set_status(a.status, RM_ERR_INDEX); c = c < 0 ? 0 : cap; }
             }
@@ -1497,7 +1497,7 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
     a.gate = la.gate;
     // Tiles of 64 neurons in this launch, when the host knows the number of active neurons (dense calls, or the
     // caller's hint); 0 = unknown.
-    const int per_episode = la.idx ? ctx->count_hint : ctx->g.I;
+    const int per_episode = la.count ? ctx->count_hint : ctx->g.I;
     const long long tiles = per_episode > 0 ? (long long)((per_episode + NT - 1) / NT) * la.B : 0;
     // Variant.  H = 1024: the lean kernel for every launch (112 KB and 107 registers: two CTAs per SM, so a cluster's
     // exchange waits are covered by its SM-mate and consecutive layers overlap); measured, 33 of its clusters are

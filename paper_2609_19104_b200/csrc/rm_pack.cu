@@ -50,7 +50,42 @@ __global__ void __launch_bounds__(256) colnorm_kernel(const __nv_bfloat16* __res
     out[n] = sqrtf(s);
 }
 
+// Compact copy of the listed neurons' packed rows: out row p = packed row idx[p], p < count.  One warp per row
+// (3H bf16, contiguous in both buffers), 16 bytes per lane and iteration.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ packed, const int32_t* __restrict__ idx,
+                                                          const int32_t* __restrict__ count, int64_t cap,
+                                                          uint4* __restrict__ out, int row_u4, int I, int* status) {
+    const int p = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    int c = *count;
+    if (c < 0 || c > cap || c > I) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) rm_set_status(status, RM_ERR_INDEX);
+        c = c < 0 ? 0 : (int)(cap < (int64_t)I ? cap : (int64_t)I);
+    }
+    if (p >= c) return;
+    const int n = idx[p];
+    if (n < 0 || n >= I) {
+        if (lane == 0) rm_set_status(status, RM_ERR_INDEX);
+        for (int e = lane; e < row_u4; e += 32) out[(size_t)p * row_u4 + e] = make_uint4(0, 0, 0, 0);
+        return;
+    }
+    const uint4* src = packed + (size_t)n * row_u4;
+    for (int e = lane; e < row_u4; e += 32) out[(size_t)p * row_u4 + e] = src[e];
+}
+
 }  // namespace
+
+int rm_launch_gather_rows(rm_ctx* ctx, const void* packed, const int32_t* idx, const int32_t* count, int64_t cap,
+                          void* out, cudaStream_t s) {
+    const rm_geom& g = ctx->g;
+    const int row_u4 = 3 * g.H * (int)sizeof(__nv_bfloat16) / 16;
+    const int64_t rows = cap < (int64_t)g.I ? cap : (int64_t)g.I;
+    if (rows <= 0) return RM_OK;
+    gather_rows_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, s>>>(static_cast<const uint4*>(packed), idx, count, cap,
+                                                                 static_cast<uint4*>(out), row_u4, g.I, ctx->d_status);
+    ctx->launches++;
+    RM_CUDA_TRY(cudaGetLastError());
+    return RM_OK;
+}
 
 int rm_launch_pack(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, void* packed, float* colnorm,
                    cudaStream_t s) {
