@@ -90,13 +90,14 @@ struct FusedArgs {
     const float* gate;
 };
 
-// r_out[0..3] += r[0..3] (+ gate * y_anchor in an update step, Eq. 4): the residual part of a layer's output
-__device__ __forceinline__ void add_residual4(const FusedArgs& a, float* o, size_t off_bt_h, int col, int b,
-                                              float r0, float r1, float r2, float r3) {
-    if (a.anchor_mode == RM_ANCHOR_UPDATE) {
-        const float4 ya = *reinterpret_cast<const float4*>(a.y_anchor + off_bt_h + col);
+// r_out[0..3] += r[0..3] (+ gate * y_anchor in an update step, Eq. 4): the residual part of a layer's output.
+// ya_update is the layer's y_anchor in update steps, else NULL.
+__device__ __forceinline__ void add_residual4(const float* ya_update, const float* gate, int H, float* o,
+                                              size_t off_bt_h, int col, int b, float r0, float r1, float r2, float r3) {
+    if (ya_update) {
+        const float4 ya = *reinterpret_cast<const float4*>(ya_update + off_bt_h + col);
         float4 g = make_float4(1.f, 1.f, 1.f, 1.f);
-        if (a.gate) g = *reinterpret_cast<const float4*>(a.gate + (size_t)b * a.H + col);
+        if (gate) g = *reinterpret_cast<const float4*>(gate + (size_t)b * H + col);
         r0 = fmaf(g.x, ya.x, r0); r1 = fmaf(g.y, ya.y, r1); r2 = fmaf(g.z, ya.z, r2); r3 = fmaf(g.w, ya.w, r3);
     }
     red_add_v4(o, r0, r1, r2, r3);
@@ -108,6 +109,35 @@ __host__ __device__ constexpr int p_row_for(int T) { return 4 * (((T + 3) / 4) |
 
 // A wait that ran out of polls records the source line of the wait and the CTA (readable as "status_detail").
 #define wait_bar(bar, parity) wait_bar_at((bar), (parity), __LINE__)
+
+// Adds one warp's share of a CTA's [T x Hs] down-projection partial (fp32 in tensor memory, lanes = output columns)
+// to the episode's residual stream, times the output gate; the anchor step of Eq. 4 also accumulates the ungated
+// partial into y_anchor.  Pointers are already offset to the episode.  wrow: which 32-lane quarter of the accumulator
+// this warp reads; token columns c0_first, c0_first + c0_step, ...
+template <int NTOK, int HS>
+__device__ __noinline__ void flush_partial(float* __restrict__ r_out, float* __restrict__ y_anchor,
+                                           const float* __restrict__ gate, bool write_anchor, uint32_t tmem_d2, int wrow,
+                                           int lane, int c0_first, int c0_step, int T, int H, int col_base) {
+#pragma unroll
+    for (int mm = 0; mm < HS / 128; ++mm) {
+        const int col = col_base + mm * 128 + wrow * 32 + lane;
+        const float gc = gate ? gate[col] : 1.f;
+        for (int c0 = c0_first; c0 < NTOK; c0 += c0_step) {
+            float v[32];
+            tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)(wrow * 32) << 16) + c0, v);
+            // explicit red.global.add: with the gate factor in front, atomicAdd() compiled to something far slower
+            // here (measured: 60 against 37 us per H = 2048 layer)
+            if (write_anchor) {
+#pragma unroll
+                for (int k = 0; k < 32; ++k)
+                    if (c0 + k < T) red_add_f32(y_anchor + (size_t)(c0 + k) * H + col, v[k]);
+            }
+#pragma unroll
+            for (int k = 0; k < 32; ++k)
+                if (c0 + k < T) red_add_f32(r_out + (size_t)(c0 + k) * H + col, gc * v[k]);
+        }
+    }
+}
 
 template <int NTOK, int HS, bool PIPE>
 struct Smem {
@@ -150,8 +180,12 @@ struct TileRef {
     bool first, last;              // first / last tile of its episode within this cluster's run
 };
 
-template <int NTOK, int HS, bool PIPE>
+// EQ4 = false compiles the anchor-relative update and the output gate out (the zero-fill step pays nothing for them)
+template <int NTOK, int HS, bool PIPE, bool EQ4>
 __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_kernel(const FusedArgs a) {
+    const int anchor_mode = EQ4 ? a.anchor_mode : (int)RM_ANCHOR_NONE;
+    const float* const gate = EQ4 ? a.gate : nullptr;
+    const float* const ya_update = anchor_mode == RM_ANCHOR_UPDATE ? a.y_anchor : nullptr;
     using S = Smem<NTOK, HS, PIPE>;
     constexpr int NB = S::NB;
     constexpr int KB = S::KB;
@@ -299,7 +333,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             float* dst = a.r_out + (size_t)b * T * H;
             for (size_t i = (size_t)blockIdx.x * FT + tid; i < (size_t)T * H / 4; i += (size_t)gridDim.x * FT) {
                 const float4 v = src[i];
-                add_residual4(a, dst + 4 * i, (size_t)b * T * H + (4 * i / H) * H, (int)(4 * i % H), b, v.x, v.y, v.z, v.w);
+                add_residual4(ya_update, gate, H, dst + 4 * i, (size_t)b * T * H + (4 * i / H) * H, (int)(4 * i % H), b, v.x, v.y, v.z, v.w);
             }
         }
     }
@@ -381,7 +415,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
                 const int col = j * HS + part * CPP;
 #pragma unroll
                 for (int i = 0; i < CPP / 4; ++i)
-                    add_residual4(a, a.r_out + row + col + 4 * i, row, col + 4 * i, b, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    add_residual4(ya_update, gate, H, a.r_out + row + col + 4 * i, row, col + 4 * i, b, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
             }
             wait_bar(bar_s, par_s);
             par_s ^= 1;
@@ -483,7 +517,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     auto anchor_prefetch = [&](int i, const TileRef& tr, float (&ha_pre)[TPL]) {
 #pragma unroll
         for (int k = 0; k < TPL; ++k) ha_pre[k] = 0.f;
-        if (a.anchor_mode != RM_ANCHOR_UPDATE) return;
+        if (anchor_mode != RM_ANCHOR_UPDATE) return;
         const int n = gN[(i & 1) * NT + j * 8 + warp];
         const int t0 = lane * TPL;
         if (n >= 0 && t0 < T) {
@@ -520,11 +554,11 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             rec += fabsf(hv[k]);
         }
         // Eq. 4: the anchor step retains h; a later step sends its difference from the anchor's h down the projection
-        if (a.anchor_mode != RM_ANCHOR_NONE) {
+        if (anchor_mode != RM_ANCHOR_NONE) {
             const int n = gN[(i & 1) * NT + j * 8 + ql];
             if (n >= 0 && t0 < T) {
                 float* hap = a.h_anchor + ((size_t)tr.b * a.I + n) * a.h_stride + t0;
-                if (a.anchor_mode == RM_ANCHOR_WRITE) {
+                if (anchor_mode == RM_ANCHOR_WRITE) {
                     if (TPL == 2) *reinterpret_cast<float2*>(hap) = make_float2(hv[0], hv[TPL - 1]);
                     else *hap = hv[0];
                 } else {
@@ -587,24 +621,9 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
 
     // ---- phase: add this CTA's [T x Hs] partial of y to the residual stream
     auto flush = [&](const TileRef& tr) {
-#pragma unroll
-        for (int mm = 0; mm < HS / 128; ++mm) {
-            for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
-                float v[32];
-                tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)((warp & 3) * 32) << 16) + c0, v);
-                const size_t off = (size_t)tr.b * T * H + (size_t)j * HS + mm * 128 + (warp & 3) * 32 + lane;
-                float* dst = a.r_out + off;
-                const float gc = a.gate ? a.gate[(size_t)tr.b * H + j * HS + mm * 128 + (warp & 3) * 32 + lane] : 1.f;
-                if (a.anchor_mode == RM_ANCHOR_WRITE) {    // the anchor step also retains its ungated FFN output
-#pragma unroll
-                    for (int k = 0; k < 32; ++k)
-                        if (c0 + k < T) atomicAdd(a.y_anchor + off + (size_t)(c0 + k) * H, v[k]);
-                }
-#pragma unroll
-                for (int k = 0; k < 32; ++k)
-                    if (c0 + k < T) atomicAdd(dst + (size_t)(c0 + k) * H, gc * v[k]);
-            }
-        }
+        flush_partial<NTOK, HS>(a.r_out + (size_t)tr.b * T * H, a.y_anchor ? a.y_anchor + (size_t)tr.b * T * H : nullptr,
+                                gate ? gate + (size_t)tr.b * H : nullptr, anchor_mode == RM_ANCHOR_WRITE, tmem_d2,
+                                warp & 3, lane, (warp >> 2) * 32, 64, T, H, j * HS);
         tc_fence_before();
         __syncthreads();
         RM_STAMP(14);
@@ -765,8 +784,11 @@ struct SmemWS {
     static int total_bytes(int T) { return OFF_P + (STAGED ? 4 : 2) * CS * 16 * p_row_for(T) * 4 + 1024; }
 };
 
-template <int NTOK, int HS>
+template <int NTOK, int HS, bool EQ4>
 __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a) {
+    const int anchor_mode = EQ4 ? a.anchor_mode : (int)RM_ANCHOR_NONE;
+    const float* const gate = EQ4 ? a.gate : nullptr;
+    const float* const ya_update = anchor_mode == RM_ANCHOR_UPDATE ? a.y_anchor : nullptr;
     using S = SmemWS<NTOK, HS>;
     constexpr int KB = S::KB;
     extern __shared__ unsigned char smem_dyn[];
@@ -1022,7 +1044,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                     const int col = j * HS + part * CPP;
 #pragma unroll
                     for (int i = 0; i < CPP / 4; ++i)
-                        add_residual4(a, a.r_out + row + col + 4 * i, row, col + 4 * i, b, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                        add_residual4(ya_update, gate, H, a.r_out + row + col + 4 * i, row, col + 4 * i, b, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
                 }
                 wait_bar(bar_s, par_s);
                 float tot = 0.f;
@@ -1102,24 +1124,9 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 const int it = it0 + seg - 1;
                 wait_bar(bar_dn(it & 1), (it >> 1) & 1);
                 tc_fence_after();
-#pragma unroll
-                for (int mm = 0; mm < HS / 128; ++mm) {
-                    for (int c0 = 0; c0 < NTOK; c0 += 32) {
-                        float v[32];
-                        tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)(warp * 32) << 16) + c0, v);
-                        const size_t off = (size_t)b * T * H + (size_t)j * HS + mm * 128 + warp * 32 + lane;
-                        float* dst = a.r_out + off;
-                        const float gc = a.gate ? a.gate[(size_t)b * H + j * HS + mm * 128 + warp * 32 + lane] : 1.f;
-                        if (a.anchor_mode == RM_ANCHOR_WRITE) {
-#pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                if (c0 + e < T) atomicAdd(a.y_anchor + off + (size_t)(c0 + e) * H, v[e]);
-                        }
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (c0 + e < T) atomicAdd(dst + (size_t)(c0 + e) * H, gc * v[e]);
-                    }
-                }
+                flush_partial<NTOK, HS>(a.r_out + (size_t)b * T * H, a.y_anchor ? a.y_anchor + (size_t)b * T * H : nullptr,
+                                        gate ? gate + (size_t)b * H : nullptr, anchor_mode == RM_ANCHOR_WRITE, tmem_d2,
+                                        warp, lane, 0, 32, T, H, j * HS);
                 tc_fence_before();
             }
         } else if (warp < 8) {
@@ -1144,9 +1151,9 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 float ha_pre[TPL];
 #pragma unroll
                 for (int e = 0; e < TPL; ++e) ha_pre[e] = 0.f;
-                const int n_own = a.anchor_mode != RM_ANCHOR_NONE ? gN[(it & 7) * NT + j * 8 + ql] : -1;
+                const int n_own = anchor_mode != RM_ANCHOR_NONE ? gN[(it & 7) * NT + j * 8 + ql] : -1;
                 float* hap = (n_own >= 0 && t0 < T) ? a.h_anchor + ((size_t)b * a.I + n_own) * a.h_stride + t0 : nullptr;
-                if (a.anchor_mode == RM_ANCHOR_UPDATE && hap) {
+                if (anchor_mode == RM_ANCHOR_UPDATE && hap) {
                     if (TPL == 4) {
                         const float4 f = *reinterpret_cast<const float4*>(hap);
                         ha_pre[0] = f.x; ha_pre[1] = f.y; ha_pre[2] = f.z; ha_pre[TPL - 1] = f.w;
@@ -1187,7 +1194,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                     rec += fabsf(hv[e]);
                 }
                 if (hap) {
-                    if (a.anchor_mode == RM_ANCHOR_WRITE) {
+                    if (anchor_mode == RM_ANCHOR_WRITE) {
                         if (TPL == 4) *reinterpret_cast<float4*>(hap) = make_float4(hv[0], hv[1], hv[2], hv[TPL - 1]);
                         else *reinterpret_cast<float2*>(hap) = make_float2(hv[0], hv[TPL - 1]);
                     } else {
@@ -1331,7 +1338,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 float* dst = a.r_out + (size_t)b * T * H;
                 for (size_t i = (size_t)blockIdx.x * 256 + tid; i < (size_t)T * H / 4; i += (size_t)gridDim.x * 256) {
                     const float4 v = src[i];
-                    add_residual4(a, dst + 4 * i, (size_t)b * T * H + (4 * i / H) * H, (int)(4 * i % H), b, v.x, v.y, v.z, v.w);
+                    add_residual4(ya_update, gate, H, dst + 4 * i, (size_t)b * T * H + (4 * i / H) * H, (int)(4 * i % H), b, v.x, v.y, v.z, v.w);
                 }
             }
         }
@@ -1351,11 +1358,13 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
 template <int NTOK, int HS>
 int launch_fused_ws(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cudaStream_t s) {
     using S = SmemWS<NTOK, HS>;
-    auto kern = fused_layer_ws_kernel<NTOK, HS>;
+    const bool eq4 = a.anchor_mode != RM_ANCHOR_NONE || a.gate != nullptr;
+    auto kern = eq4 ? fused_layer_ws_kernel<NTOK, HS, true> : fused_layer_ws_kernel<NTOK, HS, false>;
     const int smem = S::total_bytes(a.T);
     static int configured = 0;
     if (configured < smem) {
-        RM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        RM_CUDA_TRY(cudaFuncSetAttribute(fused_layer_ws_kernel<NTOK, HS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        RM_CUDA_TRY(cudaFuncSetAttribute(fused_layer_ws_kernel<NTOK, HS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         configured = smem;
     }
     cudaLaunchConfig_t cfg = {};
@@ -1380,11 +1389,13 @@ int launch_fused_ws(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, c
 template <int NTOK, int HS, bool PIPE>
 int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cudaStream_t s) {
     using S = Smem<NTOK, HS, PIPE>;
-    auto kern = fused_layer_kernel<NTOK, HS, PIPE>;
+    const bool eq4 = a.anchor_mode != RM_ANCHOR_NONE || a.gate != nullptr;
+    auto kern = eq4 ? fused_layer_kernel<NTOK, HS, PIPE, true> : fused_layer_kernel<NTOK, HS, PIPE, false>;
     const int smem = S::total_bytes(a.T);
     static int configured = 0;
     if (configured < smem) {
-        RM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        RM_CUDA_TRY(cudaFuncSetAttribute(fused_layer_kernel<NTOK, HS, PIPE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        RM_CUDA_TRY(cudaFuncSetAttribute(fused_layer_kernel<NTOK, HS, PIPE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         configured = smem;
     }
     cudaLaunchConfig_t cfg = {};
@@ -1409,7 +1420,7 @@ int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cuda
 template <int NTOK, int HS, bool PIPE>
 int max_clusters(int T, int* out) {
     using S = Smem<NTOK, HS, PIPE>;
-    auto kern = fused_layer_kernel<NTOK, HS, PIPE>;
+    auto kern = fused_layer_kernel<NTOK, HS, PIPE, false>;
     const int smem = S::total_bytes(T);
     RM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     cudaLaunchConfig_t cfg = {};
