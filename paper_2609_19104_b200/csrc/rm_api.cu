@@ -22,6 +22,20 @@ inline bool use_fused(const rm_ctx* ctx, int B, int T) {
     return ctx->path != 1 && rm_fused_supported(ctx, B, T);
 }
 
+// The streaming variant (whole tiles per CTA) pays off only when a launch has about one 64-neuron tile per SM (one SM
+// gathers at most ~38 GB/s with 16-byte cp.async and adds at most ~20 GB/s with red.global, so a tile costs it
+// ~25 us); below that the cluster kernels, which spread a tile over 8 SMs, win.  H = 1024 only: at H = 2048 the
+// warp-specialised cluster kernel is ahead at every size measured.  `masked` says whether a count is in play.
+inline bool use_stream(const rm_ctx* ctx, bool masked, int B, int T) {
+    if (ctx->path == 1 || !rm_stream_supported(ctx, B, T)) return false;
+    if (ctx->variant_override == 4) return true;
+    if (ctx->variant_override != 0 || ctx->g.H != 1024) return false;
+    const int per_episode = masked ? ctx->count_hint : ctx->g.I;
+    if (per_episode <= 0) return false;
+    const long long tiles = (long long)((per_episode + 63) / 64) * B;
+    return tiles >= ctx->stream_min_tiles;
+}
+
 }  // namespace
 
 extern "C" {
@@ -42,6 +56,7 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->g.Hs = desc->H / RM_NS;
     c->launches = 0;
     c->status_detail = 0;
+    c->stream_min_tiles = 112;             // measured: ahead of the cluster kernels from about 8 episodes x 16 tiles
     c->d_status = nullptr;
     cudaDeviceProp prop;
     if (cudaGetDevice(&c->device) != cudaSuccess || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess ||
@@ -159,6 +174,8 @@ int rm_sparse_mlp(rm_ctx* ctx, const void* packed_layer, const void* x, const fl
                                                       cudaMemcpyDeviceToDevice, s));
             else RM_CUDA_TRY(cudaMemsetAsync(y, 0, (size_t)T * ctx->g.H * sizeof(float), s));
         }
+        if (use_stream(ctx, count_dev != nullptr, 1, T))
+            return rm_launch_layer_stream(ctx, a, nullptr, false, s);
         return rm_launch_layer_fused(ctx, a, nullptr, false, false, s);
     }
     if (ctx->path == 2) return RM_ERR_UNSUPPORTED;
@@ -191,8 +208,9 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
     // Fused path: layer l reads rot[l%3] (the caller's r_in for l = 0), accumulates into rot[(l+1)%3] and clears
     // rot[(l+2)%3] for the layer after next; the last layer accumulates straight into r_out when that is a
     // different buffer from r_in.
+    const bool stream = fused && use_stream(ctx, count_dev != nullptr, B, T);
     const bool direct_out = fused && r_out != r_in;
-    if (fused) {
+    if (fused && !stream) {
         RM_CUDA_TRY(cudaMemsetAsync(g.L == 1 && direct_out ? r_out : rot[1], 0, n_bytes, s));
         if (direct_out && g.L > 1) RM_CUDA_TRY(cudaMemsetAsync(r_out, 0, n_bytes, s));
     }
@@ -221,7 +239,13 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
         a.h_stride = an.h_stride;
         a.gate = an.gate ? an.gate + (size_t)l * B * g.H : nullptr;
         int rc;
-        if (fused) {
+        if (stream) {
+            // two buffers in turn: the preparation kernel writes the residual part of the output, the tiles add theirs
+            const bool last = l == g.L - 1;
+            a.r_out = (last && direct_out) ? r_out : rot[l & 1];
+            rc = rm_launch_layer_stream(ctx, a, reinterpret_cast<__nv_bfloat16*>(layer_ws), ctx->use_pdl && l > 0, s);
+            cur = a.r_out;
+        } else if (fused) {
             const bool last = l == g.L - 1;
             a.r_out = (last && direct_out) ? r_out : rot[(l + 1) % 3];
             // the buffer cleared here is the output of layer l+1 (unless that layer writes to r_out directly); it
@@ -349,8 +373,11 @@ int rm_set_option(rm_ctx* ctx, const char* name, int value) {
         if (value < 0) return RM_ERR_INVALID_ARG;
         ctx->count_hint = value;
     } else if (n == "variant") {
-        if (value < 0 || value > 3) return RM_ERR_INVALID_ARG;
+        if (value < 0 || value > 4) return RM_ERR_INVALID_ARG;
         ctx->variant_override = value;
+    } else if (n == "stream_min_tiles") {
+        if (value < 1) return RM_ERR_INVALID_ARG;
+        ctx->stream_min_tiles = value;
     } else if (n == "l2_prefetch") {
         if (value < 0 || value > 16) return RM_ERR_INVALID_ARG;
         ctx->l2_prefetch = value;
@@ -385,6 +412,7 @@ int rm_get_info(const rm_ctx* ctx, const char* name, int* out) {
 
 int rm_debug_phase_times(rm_ctx* ctx, long long* host_out, int n) {
     if (!ctx || !host_out) return RM_ERR_INVALID_ARG;
+    if (n == -64) return rm_stream_debug_stamps(host_out);      // the streaming kernel's stamps (first tile of CTA 0)
     return rm_fused_debug_stamps(host_out, n);
 }
 

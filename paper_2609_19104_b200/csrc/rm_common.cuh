@@ -41,6 +41,7 @@ struct rm_ctx {
     int count_hint;                        // expected active neurons per layer and episode (0: unknown)
     int max_clusters_override;             // > 0: cap on clusters per launch
     int l2_prefetch;                       // L2 prefetch distance (tiles) of the warp-specialised kernel
+    int stream_min_tiles;                  // launches with at least this many 64-neuron tiles use the streaming variant
     int variant_override;                  // 0 auto, 1 lean kernel, 2 kernel with a dedicated staging buffer
 };
 
@@ -109,3 +110,7 @@ bool rm_fused_supported(const rm_ctx* ctx, int B, int T);
 int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& a, float* zero_buf, bool add_residual, bool pdl,
                           cudaStream_t s);
 int rm_launch_layer_ref(rm_ctx* ctx, const rm_layer_args& a, void* ws, cudaStream_t s);
+// Streaming tensor-core variant (whole tiles per CTA, no clusters): same shapes as the fused path.
+bool rm_stream_supported(const rm_ctx* ctx, int B, int T);
+int rm_stream_debug_stamps(long long* host_out);
+int rm_launch_layer_stream(rm_ctx* ctx, const rm_layer_args& a, __nv_bfloat16* x_scratch, bool pdl, cudaStream_t s);

@@ -51,7 +51,7 @@ def lib_const(name):
     return getattr(rm, name)
 
 
-@pytest.mark.parametrize("path,variant,max_clusters", [(1, 0, 0), (2, 0, 0), (2, 1, 3), (2, 2, 3), (2, 3, 3)])
+@pytest.mark.parametrize("path,variant,max_clusters", [(1, 0, 0), (2, 0, 0), (2, 1, 3), (2, 2, 3), (2, 3, 3), (2, 4, 0), (2, 4, 3)])
 @pytest.mark.parametrize("H,I,T,L,B", [(1024, 1024, 51, 3, 2), (2048, 512, 32, 2, 1)])
 def test_anchor_write_then_update_matches_the_oracle(lib, path, variant, max_clusters, H, I, T, L, B):
     import torch

@@ -183,7 +183,7 @@ def test_step_host_variant_matches_device_variant(lib):
     model.close()
 
 
-@pytest.mark.parametrize("variant", [1, 2, 3])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4])
 @pytest.mark.parametrize("H,I,T,B", [(1024, 2048, 51, 2), (1024, 1024, 32, 1), (2048, 1024, 51, 1),
                                      (2048, 1024, 32, 1), (1024, 1024, 64, 1), (2048, 1024, 64, 1)])
 def test_every_tensor_core_variant_and_the_portable_path_agree_with_the_oracle(lib, variant, H, I, T, B):
