@@ -167,6 +167,27 @@ int rm_action_expert_step_ex(rm_ctx* ctx, const void* const* packed_layers, cons
                              float* h_anchor, int64_t h_stride, const float* out_gate, void* ws, size_t ws_bytes,
                              rm_stream_t stream);
 
+/* ---- Context Cache: visual-token selective recomputation of one VLM FFN layer (Sec. 4.1 "Visual-Token
+ * Recomputation", Eq. 2 and Eq. 3).  This path uses the model's own weight layouts (no packing): Wg, Wu [I,H] and
+ * Wd [H,I] bf16 row-major; H and I multiples of 128.
+ *
+ * rm_context_drift (Eq. 2): score_out[p] = RMS(x_p - x_ref_p) / max(RMS(x_p), 1e-6) for the P visual rows;
+ *   x, x_ref [P,H] bf16 (FFN inputs after RMSNorm, current and reference).  The rows to recompute are then the
+ *   ceil(rho_p * P) largest scores: rm_mask_compact with RM_SRC_SCORE_F32 / RM_REDUCE_TOPK and I := P.
+ *
+ * rm_context_ffn (Eq. 3): y_out[p] = F(x_p) for the listed visual rows and for the S rows that follow the visual
+ *   rows in x (instruction and state rows, always recomputed); every other visual row keeps y_ref[p].
+ *   F(x) = Wd (gelu_tanh(Wg x) * (Wu x)), fp32 accumulation, the hidden activations rounded to bf16 between the two
+ *   products (as the model does).  x [P+S,H] bf16; rows [>= count] int32 ascending, count_dev [1] int32 (device);
+ *   y_ref [P,H] fp32; y_out [P+S,H] fp32 (may equal y_ref when that buffer has P+S rows).
+ *   R_max >= count + S is the row capacity of the call, at most 256 (RM_ERR_SHAPE above); a count that does not fit
+ *   is truncated and RM_ERR_INDEX recorded.  ws: rm_context_workspace_bytes(ctx, R_max) bytes. */
+int rm_context_drift(rm_ctx* ctx, const void* x, const void* x_ref, int P, float* score_out, rm_stream_t stream);
+size_t rm_context_workspace_bytes(const rm_ctx* ctx, int R_max);
+int rm_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, const void* x, const int32_t* rows,
+                   const int32_t* count_dev, int P, int S, int R_max, const float* y_ref, float* y_out, void* ws,
+                   size_t ws_bytes, rm_stream_t stream);
+
 /* ---- rm_sparse_mlp_static: the one-layer call of rm_sparse_mlp for callers that cannot allocate.
  * (The paper has no counterpart for this entry point; it exists for integration reasons only.)
  *

@@ -245,3 +245,47 @@ def down_colnorm(Wd):
     out = np.empty(I, dtype=np.float32)
     _load().orc_down_colnorm(_p(Wd), ctypes.c_int(H), ctypes.c_int(I), _p(out))
     return out
+
+
+# ------------------------------------------------------------------ Context Cache (Sec. 4.1 "Visual-Token Recomputation")
+def _bf16_to_f64(bits):
+    return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def drift_scores(x, x_ref):
+    """Eq. 2: d_p = RMS(x_p - xref_p) / max(RMS(x_p), 1e-6) for every row p; x, x_ref [P,H] bf16 bits; float64
+    arithmetic, rounded once to float32."""
+    a, b = _bf16_to_f64(x), _bf16_to_f64(x_ref)
+    num = np.sqrt(np.mean((a - b) ** 2, axis=1))
+    den = np.maximum(np.sqrt(np.mean(a ** 2, axis=1)), 1e-6)
+    return (num / den).astype(np.float32)
+
+
+def ffn_rows(Wg, Wu, Wd, x):
+    """F(x) = Wd (gelu_tanh(Wg x) * (Wu x)) for every row of x [R,H] (bf16 bits), in float64 with library matrix
+    products, rounded once to float32.  The hidden activations are kept in full precision."""
+    xf = _bf16_to_f64(x)
+    g = xf @ _bf16_to_f64(Wg).T
+    u = xf @ _bf16_to_f64(Wu).T
+    act = 0.5 * g * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (g + 0.044715 * g ** 3)))
+    return ((act * u) @ _bf16_to_f64(Wd).T).astype(np.float32)
+
+
+def context_select(scores, rho: float):
+    """The ceil(rho * P) rows with the largest scores, ascending; equal scores: lower index first."""
+    P = int(np.asarray(scores).shape[0])
+    k = int(min(P, max(0, np.ceil(rho * P - 1e-9))))
+    return compact_scores(np.asarray(scores, dtype=np.float32), RULE_TOPK, k=k)
+
+
+def context_ffn(Wg, Wu, Wd, x, rows, S: int, y_ref):
+    """Eq. 3: rows listed in `rows` (visual rows, indices < P) and the S rows after the P visual rows are recomputed,
+    every other visual row keeps the reference output.  x [P+S,H] bf16 bits, y_ref [P,H] float32."""
+    y_ref = np.asarray(y_ref, dtype=np.float32)
+    P, H = y_ref.shape
+    out = np.empty((P + S, H), dtype=np.float32)
+    out[:P] = y_ref
+    sel = np.concatenate([np.asarray(rows, dtype=np.int64), np.arange(P, P + S, dtype=np.int64)])
+    if sel.size:
+        out[sel] = ffn_rows(Wg, Wu, Wd, np.ascontiguousarray(x)[sel])
+    return out

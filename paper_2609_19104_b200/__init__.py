@@ -23,7 +23,8 @@ RM_ANCHOR_NONE, RM_ANCHOR_WRITE, RM_ANCHOR_UPDATE = 0, 1, 2
 
 EXPORTS = ["rm_create", "rm_destroy", "rm_packed_layer_bytes", "rm_workspace_bytes", "rm_pack_weights",
            "rm_mask_compact", "rm_sparse_mlp", "rm_action_expert_step", "rm_action_expert_step_host",
-           "rm_action_expert_step_ex", "rm_gather_weights",
+           "rm_action_expert_step_ex", "rm_gather_weights", "rm_context_drift", "rm_context_workspace_bytes",
+           "rm_context_ffn",
            "rm_device_status", "rm_launch_count", "rm_status_string", "rm_set_option", "rm_get_info",
            "rm_debug_phase_times", "rm_sparse_mlp_static"]
 
@@ -75,6 +76,10 @@ def load_library() -> ctypes.CDLL:
     lib.rm_sparse_mlp.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
     lib.rm_action_expert_step.argtypes = [vp, ctypes.POINTER(vp), vp, vp, vp, i64, vp, vp, vp, i32, i32, vp, sz, vp]
     lib.rm_action_expert_step_host.argtypes = [vp, ctypes.POINTER(vp), vp, vp, vp, i64, vp, i32, i32, vp, sz, vp]
+    lib.rm_context_drift.argtypes = [vp, vp, vp, i32, vp, vp]
+    lib.rm_context_workspace_bytes.argtypes = [vp, i32]
+    lib.rm_context_workspace_bytes.restype = sz
+    lib.rm_context_ffn.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.rm_gather_weights.argtypes = [vp, vp, vp, vp, i64, vp, vp]
     lib.rm_action_expert_step_ex.argtypes = [vp, ctypes.POINTER(vp), vp, vp, vp, i64, vp, vp, vp, i32, i32, i32, vp, vp,
                                              i64, vp, vp, sz, vp]
@@ -190,14 +195,33 @@ class Context:
 
     def rm_mask_compact(self, records: Sequence, kind: int, reduce: int, idx_out, count_out, stride: int, *,
                         n_lists: int, threshold: float = 0.0, k: int = 0, min_votes: int = 1, scale=None,
-                        scale_per_list: bool = False):
+                        scale_per_list: bool = False, I: Optional[int] = None):
         W = len(records)
         arr = (ctypes.c_void_p * max(W, 1))(*[_ptr(r) for r in records])
         src = rm_mask_src(kind, reduce, float(threshold), int(k), W, int(min_votes),
                           ctypes.cast(arr, ctypes.POINTER(ctypes.c_void_p)), _ptr(scale), int(bool(scale_per_list)),
-                          int(n_lists), self.I)
+                          int(n_lists), self.I if I is None else int(I))
         _check(self.lib.rm_mask_compact(self._h, ctypes.byref(src), _ptr(idx_out), _ptr(count_out), int(stride),
                                         _stream()), "rm_mask_compact")
+
+    def rm_context_drift(self, x, x_ref, P: int, score_out):
+        """Eq. 2: per-row drift score of the current FFN input against the reference input."""
+        _check(self.lib.rm_context_drift(self._h, _ptr(x), _ptr(x_ref), int(P), _ptr(score_out), _stream()),
+               "rm_context_drift")
+        return score_out
+
+    def rm_context_ffn(self, Wg, Wu, Wd, x, rows, count_dev, P: int, S: int, R_max: int, y_ref, y_out, ws=None):
+        """Eq. 3: recompute the listed visual rows and the S always-recomputed rows, keep y_ref elsewhere."""
+        import torch
+        need = int(self.lib.rm_context_workspace_bytes(self._h, int(R_max)))
+        if ws is None:
+            if getattr(self, "_ctx_ws", None) is None or self._ctx_ws.numel() < need:
+                self._ctx_ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+            ws = self._ctx_ws
+        _check(self.lib.rm_context_ffn(self._h, _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(x), _ptr(rows), _ptr(count_dev), int(P),
+                                       int(S), int(R_max), _ptr(y_ref), _ptr(y_out), _ptr(ws), int(ws.numel()), _stream()),
+               "rm_context_ffn")
+        return y_out
 
     def rm_gather_weights(self, packed_layer, idx, count_dev, list_cap: int, compact_out=None):
         """Compact copy of the listed neurons' packed rows (a packed layer whose leading `count` neurons are the list)."""

@@ -115,6 +115,33 @@ int rm_gather_weights(rm_ctx* ctx, const void* packed_layer, const int32_t* idx,
                                  static_cast<cudaStream_t>(stream));
 }
 
+static int context_pad(int R_max) { return R_max <= 64 ? 64 : (R_max <= 128 ? 128 : 256); }
+
+int rm_context_drift(rm_ctx* ctx, const void* x, const void* x_ref, int P, float* score_out, rm_stream_t stream) {
+    if (!ctx || !x || !x_ref || !score_out || P < 0) return RM_ERR_INVALID_ARG;
+    if (ctx->g.H % 8 != 0) return RM_ERR_UNSUPPORTED;
+    if (!all_aligned({x, x_ref, score_out})) return RM_ERR_ALIGN;
+    if (P == 0) return RM_OK;
+    return rm_launch_context_drift(ctx, x, x_ref, P, score_out, static_cast<cudaStream_t>(stream));
+}
+
+size_t rm_context_workspace_bytes(const rm_ctx* ctx, int R_max) {
+    if (!ctx || R_max < 1 || R_max > 256 || !rm_context_supported(ctx)) return 0;
+    return rm_context_workspace_bytes_impl(ctx, context_pad(R_max));
+}
+
+int rm_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, const void* x, const int32_t* rows,
+                   const int32_t* count_dev, int P, int S, int R_max, const float* y_ref, float* y_out, void* ws,
+                   size_t ws_bytes, rm_stream_t stream) {
+    if (!ctx || !Wg || !Wu || !Wd || !x || !rows || !count_dev || !y_ref || !y_out || P < 0 || S < 0) return RM_ERR_INVALID_ARG;
+    if (!rm_context_supported(ctx)) return RM_ERR_UNSUPPORTED;
+    if (R_max < 1 || R_max > 256 || S > R_max) return RM_ERR_SHAPE;
+    if (!all_aligned({Wg, Wu, Wd, x, rows, y_ref, y_out, ws})) return RM_ERR_ALIGN;
+    if (!ws || ws_bytes < rm_context_workspace_bytes(ctx, R_max)) return RM_ERR_WORKSPACE;
+    return rm_launch_context_ffn(ctx, Wg, Wu, Wd, x, rows, count_dev, P, S, context_pad(R_max), y_ref, y_out, ws,
+                                 static_cast<cudaStream_t>(stream));
+}
+
 int rm_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out, int64_t stride,
                     rm_stream_t stream) {
     if (!ctx || !src || !idx_out || !count_out || !src->records) return RM_ERR_INVALID_ARG;

@@ -77,6 +77,13 @@ int rm_launch_pack(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, 
                    cudaStream_t s);
 int rm_launch_gather_rows(rm_ctx* ctx, const void* packed, const int32_t* idx, const int32_t* count, int64_t cap,
                           void* out, cudaStream_t s);
+// Context Cache (row-sparse dense FFN on the tensor cores)
+bool rm_context_supported(const rm_ctx* ctx);
+size_t rm_context_workspace_bytes_impl(const rm_ctx* ctx, int r_pad);
+int rm_launch_context_drift(rm_ctx* ctx, const void* x, const void* x_ref, int P, float* score, cudaStream_t s);
+int rm_launch_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, const void* x, const int32_t* rows,
+                          const int32_t* count, int P, int S, int r_pad, const float* y_ref, float* y_out, void* ws,
+                          cudaStream_t s);
 int rm_launch_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out,
                            int64_t stride, cudaStream_t s);
 

@@ -33,6 +33,7 @@ _M2 = _U64(0x94D049BB133111EB)
 ROLE_WG, ROLE_WU, ROLE_WD = 1, 2, 3
 ROLE_X0, ROLE_REF_NOISE, ROLE_STEP_DIR, ROLE_RESIDUAL = 4, 5, 6, 7
 ROLE_BOOL_MASK, ROLE_RUNS, ROLE_GATE = 8, 9, 10
+ROLE_CTX_X, ROLE_CTX_DRIFT, ROLE_CTX_NOISE, ROLE_CTX_YREF = 11, 12, 13, 14
 
 
 def _mix(z: np.ndarray) -> np.ndarray:
@@ -164,6 +165,29 @@ def config5(seed: int = BASE_SEED, L: int = 18) -> Workload:
     # first step of a group is the dense anchor, the other four update the group's shared mask (top-k = 2048 of 4096)
     return Workload(5, "pi0-anchor-groups-top50", L, 1024, 4096, 51, 0.02, 10, 0.50, seed=seed,
                     extra={"weights_config": 1, "group": 5})
+
+
+def config6(seed: int = BASE_SEED, H: int = 2048, I: int = 16384, P: int = 768, S: int = 48, rho: float = 0.25) -> Workload:
+    # Context Cache: one VLM FFN layer, P visual rows (three cameras of 256 tokens) plus S instruction / state rows;
+    # the rows with the largest input drift against a reference execution are recomputed (Eq. 2, Eq. 3)
+    return Workload(6, f"context-cache-rho{rho:g}", 1, H, I, P + S, 0.015 if H >= 2048 else 0.03, 1, rho, seed=seed,
+                    extra={"P": P, "S": S})
+
+
+def context_inputs(w: Workload):
+    """(x [P+S,H], x_ref [P,H]) as bf16 bits and y_ref [P,H] float32 for the Context Cache workload.  Reference rows are
+    unit-RMS normals; the current input is reference + drift, where the drift scale of a visual row is log-normal
+    (median 0.05, sigma 1.2): most patches barely change between executions, a few (moved objects) change a lot.
+    y_ref stands for the reference execution's outputs: independent normals of the FFN's output scale."""
+    P, S, H = w.extra["P"], w.extra["S"], w.H
+    xr = normal(tensor_key(w.seed, w.config, 0, ROLE_CTX_X), (P + S) * H).reshape(P + S, H)
+    xr /= np.sqrt(np.mean(xr.astype(np.float64) ** 2, axis=1, keepdims=True)).astype(np.float32)
+    scale = np.exp(np.float32(1.2) * normal(tensor_key(w.seed, w.config, 0, ROLE_CTX_DRIFT), P)) * np.float32(0.05)
+    noise = normal(tensor_key(w.seed, w.config, 0, ROLE_CTX_NOISE), P * H).reshape(P, H)
+    x = xr.copy()
+    x[:P] += scale[:, None] * noise
+    y_ref = normal(tensor_key(w.seed, w.config, 0, ROLE_CTX_YREF), P * H).reshape(P, H) * np.float32(0.5)
+    return f32_to_bf16_bits(x), f32_to_bf16_bits(xr[:P]), y_ref.astype(np.float32)
 
 
 def scaled(w: Workload, **kw) -> Workload:

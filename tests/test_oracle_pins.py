@@ -478,3 +478,54 @@ def test_table1_products():
     assert wl.topk_count(0.5, 4096) == 2048
     assert wl.topk_count(0.25, 4096) == 1024 and wl.topk_count(0.20, 16384) == 3277
     assert wl.topk_count(0.15, 4096) == 615 and wl.topk_count(0.05, 4096) == 205
+
+
+# ------------------------------------------------------------------ Context Cache (Eq. 2, Eq. 3)
+def test_drift_score_closed_forms():
+    w = wl.config6(H=64, I=128, P=12, S=2)
+    x, xr, _ = wl.context_inputs(w)
+    P = 12
+    # identical inputs -> 0; zero reference -> exactly RMS(x)/RMS(x) = 1; scale invariance; a hand-computed row
+    assert np.all(oracle.drift_scores(x[:P], x[:P]) == 0.0)
+    assert np.allclose(oracle.drift_scores(x[:P], np.zeros_like(x[:P])), 1.0, rtol=1e-6)
+    two = lambda bits: wl.f32_to_bf16_bits(2.0 * wl.bf16_bits_to_f32(bits))          # exact in bf16
+    assert np.array_equal(oracle.drift_scores(two(x[:P]), two(xr)), oracle.drift_scores(x[:P], xr))
+    a = wl.f32_to_bf16_bits(np.array([[3.0, 4.0, 0.0, 0.0]], np.float32))
+    b = wl.f32_to_bf16_bits(np.array([[0.0, 4.0, 0.0, 4.0]], np.float32))
+    # RMS(a-b) = sqrt((9+16)/4) = 2.5, RMS(a) = sqrt(25/4) = 2.5 -> 1
+    assert oracle.drift_scores(a, b)[0] == np.float32(1.0)
+    # a zero current row: the denominator is clamped at 1e-6, not zero
+    z = wl.f32_to_bf16_bits(np.zeros((1, 4), np.float32))
+    assert np.isclose(oracle.drift_scores(z, a)[0], 2.5 / 1e-6, rtol=1e-6)
+    # larger perturbation of a row -> larger score (the quantity the selection ranks by)
+    d = oracle.drift_scores(x[:P], xr)
+    xf, xrf = wl.bf16_bits_to_f32(x[:P]), wl.bf16_bits_to_f32(xr)
+    want = np.sqrt(((xf - xrf).astype(np.float64) ** 2).mean(1)) / np.sqrt((xf.astype(np.float64) ** 2).mean(1))
+    assert np.allclose(d, want, rtol=1e-6)
+
+
+def test_context_ffn_special_cases():
+    w = wl.config6(H=64, I=128, P=20, S=3)
+    x, xr, y_ref = wl.context_inputs(w)
+    Wg, Wu, Wd = wl.layer_weights(w, 0)
+    P, S = 20, 3
+    # the FFN through library products equals the dense loop nest of the C oracle (two independent routes)
+    full = oracle.ffn_rows(Wg, Wu, Wd, x)
+    assert np.allclose(full, oracle.dense_mlp(x, Wg, Wu, Wd, None), rtol=1e-5, atol=1e-6)
+    # nothing selected: visual rows keep the reference, the S trailing rows are still recomputed
+    out = oracle.context_ffn(Wg, Wu, Wd, x, np.zeros(0, np.int32), S, y_ref)
+    assert np.array_equal(out[:P], y_ref) and np.array_equal(out[P:], full[P:])
+    # everything selected: the dense FFN of the current input
+    out = oracle.context_ffn(Wg, Wu, Wd, x, np.arange(P, dtype=np.int32), S, y_ref)
+    assert np.array_equal(out, full)
+    # a partial selection: exactly those rows change, and they equal the dense FFN's rows
+    sel = oracle.context_select(oracle.drift_scores(x[:P], xr), 0.25)
+    assert sel.size == 5 and np.all(np.diff(sel) > 0)
+    out = oracle.context_ffn(Wg, Wu, Wd, x, sel, S, y_ref)
+    keep = np.setdiff1d(np.arange(P), sel)
+    assert np.array_equal(out[keep], y_ref[keep]) and np.array_equal(out[sel], full[sel])
+    # the selection holds the rows with the largest scores
+    d = oracle.drift_scores(x[:P], xr)
+    assert d[sel].min() >= d[keep].max()
+    # ceil(rho P): 0.26 * 20 = 5.2 -> 6 rows
+    assert oracle.context_select(d, 0.26).size == 6
