@@ -53,6 +53,9 @@ def pick_workload(name: str) -> wl.Workload:
         return wl.config4()
     if name == "config5":
         return wl.config5()
+    if name.startswith("config6"):
+        parts = name.split(":")
+        return wl.config6(rho=float(parts[1]) if len(parts) > 1 else 0.25)
     if name.startswith("config3"):
         parts = name.split(":")
         rho = float(parts[1]) if len(parts) > 1 else 0.25
@@ -185,6 +188,113 @@ def max_over_ranks(values, world: int, device="cpu"):
 def job_us_per_step(total_ms: float, steps: int, world: int, B: int) -> float:
     """Whole-job metric: every rank ran `steps` steps of B episodes in `total_ms` (max over ranks)."""
     return total_ms * 1e3 / (steps * world * B)
+
+
+# ------------------------------------------------------------------------------------------------ Context Cache
+def measured_bf16_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
+
+
+def run_context(args, w: wl.Workload):
+    """The second workload (not the headline metric): one VLM FFN layer under the Context Cache.  A step = Eq. 2 drift
+    scores, top-ceil(rho P) row selection, Eq. 3 recomputation of the selected rows and scatter."""
+    import torch
+    import paper_2609_19104_b200 as rm
+    world, rank, local = rank_env()
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    P, S, H, I = w.extra["P"], w.extra["S"], w.H, w.I
+    k = wl.topk_count(w.density, P)
+    R = k + S
+    ctx = rm.Context(1, H, I, T_max=64)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed + rank)
+    mk = lambda shape: (torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32) * w.sigma).to(torch.bfloat16)
+    Wg, Wu, Wd = mk((I, H)), mk((I, H)), mk((H, I))
+    x_bits, xr_bits, y_ref = wl.context_inputs(w)
+    to = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    x, xr, yref = to(x_bits), to(xr_bits), torch.from_numpy(y_ref).cuda()
+    score = torch.empty(P, dtype=torch.float32, device="cuda")
+    rows = torch.zeros(P, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y_out = torch.empty(P + S, H, dtype=torch.float32, device="cuda")
+    pin_x = torch.from_numpy(x_bits.view(np.int16)).pin_memory()
+    pin_y = torch.empty(P + S, H, dtype=torch.float32).pin_memory()
+    flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        ctx.rm_context_drift(x, xr, P, score)
+        ctx.rm_mask_compact([score], rm.RM_SRC_SCORE_F32, rm.RM_REDUCE_TOPK, rows, cnt, P, n_lists=1, k=k, I=P)
+        ctx.rm_context_ffn(Wg, Wu, Wd, x, rows, cnt, P, S, R, yref, y_out)
+
+    for s in range(args.warmup):
+        flush.fill_(s & 0xFF)
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    l0 = ctx.launch_count()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for s in range(args.steps):
+        flush.fill_(s & 0xFF)
+        ev[s][0].record(stream)
+        step()
+        ev[s][1].record(stream)
+    torch.cuda.synchronize()
+    launches = ctx.launch_count() - l0
+    status = ctx.rm_device_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status} ({rm.status_string(status)}) after the timed steps")
+    total_ms = float(sum(a.elapsed_time(b) for a, b in ev))
+    e2e = []
+    for s in range(args.warmup + args.steps):
+        flush.fill_(s & 0xFF)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        x.view(torch.int16).copy_(pin_x, non_blocking=True)
+        step()
+        pin_y.copy_(y_out, non_blocking=True)
+        torch.cuda.synchronize()
+        if s >= args.warmup:
+            e2e.append(time.perf_counter() - t0)
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms, e2e_ms = max_over_ranks([total_ms, float(sum(e2e)) * 1e3], world, device="cuda")
+    if rank != 0:
+        return
+    us = total_ms * 1e3 / (args.steps * world)
+    hbm_peak, kind = measured_hbm_peak()
+    tf_peak, _ = measured_bf16_peak()
+    flops = 2.0 * R * 3 * H * I
+    bytes_step = 3 * H * I * 2 + (P + S) * H * 2 + P * H * 2 + 2 * R * H * 4 + 2 * R * I * 2
+    achieved = bytes_step / (us * 1e-6) / 1e9
+    line = {
+        "metric": "context_cache_us_per_ffn_layer", "value": us, "unit": "us", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 (fp32 accumulate)", "data": "synthetic",
+        "config": {"workload": w.name, "H": H, "I": I, "P": P, "S": S, "rows_recomputed": R,
+                   "l2": "flushed before every timed step (512 MB fill, outside the timed interval)",
+                   "multi_gpu": "replicas"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
+                     "traffic": None, "peak_kind": f"{kind} copy bandwidth",
+                     "kernel": "ctx_gemm_kernel (two launches: gate/up + GeLU, down with split K)",
+                     "bytes_per_launch": bytes_step, "flops_per_step": flops,
+                     "tensor_tflops": flops / (us * 1e-6) / 1e12, "tensor_frac_of_measured_bf16": flops / (us * 1e-6) / 1e12 / tf_peak,
+                     "note": f"{R} rows against {3 * H * I / 1e6:.0f} M weights: {flops / bytes_step:.0f} flop/byte, at the ridge "
+                             f"({tf_peak * 1e3 / hbm_peak:.0f} flop/byte)"},
+        "e2e": {"value": e2e_ms * 1e3 / (args.steps * world), "unit": "us",
+                "h2d_bytes_per_step": int(x_bits.nbytes), "d2h_bytes_per_step": int((P + S) * H * 4)},
+        "gpu_launches": int(launches), "clocks": clocks,
+    }
+    print(json.dumps(line))
 
 
 # ------------------------------------------------------------------------------------------------ GPU arm
@@ -446,6 +556,8 @@ def main():
     w = pick_workload(args.workload)
     if args.impl == "reference":
         run_reference(args, w)
+    elif w.config == 6:
+        run_context(args, w)
     else:
         run_gpu(args, w)
 
