@@ -67,6 +67,7 @@ __global__ void __launch_bounds__(256) drift_kernel(const __nv_bfloat16* __restr
 __global__ void __launch_bounds__(256) ctx_gather_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ rows,
                                                          const int32_t* __restrict__ count, int P, int S, int H, int r_pad,
                                                          __nv_bfloat16* __restrict__ xc, int* status) {
+    pdl_launch_dependents();               // the first product may start now: its weight loads need nothing from here
     const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= r_pad) return;
     int c = *count;
