@@ -519,7 +519,7 @@ def run_gpu(args, w: wl.Workload):
                        "multi_gpu": "replicas: each rank runs its own episodes, no collective on the data path"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name), "peak_kind": f"{peak_kind} copy bandwidth",
-                         "kernel": ("fused_layer_kernel<64,128,false>" if w.H == 1024 else "fused_layer_ws_kernel<64,256>")
+                         "kernel": ("fused_layer_kernel<64,128,false,false>" if w.H == 1024 else "fused_layer_ws_kernel<64,256,false>")
                                    + " (one launch per layer, dependent-launch chained)",
                          "bytes_per_launch": bytes_layer, "us_per_launch": in_step_layer_us,
                          "us_per_launch_isolated_cold": layer_us, "launches_per_step": launches_per_step,
