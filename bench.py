@@ -500,6 +500,14 @@ def run_gpu(args, w: wl.Workload):
             bytes_layer = wl.algorithmic_bytes_per_layer(w.H, w.T, int(round(K_mean))) * B
         bytes_step = bytes_layer * w.L
         launches_per_step = launches / args.steps                 # fused layer launches + mask compaction share
+        # the kernel the library picks for this launch shape (see the variant selection in the library)
+        tiles_per_launch = (int(round(K_mean)) + 63) // 64 * B
+        if w.H == 1024 and (args.variant == 4 or (args.variant == 0 and tiles_per_launch >= 112)):
+            kernel_name = "stream_prep_kernel + stream_tile_kernel"
+        elif w.H == 1024:
+            kernel_name = "fused_layer_kernel<NTOK,128,false,*>" if args.variant in (0, 1) else f"variant {args.variant}"
+        else:
+            kernel_name = "fused_layer_ws_kernel<NTOK,256,*>" if args.variant in (0, 3) else f"variant {args.variant}"
         in_step_layer_us = us_per_step * B / w.L                  # average duration of a layer launch inside the step
         achieved = bytes_layer / (in_step_layer_us * 1e-6) / 1e9
         io_bytes = B * w.T * w.H * 4
@@ -519,8 +527,7 @@ def run_gpu(args, w: wl.Workload):
                        "multi_gpu": "replicas: each rank runs its own episodes, no collective on the data path"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name), "peak_kind": f"{peak_kind} copy bandwidth",
-                         "kernel": ("fused_layer_kernel<64,128,false,false>" if w.H == 1024 else "fused_layer_ws_kernel<64,256,false>")
-                                   + " (one launch per layer, dependent-launch chained)",
+                         "kernel": kernel_name + " (one launch per layer, dependent-launch chained)",
                          "bytes_per_launch": bytes_layer, "us_per_launch": in_step_layer_us,
                          "us_per_launch_isolated_cold": layer_us, "launches_per_step": launches_per_step,
                          "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
