@@ -457,6 +457,41 @@ def test_step_is_the_composition_of_layers():
     assert np.array_equal(got_d, cur)
 
 
+def test_step_special_cases_that_isolate_one_layer():
+    """Special cases of the stack with known answers: zero down-projections everywhere return the input bit for bit;
+    with the down-projection of a single layer k left in place the stack equals that one layer applied to the input
+    (the other layers add exactly zero), which fixes the order of the layers and which list goes with which layer; empty
+    lists return the input; and doubling the input (exact in floating point) leaves x, hence the first layer's
+    contribution, unchanged: out(2 r) - 2 r == out(r) - r up to the rounding of the sums."""
+    L, T, H, I = 4, 5, 32, 64
+    W = [small_problem(60 + l, T=T, H=H, I=I, sigma=0.2)[1:4] for l in range(L)]
+    Wg, Wu, Wd = [w[0] for w in W], [w[1] for w in W], [w[2] for w in W]
+    zero = np.zeros_like(Wd[0])
+    r0 = wl.normal(wl.tensor_key(60, 99, 0, 7), T * H).reshape(T, H)
+    idx = np.zeros((L, I), np.int32)
+    cnt = np.zeros(L, np.int32)
+    for l in range(L):
+        s_ = np.flatnonzero(wl.uniform(wl.tensor_key(60, 99, l, 8), I) < 0.4 + 0.1 * l)
+        idx[l, :s_.size] = s_
+        cnt[l] = s_.size
+    assert np.array_equal(oracle.step(Wg, Wu, [zero] * L, r0, idx, cnt), r0)
+    assert np.array_equal(oracle.step(Wg, Wu, Wd, r0, idx, np.zeros(L, np.int32)), r0)
+    for k in range(L):
+        only_k = [Wd[l] if l == k else zero for l in range(L)]
+        got = oracle.step(Wg, Wu, only_k, r0, idx, cnt)
+        want = oracle.masked_mlp(oracle.rmsnorm_bf16(r0), Wg[k], Wu[k], Wd[k], r0, idx[k, :cnt[k]])
+        assert np.array_equal(got, want), f"layer {k}"
+    # lists swapped between two layers change the answer (so the test above cannot pass with lists mixed up)
+    sw = idx.copy(); sw[[0, 1]] = sw[[1, 0]]
+    cs = cnt.copy(); cs[[0, 1]] = cs[[1, 0]]
+    only_0 = [Wd[0]] + [zero] * (L - 1)
+    assert not np.array_equal(oracle.step(Wg, Wu, only_0, r0, sw, cs), oracle.step(Wg, Wu, only_0, r0, idx, cnt))
+    # scale: RMSNorm removes it, so a layer's contribution is the same for r and 2 r (doubling is exact)
+    one = oracle.step(Wg[:1], Wu[:1], Wd[:1], r0, idx[:1], cnt[:1]).astype(np.float64) - r0
+    two = oracle.step(Wg[:1], Wu[:1], Wd[:1], 2.0 * r0, idx[:1], cnt[:1]).astype(np.float64) - 2.0 * r0
+    assert np.max(np.abs(one - two)) <= 1e-6 * np.max(np.abs(one))  # a single layer: exactly the same x
+
+
 # ------------------------------------------------------------------ byte / flop accounting vs Table 1
 def test_table1_products():
     rows = {}
