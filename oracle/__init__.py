@@ -4,8 +4,10 @@
 compiles it with gcc and exposes it through ctypes on numpy arrays.  Only the tests, the smoke check and the
 benchmark's CPU-baseline leg may import it.  It imports nothing from the CUDA package.
 
-Parity unpinned: `step` (the L-layer stack) has no closed form; it is pinned only as the composition of the
-pinned single-layer routines and by its L=1 case.
+Parity unpinned: `step` (the L-layer stack) has no closed form; it is pinned as the composition of the pinned
+single-layer routines, by its L=1 case and by special cases that isolate one layer; the accumulation of rounding
+through a deep stack has no independent value.  The Context Cache functions at the end of this module (Eq. 2, Eq. 3)
+are written in numpy (float64, library matrix products) and pinned by closed forms and by the C loop nest.
 """
 from __future__ import annotations
 

@@ -21,8 +21,9 @@
  * (GeLU-tanh degenerates to ReLU); a library-matmul special case; additivity over disjoint sets; neuron
  * permutation invariance; linearity in W_down and r; RMSNorm unit RMS and scale invariance; compaction round
  * trips, top-k order properties and vote identities; Eq. 4 special cases.
- * Parity unpinned: the L-layer stack (orc_step) has no closed form; it is pinned only as the composition of
- * pinned single layers and by L=1 equalling the single-layer routine.
+ * Parity unpinned: the L-layer stack (orc_step) has no closed form; it is pinned as the composition of pinned
+ * single layers, by L=1 equalling the single-layer routine, and by special cases that isolate one layer (zero
+ * down-projections elsewhere); the accumulation of rounding through a deep stack has no independent value.
  */
 #include <math.h>
 #include <stdint.h>
