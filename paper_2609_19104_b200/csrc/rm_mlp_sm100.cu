@@ -320,23 +320,29 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     if (g_lo < g_hi) issue_dn(g_lo);
     cp_async_commit();
 
+    // Which of the clusters that work on an episode adds which token rows of the residual (see xprep).  Integer
+    // divisions: ~0.8 us, so the first episode's answer is worked out here, before the dependency wait.
+    auto residual_share = [&](int b, int& n_share, int& my_share) {
+        const long long e0 = gPref[b], e1 = gPref[b + 1];                  // tile range of the episode
+        // cluster c owns tiles [c*tt/na, (c+1)*tt/na); first cluster with hi > e0, last with lo < e1
+        int first_c = (int)((e0 * n_active) / tiles_total);
+        while ((long long)(first_c + 1) * tiles_total / n_active <= e0) ++first_c;
+        int last_c = (int)(((e1 - 1) * n_active) / tiles_total);
+        while (last_c + 1 < n_active && (long long)(last_c + 1) * tiles_total / n_active < e1) ++last_c;
+        n_share = last_c - first_c + 1;
+        my_share = cid - first_c;
+    };
+    int share_b = -1, share_n = 1, share_my = 0;
+    if (a.add_residual && g_lo < g_hi) {
+        share_b = tile_ref(g_lo).b;
+        residual_share(share_b, share_n, share_my);
+    }
+
     RM_WALL(1);
     pdl_wait();                            // the previous layer's output is complete and visible
     RM_STAMP(2);
     RM_WALL(2);
 
-    // episodes without a single active neuron have no cluster working on them: their residual passes through here
-    if (a.add_residual) {
-        for (int b = 0; b < a.B; ++b) {
-            if (gPref[b + 1] != gPref[b]) continue;
-            const float4* src = reinterpret_cast<const float4*>(a.r_in + (size_t)b * T * H);
-            float* dst = a.r_out + (size_t)b * T * H;
-            for (size_t i = (size_t)blockIdx.x * FT + tid; i < (size_t)T * H / 4; i += (size_t)gridDim.x * FT) {
-                const float4 v = src[i];
-                add_residual4(ya_update, gate, H, dst + 4 * i, (size_t)b * T * H + (4 * i / H) * H, (int)(4 * i % H), b, v.x, v.y, v.z, v.w);
-            }
-        }
-    }
     RM_STAMP(3);
 
     uint32_t par_dn = 0, par_s = 0;
@@ -364,17 +370,11 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
         constexpr int PARTS = FT / NTOK;                   // threads per token row
         constexpr int CPP = HS / PARTS;                    // columns per thread
         const int t = tid / PARTS, part = tid % PARTS;
-        // clusters whose runs contain tiles of this episode: first_c .. last_c (contiguous)
+        // clusters whose runs contain tiles of this episode share the addition of its residual rows
         int n_share = 1, my_share = 0;
         if (a.add_residual) {
-            const long long e0 = gPref[b], e1 = gPref[b + 1];                  // tile range of the episode
-            // cluster c owns tiles [c*tt/na, (c+1)*tt/na); first cluster with hi > e0, last with lo < e1
-            int first_c = (int)((e0 * n_active) / tiles_total);
-            while ((long long)(first_c + 1) * tiles_total / n_active <= e0) ++first_c;
-            int last_c = (int)(((e1 - 1) * n_active) / tiles_total);
-            while (last_c + 1 < n_active && (long long)(last_c + 1) * tiles_total / n_active < e1) ++last_c;
-            n_share = last_c - first_c + 1;
-            my_share = cid - first_c;
+            if (b == share_b) { n_share = share_n; my_share = share_my; }
+            else residual_share(b, n_share, my_share);
         }
         if (a.x) {
             const uint4* src = reinterpret_cast<const uint4*>(a.x + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP);
@@ -730,8 +730,20 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
 
     // ---- teardown.  Everything peers send into this CTA's shared memory is counted on barriers this CTA has waited
     // for, so nothing is in flight towards it any more and it may exit without a cluster-wide wait.
-    // ---- duty shared by all CTAs: clear the buffer the next layer accumulates into.  It sits at the very end so that
-    // no release-barrier of the exchange phases has to wait for these global stores.
+    // ---- duties shared by all CTAs, at the very end so that nothing on the exchange chain waits for their global
+    // traffic.  Episodes without a single active neuron have no cluster working on them: their residual passes
+    // through here.  Then the buffer the next layer accumulates into is cleared.
+    if (a.add_residual) {
+        for (int b = 0; b < a.B; ++b) {
+            if (gPref[b + 1] != gPref[b]) continue;
+            const float4* src = reinterpret_cast<const float4*>(a.r_in + (size_t)b * T * H);
+            float* dst = a.r_out + (size_t)b * T * H;
+            for (size_t i = (size_t)blockIdx.x * FT + tid; i < (size_t)T * H / 4; i += (size_t)gridDim.x * FT) {
+                const float4 v = src[i];
+                add_residual4(ya_update, gate, H, dst + 4 * i, (size_t)b * T * H + (4 * i / H) * H, (int)(4 * i % H), b, v.x, v.y, v.z, v.w);
+            }
+        }
+    }
     if (a.zero_buf) {
         const size_t n4 = (size_t)a.B * T * H / 4;
         float4* z = reinterpret_cast<float4*>(a.zero_buf);
@@ -994,12 +1006,11 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
             }
         } else if (warp < 8) {
             // scatter and owner warps: x slice of episode b (256-thread mapping)
-            if (!waited_prev) { pdl_wait(); waited_prev = true; }
             constexpr int PARTS = 256 / NTOK;
             constexpr int CPP = HS / PARTS;
             const int t = tid / PARTS, part = tid % PARTS;
             int n_share = 1, my_share = 0;
-            if (a.add_residual) {
+            if (a.add_residual) {          // integer divisions (~0.8 us): ahead of the dependency wait
                 const long long e0 = gPref[b], e1 = gPref[b + 1];
                 int first_c = (int)((e0 * n_active) / tiles_total);
                 while ((long long)(first_c + 1) * tiles_total / n_active <= e0) ++first_c;
@@ -1008,6 +1019,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 n_share = last_c - first_c + 1;
                 my_share = cid - first_c;
             }
+            if (!waited_prev) { pdl_wait(); waited_prev = true; }
             if (a.x) {
                 const uint4* src = reinterpret_cast<const uint4*>(a.x + ((size_t)b * T + t) * H + (size_t)j * HS + part * CPP);
 #pragma unroll
