@@ -487,7 +487,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
                         *reinterpret_cast<float4*>(row + 4 * k) = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
             }
             tc_fence_before();
-            fence_proxy_async();
+            fence_proxy_async_smem();
             __syncthreads();
             if (tid < CS)
                 bulk_copy_to_peer(map_to_rank(sP + pb * p_bytes + (j * 16 * PR) * 4, tid), smem_u32(stg) + tid * 16 * PR * 4,
@@ -589,7 +589,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             if (lane == 0 && n >= 0)
                 a.record[(size_t)tr.b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
         }
-        fence_proxy_async();
+        fence_proxy_async_smem();
         __syncthreads();
         if (tid < 2 * CS) {
             const int dst = tid >> 1, part = tid & 1;
@@ -602,7 +602,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     // ---- phase: down projection of tile i, accumulated in tensor memory across the episode's tiles
     auto mma_dn = [&](int i, const TileRef& tr) {
         if (tid == 0) {
-            fence_proxy_async();
+            fence_proxy_async_smem();
             tc_fence_after();
             const uint32_t ht = sHT + buf_of(i) * 2 * S::HT_HALF;
 #pragma unroll
@@ -636,7 +636,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             const TileRef tr = tile_ref(g_lo + i);
             open_tile(i);
             cp_async_wait<0>();            // this tile's gate/up and down rows have landed
-            fence_proxy_async();
+            fence_proxy_async_smem();
             __syncthreads();
             RM_STAMP(6);
             float ha_pre[TPL];
@@ -671,7 +671,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
         // and the down projection of tile i, so each exchange travels while the other tile's work runs.
         open_tile(0);
         cp_async_wait<0>();
-        fence_proxy_async();
+        fence_proxy_async_smem();
         __syncthreads();
         RM_STAMP(6);
         mma_gu(0);
@@ -687,7 +687,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             if (more) {
                 open_tile(i + 1);
                 if (i == 0) cp_async_wait<0>(); else cp_async_wait<1>();      // gate/up rows of tile i+1 have landed
-                fence_proxy_async();
+                fence_proxy_async_smem();
                 __syncthreads();
                 mma_gu(i + 1);
             }
@@ -709,7 +709,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             wait_bar(bar_h(buf_of(i)), phase_of(i));
             RM_STAMP(11);
             cp_async_wait<1>();            // down rows of tile i have landed
-            fence_proxy_async();
+            fence_proxy_async_smem();
             __syncthreads();
             mma_dn(i, tr);
             wait_bar(bar_dn, par_dn);
