@@ -1070,7 +1070,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                                               ((((k & 63) >> 3) ^ (t & 7)) << 4)) = pack8(v + 8 * i, inv);
                 }
             }
-            fence_proxy_async();
+            fence_proxy_async_smem();
         }
         if (!a.x) par_s ^= 1;
         __syncthreads();                   // x is in place for the mma warp
@@ -1105,7 +1105,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(d1_free(pb));
-                    fence_proxy_async();
+                    fence_proxy_async_smem();
                     named_barrier(2, 128);
                     if (tid < CS)
                         bulk_copy_to_peer(map_to_rank(sP + pb * p_bytes + (j * 16 * PR) * 4, tid),
@@ -1241,7 +1241,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                     if ((lane & 15) == 0 && n >= 0)
                         a.record[(size_t)b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
                 }
-                fence_proxy_async();
+                fence_proxy_async_smem();
                 named_barrier(1, 128);
                 if (ot < 2 * CS) {
                     const int dst = ot >> 1, part = ot & 1;
