@@ -629,6 +629,32 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
         RM_STAMP(14);
     };
 
+    // ---- duties shared by all CTAs (any time after the dependency wait).  Episodes without a single active neuron have
+    // no cluster working on them: their residual passes through here.  Then the buffer the next layer accumulates
+    // into is cleared.  CTAs with tiles do this while they wait for the first tile's partial sums, so that it is not
+    // the tail of the kernel (the next layer's dependency wait ends when the last CTA exits).
+    bool duties_done = false;
+    auto shared_duties = [&]() {
+        duties_done = true;
+        if (a.add_residual) {
+            for (int b = 0; b < a.B; ++b) {
+                if (gPref[b + 1] != gPref[b]) continue;
+                const float4* src = reinterpret_cast<const float4*>(a.r_in + (size_t)b * T * H);
+                float* dst = a.r_out + (size_t)b * T * H;
+                for (size_t i = (size_t)blockIdx.x * FT + tid; i < (size_t)T * H / 4; i += (size_t)gridDim.x * FT) {
+                    const float4 v = src[i];
+                    add_residual4(ya_update, gate, H, dst + 4 * i, (size_t)b * T * H + (4 * i / H) * H, (int)(4 * i % H), b, v.x, v.y, v.z, v.w);
+                }
+            }
+        }
+        if (a.zero_buf) {
+            const size_t n4 = (size_t)a.B * T * H / 4;
+            float4* z = reinterpret_cast<float4*>(a.zero_buf);
+            for (size_t i = (size_t)blockIdx.x * FT + tid; i < n4; i += (size_t)gridDim.x * FT)
+                z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+
     if (!PIPE) {
         // ---- one tile at a time: open, gate/up, scatter, owner work, down.  Loads of the next tile are issued as
         // soon as the stage they go to is free, so they travel during the exchanges.
@@ -649,6 +675,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             if (refill) issue_gu(g_lo + i + 1);
             cp_async_commit();
             scatter(i, refill);
+            if (i == 0) shared_duties();
             wait_bar(bar_p(0), phase_of(i));           // every source's partial sums for this CTA's neurons are here
             RM_STAMP(9);
             reduce_bcast(i, tr, ha_pre);
@@ -730,26 +757,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
 
     // ---- teardown.  Everything peers send into this CTA's shared memory is counted on barriers this CTA has waited
     // for, so nothing is in flight towards it any more and it may exit without a cluster-wide wait.
-    // ---- duties shared by all CTAs, at the very end so that nothing on the exchange chain waits for their global
-    // traffic.  Episodes without a single active neuron have no cluster working on them: their residual passes
-    // through here.  Then the buffer the next layer accumulates into is cleared.
-    if (a.add_residual) {
-        for (int b = 0; b < a.B; ++b) {
-            if (gPref[b + 1] != gPref[b]) continue;
-            const float4* src = reinterpret_cast<const float4*>(a.r_in + (size_t)b * T * H);
-            float* dst = a.r_out + (size_t)b * T * H;
-            for (size_t i = (size_t)blockIdx.x * FT + tid; i < (size_t)T * H / 4; i += (size_t)gridDim.x * FT) {
-                const float4 v = src[i];
-                add_residual4(ya_update, gate, H, dst + 4 * i, (size_t)b * T * H + (4 * i / H) * H, (int)(4 * i % H), b, v.x, v.y, v.z, v.w);
-            }
-        }
-    }
-    if (a.zero_buf) {
-        const size_t n4 = (size_t)a.B * T * H / 4;
-        float4* z = reinterpret_cast<float4*>(a.zero_buf);
-        for (size_t i = (size_t)blockIdx.x * FT + tid; i < n4; i += (size_t)gridDim.x * FT)
-            z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+    if (!duties_done) shared_duties();
     cp_async_wait<0>();
     tc_fence_before();
     if (__syncthreads_or(gave_up)) linger_after_timeout();
