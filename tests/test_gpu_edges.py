@@ -1,0 +1,64 @@
+"""Edge cases of the tensor-core path: a single token, ragged neuron counts, the largest batch, a wrong hint, and the
+same through every kernel variant."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_19104_b200 import workloads as wl
+from harness import Model, assert_close, dev, lists_to_padded
+
+pytestmark = pytest.mark.gpu
+
+
+def step_case(lib, H, I, T, L, B, density, variant=0, hint=None, max_clusters=0, config=95):
+    import torch
+    w = wl.Workload(config, "edge", L, H, I, T, 1.0 / np.sqrt(H), 1, density, B=B)
+    model = Model(lib, w, B_max=B)
+    ctx = model.ctx
+    ctx.rm_set_option("variant", variant)
+    ctx.rm_set_option("max_clusters", max_clusters)
+    if hint is not None:
+        ctx.rm_set_option("count_hint", hint)
+    r0 = np.stack([wl.bf16_bits_to_f32(wl.step_input(w, 0, episode=b)) for b in range(B)])
+    lists = [[np.flatnonzero(wl.uniform(wl.tensor_key(11, config, l, 2, b), I) < density).astype(np.int32)
+              for l in range(L)] for b in range(B)]
+    idx, cnt = lists_to_padded([s for per_b in lists for s in per_b], (I + 3) // 4 * 4)
+    out = torch.empty(B, T, H, dtype=torch.float32, device="cuda")
+    ctx.rm_action_expert_step(model.packed, dev(r0), dev(idx), dev(cnt), idx.shape[1], out, B=B, T=T)
+    got = out.cpu().numpy()
+    for b in range(B):
+        i_b, c_b = lists_to_padded(lists[b], idx.shape[1])
+        assert_close(got[b], oracle.step(model.Wg, model.Wu, model.Wd, r0[b], i_b, c_b), f"episode {b}")
+    # dense pass with records on the same model
+    rec = torch.zeros(B, L, I, dtype=torch.float32, device="cuda")
+    ctx.rm_action_expert_step(model.packed, dev(r0), None, None, 0, out, records_out=rec, B=B, T=T)
+    want, want_rec = oracle.step(model.Wg, model.Wu, model.Wd, r0[0], return_records=True)
+    assert_close(out.cpu().numpy()[0], want, "dense")
+    assert np.all(np.abs(rec.cpu().numpy()[0] - want_rec) <= 2e-2 + 1e-2 * np.abs(want_rec))
+    assert ctx.rm_device_status() == 0
+    model.close()
+
+
+@pytest.mark.parametrize("variant", [0, 1, 3, 4])
+def test_single_token_and_ragged_neuron_count(lib, variant):
+    step_case(lib, H=1024, I=1000, T=1, L=2, B=1, density=0.37, variant=variant)      # I, K not multiples of 64
+
+
+@pytest.mark.parametrize("variant", [0, 3, 4])
+def test_wide_model_ragged(lib, variant):
+    step_case(lib, H=2048, I=712, T=33, L=2, B=2, density=0.5, variant=variant)
+
+
+def test_largest_batch(lib):
+    step_case(lib, H=1024, I=256, T=7, L=1, B=64, density=0.3)
+
+
+@pytest.mark.parametrize("hint", [1, 64, 100000])
+def test_a_wrong_count_hint_only_costs_time(lib, hint):
+    # the hint sizes the launch; the lists on the device decide what is computed
+    step_case(lib, H=1024, I=1024, T=51, L=2, B=1, density=0.4, hint=hint)
+
+
+def test_streaming_variant_with_few_ctas(lib):
+    # three CTAs walk all tiles of two episodes: several tiles per CTA, episode changes inside a CTA's sequence
+    step_case(lib, H=1024, I=1024, T=40, L=2, B=2, density=0.6, variant=4, max_clusters=3)
