@@ -71,13 +71,18 @@ class ClockSampler:
 
     def __init__(self, index: int):
         self.index = index
-        self.rows = []
+        self.rows = []                     # (host time, fields)
         self.proc = None
+        self.t_begin = None
+
+    def mark_begin(self):
+        """The sampler is started before the warm-up so that nvidia-smi is already reporting; samples count from here."""
+        self.t_begin = time.time()
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100", "-i",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50", "-i",
                  str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -86,7 +91,7 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
     def stop(self):
         if self.proc is None:
@@ -98,7 +103,9 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for ts, r in self.rows:
+            if self.t_begin is not None and ts < self.t_begin:
+                continue
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
@@ -235,13 +242,14 @@ def run_context(args, w: wl.Workload):
         ctx.rm_mask_compact([score], rm.RM_SRC_SCORE_F32, rm.RM_REDUCE_TOPK, rows, cnt, P, n_lists=1, k=k, I=P)
         ctx.rm_context_ffn(Wg, Wu, Wd, x, rows, cnt, P, S, R, yref, y_out)
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     for s in range(args.warmup):
         flush.fill_(s & 0xFF)
         step()
     torch.cuda.synchronize()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
+    sampler.mark_begin()
     l0 = ctx.launch_count()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     for s in range(args.steps):
@@ -419,6 +427,9 @@ def run_gpu(args, w: wl.Workload):
         if timed_events is not None:
             timed_events[1].record(stream)
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     for s in range(args.warmup):
         one_step(s)
     torch.cuda.synchronize()
@@ -426,9 +437,7 @@ def run_gpu(args, w: wl.Workload):
         dist.barrier()
     torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
+    sampler.mark_begin()
     launches0 = ctx.launch_count()
     events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     for s in range(args.steps):
