@@ -37,6 +37,7 @@ __device__ __forceinline__ float gelu_sig(float g) {              // g * sigmoid
 // ---------------------------------------------------------------- Eq. 2: one warp per row
 __global__ void __launch_bounds__(256) drift_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ xr,
                                                     int P, int H, float* __restrict__ score) {
+    pdl_launch_dependents();               // the selection kernel behind this one may set up
     const int p = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (p >= P) return;
     const uint4* a = reinterpret_cast<const uint4*>(x + (size_t)p * H);
@@ -68,6 +69,7 @@ __global__ void __launch_bounds__(256) ctx_gather_kernel(const __nv_bfloat16* __
                                                          const int32_t* __restrict__ count, int P, int S, int H, int r_pad,
                                                          __nv_bfloat16* __restrict__ xc, int* status) {
     pdl_launch_dependents();               // the first product may start now: its weight loads need nothing from here
+    pdl_wait();                            // the row list comes from the kernel in front
     const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= r_pad) return;
     int c = *count;
@@ -87,14 +89,31 @@ __global__ void __launch_bounds__(256) ctx_gather_kernel(const __nv_bfloat16* __
     for (int e = lane; e < H / 8; e += 32) d[e] = s ? s[e] : make_uint4(0, 0, 0, 0);
 }
 
-// ---------------------------------------------------------------- scatter: reference outputs, then the recomputed rows
+// ---------------------------------------------------------------- scatter: recomputed rows and kept reference rows
+// CTAs 0 .. r_pad-1: output row of recomputed row r = sum of the K slices.  CTAs r_pad .. r_pad+P-1: visual row p keeps
+// its reference output unless it is in the (ascending) list.
 __global__ void __launch_bounds__(256) ctx_scatter_kernel(const float* __restrict__ yp, int ksplit, int r_pad,
                                                           const int32_t* __restrict__ rows, const int32_t* __restrict__ count,
-                                                          int P, int S, int H, float* __restrict__ y_out) {
-    const int r = blockIdx.x;
+                                                          int P, int S, int H, const float* __restrict__ y_ref,
+                                                          float* __restrict__ y_out) {
+    pdl_wait();                            // the partial products come from the kernel in front
     int c = *count;
     c = c < 0 ? 0 : (c > P ? P : c);
     if (c + S > r_pad) c = r_pad - S;
+    if ((int)blockIdx.x >= r_pad) {
+        const int p = (int)blockIdx.x - r_pad;
+        if (y_out == y_ref) return;
+        int lo = 0, hi = c;                // is p in rows[0 .. c)?
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (rows[mid] < p) lo = mid + 1; else hi = mid;
+        }
+        if (lo < c && rows[lo] == p) return;
+        for (int e = threadIdx.x; e < H / 4; e += blockDim.x)
+            reinterpret_cast<float4*>(y_out + (size_t)p * H)[e] = reinterpret_cast<const float4*>(y_ref + (size_t)p * H)[e];
+        return;
+    }
+    const int r = blockIdx.x;
     int dst = -1;
     if (r < c) dst = rows[r];
     else if (r < c + S) dst = P + (r - c);
@@ -374,20 +393,35 @@ int rm_launch_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const voi
     __nv_bfloat16* h1 = reinterpret_cast<__nv_bfloat16*>(w);
     w += align_up((size_t)r_pad * I * sizeof(__nv_bfloat16), 1024);
     float* yp = reinterpret_cast<float*>(w);
-    // reference outputs first (unselected rows keep them), rows to recompute gathered
-    if (y_out != y_ref)
-        RM_CUDA_TRY(cudaMemcpyAsync(y_out, y_ref, (size_t)P * H * sizeof(float), cudaMemcpyDeviceToDevice, s));
-    ctx_gather_kernel<<<(r_pad + 7) / 8, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(x), rows, count, P, S, H, r_pad, xc,
-                                                     ctx->d_status);
-    ctx->launches++;
-    RM_CUDA_TRY(cudaGetLastError());
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((r_pad + 7) / 8);
+        cfg.blockDim = dim3(256);
+        cfg.stream = s;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, ctx_gather_kernel, static_cast<const __nv_bfloat16*>(x), rows, count, P, S, H, r_pad,
+                                       xc, ctx->d_status));
+        ctx->launches++;
+    }
     int rc = RM_ERR_SHAPE;
     if (r_pad == 64) rc = run_ffn<64>(ctx, Wg, Wu, Wd, xc, h1, yp, ksplit, s);
     else if (r_pad == 128) rc = run_ffn<128>(ctx, Wg, Wu, Wd, xc, h1, yp, ksplit, s);
     else if (r_pad == 256) rc = run_ffn<256>(ctx, Wg, Wu, Wd, xc, h1, yp, ksplit, s);
     if (rc != RM_OK) return rc;
-    ctx_scatter_kernel<<<r_pad, 256, 0, s>>>(yp, ksplit, r_pad, rows, count, P, S, H, y_out);
-    ctx->launches++;
-    RM_CUDA_TRY(cudaGetLastError());
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(r_pad + P);
+        cfg.blockDim = dim3(256);
+        cfg.stream = s;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, ctx_scatter_kernel, static_cast<const float*>(yp), ksplit, r_pad, rows, count, P, S, H,
+                                       y_ref, y_out));
+        ctx->launches++;
+    }
     return RM_OK;
 }

@@ -160,6 +160,10 @@ __global__ void __launch_bounds__(MASK_THREADS) mask_compact_kernel(MaskParams p
     const int I = p.I;
 
     for (int n = threadIdx.x; n < I; n += MASK_THREADS) votes[n] = 0;
+    // programmatic dependent launch: a kernel launched behind this one may start its prologue now; the records read
+    // below may come from the kernel in front of this one
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();
 
     auto all_valid = [](int) { return true; };
@@ -246,9 +250,18 @@ int rm_launch_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out
     if (smem > 40 * 1024)
         RM_CUDA_TRY(cudaFuncSetAttribute(mask_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (src->n_lists > 0) {
-        mask_compact_kernel<<<src->n_lists, MASK_THREADS, smem, s>>>(p);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(src->n_lists);
+        cfg.blockDim = dim3(MASK_THREADS);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = s;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, mask_compact_kernel, p));
         ctx->launches++;
-        RM_CUDA_TRY(cudaGetLastError());
     }
     return RM_OK;
 }
