@@ -455,6 +455,34 @@ def run_gpu(args, w: wl.Workload):
     step_ms = [a.elapsed_time(b) for a, b in events]
     total_ms = float(sum(step_ms))
 
+    # ---- side figures (outside the timed region of the headline): the same steps with a warm L2, the mask compaction
+    # alone, and (plain workloads) the dense reference step with record emission
+    def timed(fn, reps, flush_first):
+        evs = []
+        for i in range(reps):
+            if flush_first:
+                flush.fill_(i & 0xFF)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn(i)
+            b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) * 1e3 for a, b in evs]
+
+    warm_us = timed(lambda i: run_step(1 + i % (w.steps - 1), dev_inputs[(1 + i % (w.steps - 1)) % w.steps]), min(args.steps, 20), False)
+    compact_us = timed(lambda i: compact(), 5, True)
+    dense_us = None
+    if not anchored:
+        dense_us = timed(lambda i: ctx.rm_action_expert_step(packed, refs, None, None, 0, r_out, records_out=records, B=B, T=w.T),
+                         3, True)
+        compact()                                           # the lists again, from the records just rewritten
+    union_rows = None
+    if B > 1 and not anchored:
+        h_idx, h_cnt = idx.cpu().numpy().reshape(B, w.L, -1), cnt.cpu().numpy().reshape(B, w.L)
+        union_rows = float(np.mean([len(set().union(*[set(h_idx[b, l, :h_cnt[b, l]].tolist()) for b in range(B)]))
+                                    for l in range(w.L)]))
+
     e2e_in = torch.empty(B, w.T, w.H, dtype=torch.float32, device="cuda")
     # end to end through the host-buffer entry point (H2D of the step input, step, D2H of the result, sync)
     e2e_times = []
@@ -543,7 +571,18 @@ def run_gpu(args, w: wl.Workload):
             "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes},
             "gpu_launches": int(launches),
             "clocks": clocks,
+            "per_step_us": {"median": float(np.median(step_ms)) * 1e3 / B, "p10": float(np.percentile(step_ms, 10)) * 1e3 / B,
+                            "p90": float(np.percentile(step_ms, 90)) * 1e3 / B,
+                            "note": "rank 0, per episode; the step that rebuilds the masks (one in ten) is the p90 tail"},
+            "warm_l2_us_per_step": float(np.median(warm_us)) / B,
+            "mask_compact_us": {"value": float(np.median(compact_us)), "lists": int(n_lists)},
         }
+        if dense_us is not None:
+            line["dense_step_us"] = float(np.median(dense_us)) / B
+        if union_rows is not None:
+            line["roofline"]["union_weight_bytes_per_launch"] = int(union_rows * 3 * w.H * 2)
+            line["roofline"]["note"] = ("bytes_per_launch is the sum over the episodes' lists; the union of the lists (rows that "
+                                        "must leave HBM at least once) is given beside it")
         if cpu_us is not None:
             line["cpu_baseline"] = {"value": cpu_us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}
         print(json.dumps(line))
