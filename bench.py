@@ -153,6 +153,25 @@ def time_oracle(w: wl.Workload, steps: int, warmup: int, sample_layers: int = 3)
                                       f"(K={w.K} per layer), scaled by {scale_up:g}")
 
 
+def time_oracle_config0_single_thread():
+    """The small single-layer case (Bernoulli(0.30) mask on the config-1 layer shape) on one host thread."""
+    import oracle
+    w0 = wl.config0()
+    Wg, Wu, Wd = wl.layer_weights(w0, 0)
+    x, r = wl.step_input(w0, 0), wl.residual_input(w0)
+    sel = np.flatnonzero(wl.bernoulli_mask(w0)).astype(np.int32)
+    n = oracle.num_threads()
+    oracle.set_threads(1)
+    try:
+        oracle.masked_mlp(x, Wg, Wu, Wd, r, sel)
+        t0 = time.perf_counter()
+        oracle.masked_mlp(x, Wg, Wu, Wd, r, sel)
+        dt = time.perf_counter() - t0
+    finally:
+        oracle.set_threads(n)
+    return dt * 1e6, int(sel.size)
+
+
 def run_reference(args, w: wl.Workload):
     if rank_env()[1] != 0:                 # under a multi-rank launch rank 0 alone runs and prints
         return
@@ -585,6 +604,9 @@ def run_gpu(args, w: wl.Workload):
                                         "must leave HBM at least once) is given beside it")
         if cpu_us is not None:
             line["cpu_baseline"] = {"value": cpu_us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}
+            us0, k0 = time_oracle_config0_single_thread()
+            line["cpu_baseline"]["single_layer_one_thread_us"] = us0
+            line["cpu_baseline"]["single_layer_one_thread_case"] = f"configs[0]: one layer, H=1024, I=4096, T=51, K={k0}"
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
