@@ -496,6 +496,8 @@ def run_gpu(args, w: wl.Workload):
         dense_us = timed(lambda i: ctx.rm_action_expert_step(packed, refs, None, None, 0, r_out, records_out=records, B=B, T=w.T),
                          3, True)
         compact()                                           # the lists again, from the records just rewritten
+    # the same lists through the gather-read microbenchmark (layer by layer, cold L2): how fast they can leave HBM at all
+    gather_us = timed(lambda i: [ctx.rm_debug_gather_read(packed[l], idx[l], cnt[l:l + 1], w.I) for l in range(w.L)], 5, True)
     union_rows = None
     if B > 1 and not anchored:
         h_idx, h_cnt = idx.cpu().numpy().reshape(B, w.L, -1), cnt.cpu().numpy().reshape(B, w.L)
@@ -595,6 +597,11 @@ def run_gpu(args, w: wl.Workload):
                             "note": "rank 0, per episode; the step that rebuilds the masks (one in ten) is the p90 tail"},
             "warm_l2_us_per_step": float(np.median(warm_us)) / B,
             "mask_compact_us": {"value": float(np.median(compact_us)), "lists": int(n_lists)},
+            "gather_read_microbench": {
+                "us_per_layer": float(np.median(gather_us)) / w.L,
+                "gbs": int(round(K_mean)) * 3 * w.H * 2 / (float(np.median(gather_us)) / w.L * 1e-6) / 1e9,
+                "note": "episode 0's lists read with the kernels' access pattern (8 slices per neuron, 16-byte cp.async into "
+                        "two shared-memory stages) and discarded; one plain launch per layer, cold L2"},
         }
         if dense_us is not None:
             line["dense_step_us"] = float(np.median(dense_us)) / B

@@ -215,6 +215,12 @@ int rm_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, 
 int rm_sparse_mlp_static(const void* packed_layer, const void* x, const float* residual, const int32_t* idx,
                          const int32_t* count_dev, float* y, int T, int H, int I, rm_stream_t stream);
 
+/* Measurement aid (not part of the method): reads the packed rows of the listed neurons (idx NULL: every neuron) with
+ * the layer kernels' own access pattern -- 8 column-slice pieces per neuron, 16-byte cp.async into shared memory --
+ * and discards them.  Timed by the caller it gives the rate at which this list can leave HBM with this pattern. */
+int rm_debug_gather_read(rm_ctx* ctx, const void* packed_layer, const int32_t* idx, const int32_t* count_dev,
+                         int64_t list_cap, rm_stream_t stream);
+
 /* Reads and clears the device status word (0 or the first RM_ERR_* a kernel recorded).  Synchronises `stream`. */
 int rm_device_status(rm_ctx* ctx, int* host_out, rm_stream_t stream);
 

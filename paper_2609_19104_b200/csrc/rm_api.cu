@@ -106,6 +106,14 @@ int rm_pack_weights(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd,
     return rm_launch_pack(ctx, Wg, Wu, Wd, packed_out, down_colnorm, static_cast<cudaStream_t>(stream));
 }
 
+int rm_debug_gather_read(rm_ctx* ctx, const void* packed_layer, const int32_t* idx, const int32_t* count_dev,
+                         int64_t list_cap, rm_stream_t stream) {
+    if (!ctx || !packed_layer || (idx && !count_dev) || list_cap < 0) return RM_ERR_INVALID_ARG;
+    if (!all_aligned({packed_layer, idx})) return RM_ERR_ALIGN;
+    return rm_launch_gather_read(ctx, packed_layer, idx, count_dev, idx ? list_cap : ctx->g.I,
+                                 static_cast<cudaStream_t>(stream));
+}
+
 int rm_gather_weights(rm_ctx* ctx, const void* packed_layer, const int32_t* idx, const int32_t* count_dev,
                       int64_t list_cap, void* compact_out, rm_stream_t stream) {
     if (!ctx || !packed_layer || !idx || !count_dev || !compact_out || list_cap < 0) return RM_ERR_INVALID_ARG;

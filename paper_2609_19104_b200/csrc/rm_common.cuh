@@ -84,6 +84,8 @@ int rm_launch_context_drift(rm_ctx* ctx, const void* x, const void* x_ref, int P
 int rm_launch_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, const void* x, const int32_t* rows,
                           const int32_t* count, int P, int S, int r_pad, const float* y_ref, float* y_out, void* ws,
                           cudaStream_t s);
+int rm_launch_gather_read(rm_ctx* ctx, const void* packed, const int32_t* idx, const int32_t* count, int64_t cap,
+                          cudaStream_t s);
 int rm_launch_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out,
                            int64_t stride, cudaStream_t s);
 
