@@ -62,3 +62,19 @@ def test_a_wrong_count_hint_only_costs_time(lib, hint):
 def test_streaming_variant_with_few_ctas(lib):
     # three CTAs walk all tiles of two episodes: several tiles per CTA, episode changes inside a CTA's sequence
     step_case(lib, H=1024, I=1024, T=40, L=2, B=2, density=0.6, variant=4, max_clusters=3)
+
+
+def test_gather_read_microbenchmark_runs_and_reports_bad_counts(lib):
+    import torch
+    H, I, T = 1024, 512, 8
+    w = wl.Workload(96, "edge-gather", 1, H, I, T, 0.03, 1, 0.3)
+    model = Model(lib, w)
+    ctx = model.ctx
+    sel = np.flatnonzero(wl.uniform(wl.tensor_key(12, 96, 0, 2), I) < 0.4).astype(np.int32)
+    idx, cnt = lists_to_padded([sel], I)
+    ctx.rm_debug_gather_read(model.packed[0], dev(idx[0]), dev(cnt), I)            # a list
+    ctx.rm_debug_gather_read(model.packed[0], None, None, 0)                       # every neuron
+    assert ctx.rm_device_status() == 0
+    ctx.rm_debug_gather_read(model.packed[0], dev(idx[0]), dev(np.array([I + 7], np.int32)), I)
+    assert ctx.rm_device_status() != 0                                             # count above the capacity
+    model.close()
