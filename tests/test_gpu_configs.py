@@ -89,7 +89,7 @@ def pi0(lib):
     r_ref = f32_of(wl.reference_input(w))[None]
     out, rec = gpu_dense_records(model, r_ref)
     want_out, want_rec = oracle.step(model.Wg, model.Wu, model.Wd, r_ref[0], return_records=True)
-    assert_close(out[0], want_out, "dense reference step")
+    assert_close(out[0], want_out, "dense reference step", deep_dense=True)
     records_close(rec.cpu().numpy()[0], want_rec)
     yield model, rec, want_rec
     model.close()
@@ -139,11 +139,11 @@ def test_config3_density_sweep(lib, pi0, density):
     else:
         # density 1.0 is checked against the oracle's separate dense loop, as a full list and as idx = NULL
         want = oracle.step(model.Wg, model.Wu, model.Wd, r0)
-        assert_close(got, want, "config 3 rho=1.0 (full list)")
+        assert_close(got, want, "config 3 rho=1.0 (full list)", deep_dense=True)
         import torch
         out = torch.empty(1, w.T, w.H, dtype=torch.float32, device="cuda")
         model.ctx.rm_action_expert_step(model.packed, dev(r0[None]), None, None, 0, out, B=1, T=w.T)
-        assert_close(out.cpu().numpy()[0], want, "config 3 rho=1.0 (idx NULL)")
+        assert_close(out.cpu().numpy()[0], want, "config 3 rho=1.0 (idx NULL)", deep_dense=True)
 
 
 def test_config3_batched_eight_episodes(lib, pi0):
@@ -154,7 +154,7 @@ def test_config3_batched_eight_episodes(lib, pi0):
     out, rec = gpu_dense_records(model, refs, B=B)
     for b in (0, 5):                                               # two episodes of the dense pass in full
         want_out, want_rec = oracle.step(model.Wg, model.Wu, model.Wd, refs[b], return_records=True)
-        assert_close(out[b], want_out, f"batched dense, episode {b}")
+        assert_close(out[b], want_out, f"batched dense, episode {b}", deep_dense=True)
         records_close(rec.cpu().numpy()[b], want_rec)
     K = w.K
     idx, cnt, h_idx, h_cnt = gpu_topk_lists(lib, model, [rec.view(B * w.L, w.I)], K, B * w.L)
@@ -196,7 +196,7 @@ def test_config4_run_structured_vote_window(lib, pi0):
         recs.append(rec)
         if i in (0, 4):
             want_out, want_rec = oracle.step(Wg, Wu, Wd, r_ref[0], scale=scale, return_records=True)
-            assert_close(out[0], want_out, f"config 4 dense reference {i}")
+            assert_close(out[0], want_out, f"config 4 dense reference {i}", deep_dense=True)
             records_close(rec.cpu().numpy()[0], want_rec)
     K, votes = w.K, w.extra["min_votes"]
     assert K == 615 and votes == 3
@@ -310,7 +310,7 @@ def test_config5_anchor_groups_of_five_steps(lib, pi0):
             ctx.rm_action_expert_step_ex(model.packed, dev(r0[None]), idx, cnt, I, out, lib.RM_ANCHOR_UPDATE, y_an, h_an,
                                          h_stride, out_gate=d_gate, B=1, T=T)
             want = oracle.anchor_step_update(model.Wg, model.Wu, model.Wd, r0, h_idx, h_cnt, state[0], state[1], gate)
-        rels.append(assert_close(out.cpu().numpy()[0], want, f"config 5 step {s}"))
+        rels.append(assert_close(out.cpu().numpy()[0], want, f"config 5 step {s}", deep_dense=True))
     print(f"config5: rel_l2 per step max {max(rels):.2e}")
     assert ctx.rm_device_status() == 0
 

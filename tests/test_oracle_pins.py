@@ -564,3 +564,26 @@ def test_context_ffn_special_cases():
     assert d[sel].min() >= d[keep].max()
     # ceil(rho P): 0.26 * 20 = 5.2 -> 6 rows
     assert oracle.context_select(d, 0.26).size == 6
+
+
+def test_dense_stack_amplifies_one_ulp():
+    """Conditioning of the 18-layer dense step, shown on the oracle alone: every layer re-quantises x to bf16, so a
+    relative change of 1e-6 in the fp32 input (the size of fp32 summation noise) is carried and amplified until it
+    saturates at the level of the quantisation noise, about 2e-3 in relative L2, with single elements moving by more
+    than half of the per-element bound 2e-2 + 1e-2 |ref|.  One layer is well conditioned.  This is why comparisons of
+    dense full-depth outputs allow a few elements in 10^5 outside the per-element bound."""
+    w = wl.config1()
+    W = [wl.layer_weights(w, l) for l in range(w.L)]
+    Wg, Wu, Wd = zip(*W)
+    r0 = wl.bf16_bits_to_f32(wl.reference_input(w))
+    noise = wl.normal(wl.tensor_key(w.seed, 98, 0, 5), r0.size).reshape(r0.shape)
+    r1 = (r0.astype(np.float64) * (1.0 + 1e-6 * noise)).astype(np.float32)
+    assert 0 < np.max(np.abs(r1 - r0)) <= 8e-6 * np.max(np.abs(r0))
+    base, moved = oracle.step(Wg, Wu, Wd, r0), oracle.step(Wg, Wu, Wd, r1)
+    d = np.abs(moved.astype(np.float64) - base)
+    rel = np.linalg.norm(moved.astype(np.float64) - base) / np.linalg.norm(base)
+    assert 5e-4 < rel < 5e-3, rel                            # amplified a thousandfold, still inside the L2 bound
+    assert np.max(d / (2e-2 + 1e-2 * np.abs(base))) > 0.5    # single elements come close to the per-element bound
+    one0, one1 = oracle.step(Wg[:1], Wu[:1], Wd[:1], r0), oracle.step(Wg[:1], Wu[:1], Wd[:1], r1)
+    rel1 = np.linalg.norm(one1.astype(np.float64) - one0) / np.linalg.norm(one0)
+    assert rel1 < 1e-4, rel1
