@@ -123,3 +123,6 @@ int rm_launch_layer_ref(rm_ctx* ctx, const rm_layer_args& a, void* ws, cudaStrea
 bool rm_stream_supported(const rm_ctx* ctx, int B, int T);
 int rm_stream_debug_stamps(long long* host_out);
 int rm_launch_layer_stream(rm_ctx* ctx, const rm_layer_args& a, __nv_bfloat16* x_scratch, bool pdl, cudaStream_t s);
+// Tiled tensor map (a 128-byte CUtensorMap, 64-byte aligned) of an fp32 residual buffer [B, T, H] with boxes of
+// box_rows token rows x 128 columns of one episode, not swizzled: the target of the kernels' bulk adds.
+int rm_make_out_map(void* tensor_map, const float* ptr, int B, int T, int H, int box_rows);

@@ -17,6 +17,7 @@
 // Layers are chained with programmatic dependent launch: a layer's CTAs become resident, set up, issue the loads
 // of their first tile (weight addresses depend only on the index lists) and then wait (griddepcontrol.wait) for
 // the previous layer's atomics before touching activations.
+#include <cuda.h>
 #include <cstdio>
 #include <cstdlib>
 
@@ -182,7 +183,8 @@ struct TileRef {
 
 // EQ4 = false compiles the anchor-relative update and the output gate out (the zero-fill step pays nothing for them)
 template <int NTOK, int HS, bool PIPE, bool EQ4>
-__global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_kernel(const FusedArgs a) {
+__global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_kernel(const FusedArgs a,
+                                                                                               const __grid_constant__ CUtensorMap tmOut) {
     const int anchor_mode = EQ4 ? a.anchor_mode : (int)RM_ANCHOR_NONE;
     const float* const gate = EQ4 ? a.gate : nullptr;
     const float* const ya_update = anchor_mode == RM_ANCHOR_UPDATE ? a.y_anchor : nullptr;
@@ -628,7 +630,41 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     };
 
     // ---- phase: add this CTA's [T x Hs] partial of y to the residual stream
-    auto flush = [&](const TileRef& tr) {
+    // The last flush of a run (no loads are in flight into the gate/up stage any more; the staged partial sums that
+    // may have used it have been consumed, or the owners' h could not have arrived) goes through that stage: the
+    // accumulator is laid out as [token][128 columns] per 128-column block, scaled by the gate, and the copy engine
+    // adds each block to the output as one box of the [B, T, H] tensor map.  Earlier flushes of a run (batches) and
+    // the anchor step, which also accumulates the ungated partial into y_anchor, add with red.global from registers.
+    bool bulk_pending = false;
+    auto flush = [&](const TileRef& tr, bool final_tile) {
+        if (final_tile && anchor_mode != RM_ANCHOR_WRITE) {
+            float* stage = reinterpret_cast<float*>(gbase + S::OFF_GU);
+            const int wrow = warp & 3;
+#pragma unroll
+            for (int mm = 0; mm < HS / 128; ++mm) {
+                const int cl = wrow * 32 + lane;
+                const float gc = gate ? gate[(size_t)tr.b * H + j * HS + mm * 128 + cl] : 1.f;
+                for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
+                    float v[32];
+                    tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)(wrow * 32) << 16) + c0, v);
+#pragma unroll
+                    for (int k = 0; k < 32; ++k)
+                        if (c0 + k < T) stage[(mm * NTOK + c0 + k) * 128 + cl] = gc * v[k];
+                }
+            }
+            tc_fence_before();
+            fence_proxy_async_smem();
+            __syncthreads();
+            if (tid == 0) {
+#pragma unroll
+                for (int mm = 0; mm < HS / 128; ++mm)
+                    tensor_reduce_add_3d(&tmOut, j * HS + mm * 128, 0, tr.b, smem_u32(stage + mm * NTOK * 128));
+                bulk_commit();
+                bulk_pending = true;
+            }
+            RM_STAMP(14);
+            return;
+        }
         flush_partial<NTOK, HS>(a.r_out + (size_t)tr.b * T * H, a.y_anchor ? a.y_anchor + (size_t)tr.b * T * H : nullptr,
                                 gate ? gate + (size_t)tr.b * H : nullptr, anchor_mode == RM_ANCHOR_WRITE, tmem_d2,
                                 warp & 3, lane, (warp >> 2) * 32, 64, T, H, j * HS);
@@ -696,7 +732,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             if (refill) issue_dn(g_lo + i + 1);
             cp_async_commit();
             RM_STAMP(13);
-            if (tr.last) flush(tr);
+            if (tr.last) flush(tr, !refill);
 #ifdef RM_PHASE_TIMING
             stamp_ok = false;              // first tile only
 #endif
@@ -753,7 +789,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
             if (more) issue_dn(g_lo + i + 1);
             cp_async_commit();
             RM_STAMP(13);
-            if (tr.last) flush(tr);
+            if (tr.last) flush(tr, !more);
 #ifdef RM_PHASE_TIMING
             stamp_ok = false;
 #endif
@@ -767,6 +803,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     // for, so nothing is in flight towards it any more and it may exit without a cluster-wide wait.
     if (!duties_done) shared_duties();
     cp_async_wait<0>();
+    if (bulk_pending) bulk_wait_read_all();        // the copy engine has read the staged accumulator
     tc_fence_before();
     if (__syncthreads_or(gave_up)) linger_after_timeout();
     if (warp == 0) tmem_dealloc(tmem_d1, S::TMEM_COLS);
@@ -813,7 +850,7 @@ struct SmemWS {
 };
 
 template <int NTOK, int HS, bool EQ4>
-__global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a) {
+__global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tmOut) {
     const int anchor_mode = EQ4 ? a.anchor_mode : (int)RM_ANCHOR_NONE;
     const float* const gate = EQ4 ? a.gate : nullptr;
     const float* const ya_update = anchor_mode == RM_ANCHOR_UPDATE ? a.y_anchor : nullptr;
@@ -904,6 +941,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
         return r;
     };
     bool gave_up = false;
+    bool bulk_pending = false;                 // thread 0: a bulk add of the staged accumulator is in flight
     auto wait_bar_at = [&](uint32_t bar, uint32_t parity, int line) {
         if (!mbar_wait(bar, parity)) {
             rm_set_status_at(a.status, RM_ERR_TIMEOUT, (line << 12) | (int)(blockIdx.x & 0xfffu));
@@ -1152,10 +1190,39 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                 const int it = it0 + seg - 1;
                 wait_bar(bar_dn(it & 1), (it >> 1) & 1);
                 tc_fence_after();
-                flush_partial<NTOK, HS>(a.r_out + (size_t)b * T * H, a.y_anchor ? a.y_anchor + (size_t)b * T * H : nullptr,
-                                        gate ? gate + (size_t)b * H : nullptr, anchor_mode == RM_ANCHOR_WRITE, tmem_d2,
-                                        warp, lane, 0, 32, T, H, j * HS);
-                tc_fence_before();
+                if (it == n_tiles - 1 && anchor_mode != RM_ANCHOR_WRITE) {
+                    // last flush of the run: nothing is in flight into the gate/up stage any more.  The accumulator
+                    // goes there as [token][128 columns] per 128-column block, scaled by the gate, and the copy
+                    // engine adds each block to the output as one box of the [B, T, H] tensor map.
+                    float* stage = reinterpret_cast<float*>(gbase + S::OFF_GU);
+#pragma unroll
+                    for (int mm = 0; mm < HS / 128; ++mm) {
+                        const int cl = warp * 32 + lane;
+                        const float gc = gate ? gate[(size_t)b * H + j * HS + mm * 128 + cl] : 1.f;
+                        for (int c0 = 0; c0 < NTOK; c0 += 32) {
+                            float v[32];
+                            tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)(warp * 32) << 16) + c0, v);
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (c0 + e < T) stage[(mm * NTOK + c0 + e) * 128 + cl] = gc * v[e];
+                        }
+                    }
+                    tc_fence_before();
+                    fence_proxy_async_smem();
+                    named_barrier(2, 128);
+                    if (tid == 0) {
+#pragma unroll
+                        for (int mm = 0; mm < HS / 128; ++mm)
+                            tensor_reduce_add_3d(&tmOut, j * HS + mm * 128, 0, b, smem_u32(stage + mm * NTOK * 128));
+                        bulk_commit();
+                        bulk_pending = true;
+                    }
+                } else {
+                    flush_partial<NTOK, HS>(a.r_out + (size_t)b * T * H, a.y_anchor ? a.y_anchor + (size_t)b * T * H : nullptr,
+                                            gate ? gate + (size_t)b * H : nullptr, anchor_mode == RM_ANCHOR_WRITE, tmem_d2,
+                                            warp, lane, 0, 32, T, H, j * HS);
+                    tc_fence_before();
+                }
             }
         } else if (warp < 8) {
             // ================= owner warps: warp ow handles local neurons ow and ow + 4, one per half-warp; a lane
@@ -1378,6 +1445,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
         }
     }
     cp_async_wait<0>();
+    if (bulk_pending) bulk_wait_read_all();        // the copy engine has read the staged accumulator
     tc_fence_before();
     if (__syncthreads_or(gave_up)) linger_after_timeout();
     if (warp == 8) tmem_dealloc(tmem_d1, S::TMEM_COLS);
@@ -1409,7 +1477,10 @@ int launch_fused_ws(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, c
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = pdl ? 2 : 1;
-    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, a));
+    alignas(64) CUtensorMap tm_out;
+    const int rc = rm_make_out_map(&tm_out, a.r_out, a.B, a.T, a.H, NTOK);
+    if (rc != RM_OK) return rc;
+    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, a, tm_out));
     ctx->launches++;
     return RM_OK;
 }
@@ -1440,7 +1511,10 @@ int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cuda
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = pdl ? 2 : 1;
-    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, a));
+    alignas(64) CUtensorMap tm_out;
+    const int rc = rm_make_out_map(&tm_out, a.r_out, a.B, a.T, a.H, NTOK);
+    if (rc != RM_OK) return rc;
+    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, a, tm_out));
     ctx->launches++;
     return RM_OK;
 }

@@ -608,6 +608,10 @@ int launch_tiles(rm_ctx* ctx, const StreamArgs& a, int n_ctas, cudaStream_t s) {
 
 }  // namespace
 
+int rm_make_out_map(void* tensor_map, const float* ptr, int B, int T, int H, int box_rows) {
+    return make_map_out(static_cast<CUtensorMap*>(tensor_map), ptr, (uint64_t)B, (uint64_t)T, (uint64_t)H, (uint32_t)box_rows);
+}
+
 int rm_stream_debug_stamps(long long* host_out) {
 #ifdef RM_PHASE_TIMING
     return cudaMemcpyFromSymbol(host_out, g_st_stamps, sizeof(long long) * 64) == cudaSuccess ? RM_OK : RM_ERR_CUDA;
