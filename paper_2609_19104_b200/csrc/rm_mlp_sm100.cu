@@ -115,6 +115,25 @@ __host__ __device__ constexpr int p_row_for(int T) { return 4 * (((T + 3) / 4) |
 // to the episode's residual stream, times the output gate; the anchor step of Eq. 4 also accumulates the ungated
 // partial into y_anchor.  Pointers are already offset to the episode.  wrow: which 32-lane quarter of the accumulator
 // this warp reads; token columns c0_first, c0_first + c0_step, ...
+// Width in tensor-memory columns of one 128-row block of the down accumulator.  At H = 2048 with 64-token tiles the
+// product is issued once per K step against the operand [h_hi | h_lo] (N = 128: the two h tiles lie one
+// leading-dimension step apart), so the block holds Wd*h_hi in columns 0..63 and Wd*h_lo in columns 64..127 and
+// readers add the halves; that halves the number of down-product instructions, which bound the tile rate there.
+// Elsewhere (H = 1024, where the lean kernel must stay within 128 registers and the products are not the limit, and
+// 32-token tiles) two N = NTOK products accumulate into one block.
+__host__ __device__ constexpr bool d2_wide(int ntok, int hs) { return ntok == 64 && hs == 256; }
+__host__ __device__ constexpr int d2_width(int ntok, int hs) { return d2_wide(ntok, hs) ? 128 : ntok; }
+template <int NTOK, int HS>
+__device__ __forceinline__ void ld_d2(uint32_t taddr, float (&v)[32]) {
+    tmem_ld32(taddr, v);
+    if (d2_wide(NTOK, HS)) {
+        float w[32];
+        tmem_ld32(taddr + NTOK, w);
+#pragma unroll
+        for (int k = 0; k < 32; ++k) v[k] += w[k];
+    }
+}
+
 template <int NTOK, int HS>
 __device__ __noinline__ void flush_partial(float* __restrict__ r_out, float* __restrict__ y_anchor,
                                            const float* __restrict__ gate, bool write_anchor, uint32_t tmem_d2, int wrow,
@@ -125,7 +144,7 @@ __device__ __noinline__ void flush_partial(float* __restrict__ r_out, float* __r
         const float gc = gate ? gate[col] : 1.f;
         for (int c0 = c0_first; c0 < NTOK; c0 += c0_step) {
             float v[32];
-            tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)(wrow * 32) << 16) + c0, v);
+            ld_d2<NTOK, HS>(tmem_d2 + mm * d2_width(NTOK, HS) + ((uint32_t)(wrow * 32) << 16) + c0, v);
             // explicit red.global.add: with the gate factor in front, atomicAdd() compiled to something far slower
             // here (measured: 60 against 37 us per H = 2048 layer)
             if (write_anchor) {
@@ -136,6 +155,25 @@ __device__ __noinline__ void flush_partial(float* __restrict__ r_out, float* __r
 #pragma unroll
             for (int k = 0; k < 32; ++k)
                 if (c0 + k < T) red_add_f32(r_out + (size_t)(c0 + k) * H + col, gc * v[k]);
+        }
+    }
+}
+
+// The same accumulator, scaled by the gate, laid out in shared memory as [128-column block][token][128 columns] for
+// the copy engine's bulk add (one box of the [B, T, H] tensor map per block).  Out of line for the same reason.
+template <int NTOK, int HS>
+__device__ __noinline__ void stage_partial(float* __restrict__ stage, const float* __restrict__ gate, uint32_t tmem_d2,
+                                           int wrow, int lane, int c0_first, int c0_step, int T, int col_base) {
+#pragma unroll
+    for (int mm = 0; mm < HS / 128; ++mm) {
+        const int cl = wrow * 32 + lane;
+        const float gc = gate ? gate[col_base + mm * 128 + cl] : 1.f;
+        for (int c0 = c0_first; c0 < NTOK; c0 += c0_step) {
+            float v[32];
+            ld_d2<NTOK, HS>(tmem_d2 + mm * d2_width(NTOK, HS) + ((uint32_t)(wrow * 32) << 16) + c0, v);
+#pragma unroll
+            for (int k = 0; k < 32; ++k)
+                if (c0 + k < T) stage[(mm * NTOK + c0 + k) * 128 + cl] = gc * v[k];
         }
     }
 }
@@ -159,7 +197,7 @@ struct Smem {
     static constexpr int OFF_PREF = OFF_N + 2 * NT * 4;      // [MAXB+1] tile prefix, [MAXB] counts
     static constexpr int OFF_BAR = ((OFF_PREF + (2 * MAXB + 1) * 4 + 7) / 8) * 8;
     static constexpr int OFF_P = ((OFF_BAR + 96 + 15) / 16) * 16;   // NB x [CS][16][p_row] floats (+ staging), sized at launch
-    static constexpr int TMEM_COLS_USED = NB * NTOK + (HS / 128) * NTOK;
+    static constexpr int TMEM_COLS_USED = NB * NTOK + (HS / 128) * d2_width(NTOK, HS);
     static constexpr int TMEM_COLS = TMEM_COLS_USED <= 32 ? 32 : TMEM_COLS_USED <= 64 ? 64 :
                                      TMEM_COLS_USED <= 128 ? 128 : TMEM_COLS_USED <= 256 ? 256 : 512;
     static int total_bytes(int T) { return OFF_P + (NB + (STAGED ? 1 : 0)) * CS * 16 * p_row_for(T) * 4 + 1024; }
@@ -356,7 +394,7 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
 
     uint32_t par_dn = 0, par_s = 0;
     constexpr uint32_t IDESC_GU = idesc_bf16_f32(128, NTOK, false, false);
-    constexpr uint32_t IDESC_DN = idesc_bf16_f32(128, NTOK, true, true);
+    constexpr uint32_t IDESC_DN = idesc_bf16_f32(128, d2_width(NTOK, HS), true, true);
     const uint64_t desc_k = smem_desc_sw128(0, 16, 1024);        // K-major operand: 8-row groups 1024 B apart
     const uint64_t desc_mn = smem_desc_sw128(0, 8192, 1024);     // MN-major operand: 64-element blocks 8192 B apart
     const int n_tiles = g_hi - g_lo;
@@ -620,9 +658,10 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
                     const uint64_t aa = desc_mn | desc_addr(sDN + mm * 16384 + ks * 2048);
-                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + ks * 2048), IDESC_DN,
+                    mma_bf16_ss(tmem_d2 + mm * d2_width(NTOK, HS), aa, desc_mn | desc_addr(ht + ks * 2048), IDESC_DN,
                                 !(tr.first && ks == 0));
-                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + S::HT_HALF + ks * 2048), IDESC_DN, true);
+                    if (!d2_wide(NTOK, HS))
+                        mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + S::HT_HALF + ks * 2048), IDESC_DN, true);
                 }
             mma_commit(bar_dn);
         }
@@ -639,19 +678,8 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
     auto flush = [&](const TileRef& tr, bool final_tile) {
         if (final_tile && anchor_mode != RM_ANCHOR_WRITE) {
             float* stage = reinterpret_cast<float*>(gbase + S::OFF_GU);
-            const int wrow = warp & 3;
-#pragma unroll
-            for (int mm = 0; mm < HS / 128; ++mm) {
-                const int cl = wrow * 32 + lane;
-                const float gc = gate ? gate[(size_t)tr.b * H + j * HS + mm * 128 + cl] : 1.f;
-                for (int c0 = (warp >> 2) * 32; c0 < NTOK; c0 += 64) {
-                    float v[32];
-                    tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)(wrow * 32) << 16) + c0, v);
-#pragma unroll
-                    for (int k = 0; k < 32; ++k)
-                        if (c0 + k < T) stage[(mm * NTOK + c0 + k) * 128 + cl] = gc * v[k];
-                }
-            }
+            stage_partial<NTOK, HS>(stage, gate ? gate + (size_t)tr.b * H : nullptr, tmem_d2, warp & 3, lane, (warp >> 2) * 32,
+                                    64, T, j * HS);
             tc_fence_before();
             fence_proxy_async_smem();
             __syncthreads();
@@ -845,7 +873,7 @@ struct SmemWS {
                                                             // to six tiles ahead of the owner warps that read them
     static constexpr int OFF_BAR = ((OFF_PREF + (2 * MAXB + 1) * 4 + 7) / 8) * 8;
     static constexpr int OFF_P = ((OFF_BAR + 224 + 15) / 16) * 16;  // [2][CS][16][p_row] (+ [2] staging), sized at launch
-    static constexpr int TMEM_COLS = 256;                    // D1 x 2 (NTOK each) + D2 (HS/128 x NTOK) <= 256
+    static constexpr int TMEM_COLS = 2 * NTOK + (HS / 128) * d2_width(NTOK, HS) <= 256 ? 256 : 512;   // D1 x 2 + D2 blocks
     static int total_bytes(int T) { return OFF_P + (STAGED ? 4 : 2) * CS * 16 * p_row_for(T) * 4 + 1024; }
 };
 
@@ -1032,7 +1060,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
     __syncthreads();                       // gPref / gCnt
 
     constexpr uint32_t IDESC_GU = idesc_bf16_f32(128, NTOK, false, false);
-    constexpr uint32_t IDESC_DN = idesc_bf16_f32(128, NTOK, true, true);
+    constexpr uint32_t IDESC_DN = idesc_bf16_f32(128, d2_width(NTOK, HS), true, true);
     const uint64_t desc_k = smem_desc_sw128(0, 16, 1024);
     const uint64_t desc_mn = smem_desc_sw128(0, 8192, 1024);
     const int n_tiles = g_hi - g_lo;
@@ -1195,18 +1223,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                     // goes there as [token][128 columns] per 128-column block, scaled by the gate, and the copy
                     // engine adds each block to the output as one box of the [B, T, H] tensor map.
                     float* stage = reinterpret_cast<float*>(gbase + S::OFF_GU);
-#pragma unroll
-                    for (int mm = 0; mm < HS / 128; ++mm) {
-                        const int cl = warp * 32 + lane;
-                        const float gc = gate ? gate[(size_t)b * H + j * HS + mm * 128 + cl] : 1.f;
-                        for (int c0 = 0; c0 < NTOK; c0 += 32) {
-                            float v[32];
-                            tmem_ld32(tmem_d2 + mm * NTOK + ((uint32_t)(warp * 32) << 16) + c0, v);
-#pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                if (c0 + e < T) stage[(mm * NTOK + c0 + e) * 128 + cl] = gc * v[e];
-                        }
-                    }
+                    stage_partial<NTOK, HS>(stage, gate ? gate + (size_t)b * H : nullptr, tmem_d2, warp, lane, 0, 32, T, j * HS);
                     tc_fence_before();
                     fence_proxy_async_smem();
                     named_barrier(2, 128);
@@ -1379,8 +1396,10 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                             for (int k2 = 0; k2 < 2; ++k2) {
                                 const int ks = h * 2 + k2;
                                 const uint64_t aa = desc_mn | desc_addr(sDN + mm * 16384 + ks * 2048);
-                                mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + ks * 2048), IDESC_DN, !(k == 0 && ks == 0));
-                                mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + S::HT_HALF + ks * 2048), IDESC_DN, true);
+                                mma_bf16_ss(tmem_d2 + mm * d2_width(NTOK, HS), aa, desc_mn | desc_addr(ht + ks * 2048), IDESC_DN,
+                                            !(k == 0 && ks == 0));
+                                if (!d2_wide(NTOK, HS))
+                                    mma_bf16_ss(tmem_d2 + mm * NTOK, aa, desc_mn | desc_addr(ht + S::HT_HALF + ks * 2048), IDESC_DN, true);
                             }
                         mma_commit(dnh_free(h));
                         if (h == 0) RM_WS(it, 9);

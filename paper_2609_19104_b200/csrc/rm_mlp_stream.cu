@@ -134,13 +134,6 @@ __device__ __forceinline__ long long st_now() {
 #define RM_ST(i) do { } while (0)
 #endif
 
-// One box of a tiled tensor map into shared memory; its bytes are counted on an mbarrier of this CTA.  The innermost
-// coordinate times the element size must be a multiple of 16 bytes (here: multiples of 64 bf16 columns).
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t mbar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(mbar) : "memory");
-}
-
 // GeLU-tanh(g) through the identity 0.5 (1 + tanh z) = 1 / (1 + exp(-2 z)): one exponential and one division
 __device__ __forceinline__ float gelu_tanh_sig(float g) {
     const float z2 = 1.5957691216057308f * (g + 0.044715f * g * g * g);       // 2 sqrt(2/pi) (g + 0.044715 g^3)
