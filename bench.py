@@ -82,7 +82,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50", "-i",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20", "-i",
                  str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -101,21 +101,31 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ts, r in self.rows:
-            if self.t_begin is not None and ts < self.t_begin:
-                continue
-            try:
-                sm.append(float(r[0]))
-                mx.append(float(r[1]))
-                for n, v in zip(names, r[2:6]):
-                    if v.lower().startswith("active"):
-                        reasons.add(n)
-            except Exception:
-                continue
+
+        def summarise(rows):
+            sm, mx, reasons = [], [], set()
+            for _, r in rows:
+                try:
+                    sm.append(float(r[0]))
+                    mx.append(float(r[1]))
+                    for n, v in zip(names, r[2:6]):
+                        if v.lower().startswith("active"):
+                            reasons.add(n)
+                except Exception:
+                    continue
+            return sm, mx, reasons
+
+        # samples from the start of the timed steps to the end of the run (the side figures and the end-to-end steps
+        # keep the GPU on the same work); a run too short for one such sample falls back to every sample taken
+        # since the warm-up began, and says so
+        window = "timed steps onward"
+        sm, mx, reasons = summarise([x for x in self.rows if self.t_begin is None or x[0] >= self.t_begin])
+        if not sm:
+            window = "whole run including warm-up"
+            sm, mx, reasons = summarise(self.rows)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "window": window}
 
 
 # ------------------------------------------------------------------------------------------------ reference arm
