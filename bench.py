@@ -32,7 +32,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused layer launch, from the ncu capture summarised in
 # profiles/fused_layer_kernel_config1.md
-TRAFFIC_BYTES_PER_LAUNCH = {"pi0-stack-top25": 6.797e6}
+TRAFFIC_BYTES_PER_LAUNCH = {"pi0-stack-top25": 6.794e6}
 
 
 def measured_hbm_peak():
