@@ -8,14 +8,17 @@
 //                  stage), accumulates D1[128 x T_pad] over the whole width H in tensor memory, applies GeLU-tanh(g)*u
 //                  (record, Eq. 4 bookkeeping), keeps h = hi + lo (bf16 pair) in shared memory, then streams the tile's
 //                  down rows 128 output columns at a time, D2 = Wd_block * h in tensor memory (two slots), and adds
-//                  each finished block to the output with red.global.add.
-//                  One warp loads (cp.async.bulk.tensor boxes of one 128-byte row piece per neuron, straight into the
-//                  swizzled operand layout; 16-byte cp.async gathers top out near 16 bytes per clock and SM, far too
-//                  little when one SM has to pull a whole tile), four warps read tensor memory and do the arithmetic,
-//                  one thread issues the tcgen05.mma instructions.
+//                  each finished block to the output: transposed through shared memory and added by the copy engine
+//                  as one box of the [B, T, H] tensor map (red.global.add in the anchor step, which also accumulates
+//                  the ungated block into y_anchor).
+//                  Four warps load: 16-byte cp.async gathers straight into the swizzled operand layout for index
+//                  lists (they top out near 16 bytes per clock and SM), cp.async.bulk.tensor boxes of 64 neurons x 64
+//                  columns for runs of consecutive neurons (one-row boxes were tried for lists and are far slower);
+//                  four warps read tensor memory and do the arithmetic, one thread issues the tcgen05.mma
+//                  instructions.
 //
 // Compared with the cluster kernels this trades the exchange latency (three hops per tile) for re-reading x from L2
-// once per tile and for T*H atomic adds per tile; it wins when there are enough tiles to occupy the SMs.
+// once per tile and for T*H added elements per tile; it wins when there are enough tiles to occupy the SMs.
 #include <cuda.h>
 
 #include <mutex>
@@ -36,7 +39,7 @@ constexpr int STAGE = 24576;           // + x block: up to 64 token rows x 128 b
 struct StreamArgs {
     const __nv_bfloat16* packed;
     const __nv_bfloat16* x;            // [B,T,H] bf16 (normalised)
-    float* r_out;                      // [B,T,H] fp32, already holding the residual part; tiles are added with red
+    float* r_out;                      // [B,T,H] fp32, already holding the residual part; tiles are added to it
     const int32_t* idx;
     const int32_t* count;
     int64_t idx_stride, list_cap, count_stride;
