@@ -52,6 +52,15 @@ extern int rm_last_cuda_error;            // cudaError_t of the last failed runt
         if (_e != cudaSuccess) { rm_last_cuda_error = (int)_e; return RM_ERR_CUDA; } \
     } while (0)
 
+// Dynamic shared-memory size a kernel has been configured for, per device: cudaFuncSetAttribute applies to the
+// current device only, and one process may hold contexts on several devices.  (A race between two threads costs a
+// redundant call, nothing else.)
+struct rm_smem_configured {
+    int bytes[64];
+    bool covers(int device, int need) const { return device >= 0 && device < 64 && bytes[device] >= need; }
+    void set(int device, int need) { if (device >= 0 && device < 64) bytes[device] = need; }
+};
+
 static inline bool rm_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 __device__ __forceinline__ void rm_set_status(int* status, int code) {

@@ -309,11 +309,11 @@ int run_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, const _
     const int H = ctx->g.H, I = ctx->g.I;
     using SA = SmemCtx<NR, true>;
     using SB = SmemCtx<NR, false>;
-    static bool configured = false;
-    if (!configured) {
+    static rm_smem_configured configured = {};
+    if (!configured.covers(ctx->device, SA::TOTAL)) {
         RM_CUDA_TRY(cudaFuncSetAttribute(ctx_gemm_kernel<NR, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SA::TOTAL));
         RM_CUDA_TRY(cudaFuncSetAttribute(ctx_gemm_kernel<NR, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SB::TOTAL));
-        configured = true;
+        configured.set(ctx->device, SA::TOTAL);
     }
     CUtensorMap tg, tu, tx, td, th;
     int rc;

@@ -51,10 +51,10 @@ int rm_launch_gather_read(rm_ctx* ctx, const void* packed, const int32_t* idx, c
     if (g.H % 64 != 0) return RM_ERR_UNSUPPORTED;
     const int smem = 2 * GNT * 3 * g.Hs * 2 + 128;
     if (smem > 200 * 1024) return RM_ERR_UNSUPPORTED;
-    static int configured = 0;
-    if (configured < smem) {
+    static rm_smem_configured configured = {};
+    if (!configured.covers(ctx->device, smem)) {
         RM_CUDA_TRY(cudaFuncSetAttribute(gather_read_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        configured = smem;
+        configured.set(ctx->device, smem);
     }
     const int groups = ctx->sm_count >= 8 ? ctx->sm_count / 8 : 1;             // 18 groups of 8 CTAs on 148 SMs
     gather_read_kernel<<<groups * 8, GT, smem, s>>>(static_cast<const __nv_bfloat16*>(packed), idx, count, cap, g.H, g.I,

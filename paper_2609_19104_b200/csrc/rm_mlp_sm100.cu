@@ -1476,11 +1476,11 @@ int launch_fused_ws(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, c
     const bool eq4 = a.anchor_mode != RM_ANCHOR_NONE || a.gate != nullptr;
     auto kern = eq4 ? fused_layer_ws_kernel<NTOK, HS, true> : fused_layer_ws_kernel<NTOK, HS, false>;
     const int smem = S::total_bytes(a.T);
-    static int configured = 0;
-    if (configured < smem) {
+    static rm_smem_configured configured = {};
+    if (!configured.covers(ctx->device, smem)) {
         RM_CUDA_TRY(cudaFuncSetAttribute(fused_layer_ws_kernel<NTOK, HS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         RM_CUDA_TRY(cudaFuncSetAttribute(fused_layer_ws_kernel<NTOK, HS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        configured = smem;
+        configured.set(ctx->device, smem);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_clusters * CS);
@@ -1510,11 +1510,11 @@ int launch_fused(rm_ctx* ctx, const FusedArgs& a, int n_clusters, bool pdl, cuda
     const bool eq4 = a.anchor_mode != RM_ANCHOR_NONE || a.gate != nullptr;
     auto kern = eq4 ? fused_layer_kernel<NTOK, HS, PIPE, true> : fused_layer_kernel<NTOK, HS, PIPE, false>;
     const int smem = S::total_bytes(a.T);
-    static int configured = 0;
-    if (configured < smem) {
+    static rm_smem_configured configured = {};
+    if (!configured.covers(ctx->device, smem)) {
         RM_CUDA_TRY(cudaFuncSetAttribute(fused_layer_kernel<NTOK, HS, PIPE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         RM_CUDA_TRY(cudaFuncSetAttribute(fused_layer_kernel<NTOK, HS, PIPE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        configured = smem;
+        configured.set(ctx->device, smem);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_clusters * CS);

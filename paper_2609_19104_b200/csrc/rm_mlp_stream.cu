@@ -572,13 +572,13 @@ int launch_tiles(rm_ctx* ctx, const StreamArgs& a, int n_ctas, cudaStream_t s) {
     const bool gather = a.idx != nullptr;
     auto kern = gather ? (eq4 ? stream_tile_kernel<NTOK, true, true> : stream_tile_kernel<NTOK, false, true>)
                        : (eq4 ? stream_tile_kernel<NTOK, true, false> : stream_tile_kernel<NTOK, false, false>);
-    static bool configured = false;
-    if (!configured) {
+    static rm_smem_configured configured = {};
+    if (!configured.covers(ctx->device, S::TOTAL)) {
         RM_CUDA_TRY(cudaFuncSetAttribute(stream_tile_kernel<NTOK, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
         RM_CUDA_TRY(cudaFuncSetAttribute(stream_tile_kernel<NTOK, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
         RM_CUDA_TRY(cudaFuncSetAttribute(stream_tile_kernel<NTOK, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
         RM_CUDA_TRY(cudaFuncSetAttribute(stream_tile_kernel<NTOK, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
-        configured = true;
+        configured.set(ctx->device, S::TOTAL);
     }
     CUtensorMap tmW, tmX, tmOut;
     int rc = make_map(&tmW, a.packed, (uint64_t)a.I, (uint64_t)3 * a.H, NT);       // used without a list only
