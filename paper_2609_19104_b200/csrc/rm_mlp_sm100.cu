@@ -1364,7 +1364,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                         if (h == 0 || !both) {
                             wait_bar(guh_full(h), it & 1);
                             if (h == 0) both = mbar_try_wait(guh_full(1), it & 1);
-                            fence_proxy_async();
+                            fence_proxy_async_smem();
                         }
                         if (h == 0) RM_WS(it, 1);
                         tc_fence_after();
@@ -1396,7 +1396,7 @@ __global__ void __launch_bounds__(WT, 1) fused_layer_ws_kernel(const FusedArgs a
                         if (h == 0 || !both) {
                             wait_bar(dnh_full(h), it & 1);
                             if (h == 0) both = mbar_try_wait(dnh_full(1), it & 1);
-                            fence_proxy_async();
+                            fence_proxy_async_smem();
                         }
                         RM_WS(it, 8 + 2 * h);
                         tc_fence_after();
