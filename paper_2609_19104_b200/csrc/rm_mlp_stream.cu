@@ -414,7 +414,7 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
                     *reinterpret_cast<uint4*>(rowp + NT * 128 + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                 }
             }
-            fence_proxy_async();
+            fence_proxy_async_smem();
             mbar_arrive(h_full);
             if (m == 0) RM_ST(9);
             // finished down blocks: lane = output column, token columns.  Transposed through shared memory into
@@ -480,7 +480,7 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
                 wait_bar(full(blk % NSTAGE), (blk / NSTAGE) & 1);
                 if (kb == 0) RM_ST(3);
                 if (kb == KBN - 1) RM_ST(4);
-                if (GATHER) fence_proxy_async();
+                if (GATHER) fence_proxy_async_smem();
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
@@ -497,7 +497,7 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
                 const uint32_t st = sRing + (blk % NSTAGE) * STAGE;
                 if (mbc >= 2) wait_bar(d2_free(slot), ((mbc >> 1) - 1) & 1);
                 wait_bar(full(blk % NSTAGE), (blk / NSTAGE) & 1);
-                if (GATHER) fence_proxy_async();
+                if (GATHER) fence_proxy_async_smem();
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
