@@ -26,14 +26,16 @@ inline bool use_fused(const rm_ctx* ctx, int B, int T) {
 // gathers at most ~38 GB/s with 16-byte cp.async and adds at most ~20 GB/s with red.global, so a tile costs it
 // ~25 us); below that the cluster kernels, which spread a tile over 8 SMs, win.  H = 1024 only: at H = 2048 the
 // warp-specialised cluster kernel is ahead at every size measured.  `masked` says whether a count is in play.
-inline bool use_stream(const rm_ctx* ctx, bool masked, int B, int T) {
+// anchor_write: the anchor step of Eq. 4 adds its blocks with per-thread reds (it also accumulates y_anchor), which
+// keeps the streaming variant behind the cluster kernels until there is about a tile per SM
+inline bool use_stream(const rm_ctx* ctx, bool masked, int B, int T, bool anchor_write = false) {
     if (ctx->path == 1 || !rm_stream_supported(ctx, B, T)) return false;
     if (ctx->variant_override == 4) return true;
-    if (ctx->variant_override != 0 || ctx->g.H != 1024) return false;
+    if (ctx->variant_override != 0) return false;
     const int per_episode = masked ? ctx->count_hint : ctx->g.I;
     if (per_episode <= 0) return false;
     const long long tiles = (long long)((per_episode + 63) / 64) * B;
-    return tiles >= ctx->stream_min_tiles;
+    return tiles >= (anchor_write && ctx->stream_min_tiles < 112 ? 112 : ctx->stream_min_tiles);
 }
 
 }  // namespace
@@ -56,7 +58,9 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->g.Hs = desc->H / RM_NS;
     c->launches = 0;
     c->status_detail = 0;
-    c->stream_min_tiles = 112;             // measured: ahead of the cluster kernels from about 8 episodes x 16 tiles
+    // measured crossover with the cluster kernels: from the point where their clusters would walk a second tile
+    // (H = 1024: 40 tiles, 24 against 25 us per layer) or a third (H = 2048: 64 tiles, 39 against 39 us; 96: 40 against 50)
+    c->stream_min_tiles = desc->H == 2048 ? 64 : 40;
     c->d_status = nullptr;
     cudaDeviceProp prop;
     if (cudaGetDevice(&c->device) != cudaSuccess || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess ||
@@ -243,7 +247,7 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
     // Fused path: layer l reads rot[l%3] (the caller's r_in for l = 0), accumulates into rot[(l+1)%3] and clears
     // rot[(l+2)%3] for the layer after next; the last layer accumulates straight into r_out when that is a
     // different buffer from r_in.
-    const bool stream = fused && use_stream(ctx, count_dev != nullptr, B, T);
+    const bool stream = fused && use_stream(ctx, count_dev != nullptr, B, T, an.mode == RM_ANCHOR_WRITE);
     const bool direct_out = fused && r_out != r_in;
     if (fused && !stream) {
         RM_CUDA_TRY(cudaMemsetAsync(g.L == 1 && direct_out ? r_out : rot[1], 0, n_bytes, s));

@@ -114,12 +114,14 @@ template <int NTOK>
 struct SmemST {
     static constexpr int OFF_RING = 0;
     static constexpr int OFF_HT = OFF_RING + NSTAGE * STAGE;       // h tile: hi 8 KB, lo 8 KB (64 neurons x 128 bytes)
-    static constexpr int OFF_Y = OFF_HT + 2 * NT * 128;            // 32 KB: GeLU exchange [2][token][neuron] fp32, then
-                                                                   // the transposed down block [token][128 columns] fp32
-    static constexpr int OFF_REC = OFF_Y + 32768;                  // record halves of the second token half
+    static constexpr int OFF_Y = OFF_HT + 2 * NT * 128;            // 2 x 32 KB: GeLU exchange [2][token][neuron] fp32 (first
+                                                                   // buffer), then the transposed down blocks [token][128
+                                                                   // columns] fp32, alternating between the two buffers
+    static constexpr int OFF_REC = OFF_Y + 65536;                  // record halves of the second token half
     static constexpr int OFF_PREF = OFF_REC + NT * 4;              // tile prefix per episode, counts
     static constexpr int OFF_BAR = ((OFF_PREF + (2 * MAXB + 1) * 4 + 7) / 8) * 8;
     static constexpr int TOTAL = OFF_BAR + 256 + 1024;             // + slack for the 1024-byte alignment
+    static_assert(TOTAL <= 232448, "the streaming kernel's buffers exceed the 227 KB a CTA may use");
     static constexpr int TMEM_COLS = NTOK == 64 ? 256 : 128;       // D1 + two D2 slots, power of two
 };
 
@@ -435,17 +437,18 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
                               *reinterpret_cast<float(*)[32]>(y + c0));
                 tc_fence_before();
                 mbar_arrive(d2_free(slot));
-                if (m == 0) bulk_wait_read_all();                  // the previous box has left shared memory
+                if (m == 0) bulk_wait_read_but_one();              // the box sent from this buffer two blocks ago has left it
                 named_barrier(1, 128);                             // the previous block's rows have been read
                 if (!ya_b) {
+                    float* gYb = gY + (mbc & 1) * 8192;            // the copy engine reads one buffer while the other fills
                     const float gm = gate ? gate[(size_t)b * H + mb * 128 + m] : 1.f;
 #pragma unroll
                     for (int t = 0; t < NTOK; ++t)
-                        if (t < T) gY[t * 128 + m] = gm * y[t];
+                        if (t < T) gYb[t * 128 + m] = gm * y[t];
                     fence_proxy_async_smem();
                     named_barrier(1, 128);
                     if (m == 0) {
-                        tensor_reduce_add_3d(&tmOut, mb * 128, 0, b, smem_u32(gY));
+                        tensor_reduce_add_3d(&tmOut, mb * 128, 0, b, smem_u32(gYb));
                         bulk_commit();
                     }
                 } else {
