@@ -103,7 +103,10 @@ int rm_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32
 /* ---- rm_gather_weights: the paper's own preparation of the selected weights (Sec. 4.1: "Selected weights are
  * prepared in shared compact buffers and reused across each group's steps"; Sec. 5 "Overlapping Retrieval and Weight
  * Gathering"), as a comparison variant to gathering inside the products.  Copies the packed rows of the listed
- * neurons to the front of compact_out: compact row p = packed row idx[p] for p < count.  compact_out holds at least
+ * neurons to the front of compact_out: compact row p = packed row idx[p] for p < count; the rows from count up to the
+ * next multiple of 64 (where the buffer has them) are cleared, because a kernel may fetch the last 64-neuron tile whole
+ * and multiply its unused rows by zero -- a compact layer built by other means must hold finite values there too.
+ * compact_out holds at least
  * min(list_cap, I) rows of 3*H bf16 (rm_packed_layer_bytes is always enough) and is itself a packed layer: pass it to
  * rm_sparse_mlp / rm_action_expert_step with idx = NULL and the same count_dev ("the leading count neurons"), and the
  * result is the masked layer over the listed neurons.  Activation records and anchor activations of such a call are

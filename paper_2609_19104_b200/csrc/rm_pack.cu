@@ -50,7 +50,8 @@ __global__ void __launch_bounds__(256) colnorm_kernel(const __nv_bfloat16* __res
     out[n] = sqrtf(s);
 }
 
-// Compact copy of the listed neurons' packed rows: out row p = packed row idx[p], p < count.  One warp per row
+// Compact copy of the listed neurons' packed rows: out row p = packed row idx[p], p < count (rows up to the next
+// multiple of 64 are cleared, later rows are left alone).  One warp per row
 // (3H bf16, contiguous in both buffers), 16 bytes per lane and iteration.
 __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ packed, const int32_t* __restrict__ idx,
                                                           const int32_t* __restrict__ count, int64_t cap,
@@ -61,7 +62,14 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restric
         if (blockIdx.x == 0 && threadIdx.x == 0) rm_set_status(status, RM_ERR_INDEX);
         c = c < 0 ? 0 : (int)(cap < (int64_t)I ? cap : (int64_t)I);
     }
-    if (p >= c) return;
+    if (p >= c) {
+        // the rest of the last 64-neuron tile is zero-filled: kernels that fetch a compact layer in whole-tile boxes
+        // multiply those rows by h = 0, which must not meet a NaN left in the buffer
+        const int64_t rows = cap < (int64_t)I ? cap : (int64_t)I;
+        if (p < ((c + 63) & ~63) && p < rows)
+            for (int e = lane; e < row_u4; e += 32) out[(size_t)p * row_u4 + e] = make_uint4(0, 0, 0, 0);
+        return;
+    }
     const int n = idx[p];
     if (n < 0 || n >= I) {
         if (lane == 0) rm_set_status(status, RM_ERR_INDEX);

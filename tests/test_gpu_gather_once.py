@@ -64,3 +64,32 @@ def test_gather_reports_bad_indices_and_counts(lib):
     ctx.rm_gather_weights(model.packed[0], bad, dev(np.array([I + 1], np.int32)), I)     # count above the capacity
     assert ctx.rm_device_status() != 0
     model.close()
+
+
+@pytest.mark.parametrize("variant", [0, 1, 3, 4])
+def test_compact_layers_in_buffers_full_of_nan(lib, variant):
+    """Kernels that fetch a compact layer in whole 64-neuron tiles read rows past the count of the last tile and
+    multiply them by h = 0.  The compact buffers here start as bf16 NaN patterns and the counts are not multiples of
+    64: rm_gather_weights clears the rest of the last tile, so every variant must return the masked step, finite."""
+    import torch
+    H, I, T, L = 1024, 4096, 51, 2
+    w = wl.Workload(94, "tiny-gather-nan", L, H, I, T, 1.0 / np.sqrt(H), 1, 0.8)
+    model = Model(lib, w)
+    ctx = model.ctx
+    lists = [np.flatnonzero(wl.uniform(wl.tensor_key(9, 94, l, 3), I) < 0.8).astype(np.int32) for l in range(L)]
+    lists = [s[:-1] if s.size % 64 == 0 else s for s in lists]
+    assert all(s.size % 64 != 0 and s.size > 40 * 64 for s in lists)      # enough tiles for the streaming variant
+    idx, cnt = lists_to_padded(lists, I)
+    d_idx, d_cnt = dev(idx), dev(cnt)
+    compact = []
+    for l in range(L):
+        buf = torch.full((ctx.packed_layer_bytes() // 2,), 0x7FC0, dtype=torch.int16, device="cuda").view(torch.uint8)
+        compact.append(ctx.rm_gather_weights(model.packed[l], d_idx[l], d_cnt[l:l + 1], I, compact_out=buf))
+    ctx.rm_set_option("variant", variant)
+    ctx.rm_set_option("count_hint", int(cnt.max()))
+    r0 = wl.bf16_bits_to_f32(wl.step_input(w, 0))
+    out = torch.empty(1, T, H, dtype=torch.float32, device="cuda")
+    ctx.rm_action_expert_step(compact, dev(r0[None]), None, d_cnt, 0, out, B=1, T=T)
+    assert_close(out.cpu().numpy()[0], oracle.step(model.Wg, model.Wu, model.Wd, r0, idx, cnt), f"variant {variant}")
+    assert ctx.rm_device_status() == 0
+    model.close()
