@@ -225,9 +225,11 @@ def test_every_tensor_core_variant_and_the_portable_path_agree_with_the_oracle(l
     model.close()
 
 
+@pytest.mark.parametrize("masked", [False, True])
 @pytest.mark.parametrize("H,I,T", [(1024, 1024, 64), (1024, 1024, 62), (1024, 2048, 51), (2048, 2048, 51)])
-def test_repeated_dense_stacks_agree_across_runs_and_variants(lib, H, I, T):
-    """Races show up as rare wrong token rows, not as a steady error: the same two-layer dense stack is run 60 times
+def test_repeated_dense_stacks_agree_across_runs_and_variants(lib, H, I, T, masked):
+    """Races show up as rare wrong token rows, not as a steady error: the same two-layer stack (dense, or masked with
+    index lists) is run 60 times
     through every tensor-core variant (default clusters: one or two tiles per cluster) and every result must match
     the first lean-kernel result.  (The two-tile variant once produced wrong rows in ~7 % of such runs for T > 60; it
     is no longer selected there.)"""
@@ -238,15 +240,22 @@ def test_repeated_dense_stacks_agree_across_runs_and_variants(lib, H, I, T):
     ctx = model.ctx
     r0 = dev(wl.bf16_bits_to_f32(wl.step_input(w, 0))[None])
     out = torch.empty(1, T, H, dtype=torch.float32, device="cuda")
+    idx = cnt = d_idx = d_cnt = None
+    if masked:                                             # index lists of ~70 % of the neurons: the gathering loaders
+        lists = [np.flatnonzero(wl.uniform(wl.tensor_key(4, 92, l, 8), I) < 0.7).astype(np.int32) for l in range(L)]
+        idx, cnt = lists_to_padded(lists, I)
+        d_idx, d_cnt = dev(idx), dev(cnt)
+        ctx.rm_set_option("count_hint", int(cnt.max()))
 
     def run(variant):
         ctx.rm_set_option("path", 2)
         ctx.rm_set_option("variant", variant)
-        ctx.rm_action_expert_step(model.packed, r0, None, None, 0, out, B=1, T=T)
+        ctx.rm_action_expert_step(model.packed, r0, d_idx, d_cnt, I if masked else 0, out, B=1, T=T)
         return out.cpu().numpy()[0].copy()
 
     ref = run(1)
-    assert_close(ref, oracle.step(model.Wg, model.Wu, model.Wd, wl.bf16_bits_to_f32(wl.step_input(w, 0))), "lean kernel")
+    assert_close(ref, oracle.step(model.Wg, model.Wu, model.Wd, wl.bf16_bits_to_f32(wl.step_input(w, 0)), idx, cnt),
+                 "lean kernel")
     for variant in (1, 2, 3, 4):
         for rep in range(60):
             got = run(variant)
