@@ -801,6 +801,10 @@ __global__ void __launch_bounds__(FT, (HS == 128 && !PIPE ? 2 : 1)) fused_layer_
                 const bool refill = i + 2 < n_tiles;
                 if (refill) issue_gu(g_lo + i + 2);
                 cp_async_commit();
+                // The staging area (and, without one, the gate/up stage of a last tile) is shared by consecutive
+                // tiles: this CTA's copies of tile i's partial sums must all have been read before tile i+1 is staged
+                // over them.  They have once h(i) is complete here: every owner has then finished its reduction.
+                if (S::STAGED || !refill) wait_bar(bar_h(buf_of(i)), phase_of(i));
                 scatter(i + 1, refill);
             } else {
                 cp_async_commit();
@@ -1658,11 +1662,6 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
         if (fits_t > 232448) variant = 2;
         else if (ctx->max_clusters_override <= 0 || cap > ctx->fused_clusters) cap = ctx->fused_clusters;
     }
-    // The two-tile variant is not used for T > 60 (64-float rows in the exchange buffers): there, and only there, a
-    // stack of two or more layers with two tiles per cluster came out with wrong token rows in ~7 % of the runs
-    // (one layer alone never did; the lean kernel on the same shapes never did in thousands of runs).  The cause has
-    // not been found; the variant is a test and fallback variant, and the lean kernel takes these launches.
-    if (variant == 2 && la.T > 60) variant = 1;
     if (variant == 2 && ctx->max_clusters_override <= 0) cap = ctx->fused_clusters;      // one CTA per SM
     // Clusters: no more than the cap, and when the tile count is known, the fewest that keep the longest run of
     // tiles per cluster as short as the cap allows (40 tiles under a cap of 32: 20 clusters of 2, not 32 of 1 or 2).

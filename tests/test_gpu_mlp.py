@@ -231,8 +231,8 @@ def test_repeated_dense_stacks_agree_across_runs_and_variants(lib, H, I, T, mask
     """Races show up as rare wrong token rows, not as a steady error: the same two-layer stack (dense, or masked with
     index lists) is run 60 times
     through every tensor-core variant (default clusters: one or two tiles per cluster) and every result must match
-    the first lean-kernel result.  (The two-tile variant once produced wrong rows in ~7 % of such runs for T > 60; it
-    is no longer selected there.)"""
+    the first lean-kernel result.  (The two-tile variant once produced wrong rows in ~7 % of such runs for T > 60: it
+    staged a tile's partial sums over the previous tile's while those were still being copied out.)"""
     import torch
     L = 2
     w = tiny(H=H, I=I, T=T, L=L, sigma=1.0 / np.sqrt(H), B=1, config=92)
