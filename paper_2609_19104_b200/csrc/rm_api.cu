@@ -58,9 +58,10 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->g.Hs = desc->H / RM_NS;
     c->launches = 0;
     c->status_detail = 0;
-    // measured crossover with the cluster kernels: from the point where their clusters would walk a second tile
-    // (H = 1024: 40 tiles, 24 against 25 us per layer) or a third (H = 2048: 64 tiles, 39 against 39 us; 96: 40 against 50)
-    c->stream_min_tiles = desc->H == 2048 ? 64 : 40;
+    // measured crossover with the cluster kernels.  H = 1024: at 48 tiles the lean kernel is level or ahead (3 episodes
+    // x 16 tiles: 126 against 134 us per step; one episode of 48 tiles: 378 against 373), at 64 the streaming variant
+    // is 5-7 % ahead, at 80 by 28 %.  H = 2048: level at 64 tiles (39 against 39 us per layer), 40 against 50 at 96.
+    c->stream_min_tiles = desc->H == 2048 ? 64 : 56;
     c->d_status = nullptr;
     cudaDeviceProp prop;
     if (cudaGetDevice(&c->device) != cudaSuccess || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess ||
