@@ -29,11 +29,6 @@ __device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* tm, int
                  ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(mbar) : "memory");
 }
 
-__device__ __forceinline__ float gelu_sig(float g) {              // g * sigmoid(2 sqrt(2/pi) (g + 0.044715 g^3))
-    const float z2 = 1.5957691216057308f * (g + 0.044715f * g * g * g);
-    return __fdividef(g, 1.0f + __expf(-z2));
-}
-
 // ---------------------------------------------------------------- Eq. 2: one warp per row
 __global__ void __launch_bounds__(256) drift_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ xr,
                                                     int P, int H, float* __restrict__ score) {
@@ -248,9 +243,15 @@ __global__ void __launch_bounds__(CT, 1) ctx_gemm_kernel(const CtxGemmArgs a, co
                 tmem_ld32(tmem + NR + ((uint32_t)(warp * 32) << 16) + c0, u);
                 // h for 32 activation rows x this neuron -> staging [row][128 neurons] bf16, then 16-byte stores
                 named_barrier(1, 128);
+                // in stages over the 32 values, so that the exponentials and divisions of different rows overlap
+                // (one warp per scheduler runs this; a value-by-value chain costs ~140 clocks per value)
+                float e[32];
 #pragma unroll
-                for (int t = 0; t < 32; ++t)
-                    reinterpret_cast<__nv_bfloat16*>(stg)[t * 128 + m] = __float2bfloat16_rn(gelu_sig(v[t]) * u[t]);
+                for (int t = 0; t < 32; ++t) e[t] = __expf(-1.5957691216057308f * (v[t] + 0.044715f * v[t] * v[t] * v[t]));
+#pragma unroll
+                for (int t = 0; t < 32; ++t) e[t] = __fdividef(v[t], 1.0f + e[t]) * u[t];
+#pragma unroll
+                for (int t = 0; t < 32; ++t) reinterpret_cast<__nv_bfloat16*>(stg)[t * 128 + m] = __float2bfloat16_rn(e[t]);
                 named_barrier(1, 128);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {

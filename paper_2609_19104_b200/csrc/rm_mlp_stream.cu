@@ -139,12 +139,6 @@ __device__ __forceinline__ long long st_now() {
 #define RM_ST(i) do { } while (0)
 #endif
 
-// GeLU-tanh(g) through the identity 0.5 (1 + tanh z) = 1 / (1 + exp(-2 z)): one exponential and one division
-__device__ __forceinline__ float gelu_tanh_sig(float g) {
-    const float z2 = 1.5957691216057308f * (g + 0.044715f * g * g * g);       // 2 sqrt(2/pi) (g + 0.044715 g^3)
-    return __fdividef(g, 1.0f + __expf(-z2));
-}
-
 constexpr int SE = 288;                // threads: 4 epilogue warps (0-3), 4 loader warps (4-7), issuer warp (8)
 
 // GATHER: the tile's neurons come from an index list, their rows are gathered with 16-byte cp.async (about 16 bytes
@@ -347,6 +341,7 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
                 tmem_ld32(tmem_d1 + ((uint32_t)(w4 * 32) << 16) + c0, *reinterpret_cast<float(*)[32]>(v + c0));
             tc_fence_before();
             mbar_arrive(d1_free);
+            if (m == 0) RM_ST(40);
             // lanes 0..63 hold the gate rows, lanes 64..127 the up rows.  Thread (q, half 0) finishes tokens 0..TH-1
             // of neuron q, thread (q, half 1) tokens TH..NTOK-1: each passes the other the half it does not need.
             float* xg = gY;                                        // gate values of the second token half [t][q]
@@ -359,15 +354,28 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
                 for (int t = 0; t < TH; ++t) xu[t * NT + q] = v[t];
             }
             named_barrier(1, 128);
+            if (m == 0) RM_ST(41);
             const int tb = half * TH;                              // first token of this thread
             float hv[TH];
             float rec = 0.f;
+            // in stages over all TH elements, so that the exponentials and divisions of different tokens overlap (one
+            // warp per scheduler runs this: a token-by-token chain costs ~140 clocks per token)
+            {
+                float e[TH];
 #pragma unroll
-            for (int t = 0; t < TH; ++t) {
-                const float gg = half == 0 ? v[t] : xg[t * NT + q];
-                const float uu = half == 0 ? xu[t * NT + q] : v[TH + t];
-                hv[t] = (tb + t < T && n >= 0) ? gelu_tanh_sig(gg) * uu : 0.f;
-                rec += fabsf(hv[t]);
+                for (int t = 0; t < TH; ++t) {
+                    const float gg = half == 0 ? v[t] : xg[t * NT + q];
+                    hv[t] = gg;
+                    e[t] = __expf(-1.5957691216057308f * (gg + 0.044715f * gg * gg * gg));
+                }
+#pragma unroll
+                for (int t = 0; t < TH; ++t) e[t] = __fdividef(hv[t], 1.0f + e[t]);     // GeLU-tanh(g) = g / (1 + exp(-2z))
+#pragma unroll
+                for (int t = 0; t < TH; ++t) {
+                    const float uu = half == 0 ? xu[t * NT + q] : v[TH + t];
+                    hv[t] = (tb + t < T && n >= 0) ? e[t] * uu : 0.f;
+                    rec += fabsf(hv[t]);
+                }
             }
             if (anchor_mode != RM_ANCHOR_NONE && n >= 0) {
                 float* hap = a.h_anchor + ((size_t)b * a.I + n) * a.h_stride + tb;
@@ -395,6 +403,7 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
                     a.record[(size_t)b * a.record_stride + n] = a.record_scale ? rec * a.record_scale[n] : rec;
                 }
             }
+            if (m == 0) RM_ST(42);
             if (k > 0) wait_bar(h_free, (k - 1) & 1);              // the previous tile's down products are complete
             // row q of the h tile: 64 tokens in bf16, 16-byte chunks swizzled by the row; hi at 0, lo at 8 KB
             {
