@@ -570,7 +570,7 @@ def run_gpu(args, w: wl.Workload):
         launches_per_step = launches / args.steps                 # fused layer launches + mask compaction share
         # the kernel the library picks for this launch shape (see the variant selection in the library)
         tiles_per_launch = (int(round(K_mean)) + 63) // 64 * B
-        stream_from = 56 if w.H == 1024 else 64                   # the library's default crossover ("stream_min_tiles")
+        stream_from = 48 if w.H == 1024 else 64                   # the library's default crossover ("stream_min_tiles")
         if args.variant == 4 or (args.variant == 0 and tiles_per_launch >= stream_from):
             kernel_name = "stream_prep_kernel + stream_tile_kernel"
         elif w.H == 1024:

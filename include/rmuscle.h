@@ -245,7 +245,7 @@ int64_t rm_launch_count(const rm_ctx* ctx);
  *                         of consecutive tiles run concurrently; for clusters that walk many tiles), 4 = streaming
  *                         (no clusters: every CTA owns whole tiles; for launches with many tiles)
  *   "stream_min_tiles"    launches with at least this many 64-neuron tiles use variant 4 when the variant is chosen
- *                         per launch (default 56 at H = 1024, 64 at H = 2048)                                   */
+ *                         per launch (default 48 at H = 1024, 64 at H = 2048)                                   */
 int rm_set_option(rm_ctx* ctx, const char* name, int value);
 
 /* Read-only facts: "fused_clusters" (co-resident clusters of the tcgen05 kernel, 0 when that path is

@@ -58,10 +58,12 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->g.Hs = desc->H / RM_NS;
     c->launches = 0;
     c->status_detail = 0;
-    // measured crossover with the cluster kernels.  H = 1024: at 48 tiles the lean kernel is level or ahead (3 episodes
-    // x 16 tiles: 126 against 134 us per step; one episode of 48 tiles: 378 against 373), at 64 the streaming variant
-    // is 5-7 % ahead, at 80 by 28 %.  H = 2048: level at 64 tiles (39 against 39 us per layer), 40 against 50 at 96.
-    c->stream_min_tiles = desc->H == 2048 ? 64 : 56;
+    // measured crossover with the cluster kernels.  H = 1024: at 32 tiles the lean kernel is far ahead (270 against
+    // 370 us per step); at 48 the two are level on 3 episodes x 16 tiles (127 against 126) and the streaming variant
+    // is 7 % ahead on one episode of 48 tiles (378 against 350); at 64 it is 10 % ahead, at 80 by 30 %.
+    // H = 2048: the warp-specialised kernel is ahead at 52 tiles (512 against 582), level at 64, behind at 96 (50
+    // against 38 us per layer).
+    c->stream_min_tiles = desc->H == 2048 ? 64 : 48;
     c->d_status = nullptr;
     cudaDeviceProp prop;
     if (cudaGetDevice(&c->device) != cudaSuccess || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess ||
