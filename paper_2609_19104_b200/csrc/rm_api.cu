@@ -26,8 +26,9 @@ inline bool use_fused(const rm_ctx* ctx, int B, int T) {
 // gathers at most ~38 GB/s with 16-byte cp.async and adds at most ~20 GB/s with red.global, so a tile costs it
 // ~25 us); below that the cluster kernels, which spread a tile over 8 SMs, win.  H = 1024 only: at H = 2048 the
 // warp-specialised cluster kernel is ahead at every size measured.  `masked` says whether a count is in play.
-// anchor_write: the anchor step of Eq. 4 adds its blocks with per-thread reds (it also accumulates y_anchor), which
-// keeps the streaming variant behind the cluster kernels until there is about a tile per SM
+// anchor_write: the anchor step of Eq. 4 adds two boxes per block (y_anchor and the output) and stores h_anchor; measured
+// on the anchor schedule it stays behind the cluster kernels at 64 tiles (352 against 334 us per step), so it keeps
+// the threshold of about a tile per SM
 inline bool use_stream(const rm_ctx* ctx, bool masked, int B, int T, bool anchor_write = false) {
     if (ctx->path == 1 || !rm_stream_supported(ctx, B, T)) return false;
     if (ctx->variant_override == 4) return true;

@@ -147,7 +147,8 @@ constexpr int SE = 288;                // threads: 4 epilogue warps (0-3), 4 loa
 template <int NTOK, bool EQ4, bool GATHER>
 __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, const __grid_constant__ CUtensorMap tmW,
                                                             const __grid_constant__ CUtensorMap tmX,
-                                                            const __grid_constant__ CUtensorMap tmOut) {
+                                                            const __grid_constant__ CUtensorMap tmOut,
+                                                            const __grid_constant__ CUtensorMap tmYa) {
     using S = SmemST<NTOK>;
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -430,10 +431,10 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
             if (m == 0) RM_ST(9);
             // finished down blocks: lane = output column, token columns.  Transposed through shared memory into
             // [token][128 columns]; the copy engine adds the block to the output as one box of the [B, T, H] tensor
-            // map (rows past T fall outside the map and are dropped).  The anchor step, which also accumulates the
-            // ungated block into y_anchor, adds with vector reds instead.
-            float* out_b = a.r_out + (size_t)b * T * H;
-            float* ya_b = (anchor_mode == RM_ANCHOR_WRITE) ? a.y_anchor + (size_t)b * T * H : nullptr;
+            // map (rows past T fall outside the map and are dropped).  The two staging buffers alternate, so one is
+            // read while the other fills; the anchor step fills both per block, the ungated block for y_anchor and
+            // the gated one for the output.
+            const bool ya_b = anchor_mode == RM_ANCHOR_WRITE;
             for (int mb = 0; mb < MBN; ++mb, ++mbc) {
                 const int slot = mbc & 1;
                 wait_bar(d2_full(slot), (mbc >> 1) & 1);
@@ -446,7 +447,10 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
                               *reinterpret_cast<float(*)[32]>(y + c0));
                 tc_fence_before();
                 mbar_arrive(d2_free(slot));
-                if (m == 0) bulk_wait_read_but_one();              // the box sent from this buffer two blocks ago has left it
+                if (m == 0) {                                      // the box(es) sent from the buffer(s) about to be filled have left
+                    if (ya_b) bulk_wait_read_all();
+                    else bulk_wait_read_but_one();
+                }
                 named_barrier(1, 128);                             // the previous block's rows have been read
                 if (!ya_b) {
                     float* gYb = gY + (mbc & 1) * 8192;            // the copy engine reads one buffer while the other fills
@@ -461,17 +465,19 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
                         bulk_commit();
                     }
                 } else {
+                    const float gm = gate ? gate[(size_t)b * H + mb * 128 + m] : 1.f;
 #pragma unroll
                     for (int t = 0; t < NTOK; ++t)
-                        if (t < T) gY[t * 128 + m] = y[t];
+                        if (t < T) {
+                            gY[t * 128 + m] = y[t];
+                            gY[8192 + t * 128 + m] = gm * y[t];
+                        }
+                    fence_proxy_async_smem();
                     named_barrier(1, 128);
-                    const int c4 = (m & 31) * 4;                   // four columns of this block
-                    float4 gc = make_float4(1.f, 1.f, 1.f, 1.f);
-                    if (gate) gc = *reinterpret_cast<const float4*>(gate + (size_t)b * H + mb * 128 + c4);
-                    for (int t = m >> 5; t < T; t += 4) {
-                        const float4 f = *reinterpret_cast<const float4*>(gY + t * 128 + c4);
-                        red_add_v4(ya_b + (size_t)t * H + mb * 128 + c4, f.x, f.y, f.z, f.w);
-                        red_add_v4(out_b + (size_t)t * H + mb * 128 + c4, gc.x * f.x, gc.y * f.y, gc.z * f.z, gc.w * f.w);
+                    if (m == 0) {
+                        tensor_reduce_add_3d(&tmYa, mb * 128, 0, b, smem_u32(gY));
+                        tensor_reduce_add_3d(&tmOut, mb * 128, 0, b, smem_u32(gY + 8192));
+                        bulk_commit();
                     }
                 }
                 if (m == 0) RM_ST(30 + mb);
@@ -592,12 +598,16 @@ int launch_tiles(rm_ctx* ctx, const StreamArgs& a, int n_ctas, cudaStream_t s) {
         RM_CUDA_TRY(cudaFuncSetAttribute(stream_tile_kernel<NTOK, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
         configured.set(ctx->device, S::TOTAL);
     }
-    CUtensorMap tmW, tmX, tmOut;
+    CUtensorMap tmW, tmX, tmOut, tmYa;
     int rc = make_map(&tmW, a.packed, (uint64_t)a.I, (uint64_t)3 * a.H, NT);       // used without a list only
     if (rc != RM_OK) return rc;
     rc = make_map(&tmX, a.x, (uint64_t)a.B * a.T, (uint64_t)a.H, NTOK);
     if (rc != RM_OK) return rc;
     rc = make_map_out(&tmOut, a.r_out, (uint64_t)a.B, (uint64_t)a.T, (uint64_t)a.H, NTOK);
+    if (rc != RM_OK) return rc;
+    // the anchor step's second target; any valid map otherwise (not used)
+    rc = make_map_out(&tmYa, a.anchor_mode == RM_ANCHOR_WRITE ? a.y_anchor : a.r_out, (uint64_t)a.B, (uint64_t)a.T,
+                      (uint64_t)a.H, NTOK);
     if (rc != RM_OK) return rc;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_ctas);
@@ -609,7 +619,7 @@ int launch_tiles(rm_ctx* ctx, const StreamArgs& a, int n_ctas, cudaStream_t s) {
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, a, tmW, tmX, tmOut));
+    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, a, tmW, tmX, tmOut, tmYa));
     ctx->launches++;
     return RM_OK;
 }
