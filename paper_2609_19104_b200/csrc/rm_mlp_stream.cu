@@ -9,8 +9,8 @@
 //                  (record, Eq. 4 bookkeeping), keeps h = hi + lo (bf16 pair) in shared memory, then streams the tile's
 //                  down rows 128 output columns at a time, D2 = Wd_block * h in tensor memory (two slots), and adds
 //                  each finished block to the output: transposed through shared memory and added by the copy engine
-//                  as one box of the [B, T, H] tensor map (red.global.add in the anchor step, which also accumulates
-//                  the ungated block into y_anchor).
+//                  as one box of the [B, T, H] tensor map (two boxes in the anchor step, which also accumulates the
+//                  ungated block into y_anchor).
 //                  Four warps load: 16-byte cp.async gathers straight into the swizzled operand layout for index
 //                  lists (they top out near 16 bytes per clock and SM), cp.async.bulk.tensor boxes of 64 neurons x 64
 //                  columns for runs of consecutive neurons (one-row boxes were tried for lists and are far slower);
