@@ -22,6 +22,18 @@ inline bool use_fused(const rm_ctx* ctx, int B, int T) {
     return ctx->path != 1 && rm_fused_supported(ctx, B, T);
 }
 
+// The whole-step kernel (variant 5) runs every step it covers unless a per-layer variant is forced.
+inline bool use_persist(const rm_ctx* ctx, int B, int T) {
+    if (ctx->path == 1 || !rm_persist_supported(ctx, B, T)) return false;
+    if (ctx->variant_override == 5) return true;
+    return ctx->variant_override == 0 && B <= ctx->persist_max_b;
+}
+
+inline void* persist_ws(const rm_ctx* ctx, void* ws, int B, int T) {
+    const size_t r_bytes = align_up((size_t)B * T * ctx->g.H * sizeof(float), 256);
+    return static_cast<char*>(ws) + 4 * r_bytes + align_up(rm_ref_workspace_bytes(ctx, B, T), 256);
+}
+
 // The streaming variant (whole tiles per CTA) pays off only when a launch has about one 64-neuron tile per SM (one SM
 // gathers at most ~38 GB/s with 16-byte cp.async and adds at most ~20 GB/s with red.global, so a tile costs it
 // ~25 us); below that the cluster kernels, which spread a tile over 8 SMs, win.  H = 1024 only: at H = 2048 the
@@ -83,7 +95,11 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->l2_prefetch = 0;
     c->fused_clusters = 0;
     c->fused_blocks_per_sm = 0;
-    if (prop.major == 10) rm_fused_init(c);                 // failure leaves the portable path in charge
+    c->last_variant = 0;
+    c->persist_clusters = 0;
+    c->persist_max_b = 1;
+    c->persist_xbuf = nullptr;
+    if (prop.major == 10) { rm_fused_init(c); rm_persist_init(c); }   // failure leaves the portable path in charge
     cudaGetLastError();
     *out = c;
     return RM_OK;
@@ -104,7 +120,7 @@ size_t rm_workspace_bytes(const rm_ctx* ctx, int B, int T) {
     if (!ctx || B < 1 || T < 1) return 0;
     // three rotating residual-stream buffers, the host variant's staging buffer, then the portable path's scratch
     size_t r_bytes = align_up((size_t)B * T * ctx->g.H * sizeof(float), 256);
-    return 4 * r_bytes + rm_ref_workspace_bytes(ctx, B, T);
+    return 4 * r_bytes + align_up(rm_ref_workspace_bytes(ctx, B, T), 256) + rm_persist_workspace_bytes(ctx);
 }
 
 int rm_pack_weights(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, void* packed_out,
@@ -217,11 +233,36 @@ int rm_sparse_mlp(rm_ctx* ctx, const void* packed_layer, const void* x, const fl
                                                       cudaMemcpyDeviceToDevice, s));
             else RM_CUDA_TRY(cudaMemsetAsync(y, 0, (size_t)T * ctx->g.H * sizeof(float), s));
         }
-        if (use_stream(ctx, count_dev != nullptr, 1, T))
+        if (use_persist(ctx, 1, T)) {
+            // the whole-step kernel on a stack of one layer whose input is the caller's x
+            const void* one[1] = {packed_layer};
+            rm_step_args sa{};
+            sa.packed_layers = one;
+            sa.L = 1;
+            sa.r = y;
+            sa.idx = idx;
+            sa.count = count_dev;
+            sa.idx_b_stride = 0;
+            sa.idx_l_stride = 0;
+            sa.list_cap = ctx->g.I;
+            sa.count_b_stride = 0;
+            sa.record = record_out;
+            sa.rec_b_stride = 0;
+            sa.record_scale = record_scale;
+            sa.B = 1;
+            sa.T = T;
+            sa.x_ext = x;
+            ctx->last_variant = 5;
+            return rm_launch_step_persist(ctx, sa, persist_ws(ctx, ws, 1, T), s);
+        }
+        if (use_stream(ctx, count_dev != nullptr, 1, T)) {
+            ctx->last_variant = 4;
             return rm_launch_layer_stream(ctx, a, nullptr, false, s);
+        }
         return rm_launch_layer_fused(ctx, a, nullptr, false, false, s);
     }
     if (ctx->path == 2) return RM_ERR_UNSUPPORTED;
+    ctx->last_variant = 0;
     return rm_launch_layer_ref(ctx, a, static_cast<char*>(ws) + 4 * r_bytes, s);
 }
 
@@ -243,6 +284,27 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
     const size_t n_bytes = (size_t)B * T * g.H * sizeof(float);
     const size_t r_bytes = align_up(n_bytes, 256);
     char* layer_ws = static_cast<char*>(ws) + 4 * r_bytes;
+    if (use_persist(ctx, B, T) && an.mode == RM_ANCHOR_NONE && !an.gate) {
+        // the whole step in one launch: the layers add into r_out in place
+        if (r_out != r_in) RM_CUDA_TRY(cudaMemcpyAsync(r_out, r_in, n_bytes, cudaMemcpyDeviceToDevice, s));
+        rm_step_args sa{};
+        sa.packed_layers = packed_layers;
+        sa.L = g.L;
+        sa.r = r_out;
+        sa.idx = idx;
+        sa.count = count_dev;
+        sa.idx_b_stride = (int64_t)g.L * stride;
+        sa.idx_l_stride = stride;
+        sa.list_cap = idx ? stride : g.I;
+        sa.count_b_stride = g.L;
+        sa.record = records_out;
+        sa.rec_b_stride = (int64_t)g.L * g.I;
+        sa.record_scale = record_scale;
+        sa.B = B;
+        sa.T = T;
+        ctx->last_variant = 5;
+        return rm_launch_step_persist(ctx, sa, persist_ws(ctx, ws, B, T), s);
+    }
     const bool fused = use_fused(ctx, B, T);
     if (!fused && ctx->path == 2) return RM_ERR_UNSUPPORTED;
     float* rot[3] = {reinterpret_cast<float*>(static_cast<char*>(ws)),
@@ -286,6 +348,7 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
             // two buffers in turn: the preparation kernel writes the residual part of the output, the tiles add theirs
             const bool last = l == g.L - 1;
             a.r_out = (last && direct_out) ? r_out : rot[l & 1];
+            ctx->last_variant = 4;
             rc = rm_launch_layer_stream(ctx, a, reinterpret_cast<__nv_bfloat16*>(layer_ws), ctx->use_pdl && l > 0, s);
             cur = a.r_out;
         } else if (fused) {
@@ -298,6 +361,7 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
             cur = a.r_out;
         } else {
             a.r_out = r_out;                               // in place after the first layer
+            ctx->last_variant = 0;
             rc = rm_launch_layer_ref(ctx, a, layer_ws, s);
             cur = r_out;
         }
@@ -416,8 +480,11 @@ int rm_set_option(rm_ctx* ctx, const char* name, int value) {
         if (value < 0) return RM_ERR_INVALID_ARG;
         ctx->count_hint = value;
     } else if (n == "variant") {
-        if (value < 0 || value > 4) return RM_ERR_INVALID_ARG;
+        if (value < 0 || value > 5) return RM_ERR_INVALID_ARG;
         ctx->variant_override = value;
+    } else if (n == "persist_max_batch") {
+        if (value < 0 || value > 16) return RM_ERR_INVALID_ARG;
+        ctx->persist_max_b = value;
     } else if (n == "stream_min_tiles") {
         if (value < 1) return RM_ERR_INVALID_ARG;
         ctx->stream_min_tiles = value;
@@ -441,6 +508,8 @@ int rm_get_info(const rm_ctx* ctx, const char* name, int* out) {
     if (n == "fused_clusters") *out = ctx->fused_clusters;
     else if (n == "fused_blocks_per_sm") *out = ctx->fused_blocks_per_sm;
     else if (n == "sm_count") *out = ctx->sm_count;
+    else if (n == "persist_clusters") *out = ctx->persist_clusters;
+    else if (n == "last_variant") *out = ctx->last_variant;
     else if (n == "path") *out = ctx->path;
     else if (n == "status_detail") *out = ctx->status_detail;
     else if (n == "status_log_count") *out = ctx->status_log[2] < RM_STATUS_LOG ? ctx->status_log[2] : RM_STATUS_LOG;
@@ -456,6 +525,7 @@ int rm_get_info(const rm_ctx* ctx, const char* name, int* out) {
 int rm_debug_phase_times(rm_ctx* ctx, long long* host_out, int n) {
     if (!ctx || !host_out) return RM_ERR_INVALID_ARG;
     if (n == -64) return rm_stream_debug_stamps(host_out);      // the streaming kernel's stamps (first tile of CTA 0)
+    if (n <= -(1 << 20)) return rm_persist_debug_stamps(host_out, -n - (1 << 20));   // the whole-step kernel's stamps
     return rm_fused_debug_stamps(host_out, n);
 }
 

@@ -43,6 +43,12 @@ struct rm_ctx {
     int l2_prefetch;                       // L2 prefetch distance (tiles) of the warp-specialised kernel
     int stream_min_tiles;                  // launches with at least this many 64-neuron tiles use the streaming variant
     int variant_override;                  // 0 auto, 1 lean kernel, 2 kernel with a dedicated staging buffer
+    int last_variant;                      // kernel family of the last layer or step launched (see rm_get_info)
+    // whole-step kernel (rm_mlp_persist.cu)
+    int persist_clusters;                  // co-resident 8-CTA clusters of the whole-step kernel (0: unavailable)
+    int persist_max_b;                     // largest batch the whole-step kernel is chosen for when the variant is automatic
+    const void* persist_xbuf;              // buffer the cached tensor map below describes
+    alignas(64) unsigned char persist_tm[128];   // CUtensorMap of the clusters' x copies in the workspace
 };
 
 extern int rm_last_cuda_error;            // cudaError_t of the last failed runtime call (diagnostics; "last_cuda_error")
@@ -132,6 +138,25 @@ int rm_launch_layer_ref(rm_ctx* ctx, const rm_layer_args& a, void* ws, cudaStrea
 bool rm_stream_supported(const rm_ctx* ctx, int B, int T);
 int rm_stream_debug_stamps(long long* host_out);
 int rm_launch_layer_stream(rm_ctx* ctx, const rm_layer_args& a, __nv_bfloat16* x_scratch, bool pdl, cudaStream_t s);
+// Whole-step kernel: every layer of a step in one launch.  H in {1024, 2048}, T <= 64, B <= 16, L <= 64, zero-fill form.
+struct rm_step_args {
+    const void* const* packed_layers;      // host array of L device pointers
+    int L;
+    float* r;                              // [B,T,H] fp32: r_0 on entry, r_L on exit
+    const int32_t* idx;                    // list (b, l) at idx + b * idx_b_stride + l * idx_l_stride; NULL: positions
+    const int32_t* count;                  // count (b, l) at count[b * count_b_stride + l]; NULL: every neuron
+    int64_t idx_b_stride, idx_l_stride, list_cap, count_b_stride;
+    float* record;                         // record (b, l, n) at record[b * rec_b_stride + l * I + n]; NULL: none
+    int64_t rec_b_stride;
+    const float* record_scale;             // [L, I] or NULL
+    int B, T;
+    const void* x_ext;                     // [T,H] bf16: layer 0 takes this as its input instead of normalising r (L = 1 calls)
+};
+int rm_persist_init(rm_ctx* ctx);
+bool rm_persist_supported(const rm_ctx* ctx, int B, int T);
+size_t rm_persist_workspace_bytes(const rm_ctx* ctx);
+int rm_launch_step_persist(rm_ctx* ctx, const rm_step_args& sa, void* ws, cudaStream_t s);
+int rm_persist_debug_stamps(long long* host_out, int n);
 // Tiled tensor map (a 128-byte CUtensorMap, 64-byte aligned) of an fp32 residual buffer [B, T, H] with boxes of
 // box_rows token rows x 128 columns of one episode, not swizzled: the target of the kernels' bulk adds.
 int rm_make_out_map(void* tensor_map, const float* ptr, int B, int T, int H, int box_rows);

@@ -1672,6 +1672,7 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
         nc = variant == 3 ? (int)(tiles < cap ? tiles : cap) : (int)((tiles + run - 1) / run);
     }
     const bool small_t = la.T <= 32;
+    ctx->last_variant = variant;
     if (variant == 3) {
         if (ctx->g.H == 1024)
             return small_t ? launch_fused_ws<32, 128>(ctx, a, nc, pdl, s) : launch_fused_ws<64, 128>(ctx, a, nc, pdl, s);
