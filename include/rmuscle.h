@@ -183,8 +183,11 @@ int rm_action_expert_step_ex(rm_ctx* ctx, const void* const* packed_layers, cons
  *   F(x) = Wd (gelu_tanh(Wg x) * (Wu x)), fp32 accumulation, the hidden activations rounded to bf16 between the two
  *   products (as the model does).  x [P+S,H] bf16; rows [>= count] int32 ascending, count_dev [1] int32 (device);
  *   y_ref [P,H] fp32; y_out [P+S,H] fp32 (may equal y_ref when that buffer has P+S rows).
- *   R_max >= count + S is the row capacity of the call, at most 256 (RM_ERR_SHAPE above); a count that does not fit
- *   is truncated and RM_ERR_INDEX recorded.  ws: rm_context_workspace_bytes(ctx, R_max) bytes. */
+ *   R_max >= count + S is the row capacity of the call, at most 1024 (RM_ERR_SHAPE above); a count that does not fit
+ *   is truncated and RM_ERR_INDEX recorded.  Up to 256 rows go through the two products at once; a larger capacity
+ *   takes one pass over the weights per 256 rows (the setting of the paper's Context Cache table, rho_p = 0.4 of 768
+ *   visual rows plus 48 others = 356 rows, takes two).  A listed index outside [0, P) is skipped and RM_ERR_INDEX
+ *   recorded.  ws: rm_context_workspace_bytes(ctx, R_max) bytes. */
 int rm_context_drift(rm_ctx* ctx, const void* x, const void* x_ref, int P, float* score_out, rm_stream_t stream);
 size_t rm_context_workspace_bytes(const rm_ctx* ctx, int R_max);
 int rm_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, const void* x, const int32_t* rows,
@@ -202,10 +205,12 @@ int rm_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, 
  * How: the scratch that the two-kernel portable path needs (the compact hidden activations h [T, I] in fp32) is a
  * fixed 4 MiB array that is part of the library image; every GPU that loads the library carries it until the
  * process exits.  Limit: T * I <= 1,048,576 (for example T = 64 with I = 16384); larger requests return
- * RM_ERR_SHAPE.  H must be a multiple of 64.
+ * RM_ERR_SHAPE.  H must be a multiple of 64 and at most 7232 (the gate/up kernel stages 32 * H bytes of x per CTA;
+ * RM_ERR_SHAPE above).
  *
  * Arguments as for rm_sparse_mlp (packed_layer from rm_pack_weights with the same H and I; x [T,H] bf16; residual
- * [T,H] fp32 or NULL; idx ascending int32 or NULL for dense; count_dev [1] int32 on the device; y [T,H] fp32, may
+ * [T,H] fp32 or NULL; idx ascending int32 or NULL for dense; count_dev [1] int32 on the device, required with idx,
+ * and with idx NULL it selects the leading count neurons of the layer exactly as in rm_sparse_mlp; y [T,H] fp32, may
  * equal residual).  All pointers are device pointers, 16-byte aligned; the caller passes inputs and outputs as usual.
  * No activation record is produced.  Out-of-range indices are skipped silently (there is no status word without a
  * context).  The work is enqueued on `stream`; the call does not wait for it.
@@ -218,11 +223,23 @@ int rm_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, 
 int rm_sparse_mlp_static(const void* packed_layer, const void* x, const float* residual, const int32_t* idx,
                          const int32_t* count_dev, float* y, int T, int H, int I, rm_stream_t stream);
 
-/* Measurement aid (not part of the method): reads the packed rows of the listed neurons (idx NULL: every neuron) with
- * the layer kernels' own access pattern -- 8 column-slice pieces per neuron, 16-byte cp.async into shared memory --
- * and discards them.  Timed by the caller it gives the rate at which this list can leave HBM with this pattern. */
+/* Measurement aids (not part of the method; the paper has no counterpart).
+ * rm_debug_gather_read: reads the whole packed rows (6*H bytes each) of the listed neurons (idx NULL: every neuron) with
+ * the instruction the layer kernels gather with -- 16-byte cp.async into shared memory, one CTA per SM, 12 rows in
+ * flight per CTA -- and discards them.  Timed by the caller it gives the rate at which this list can leave HBM at all.
+ * rm_debug_gather_read_step: the same for the L lists of one episode's step in ONE launch (packed_layers: host array of
+ * L device pointers; list l at idx + l * stride, its count at count_dev[l]; idx NULL: every neuron of every layer). */
 int rm_debug_gather_read(rm_ctx* ctx, const void* packed_layer, const int32_t* idx, const int32_t* count_dev,
                          int64_t list_cap, rm_stream_t stream);
+int rm_debug_gather_read_step(rm_ctx* ctx, const void* const* packed_layers, const int32_t* idx, const int32_t* count_dev,
+                              int64_t stride, rm_stream_t stream);
+
+/* Test aid for the failure path: launches one CTA that waits on a barrier nobody arrives at, with a budget of `polls`
+ * polls (1 .. 2^20; a few thousand take microseconds).  The wait runs out, the kernel records RM_ERR_TIMEOUT and the
+ * place where it gave up exactly as the layer kernels' bounded waits do, and returns: rm_device_status then reports
+ * RM_ERR_TIMEOUT, rm_get_info("status_detail") the source line and CTA, and the next rm_device_status is clean.
+ * Nothing is left waiting and the context stays usable. */
+int rm_debug_wait_timeout(rm_ctx* ctx, int polls, rm_stream_t stream);
 
 /* Reads and clears the device status word (0 or the first RM_ERR_* a kernel recorded).  Synchronises `stream`. */
 int rm_device_status(rm_ctx* ctx, int* host_out, rm_stream_t stream);
@@ -243,13 +260,20 @@ int64_t rm_launch_count(const rm_ctx* ctx);
  *   "variant"             tcgen05 kernel variant: 0 = choose per launch, 1 = lean (one tile at a time, two CTAs per
  *                         SM at H = 1024), 2 = two tiles in flight per cluster, 3 = warp-specialised (the phases
  *                         of consecutive tiles run concurrently; for clusters that walk many tiles), 4 = streaming
- *                         (no clusters: every CTA owns whole tiles; for launches with many tiles)
+ *                         (no clusters: every CTA owns whole tiles; for launches with many tiles), 5 = the whole-step
+ *                         kernel (every layer of a step in one launch; zero-fill form, B <= 16; calls it does not
+ *                         cover are chosen per launch)
  *   "stream_min_tiles"    launches with at least this many 64-neuron tiles use variant 4 when the variant is chosen
- *                         per launch (default 48 at H = 1024, 64 at H = 2048)                                   */
+ *                         per launch (default 48 at H = 1024, 64 at H = 2048)
+ *   "persist_max_batch"   largest B for which the whole-step kernel may be chosen per call (default 1)
+ *   "persist_prefetch_kb" whole-step kernel: KB of weight rows a CTA may ask into L2 ahead of its loaders (default 0:
+ *                         measured slower than no prefetch)                                                    */
 int rm_set_option(rm_ctx* ctx, const char* name, int value);
 
 /* Read-only facts: "fused_clusters" (co-resident clusters of the tcgen05 kernel, 0 when that path is
- * unavailable for this geometry or device), "fused_blocks_per_sm", "sm_count", "path", and "status_detail": for
+ * unavailable for this geometry or device), "fused_blocks_per_sm", "persist_clusters" (co-resident clusters of the
+ * whole-step kernel), "sm_count", "path", "last_variant" (kernel family of the last layer or step launched through this
+ * context: 0 portable, 1-5 as for the "variant" option), and "status_detail": for
  * the last non-zero status that rm_device_status returned, where the kernel gave up (a bounded wait that ran out:
  * source line of the wait << 12 | CTA index & 0xfff); 0 when that status carried no detail.
  * "last_cuda_error" (ctx may be NULL) is the cudaError_t of the last runtime call that made an entry point return

@@ -24,7 +24,7 @@ RM_ANCHOR_NONE, RM_ANCHOR_WRITE, RM_ANCHOR_UPDATE = 0, 1, 2
 EXPORTS = ["rm_create", "rm_destroy", "rm_packed_layer_bytes", "rm_workspace_bytes", "rm_pack_weights",
            "rm_mask_compact", "rm_sparse_mlp", "rm_action_expert_step", "rm_action_expert_step_host",
            "rm_action_expert_step_ex", "rm_gather_weights", "rm_context_drift", "rm_context_workspace_bytes",
-           "rm_context_ffn", "rm_debug_gather_read",
+           "rm_context_ffn", "rm_debug_gather_read", "rm_debug_gather_read_step", "rm_debug_wait_timeout",
            "rm_device_status", "rm_launch_count", "rm_status_string", "rm_set_option", "rm_get_info",
            "rm_debug_phase_times", "rm_sparse_mlp_static"]
 
@@ -82,6 +82,8 @@ def load_library() -> ctypes.CDLL:
     lib.rm_context_ffn.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.rm_debug_gather_read.argtypes = [vp, vp, vp, vp, i64, vp]
     lib.rm_gather_weights.argtypes = [vp, vp, vp, vp, i64, vp, vp]
+    lib.rm_debug_gather_read_step.argtypes = [vp, ctypes.POINTER(vp), vp, vp, i64, vp]
+    lib.rm_debug_wait_timeout.argtypes = [vp, i32, vp]
     lib.rm_action_expert_step_ex.argtypes = [vp, ctypes.POINTER(vp), vp, vp, vp, i64, vp, vp, vp, i32, i32, i32, vp, vp,
                                              i64, vp, vp, sz, vp]
     lib.rm_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
@@ -228,6 +230,15 @@ class Context:
         """Measurement aid: read the listed neurons' rows with the kernels' access pattern and discard them."""
         _check(self.lib.rm_debug_gather_read(self._h, _ptr(packed_layer), _ptr(idx), _ptr(count_dev), int(list_cap),
                                              _stream()), "rm_debug_gather_read")
+
+    def rm_debug_gather_read_step(self, packed_layers, idx, count_dev, stride: int):
+        """Measurement aid: the L lists of one episode's step read in one launch and discarded."""
+        _check(self.lib.rm_debug_gather_read_step(self._h, self._layer_ptrs(packed_layers), _ptr(idx), _ptr(count_dev),
+                                                  int(stride), _stream()), "rm_debug_gather_read_step")
+
+    def rm_debug_wait_timeout(self, polls: int = 4096):
+        """Test aid: one CTA whose bounded wait runs out (records RM_ERR_TIMEOUT and returns)."""
+        _check(self.lib.rm_debug_wait_timeout(self._h, int(polls), _stream()), "rm_debug_wait_timeout")
 
     def rm_gather_weights(self, packed_layer, idx, count_dev, list_cap: int, compact_out=None):
         """Compact copy of the listed neurons' packed rows (a packed layer whose leading `count` neurons are the list)."""

@@ -22,11 +22,18 @@ inline bool use_fused(const rm_ctx* ctx, int B, int T) {
     return ctx->path != 1 && rm_fused_supported(ctx, B, T);
 }
 
-// The whole-step kernel (variant 5) runs every step it covers unless a per-layer variant is forced.
-inline bool use_persist(const rm_ctx* ctx, int B, int T) {
+// The whole-step kernel (variant 5).  Chosen by itself where it is measured ahead of the per-layer kernels: masked
+// steps of single episodes at H = 2048 (config 2: 395 against 509 us per step); it adapts to the counts on the device,
+// so it needs no hint.  At H = 1024 the lean per-layer kernel, which overlaps consecutive layers with two CTAs per SM,
+// is still ahead on masked steps (210 against 236 us at config 1), and the streaming kernel on dense passes (341 / 1151
+// against 360 / 1256 us at H = 1024 / 2048) and on batches.  `steps`: a whole stack (false: the one-layer entry, which
+// pays the kernel's set-up for a single layer).
+inline bool use_persist(const rm_ctx* ctx, int B, int T, bool masked, bool steps) {
     if (ctx->path == 1 || !rm_persist_supported(ctx, B, T)) return false;
     if (ctx->variant_override == 5) return true;
-    return ctx->variant_override == 0 && B <= ctx->persist_max_b;
+    if (ctx->variant_override != 0 || B > ctx->persist_max_b || !steps || !masked) return false;
+    if (ctx->count_hint > 0 && (long long)ctx->count_hint * 10 > (long long)ctx->g.I * 6) return false;   // nearly dense lists
+    return ctx->g.H == 2048;
 }
 
 inline void* persist_ws(const rm_ctx* ctx, void* ws, int B, int T) {
@@ -44,7 +51,7 @@ inline void* persist_ws(const rm_ctx* ctx, void* ws, int B, int T) {
 inline bool use_stream(const rm_ctx* ctx, bool masked, int B, int T, bool anchor_write = false) {
     if (ctx->path == 1 || !rm_stream_supported(ctx, B, T)) return false;
     if (ctx->variant_override == 4) return true;
-    if (ctx->variant_override != 0) return false;
+    if (ctx->variant_override != 0 && ctx->variant_override != 5) return false;   // 5: a call the whole-step kernel does not cover
     const int per_episode = masked ? ctx->count_hint : ctx->g.I;
     if (per_episode <= 0) return false;
     const long long tiles = (long long)((per_episode + 63) / 64) * B;
@@ -98,6 +105,7 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->last_variant = 0;
     c->persist_clusters = 0;
     c->persist_max_b = 1;
+    c->persist_prefetch_kb = 0;
     c->persist_xbuf = nullptr;
     if (prop.major == 10) { rm_fused_init(c); rm_persist_init(c); }   // failure leaves the portable path in charge
     cudaGetLastError();
@@ -138,6 +146,22 @@ int rm_debug_gather_read(rm_ctx* ctx, const void* packed_layer, const int32_t* i
                                  static_cast<cudaStream_t>(stream));
 }
 
+int rm_debug_gather_read_step(rm_ctx* ctx, const void* const* packed_layers, const int32_t* idx, const int32_t* count_dev,
+                              int64_t stride, rm_stream_t stream) {
+    if (!ctx || !packed_layers || (idx && (!count_dev || stride < 1))) return RM_ERR_INVALID_ARG;
+    for (int l = 0; l < ctx->g.L; ++l) {
+        if (!packed_layers[l]) return RM_ERR_INVALID_ARG;
+        if (!rm_aligned16(packed_layers[l])) return RM_ERR_ALIGN;
+    }
+    if (!all_aligned({idx})) return RM_ERR_ALIGN;
+    return rm_launch_gather_read_step(ctx, packed_layers, idx, count_dev, stride, static_cast<cudaStream_t>(stream));
+}
+
+int rm_debug_wait_timeout(rm_ctx* ctx, int polls, rm_stream_t stream) {
+    if (!ctx || polls < 1 || polls > (1 << 20)) return RM_ERR_INVALID_ARG;
+    return rm_launch_wait_timeout(ctx, (unsigned)polls, static_cast<cudaStream_t>(stream));
+}
+
 int rm_gather_weights(rm_ctx* ctx, const void* packed_layer, const int32_t* idx, const int32_t* count_dev,
                       int64_t list_cap, void* compact_out, rm_stream_t stream) {
     if (!ctx || !packed_layer || !idx || !count_dev || !compact_out || list_cap < 0) return RM_ERR_INVALID_ARG;
@@ -157,8 +181,10 @@ int rm_context_drift(rm_ctx* ctx, const void* x, const void* x_ref, int P, float
     return rm_launch_context_drift(ctx, x, x_ref, P, score_out, static_cast<cudaStream_t>(stream));
 }
 
+constexpr int RM_CONTEXT_MAX_ROWS = 1024;      // four passes of 256 rows over the weights
+
 size_t rm_context_workspace_bytes(const rm_ctx* ctx, int R_max) {
-    if (!ctx || R_max < 1 || R_max > 256 || !rm_context_supported(ctx)) return 0;
+    if (!ctx || R_max < 1 || R_max > RM_CONTEXT_MAX_ROWS || !rm_context_supported(ctx)) return 0;
     return rm_context_workspace_bytes_impl(ctx, context_pad(R_max));
 }
 
@@ -167,11 +193,12 @@ int rm_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, 
                    size_t ws_bytes, rm_stream_t stream) {
     if (!ctx || !Wg || !Wu || !Wd || !x || !rows || !count_dev || !y_ref || !y_out || P < 0 || S < 0) return RM_ERR_INVALID_ARG;
     if (!rm_context_supported(ctx)) return RM_ERR_UNSUPPORTED;
-    if (R_max < 1 || R_max > 256 || S > R_max) return RM_ERR_SHAPE;
+    if (R_max < 1 || R_max > RM_CONTEXT_MAX_ROWS || S > R_max) return RM_ERR_SHAPE;
     if (!all_aligned({Wg, Wu, Wd, x, rows, y_ref, y_out, ws})) return RM_ERR_ALIGN;
     if (!ws || ws_bytes < rm_context_workspace_bytes(ctx, R_max)) return RM_ERR_WORKSPACE;
-    return rm_launch_context_ffn(ctx, Wg, Wu, Wd, x, rows, count_dev, P, S, context_pad(R_max), y_ref, y_out, ws,
-                                 static_cast<cudaStream_t>(stream));
+    // rows beyond 256 take further passes; a single pass rounds its capacity up to the tile it runs in
+    return rm_launch_context_ffn(ctx, Wg, Wu, Wd, x, rows, count_dev, P, S, R_max <= 256 ? context_pad(R_max) : R_max, y_ref,
+                                 y_out, ws, static_cast<cudaStream_t>(stream));
 }
 
 int rm_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out, int64_t stride,
@@ -233,7 +260,7 @@ int rm_sparse_mlp(rm_ctx* ctx, const void* packed_layer, const void* x, const fl
                                                       cudaMemcpyDeviceToDevice, s));
             else RM_CUDA_TRY(cudaMemsetAsync(y, 0, (size_t)T * ctx->g.H * sizeof(float), s));
         }
-        if (use_persist(ctx, 1, T)) {
+        if (use_persist(ctx, 1, T, count_dev != nullptr, false)) {
             // the whole-step kernel on a stack of one layer whose input is the caller's x
             const void* one[1] = {packed_layer};
             rm_step_args sa{};
@@ -284,7 +311,7 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
     const size_t n_bytes = (size_t)B * T * g.H * sizeof(float);
     const size_t r_bytes = align_up(n_bytes, 256);
     char* layer_ws = static_cast<char*>(ws) + 4 * r_bytes;
-    if (use_persist(ctx, B, T) && an.mode == RM_ANCHOR_NONE && !an.gate) {
+    if (use_persist(ctx, B, T, count_dev != nullptr, true) && an.mode == RM_ANCHOR_NONE && !an.gate) {
         // the whole step in one launch: the layers add into r_out in place
         if (r_out != r_in) RM_CUDA_TRY(cudaMemcpyAsync(r_out, r_in, n_bytes, cudaMemcpyDeviceToDevice, s));
         rm_step_args sa{};
@@ -482,6 +509,9 @@ int rm_set_option(rm_ctx* ctx, const char* name, int value) {
     } else if (n == "variant") {
         if (value < 0 || value > 5) return RM_ERR_INVALID_ARG;
         ctx->variant_override = value;
+    } else if (n == "persist_prefetch_kb") {
+        if (value < 0 || value > 4096) return RM_ERR_INVALID_ARG;
+        ctx->persist_prefetch_kb = value;
     } else if (n == "persist_max_batch") {
         if (value < 0 || value > 16) return RM_ERR_INVALID_ARG;
         ctx->persist_max_b = value;

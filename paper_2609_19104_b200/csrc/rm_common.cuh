@@ -46,6 +46,7 @@ struct rm_ctx {
     int last_variant;                      // kernel family of the last layer or step launched (see rm_get_info)
     // whole-step kernel (rm_mlp_persist.cu)
     int persist_clusters;                  // co-resident 8-CTA clusters of the whole-step kernel (0: unavailable)
+    int persist_prefetch_kb;               // weight KB a CTA of the whole-step kernel may ask into L2 ahead of its loaders
     int persist_max_b;                     // largest batch the whole-step kernel is chosen for when the variant is automatic
     const void* persist_xbuf;              // buffer the cached tensor map below describes
     alignas(64) unsigned char persist_tm[128];   // CUtensorMap of the clusters' x copies in the workspace
@@ -97,10 +98,13 @@ bool rm_context_supported(const rm_ctx* ctx);
 size_t rm_context_workspace_bytes_impl(const rm_ctx* ctx, int r_pad);
 int rm_launch_context_drift(rm_ctx* ctx, const void* x, const void* x_ref, int P, float* score, cudaStream_t s);
 int rm_launch_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, const void* x, const int32_t* rows,
-                          const int32_t* count, int P, int S, int r_pad, const float* y_ref, float* y_out, void* ws,
+                          const int32_t* count, int P, int S, int cap, const float* y_ref, float* y_out, void* ws,
                           cudaStream_t s);
 int rm_launch_gather_read(rm_ctx* ctx, const void* packed, const int32_t* idx, const int32_t* count, int64_t cap,
                           cudaStream_t s);
+int rm_launch_gather_read_step(rm_ctx* ctx, const void* const* packed_layers, const int32_t* idx, const int32_t* count,
+                               int64_t stride, cudaStream_t s);
+int rm_launch_wait_timeout(rm_ctx* ctx, unsigned polls, cudaStream_t s);
 int rm_launch_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out,
                            int64_t stride, cudaStream_t s);
 

@@ -59,25 +59,33 @@ __global__ void __launch_bounds__(256) drift_kernel(const __nv_bfloat16* __restr
 }
 
 // ---------------------------------------------------------------- gather of the rows to recompute
-// Row r < count: visual row rows[r]; count <= r < count + S: always-recomputed row P + (r - count); beyond: zero.
+// The rows to recompute form one sequence q = 0, 1, ...: q < count is the visual row rows[q], count <= q < count + S the
+// always-recomputed row P + (q - count).  A call holds at most `cap` of them (a longer list is cut and reported); one
+// pass of the kernels handles the window q_lo <= q < q_lo + r_pad, compact row r = q - q_lo; rows beyond the sequence
+// are zero.
+__device__ __forceinline__ int ctx_count(const int32_t* count, int P, int S, int cap, bool* bad) {
+    int c = *count;
+    *bad = c < 0 || c > P || c + S > cap;
+    if (*bad) c = c < 0 ? 0 : (P < cap - S ? P : cap - S);
+    return c;
+}
 __global__ void __launch_bounds__(256) ctx_gather_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ rows,
                                                          const int32_t* __restrict__ count, int P, int S, int H, int r_pad,
-                                                         __nv_bfloat16* __restrict__ xc, int* status) {
+                                                         int q_lo, int cap, __nv_bfloat16* __restrict__ xc, int* status) {
     pdl_launch_dependents();               // the first product may start now: its weight loads need nothing from here
     pdl_wait();                            // the row list comes from the kernel in front
     const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= r_pad) return;
-    int c = *count;
-    if (c < 0 || c > P || c + S > r_pad) {
-        if (r == 0 && lane == 0) rm_set_status(status, RM_ERR_INDEX);
-        c = c < 0 ? 0 : (P < r_pad - S ? P : r_pad - S);
-    }
+    bool bad;
+    const int c = ctx_count(count, P, S, cap, &bad);
+    if (bad && r == 0 && lane == 0) rm_set_status(status, RM_ERR_INDEX);
+    const int q = q_lo + r;
     int src = -1;
-    if (r < c) {
-        src = rows[r];
+    if (q < c) {
+        src = rows[q];
         if (src < 0 || src >= P) { if (lane == 0) rm_set_status(status, RM_ERR_INDEX); src = -1; }
-    } else if (r < c + S) {
-        src = P + (r - c);
+    } else if (q < c + S) {
+        src = P + (q - c);
     }
     uint4* d = reinterpret_cast<uint4*>(xc + (size_t)r * H);
     const uint4* s = src >= 0 ? reinterpret_cast<const uint4*>(x + (size_t)src * H) : nullptr;
@@ -89,13 +97,12 @@ __global__ void __launch_bounds__(256) ctx_gather_kernel(const __nv_bfloat16* __
 // its reference output unless it is in the (ascending) list.
 __global__ void __launch_bounds__(256) ctx_scatter_kernel(const float* __restrict__ yp, int ksplit, int r_pad,
                                                           const int32_t* __restrict__ rows, const int32_t* __restrict__ count,
-                                                          int P, int S, int H, const float* __restrict__ y_ref,
+                                                          int P, int S, int H, int q_lo, int cap, const float* __restrict__ y_ref,
                                                           float* __restrict__ y_out) {
     pdl_wait();                            // the partial products come from the kernel in front
-    int c = *count;
-    c = c < 0 ? 0 : (c > P ? P : c);
-    if (c + S > r_pad) c = r_pad - S;
-    if ((int)blockIdx.x >= r_pad) {
+    bool bad;
+    const int c = ctx_count(count, P, S, cap, &bad);
+    if ((int)blockIdx.x >= r_pad) {       // (the first pass of a call only: its grid alone has these CTAs)
         const int p = (int)blockIdx.x - r_pad;
         if (y_out == y_ref) return;
         int lo = 0, hi = c;                // is p in rows[0 .. c)?
@@ -108,10 +115,13 @@ __global__ void __launch_bounds__(256) ctx_scatter_kernel(const float* __restric
             reinterpret_cast<float4*>(y_out + (size_t)p * H)[e] = reinterpret_cast<const float4*>(y_ref + (size_t)p * H)[e];
         return;
     }
-    const int r = blockIdx.x;
+    const int r = blockIdx.x, q = q_lo + r;
     int dst = -1;
-    if (r < c) dst = rows[r];
-    else if (r < c + S) dst = P + (r - c);
+    if (q < c) {
+        dst = rows[q];
+        if (dst >= P) dst = -1;            // a listed row must be a visual row: the gather zeroed it and recorded the error;
+                                           // writing it would race with the always-recomputed row of the same number
+    } else if (q < c + S) dst = P + (q - c);
     if (dst < 0 || dst >= P + S) return;
     for (int e = threadIdx.x; e < H / 4; e += blockDim.x) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -384,45 +394,51 @@ int rm_launch_context_drift(rm_ctx* ctx, const void* x, const void* x_ref, int P
 }
 
 int rm_launch_context_ffn(rm_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, const void* x, const int32_t* rows,
-                          const int32_t* count, int P, int S, int r_pad, const float* y_ref, float* y_out, void* ws,
+                          const int32_t* count, int P, int S, int cap, const float* y_ref, float* y_out, void* ws,
                           cudaStream_t s) {
     const int H = ctx->g.H, I = ctx->g.I;
     const int ksplit = pick_ksplit(ctx);
-    char* w = static_cast<char*>(ws);
-    __nv_bfloat16* xc = reinterpret_cast<__nv_bfloat16*>(w);
-    w += align_up((size_t)r_pad * H * sizeof(__nv_bfloat16), 1024);
-    __nv_bfloat16* h1 = reinterpret_cast<__nv_bfloat16*>(w);
-    w += align_up((size_t)r_pad * I * sizeof(__nv_bfloat16), 1024);
-    float* yp = reinterpret_cast<float*>(w);
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
-    {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((r_pad + 7) / 8);
-        cfg.blockDim = dim3(256);
-        cfg.stream = s;
-        cfg.attrs = at;
-        cfg.numAttrs = 1;
-        RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, ctx_gather_kernel, static_cast<const __nv_bfloat16*>(x), rows, count, P, S, H, r_pad,
-                                       xc, ctx->d_status));
-        ctx->launches++;
-    }
-    int rc = RM_ERR_SHAPE;
-    if (r_pad == 64) rc = run_ffn<64>(ctx, Wg, Wu, Wd, xc, h1, yp, ksplit, s);
-    else if (r_pad == 128) rc = run_ffn<128>(ctx, Wg, Wu, Wd, xc, h1, yp, ksplit, s);
-    else if (r_pad == 256) rc = run_ffn<256>(ctx, Wg, Wu, Wd, xc, h1, yp, ksplit, s);
-    if (rc != RM_OK) return rc;
-    {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(r_pad + P);
-        cfg.blockDim = dim3(256);
-        cfg.stream = s;
-        cfg.attrs = at;
-        cfg.numAttrs = 1;
-        RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, ctx_scatter_kernel, static_cast<const float*>(yp), ksplit, r_pad, rows, count, P, S, H,
-                                       y_ref, y_out));
-        ctx->launches++;
+    // Up to 256 rows go through the products at once; a longer sequence takes further passes over the weights (the
+    // paper's own setting, 40 % of 768 visual rows plus 48 others = 356 rows, takes two).
+    for (int q_lo = 0; q_lo < cap; q_lo += 256) {
+        const int left = cap - q_lo;
+        const int r_pad = left <= 64 ? 64 : (left <= 128 ? 128 : 256);
+        char* w = static_cast<char*>(ws);
+        __nv_bfloat16* xc = reinterpret_cast<__nv_bfloat16*>(w);
+        w += align_up((size_t)r_pad * H * sizeof(__nv_bfloat16), 1024);
+        __nv_bfloat16* h1 = reinterpret_cast<__nv_bfloat16*>(w);
+        w += align_up((size_t)r_pad * I * sizeof(__nv_bfloat16), 1024);
+        float* yp = reinterpret_cast<float*>(w);
+        {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((r_pad + 7) / 8);
+            cfg.blockDim = dim3(256);
+            cfg.stream = s;
+            cfg.attrs = at;
+            cfg.numAttrs = 1;
+            RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, ctx_gather_kernel, static_cast<const __nv_bfloat16*>(x), rows, count, P, S, H, r_pad,
+                                           q_lo, cap, xc, ctx->d_status));
+            ctx->launches++;
+        }
+        int rc = RM_ERR_SHAPE;
+        if (r_pad == 64) rc = run_ffn<64>(ctx, Wg, Wu, Wd, xc, h1, yp, ksplit, s);
+        else if (r_pad == 128) rc = run_ffn<128>(ctx, Wg, Wu, Wd, xc, h1, yp, ksplit, s);
+        else if (r_pad == 256) rc = run_ffn<256>(ctx, Wg, Wu, Wd, xc, h1, yp, ksplit, s);
+        if (rc != RM_OK) return rc;
+        {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(r_pad + (q_lo == 0 ? P : 0));      // the first pass also copies the kept reference rows
+            cfg.blockDim = dim3(256);
+            cfg.stream = s;
+            cfg.attrs = at;
+            cfg.numAttrs = 1;
+            RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, ctx_scatter_kernel, static_cast<const float*>(yp), ksplit, r_pad, rows, count, P, S, H,
+                                           q_lo, cap, y_ref, y_out));
+            ctx->launches++;
+        }
     }
     return RM_OK;
 }

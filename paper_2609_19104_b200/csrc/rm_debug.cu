@@ -1,8 +1,13 @@
-// Gather-read microbenchmark: the access pattern of the layer kernels' loaders and nothing else.  For a list of
-// neurons, CTA (group g, slice j) reads the 3*Hs*2-byte piece j of every neuron of tiles g, g + G, ... with 16-byte
-// cp.async into two shared-memory stages and throws the data away.  Timed by the caller, it says how fast this list
-// can leave HBM at all with this pattern -- the ceiling the layer kernels are measured against besides the copy
-// bandwidth.
+// Measurement and test aids (not part of the method).
+//
+// gather_read_kernel: the practical ceiling of reading the listed neurons' packed rows and nothing else.  One CTA per SM;
+// CTA c takes list positions c, c + G, ... of every layer handed to it and pulls each neuron's whole 6*H-byte row into a
+// ring of shared-memory stages with 16-byte cp.async (the instruction the layer kernels gather with), 12 rows in
+// flight, then throws the data away.  One launch covers one layer or a whole step's layers back to back.  Timed by the
+// caller it says how fast these lists can leave HBM at all.
+//
+// wait_timeout_kernel: one CTA waits on an mbarrier that nobody arrives at, with a small poll budget, records
+// RM_ERR_TIMEOUT with the source line of the wait like the layer kernels' bounded waits do, and returns.
 #include "rm_common.cuh"
 #include "rm_sm100.cuh"
 
@@ -10,55 +15,106 @@ using namespace sm100;
 
 namespace {
 
-constexpr int GT = 128;                // threads per CTA
-constexpr int GNT = 64;                // neurons per tile
+constexpr int GT = 256;                // threads per CTA
+constexpr int DEPTH = 12;              // rows in flight per CTA
+constexpr int MAXL_DBG = 64;
 
-__global__ void __launch_bounds__(GT) gather_read_kernel(const __nv_bfloat16* __restrict__ packed,
-                                                         const int32_t* __restrict__ idx, const int32_t* __restrict__ count,
-                                                         int64_t cap, int H, int I, int* status) {
+struct GatherArgs {
+    const __nv_bfloat16* packed[MAXL_DBG];
+    const int32_t* idx;                // list of layer l at idx + l * stride; NULL: every neuron
+    const int32_t* count;              // count of layer l at count[l]
+    int64_t stride, cap;
+    int L, H, I;
+    int* status;
+};
+
+__global__ void __launch_bounds__(GT) gather_read_kernel(const __grid_constant__ GatherArgs a) {
     extern __shared__ unsigned char smem[];
-    const int j = blockIdx.x & 7, g = blockIdx.x >> 3, G = gridDim.x >> 3;
-    const int Hs = H / 8, chunks = 3 * Hs * 2 / 16;        // 16-byte chunks per piece
     const uint32_t base = (smem_u32(smem) + 127u) & ~127u;
-    const int stage_bytes = GNT * chunks * 16;
-    int c = idx ? *count : I;
-    if (c < 0 || c > cap || c > I) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) rm_set_status(status, RM_ERR_INDEX);
-        c = c < 0 ? 0 : (int)(cap < (int64_t)I ? cap : (int64_t)I);
-    }
-    const int tiles = (c + GNT - 1) / GNT;
+    const int row_bytes = 6 * a.H, pieces = row_bytes / 16;
     int k = 0;
-    for (int t = g; t < tiles; t += G, ++k) {
-        const uint32_t st = base + (k & 1) * stage_bytes;
-        if (k >= 2) cp_async_wait<1>();                    // the stage's previous tile has landed
-        for (int e = threadIdx.x; e < GNT * chunks; e += GT) {
-            const int q = e / chunks, ch = e - q * chunks;
-            const int p = t * GNT + q;
-            int n = p < c ? (idx ? idx[p] : p) : -1;
-            if (n >= I) n = -1;
-            cp_async16(st + e * 16, packed + (size_t)(n < 0 ? 0 : n) * 3 * H + (size_t)j * 3 * Hs + ch * 8, n >= 0);
+    for (int l = 0; l < a.L; ++l) {
+        int c = a.idx ? a.count[l] : a.I;
+        if (c < 0 || c > a.cap || c > a.I) {
+            if (blockIdx.x == 0 && threadIdx.x == 0) rm_set_status(a.status, RM_ERR_INDEX);
+            c = c < 0 ? 0 : (int)(a.cap < (int64_t)a.I ? a.cap : (int64_t)a.I);
         }
-        cp_async_commit();
+        const int32_t* list = a.idx ? a.idx + (size_t)l * a.stride : nullptr;
+        for (int p = blockIdx.x; p < c; p += gridDim.x, ++k) {
+            int n = list ? list[p] : p;
+            if (n < 0 || n >= a.I) n = -1;
+            const uint32_t st = base + (k % DEPTH) * row_bytes;
+            if (k >= DEPTH) cp_async_wait<DEPTH - 1>();        // the stage's previous row has landed
+            const __nv_bfloat16* src = a.packed[l] + (size_t)(n < 0 ? 0 : n) * 3 * a.H;
+            for (int e = threadIdx.x; e < pieces; e += GT) cp_async16(st + e * 16, src + e * 8, n >= 0);
+            cp_async_commit();
+        }
     }
     cp_async_wait<0>();
+}
+
+__global__ void __launch_bounds__(32) wait_timeout_kernel(int* status, unsigned polls) {
+    __shared__ __align__(8) unsigned long long bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        fence_mbar_init();
+        // nobody arrives: the wait runs out of its budget, records where it gave up, and the kernel returns
+        if (!mbar_wait(b, 0, polls)) rm_set_status_at(status, RM_ERR_TIMEOUT, (__LINE__ << 12) | (int)(blockIdx.x & 0xfffu));
+    }
+}
+
+int launch_gather(rm_ctx* ctx, const GatherArgs& a, cudaStream_t s) {
+    const rm_geom& g = ctx->g;
+    if (g.H % 64 != 0) return RM_ERR_UNSUPPORTED;
+    const int smem = DEPTH * 6 * g.H + 128;
+    if (smem > 227 * 1024) return RM_ERR_UNSUPPORTED;
+    static rm_smem_configured configured = {};
+    if (!configured.covers(ctx->device, smem)) {
+        RM_CUDA_TRY(cudaFuncSetAttribute(gather_read_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        configured.set(ctx->device, smem);
+    }
+    gather_read_kernel<<<ctx->sm_count > 0 ? ctx->sm_count : 148, GT, smem, s>>>(a);
+    ctx->launches++;
+    RM_CUDA_TRY(cudaGetLastError());
+    return RM_OK;
 }
 
 }  // namespace
 
 int rm_launch_gather_read(rm_ctx* ctx, const void* packed, const int32_t* idx, const int32_t* count, int64_t cap,
                           cudaStream_t s) {
-    const rm_geom& g = ctx->g;
-    if (g.H % 64 != 0) return RM_ERR_UNSUPPORTED;
-    const int smem = 2 * GNT * 3 * g.Hs * 2 + 128;
-    if (smem > 200 * 1024) return RM_ERR_UNSUPPORTED;
-    static rm_smem_configured configured = {};
-    if (!configured.covers(ctx->device, smem)) {
-        RM_CUDA_TRY(cudaFuncSetAttribute(gather_read_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        configured.set(ctx->device, smem);
-    }
-    const int groups = ctx->sm_count >= 8 ? ctx->sm_count / 8 : 1;             // 18 groups of 8 CTAs on 148 SMs
-    gather_read_kernel<<<groups * 8, GT, smem, s>>>(static_cast<const __nv_bfloat16*>(packed), idx, count, cap, g.H, g.I,
-                                                    ctx->d_status);
+    GatherArgs a{};
+    a.packed[0] = static_cast<const __nv_bfloat16*>(packed);
+    a.idx = idx;
+    a.count = count;
+    a.stride = 0;
+    a.cap = cap;
+    a.L = 1;
+    a.H = ctx->g.H;
+    a.I = ctx->g.I;
+    a.status = ctx->d_status;
+    return launch_gather(ctx, a, s);
+}
+
+int rm_launch_gather_read_step(rm_ctx* ctx, const void* const* packed_layers, const int32_t* idx, const int32_t* count,
+                               int64_t stride, cudaStream_t s) {
+    if (ctx->g.L > MAXL_DBG) return RM_ERR_UNSUPPORTED;
+    GatherArgs a{};
+    for (int l = 0; l < ctx->g.L; ++l) a.packed[l] = static_cast<const __nv_bfloat16*>(packed_layers[l]);
+    a.idx = idx;
+    a.count = count;
+    a.stride = stride;
+    a.cap = idx ? stride : ctx->g.I;
+    a.L = ctx->g.L;
+    a.H = ctx->g.H;
+    a.I = ctx->g.I;
+    a.status = ctx->d_status;
+    return launch_gather(ctx, a, s);
+}
+
+int rm_launch_wait_timeout(rm_ctx* ctx, unsigned polls, cudaStream_t s) {
+    wait_timeout_kernel<<<1, 32, 0, s>>>(ctx->d_status, polls);
     ctx->launches++;
     RM_CUDA_TRY(cudaGetLastError());
     return RM_OK;

@@ -7,9 +7,13 @@
 // Grid: clusters of 8 CTAs, all co-resident (one CTA per SM).  Per layer and episode (an "item") the active list is
 // cut evenly over the clusters; a cluster walks its run in tiles of up to 256 neurons.  Inside a tile
 //   gate/up : CTA j takes up to 32 of the tile's neurons and computes their gate and up rows against the whole
-//             width H -- A = the neurons' weight rows (64 rows: gate and up interleaved, K-major, 128-byte swizzle,
-//             gathered by 16-byte cp.async), B = x (64 token rows, one tensor-map box per 64 columns),
-//             D1[64 x 64] in tensor memory.  No partial sums cross CTAs.
+//             width H -- A = the neurons' weight rows (gate and up interleaved, K-major, 128-byte swizzle, gathered by
+//             16-byte cp.async), B = x (64 token rows).  One tcgen05.mma costs the same ~64 clocks whatever its
+//             shape up to 128 x 128, so an instruction carries two 16-column steps at once, one from each half of
+//             H: A = [rows over columns of the first half ; the same rows over columns of the second half]
+//             (M = 128), B = [x columns of the first half ; of the second half] (N = 128); the two diagonal
+//             64 x 64 blocks of D1 are the two halves' partial sums (the off-diagonal blocks are ignored) and are
+//             added in the epilogue.  No partial sums cross CTAs.
 //   GLU     : h = gelu_tanh(g) * u from tensor memory, split into a bf16 pair hi + lo, written to this CTA's h tile
 //             and copied to the 7 peers' h tiles (bulk copies counted on the receivers' mbarriers).
 //   down    : CTA j owns output columns [j H/8, (j+1) H/8): D2[H/8 x (hi | lo tokens)] += Wd-slice * h over ALL the
@@ -37,19 +41,23 @@ constexpr int CS = 8;                  // CTAs per cluster = column slices of th
 constexpr int NT = 32;                 // neurons whose gate/up rows one CTA computes per tile
 constexpr int CT = CS * NT;            // slots of a cluster tile
 constexpr int NTOK = 64;               // token rows (padded)
-constexpr int XS = 4;                  // x ring: stages of one 64-column box (8 KB)
-constexpr int X_BYTES = NTOK * 128;
-constexpr int W_RING = 96 * 1024;      // weight ring
-constexpr int H_HALF = CT * 128;       // h tile: hi block, then lo block (each 256 slots x 64 tokens bf16)
+constexpr int X_BYTES = NTOK * 128;    // one 64-column block of x: 64 token rows x 128 bytes
+constexpr int XSB = 2 * X_BYTES;       // x ring stage: the blocks of columns c and c + H/2
+constexpr int XS_MAX = 8;
+constexpr int SB = 16384;              // weight ring stage: 128 rows x 128 bytes
+constexpr int EXCH = 16384;            // second-half partial sums of a tile on their way to the threads that finish them
 constexpr int MAXL = 64, MAXB = 16;
-constexpr int NTHREADS = 576;          // warps: 0-7 epilogue, 8-11 loaders, 12-15 normalisation, 16 issuer, 17 x boxes
-constexpr int W_LOAD0 = 8, W_NORM0 = 12, W_MMA = 16, W_XTMA = 17;
+constexpr int NXW = 4;                 // warps that issue the x copies (copies of one issuing thread do not overlap much)
+constexpr int NTHREADS = 608;          // warps: 0-7 epilogue and normalisation, 8-11 loaders, 12 issuer, 13-16 x copies, 17 L2 prefetch,
+                                       // 18 stage watcher
+constexpr int W_LOAD0 = 8, W_MMA = 12, W_X0 = 13, W_PF = 17, W_WATCH = 18;
 constexpr int SYNC_ABORT = MAXB;       // sync[0..MAXB): per-episode arrival counters; sync[MAXB]: abort flag
 
 struct PArgs {
     const __nv_bfloat16* packed[MAXL];
     float* r;                          // [B,T,H] fp32: holds r_0 on entry and r_L on exit (layers add in place)
-    __nv_bfloat16* xbuf;               // [clusters][2][64][H] bf16: the clusters' own copies of x
+    __nv_bfloat16* xbuf;               // [clusters][2][H/64][64 rows x 128 bytes]: the clusters' own copies of x, stored as
+                                       // the shared-memory image of each 64-column block (128-byte swizzle)
     const int32_t* idx;                // list (b, l) at idx + b * idx_b_stride + l * idx_l_stride; NULL: positions
     const int32_t* count;              // count (b, l) at count[b * count_b_stride + l]; NULL: every neuron
     int64_t idx_b_stride, idx_l_stride, list_cap, count_b_stride;
@@ -60,24 +68,37 @@ struct PArgs {
     int* status;
     int L, B, T, I;
     int x_ext;                         // layer 0 takes x from the caller's buffer (single-layer entry): no normalisation
+    int pf_bytes;                      // weight bytes a CTA may have asked into L2 ahead of its loaders (0: no prefetch)
 };
 
 #ifdef RM_PHASE_TIMING
-__device__ long long g_ps_stamps[64 * 128 * 16];
+__device__ long long g_ps_stamps[64 * 128 * 32];
 __device__ __forceinline__ long long ps_now() {
     long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-#define RM_PS(item, slot) do { if ((item) < 64 && blockIdx.x < 128) g_ps_stamps[((item) * 128 + blockIdx.x) * 16 + (slot)] = ps_now(); } while (0)
+#define RM_PS(item, slot) do { if ((item) < 64 && blockIdx.x < 128) g_ps_stamps[((item) * 128 + blockIdx.x) * 32 + (slot)] = ps_now(); } while (0)
+#define RM_PC(item, slot, v) do { if ((item) < 64 && blockIdx.x < 128) g_ps_stamps[((item) * 128 + blockIdx.x) * 32 + (slot)] = (v); } while (0)
+#define RM_CLK() clock64()
 #else
 #define RM_PS(item, slot) do { } while (0)
+#define RM_PC(item, slot, v) do { } while (0)
+#define RM_CLK() 0ll
 #endif
 
 __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
+}
+__device__ __forceinline__ int ld_acquire_cta(const int* p) {          // shared memory
+    int v;
+    asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_cta(int* p, int v) {         // shared memory
+    asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
 __device__ __forceinline__ void red_release_gpu(int* p, int v) {
     asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -157,6 +178,11 @@ __device__ __forceinline__ void cur_init(Cur& k, const Env& e) {
     k.item = 0; k.seq = 0; k.ni = 0; k.use = 0; k.i = 0;
     cur_seek(k, e);
 }
+// The gate/up products of tile g may be issued before the down products of tile d (the tile in front of it) when g
+// does not need d's result: the same item, or another episode.  (The next layer of the same episode does: its input is
+// normalised from the residual stream that d's item adds into.  With empty lists in between, the next non-empty item
+// can be that even when several episodes are in the batch.)
+__device__ __forceinline__ bool may_run_ahead(const Cur& g, const Cur& d) { return g.item == d.item || g.b != d.b; }
 __device__ __forceinline__ void cur_next(Cur& k, const Env& e) {
     ++k.seq;
     if (++k.i < k.run.ntiles) return;
@@ -166,51 +192,65 @@ __device__ __forceinline__ void cur_next(Cur& k, const Env& e) {
     cur_seek(k, e);
 }
 
+// Shared memory: a fixed head (item counts, the tiles' neuron ids, barriers), the weight ring, then the h tile and the x
+// ring, which share what is left: the h tile is sized for the largest tile of the step, the x ring takes the rest.
 template <int HS8>
 struct Geo {
     static constexpr int H = 8 * HS8;
+    // weight ring stages: the wide model streams twice as much x per tile, so its x ring gets some of the space
+    static constexpr int NW = HS8 == 256 ? 5 : 6;
+    static constexpr int W_RING = NW * SB;
     static constexpr int NSB = HS8 / 64;               // 64-column boxes per column slice
     static constexpr int NMB = HS8 / 128;              // 128-column output blocks per slice
-    static constexpr int SB = HS8 * 128;               // bytes of a weight stage: 64 rows x HS8 columns
-    static constexpr int NW = W_RING / SB;
+    static constexpr int NCH = H / 64;                 // 64-column blocks of H
+    static constexpr int SPS = SB / (HS8 * 2);         // slots (neurons) of one down stage: 32 or 64
+    static constexpr int KPS = SPS / 16;               // product steps of one down stage
     static constexpr int ND2 = NMB == 1 ? 2 : 1;       // down accumulators (an item's flush overlaps the next item's products)
-    static constexpr int D2_COL = 2 * NTOK;            // tensor memory: D1[2] at 0 and 64, D2 from 128
-    static constexpr int OFF_W = 0;
-    static constexpr int OFF_X = OFF_W + W_RING;
-    static constexpr int OFF_H = OFF_X + XS * X_BYTES;
-    static constexpr int OFF_K = OFF_H + 2 * H_HALF;   // counts of the items
-    static constexpr int OFF_REC = OFF_K + MAXL * MAXB * 4;
-    static constexpr int OFF_BAR = OFF_REC + NT * 4;
-    static constexpr int TOTAL = OFF_BAR + 512 + 1024; // + slack for the 1024-byte alignment
+    static constexpr int D2_COL = 4 * NTOK;            // tensor memory: D1[2] at 0 and 128 (128 columns each), D2 from 256
+    static constexpr int OFF_K = 0;                    // counts of the items
+    static constexpr int OFF_IDX = OFF_K + MAXL * MAXB * 4;     // neuron ids of three tiles in turn
+    static constexpr int OFF_REC = OFF_IDX + 3 * CT * 4;
+    static constexpr int OFF_MISC = OFF_REC + 4 * NT * 4;
+    static constexpr int OFF_BAR = OFF_MISC + 128;
+    static constexpr int OFF_W = 9 * 1024;
+    static constexpr int OFF_EX = OFF_W + W_RING;
+    static constexpr int OFF_HX = OFF_EX + EXCH;
+    static constexpr int END = 231424;
+    static constexpr int TOTAL = END + 1024;           // + slack for the 1024-byte alignment
+    static_assert(OFF_BAR + 640 <= OFF_W, "fixed head overflows");
     static_assert(TOTAL <= 232448, "buffers exceed the shared memory of a CTA");
 };
 
 template <int HS8>
 __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant__ PArgs a,
-                                                          const __grid_constant__ CUtensorMap tmX,
                                                           const __grid_constant__ CUtensorMap tmXext) {
     using G = Geo<HS8>;
-    constexpr int H = G::H, NSB = G::NSB, NMB = G::NMB, SB = G::SB, NW = G::NW, ND2 = G::ND2;
+    constexpr int H = G::H, NSB = G::NSB, NMB = G::NMB, SPS = G::SPS, KPS = G::KPS, ND2 = G::ND2, NCH = G::NCH, NW = G::NW;
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* gbase = smem_dyn + (base - smem_u32(smem_dyn));
-    const uint32_t sW = base + G::OFF_W, sX = base + G::OFF_X, sH = base + G::OFF_H;
+    const uint32_t sW = base + G::OFF_W, sH = base + G::OFF_HX;
     int* sK = reinterpret_cast<int*>(gbase + G::OFF_K);
+    int* sIdx = reinterpret_cast<int*>(gbase + G::OFF_IDX);
     float* sRec = reinterpret_cast<float*>(gbase + G::OFF_REC);
+    volatile int* sMisc = reinterpret_cast<volatile int*>(gbase + G::OFF_MISC);
+    volatile uint32_t* g_tmem = reinterpret_cast<volatile uint32_t*>(gbase + G::OFF_MISC);      // [0] tensor-memory base
+    volatile int* sAbort = sMisc + 1;                              // [1] a wait of this CTA gave up
+    volatile int* sHslots = sMisc + 2;                             // [2] slots of the h tile (largest tile, rounded to 16)
+    volatile int* sLoaded = sMisc + 3;                             // [3] neurons whose gate/up rows the loaders have started on
+    int* sReady = const_cast<int*>(sMisc) + 4;                     // [4] ring stages (in consumption order) whose data has landed
+    const uint32_t s_tmem = base + G::OFF_MISC;
     const uint32_t bar0 = base + G::OFF_BAR;
-    auto w_full = [&](int s) { return bar0 + 8 * s; };              // up to 6
-    auto w_empty = [&](int s) { return bar0 + 48 + 8 * s; };
-    auto x_full = [&](int s) { return bar0 + 96 + 8 * s; };         // 4
-    auto x_empty = [&](int s) { return bar0 + 128 + 8 * s; };
-    auto d1_full = [&](int s) { return bar0 + 160 + 8 * s; };       // 2
-    auto d2_full = [&](int s) { return bar0 + 176 + 8 * s; };       // 2
-    auto d2_empty = [&](int s) { return bar0 + 192 + 8 * s; };
-    auto x_ready = [&](int s) { return bar0 + 208 + 8 * s; };       // 2
-    auto x_free = [&](int s) { return bar0 + 224 + 8 * s; };
-    const uint32_t h_full = bar0 + 240, h_free = bar0 + 248;
-    const uint32_t s_tmem = bar0 + 256;
-    volatile uint32_t* g_tmem = reinterpret_cast<volatile uint32_t*>(gbase + G::OFF_BAR + 256);
-    volatile int* sAbort = reinterpret_cast<volatile int*>(gbase + G::OFF_BAR + 264);
+    auto w_full = [&](int s) { return bar0 + 8 * s; };              // NW <= 6
+    auto w_empty = [&](int s) { return bar0 + 96 + 8 * s; };
+    auto x_full = [&](int s) { return bar0 + 192 + 8 * s; };        // up to XS_MAX = 8
+    auto x_empty = [&](int s) { return bar0 + 320 + 8 * s; };
+    auto d1_full = [&](int s) { return bar0 + 448 + 8 * s; };       // 2
+    auto d2_full = [&](int s) { return bar0 + 464 + 8 * s; };       // 2
+    auto d2_empty = [&](int s) { return bar0 + 480 + 8 * s; };
+    auto x_ready = [&](int s) { return bar0 + 496 + 8 * s; };       // 2
+    auto x_free = [&](int s) { return bar0 + 512 + 8 * s; };
+    const uint32_t h_full = bar0 + 528, h_free = bar0 + 536;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int j = (int)cluster_ctarank(), c = (int)cluster_id_x(), NC = (int)cluster_count_x();
@@ -218,17 +258,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     const int n_ctas = (int)gridDim.x;
     const int n_items = L * B;
 
-    if (tid == 0) {
-        for (int s = 0; s < NW; ++s) { mbar_init(w_full(s), 128); mbar_init(w_empty(s), 1); }
-        for (int s = 0; s < XS; ++s) { mbar_init(x_full(s), 1); mbar_init(x_empty(s), 1); }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(d1_full(s), 1); mbar_init(d2_full(s), 1); mbar_init(d2_empty(s), 256);
-            mbar_init(x_ready(s), CS); mbar_init(x_free(s), CS);
-        }
-        mbar_init(h_full, 1); mbar_init(h_free, CS);
-        fence_mbar_init();
-        *sAbort = 0;
-    }
     {
         const int cap = (int)(a.list_cap < (int64_t)I ? a.list_cap : (int64_t)I);
         for (int it = tid; it < n_items; it += NTHREADS) {
@@ -241,16 +270,37 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             sK[it] = k;
         }
     }
+    __syncthreads();
+    if (tid == 0) {
+        for (int s = 0; s < NW; ++s) { mbar_init(w_full(s), 128); mbar_init(w_empty(s), 1); }
+        for (int s = 0; s < XS_MAX; ++s) { mbar_init(x_full(s), 2); mbar_init(x_empty(s), 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(d1_full(s), 1); mbar_init(d2_full(s), 1); mbar_init(d2_empty(s), 256);
+            mbar_init(x_ready(s), CS); mbar_init(x_free(s), CS);
+        }
+        mbar_init(h_full, 1); mbar_init(h_free, CS);
+        fence_mbar_init();
+        *sAbort = 0;
+        *sLoaded = 0;
+        *sReady = 0;
+        int ts_max = 16;
+        for (int it = 0; it < n_items; ++it) {
+            const Run r = cluster_run(sK[it], c, NC);
+            if (r.ntiles > 0) { const int ts = (r.n + r.ntiles - 1) / r.ntiles; ts_max = ts > ts_max ? ts : ts_max; }
+        }
+        *sHslots = (ts_max + 15) & ~15;
+    }
     if (warp == W_MMA) tmem_alloc(s_tmem, 512);
-    if (warp >= W_NORM0 && warp < W_NORM0 + 4) {
-        // token rows T..63 of the cluster's x copies stay zero for the whole step
-        const int nw = warp - W_NORM0;
-        for (int slot = 0; slot < 2; ++slot)
-            for (int row = T + nw; row < NTOK; row += 4) {
-                if ((row & 7) != j) continue;
-                uint2* dst = reinterpret_cast<uint2*>(a.xbuf + ((size_t)(c * 2 + slot) * NTOK + row) * H);
-                for (int e = lane; e < H / 4; e += 32) dst[e] = make_uint2(0u, 0u);
-            }
+    // the x copies bring token rows 0..T-1 only: the other rows of every ring stage stay zero from here on
+    for (int e = tid; e < (G::END - G::OFF_HX) / 16; e += NTHREADS)
+        reinterpret_cast<uint4*>(gbase + G::OFF_HX)[e] = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+    if (warp < 8) {
+        // token rows T..63 of the cluster's x copies stay zero for the whole step (CTA j clears every 8th block)
+        for (int blk = j + CS * warp; blk < 2 * (H / 64); blk += CS * 8) {
+            unsigned char* img = reinterpret_cast<unsigned char*>(a.xbuf) + ((size_t)c * 2 * (H / 64) + blk) * X_BYTES;
+            for (int e = T * 8 + lane; e < NTOK * 8; e += 32) reinterpret_cast<uint4*>(img)[e] = make_uint4(0u, 0u, 0u, 0u);
+        }
         __threadfence();
         fence_proxy_async();
     }
@@ -259,6 +309,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     cluster_sync();
     tc_fence_after();
     const uint32_t tmem = *g_tmem;
+    const int h_half = *sHslots * 128;                             // bytes of the hi block (= of the lo block) of the h tile
+    const uint32_t sX = sH + 2 * h_half;
+    int xs_n = (G::END - G::OFF_HX - 2 * h_half) / XSB;
+    const int XS = xs_n > XS_MAX ? XS_MAX : xs_n;                    // >= 2
     Env env{sK, L, B, c, NC, a.x_ext};
 
     bool gave_up = false;
@@ -270,6 +324,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     };
     auto wait_at = [&](uint32_t bar, uint32_t parity, int line) {
         if (gave_up) return;
+        if (mbar_test_wait(bar, parity)) return;
         for (uint32_t i = 0; i < (1u << 22); ++i) {
             if (mbar_try_wait(bar, parity)) return;
             if (i > 64) __nanosleep(32);
@@ -284,9 +339,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
 #define WAIT(bar, parity) wait_at((bar), (parity), __LINE__)
 
     const uint64_t desc_k = smem_desc_sw128(0, 16, 1024);
-    const uint64_t desc_mn_a = smem_desc_sw128(0, 8192, 1024);
-    const uint64_t desc_mn_b = smem_desc_sw128(0, H_HALF, 1024);
-    constexpr uint32_t IDESC_G = idesc_bf16_f32(64, NTOK, false, false);
+    const uint64_t desc_mn_a = smem_desc_sw128(0, SPS * 128, 1024);
+    const uint64_t desc_mn_b = smem_desc_sw128(0, (uint32_t)h_half, 1024);
+    constexpr uint32_t IDESC_G = idesc_bf16_f32(128, 2 * NTOK, false, false);
     constexpr uint32_t IDESC_D = idesc_bf16_f32(128, 2 * NTOK, true, true);
 
     if (warp >= W_LOAD0 && warp < W_LOAD0 + 4) {
@@ -295,43 +350,57 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         const int lt = tid - W_LOAD0 * 32, lw = lt >> 5;
         const int pc = lt & 7, r0 = lt >> 3;                       // gate/up: 16-byte piece, rows r0 + 16 q
         uint32_t wcnt = 0;
+        int loaded = 0;
+        bool stop = false;                                         // agreed by all loader threads at the start of a tile
+        // one lane per warp waits for the stage (128 threads testing one mbarrier take several hundred clocks)
         auto acquire = [&]() {
             const int ws = wcnt % NW;
-            if (wcnt >= (uint32_t)NW) WAIT(w_empty(ws), ((wcnt / NW) - 1) & 1);
+            if (wcnt >= (uint32_t)NW) {
+                if (lane == 0) WAIT(w_empty(ws), ((wcnt / NW) - 1) & 1);
+                __syncwarp();
+            }
             return sW + ws * SB;
-        };
-        auto list_of = [&](const Cur& k) {
-            return a.idx ? a.idx + (size_t)k.b * a.idx_b_stride + (size_t)k.l * a.idx_l_stride : nullptr;
-        };
-        auto neuron = [&](const int32_t* list, int pos) {
-            int n = list ? __ldg(list + pos) : pos;
-            if (n < 0 || n >= I) { rm_set_status(a.status, RM_ERR_INDEX); n = -1; }
-            return n;
         };
         auto load_g = [&](const Cur& k) {
             int t0, ts, off, nj;
             tile_span(k.run, k.i, t0, ts);
             cta_span(ts, j, off, nj);
-            const int32_t* list = list_of(k);
+            // the tile's neuron ids, for these rows and for the tile's down stages
+            const int32_t* list = a.idx ? a.idx + (size_t)k.b * a.idx_b_stride + (size_t)k.l * a.idx_l_stride : nullptr;
+            int* ids = sIdx + (k.seq % 3) * CT;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int kk = lt + 128 * e;
+                int n = -1;
+                if (kk < ts) {
+                    n = list ? __ldg(list + t0 + kk) : t0 + kk;
+                    if (n < 0 || n >= I) { rm_set_status(a.status, RM_ERR_INDEX); n = -1; }
+                }
+                ids[kk] = n;
+            }
+            stop = named_barrier_or(3, 128, gave_up || *sAbort);
+            if (lt == 0) { loaded += nj; *sLoaded = loaded; }
             const __nv_bfloat16* src[4];
             bool ok[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const int r = r0 + 16 * q, i = r >> 1;
-                int n = -1;
-                if (i < nj) n = neuron(list, t0 + off + i);
+                const int n = i < nj ? ids[off + i] : -1;
                 ok[q] = n >= 0;
                 src[q] = a.packed[k.l] + (size_t)(n < 0 ? 0 : n) * 3 * H + (r & 1) * HS8 + pc * 8;
             }
-            for (int cc = 0; cc < CS; ++cc) {
+            // stage cc: the rows over the 64-column blocks cc (first 8 KB) and cc + NCH/2 (second 8 KB)
+            for (int cc = 0; cc < NCH / 2; ++cc) {
                 const uint32_t st = acquire();
+                const int c1 = cc + NCH / 2;
+                const int so0 = (cc / NSB) * 3 * HS8 + (cc % NSB) * 64, so1 = (c1 / NSB) * 3 * HS8 + (c1 % NSB) * 64;
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const int r = r0 + 16 * q;
                     const uint32_t d = st + (r >> 3) * 1024 + (r & 7) * 128 + ((pc ^ (r & 7)) << 4);
                     if (ok[q]) {
-#pragma unroll
-                        for (int sb = 0; sb < NSB; ++sb) cp_async16(d + sb * 8192, src[q] + cc * 3 * HS8 + sb * 64, true);
+                        cp_async16(d, src[q] + so0, true);
+                        cp_async16(d + 8192, src[q] + so1, true);
                     }
                 }
                 cp_async_arrive_noinc(w_full(wcnt % NW));
@@ -341,27 +410,21 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         auto load_d = [&](const Cur& k) {
             int t0, ts;
             tile_span(k.run, k.i, t0, ts);
-            const int32_t* list = list_of(k);
-            const int kst = (ts + 15) >> 4, nst = (ts + 63) >> 6;
+            const int* ids = sIdx + (k.seq % 3) * CT;
+            const int kst = (ts + 15) >> 4, nst = (ts + SPS - 1) / SPS;
             constexpr int PPS = HS8 / 8;                           // 16-byte pieces of a neuron's down slice
             constexpr int SPW = 32 / PPS;                          // slots one warp instruction covers
-            constexpr int NIT = 64 / (4 * SPW);
             const int piece = lane % PPS;
+            const __nv_bfloat16* wl = a.packed[k.l] + j * 3 * HS8 + 2 * HS8 + piece * 8;
             for (int s = 0; s < nst; ++s) {
                 const uint32_t st = acquire();
-                int nn[NIT];
 #pragma unroll
-                for (int m = 0; m < NIT; ++m) {
-                    const int slot = (lw + 4 * m) * SPW + lane / PPS, kk = 64 * s + slot;
-                    nn[m] = kk < ts ? neuron(list, t0 + kk) : -1;
-                }
-#pragma unroll
-                for (int m = 0; m < NIT; ++m) {
-                    const int slot = (lw + 4 * m) * SPW + lane / PPS, kk = 64 * s + slot;
+                for (int m = 0; m < 8; ++m) {
+                    const int slot = (lw + 4 * m) * SPW + lane / PPS, kk = SPS * s + slot;
                     if (kk >= 16 * kst) continue;                  // beyond the last product step of the tile
-                    const uint32_t d = st + (piece >> 3) * 8192 + slot * 128 + (((piece & 7) ^ (slot & 7)) << 4);
-                    const __nv_bfloat16* p = a.packed[k.l] + (size_t)(nn[m] < 0 ? 0 : nn[m]) * 3 * H + j * 3 * HS8 + 2 * HS8 + piece * 8;
-                    cp_async16(d, p, nn[m] >= 0);                  // unused slots of the last step: zeros
+                    const int n = kk < ts ? ids[kk] : -1;
+                    const uint32_t d = st + (piece >> 3) * (SPS * 128) + slot * 128 + (((piece & 7) ^ (slot & 7)) << 4);
+                    cp_async16(d, wl + (size_t)(n < 0 ? 0 : n) * 3 * H, n >= 0);      // unused slots of the last step: zeros
                 }
                 cp_async_arrive_noinc(w_full(wcnt % NW));
                 ++wcnt;
@@ -371,18 +434,51 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         cur_init(g, env);
         d = g;
         if (g.valid) { load_g(g); cur_next(g, env); }
-        while (d.valid && !gave_up) {
-            const bool ahead = g.valid && (g.item == d.item || B >= 2);
+        while (d.valid && !stop) {
+            const bool ahead = g.valid && may_run_ahead(g, d);
             if (ahead) { load_g(g); cur_next(g, env); }
             load_d(d);
             cur_next(d, env);
             if (!ahead && g.valid) { load_g(g); cur_next(g, env); }
         }
         cp_async_wait<0>();
-    } else if (warp == W_XTMA) {
-        // ================================================================ x boxes (one thread)
+    } else if (warp == W_PF) {
+        // ================================================================ L2 prefetch: while the loaders wait for ring
+        // space (the arithmetic is held up at a layer boundary), the rows of the tiles ahead are asked into L2, so
+        // that HBM keeps streaming.  A CTA asks for the whole rows of its own neurons; the cluster's CTAs together
+        // cover every slice that any of them will read.
+        Cur k;
+        cur_init(k, env);
+        int asked = 0;
+        const int ahead_n = a.pf_bytes / (6 * H);
+        while (k.valid && a.pf_bytes > 0) {
+            int t0, ts, off, nj;
+            tile_span(k.run, k.i, t0, ts);
+            cta_span(ts, j, off, nj);
+            bool go = false;
+            for (uint32_t i = 0; i < (1u << 20); ++i) {
+                if (asked - *sLoaded <= ahead_n) { go = true; break; }
+                if (*sAbort) break;
+                __nanosleep(200);
+            }
+            if (!go) break;                                        // a hint only: giving up costs nothing
+            if (lane < nj) {
+                const int32_t* list = a.idx ? a.idx + (size_t)k.b * a.idx_b_stride + (size_t)k.l * a.idx_l_stride : nullptr;
+                const int n = list ? __ldg(list + t0 + off + lane) : t0 + off + lane;
+                if (n >= 0 && n < I) prefetch_l2(a.packed[k.l] + (size_t)n * 3 * H, 6 * H);
+            }
+            asked += nj;
+            cur_next(k, env);
+        }
+    } else if (warp >= W_X0 && warp < W_X0 + NXW) {
+        // ================================================================ x copies: one thread of each of four warps,
+        // block n of the stream by thread n mod 4.  The cluster's own x is stored as shared-memory images, so a block
+        // is one contiguous 8 KB copy; the caller's x (single-layer entry) comes as one tensor-map box.
         if (lane == 0) {
-            uint32_t xcnt = 0;
+            // thread xq copies the half (xq & 1) of every second stage, starting with stage xq >> 1
+            const int xq = warp - W_X0, half = xq & 1;
+            uint32_t n = xq >> 1, ph = 0;                          // stage number in the stream; ring pass parity
+            int xs = (xq >> 1) % XS;                               // (XS >= 2)
             Cur k;
             cur_init(k, env);
             int cur_item = -1;
@@ -394,114 +490,202 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     ext = item_ext(env, k.l);
                     slot = k.use & 1;
                     if (!ext) {
-                        const uint32_t ph = (k.use >> 1) & 1;
+                        const uint32_t rph = (k.use >> 1) & 1;
                         bool ok = false;
                         for (uint32_t i = 0; i < (1u << 22) && !ok; ++i) {
-                            ok = mbar_try_wait_cluster(x_ready(slot), ph);
+                            ok = mbar_try_wait_cluster(x_ready(slot), rph);
                             if (!ok && i > 64) __nanosleep(32);
                             if ((i & 1023u) == 1023u && *sAbort) break;
                         }
                         if (!ok) { if (!*sAbort) timed_out(__LINE__); gave_up = true; break; }
-                        fence_proxy_async();
-                        RM_PS(k.item, 0);
+                        if (xq == 0) RM_PS(k.item, 0);
                     }
                 }
-                const int row = ext ? 0 : (c * 2 + slot) * NTOK;
-                for (int cc = 0; cc < CS * NSB; ++cc) {
-                    const int xs = xcnt % XS;
-                    if (xcnt >= (uint32_t)XS) WAIT(x_empty(xs), ((xcnt / XS) - 1) & 1);
-                    mbar_arrive_expect_tx(x_full(xs), X_BYTES);
-                    tma_load_2d(sX + xs * X_BYTES, ext ? &tmXext : &tmX, cc * 64, row, x_full(xs));
-                    ++xcnt;
+                const unsigned char* img = reinterpret_cast<const unsigned char*>(a.xbuf) + (size_t)(c * 2 + slot) * NCH * X_BYTES;
+                for (int cc = xq >> 1; cc < NCH / 2; cc += 2) {
+                    if (n >= (uint32_t)XS) WAIT(x_empty(xs), ph ^ 1);
+                    const int blk = cc + half * (NCH / 2);
+                    const uint32_t dst = sX + xs * XSB + half * X_BYTES;
+                    if (ext) {
+                        mbar_arrive_expect_tx(x_full(xs), X_BYTES);
+                        tma_load_2d(dst, &tmXext, blk * 64, 0, x_full(xs));
+                    } else {
+                        mbar_arrive_expect_tx(x_full(xs), (uint32_t)T * 128u);
+                        bulk_load(dst, img + (size_t)blk * X_BYTES, (uint32_t)T * 128u, x_full(xs));
+                    }
+                    n += 2;
+                    xs += 2;
+                    if (xs >= XS) { xs -= XS; ph ^= 1; }
                 }
                 cur_next(k, env);
+            }
+        }
+    } else if (warp == W_WATCH) {
+        // ================================================================ stage watcher (one thread): waits for the ring
+        // stages in the order in which the issuer consumes them, fences their cp.async data for the tensor core, and
+        // publishes the count
+        if (lane == 0) {
+            uint32_t wcnt = 0, xph = 0, stage = 0;
+            int xs = 0;
+            auto watch_g = [&](const Cur& k) {
+                long long c_w = 0, c_x = 0, c_f = 0;
+                for (int cc = 0; cc < NCH / 2; ++cc) {
+                    const long long q0 = RM_CLK();
+                    WAIT(w_full(wcnt % NW), (wcnt / NW) & 1);
+                    const long long q1 = RM_CLK();
+                    WAIT(x_full(xs), xph);
+                    const long long q2 = RM_CLK();
+                    fence_proxy_async_smem();
+                    st_release_cta(sReady, (int)++stage);
+                    const long long q3 = RM_CLK();
+                    if (cc > 0) { c_w += q1 - q0; c_x += q2 - q1; c_f += q3 - q2; }
+                    if (++xs == XS) { xs = 0; xph ^= 1; }
+                    ++wcnt;
+                }
+                if (k.i == 0) { RM_PC(k.item, 13, c_w); RM_PC(k.item, 14, c_x); RM_PC(k.item, 15, c_f); }
+            };
+            auto watch_d = [&](const Cur& k) {
+                int t0, ts;
+                tile_span(k.run, k.i, t0, ts);
+                const int nst = (ts + SPS - 1) / SPS;
+                for (int s = 0; s < nst; ++s) {
+                    WAIT(w_full(wcnt % NW), (wcnt / NW) & 1);
+                    fence_proxy_async_smem();
+                    st_release_cta(sReady, (int)++stage);
+                    ++wcnt;
+                }
+            };
+            Cur g, d;
+            cur_init(g, env);
+            d = g;
+            if (g.valid) { watch_g(g); cur_next(g, env); }
+            while (d.valid && !gave_up) {
+                const bool ahead = g.valid && may_run_ahead(g, d);
+                if (ahead) { watch_g(g); cur_next(g, env); }
+                watch_d(d);
+                cur_next(d, env);
+                if (!ahead && g.valid) { watch_g(g); cur_next(g, env); }
             }
         }
     } else if (warp == W_MMA) {
         // ================================================================ issuer (one thread)
         if (lane == 0) {
-            uint32_t wcnt = 0, xcnt = 0;
+            uint32_t wcnt = 0;
+            int xs = 0;
+            // Testing an mbarrier costs ~170 clocks even when its phase is long complete, which is more than the ~140
+            // clocks of a stage's two product instructions.  So the watcher thread does the waiting (and the proxy fence
+            // for the cp.async data) and publishes how many stages of the stream have landed; the issuer only reads that
+            // count, and reads it again only when it has used up what it knows of.
+            uint32_t stage = 0, ready = 0;                         // stages issued; stages known to have landed
+            int ready_next = 0;                                    // a read of the count started before the last products
+            auto peek = [&]() { if (stage + 1 >= ready) ready_next = ld_acquire_cta(sReady); };
+            auto need = [&](int line) {
+                if (stage >= ready) ready = (uint32_t)ready_next > ready ? (uint32_t)ready_next : ready;
+                if (stage < ready || gave_up) return;
+                for (uint32_t i = 0; i < (1u << 24); ++i) {
+                    ready = (uint32_t)ld_acquire_cta(sReady);
+                    if (stage < ready) return;
+                    if ((i & 4095u) == 4095u && *sAbort) { gave_up = true; return; }
+                }
+                timed_out(line);
+            };
             auto issue_g = [&](const Cur& k) {
                 const int buf = k.seq & 1;
-                for (int cc = 0; cc < CS; ++cc) {
+                long long c_n = 0, c_m = 0, c_c = 0;
+                for (int cc = 0; cc < NCH / 2; ++cc) {
                     const int ws = wcnt % NW;
-                    const uint32_t st = sW + ws * SB;
-                    WAIT(w_full(ws), (wcnt / NW) & 1);
-                    fence_proxy_async_smem();
+                    const uint32_t st = sW + ws * SB, xt = sX + xs * XSB;
+                    const long long q0 = RM_CLK();
+                    need(__LINE__);
+                    if (cc == 0 && k.i == 0) RM_PS(k.item, 1);
+                    tc_fence_after();
+                    peek();
+                    const long long q1 = RM_CLK();
 #pragma unroll
-                    for (int sb = 0; sb < NSB; ++sb) {
-                        const int xs = xcnt % XS;
-                        const uint32_t xt = sX + xs * X_BYTES;
-                        WAIT(x_full(xs), (xcnt / XS) & 1);
-                        if (cc == 0 && sb == 0 && k.i == 0) RM_PS(k.item, 1);
-                        tc_fence_after();
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            mma_bf16_ss(tmem + buf * NTOK, desc_k | desc_addr(st + sb * 8192 + ks * 32),
-                                        desc_k | desc_addr(xt + ks * 32), IDESC_G, (cc | sb | ks) != 0);
-                        mma_commit(x_empty(xs));
-                        ++xcnt;
-                    }
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_bf16_ss(tmem + buf * (2 * NTOK), desc_k | desc_addr(st + ks * 32), desc_k | desc_addr(xt + ks * 32),
+                                    IDESC_G, (cc | ks) != 0);
+                    const long long q2 = RM_CLK();
+                    mma_commit(x_empty(xs));
                     mma_commit(w_empty(ws));
+                    const long long q3 = RM_CLK();
+                    if (cc > 0) { c_n += q1 - q0; c_m += q2 - q1; c_c += q3 - q2; }
+                    if (++xs == XS) xs = 0;
                     ++wcnt;
+                    ++stage;
                 }
                 mma_commit(d1_full(buf));
+                if (k.i == 0) { RM_PS(k.item, 24); RM_PC(k.item, 10, c_n); RM_PC(k.item, 11, c_m); RM_PC(k.item, 12, c_c); }
                 if (k.i == k.run.ntiles - 1 && !item_ext(env, k.l)) mma_commit_mc(x_free(k.use & 1), 0xff);
             };
             auto issue_d = [&](const Cur& k) {
                 int t0, ts;
                 tile_span(k.run, k.i, t0, ts);
-                const int kst = (ts + 15) >> 4, nst = (ts + 63) >> 6;
+                const int kst = (ts + 15) >> 4, nst = (ts + SPS - 1) / SPS;
                 const int d2b = ND2 == 2 ? (k.ni & 1) : 0, nu = ND2 == 2 ? (k.ni >> 1) : k.ni;
                 if (k.i == 0 && nu >= 1) WAIT(d2_empty(d2b), (nu - 1) & 1);
                 WAIT(h_full, k.seq & 1);
                 RM_PS(k.item, 4);
-                tc_fence_after();
                 const uint32_t d2 = tmem + G::D2_COL + d2b * (2 * NTOK);
                 for (int s = 0; s < nst; ++s) {
                     const int ws = wcnt % NW;
                     const uint32_t st = sW + ws * SB;
-                    WAIT(w_full(ws), (wcnt / NW) & 1);
-                    fence_proxy_async_smem();
+                    need(__LINE__);
                     tc_fence_after();
-                    const int nks = kst - 4 * s < 4 ? kst - 4 * s : 4;
-                    for (int ks = 0; ks < nks; ++ks) {
-                        const int kk = 4 * s + ks;
+                    peek();
 #pragma unroll
-                        for (int mb = 0; mb < NMB; ++mb)
-                            mma_bf16_ss(d2 + mb * (2 * NTOK), desc_mn_a | desc_addr(st + mb * 16384 + ks * 2048),
-                                        desc_mn_b | desc_addr(sH + kk * 2048), IDESC_D, !(k.i == 0 && kk == 0));
+                    for (int ks = 0; ks < KPS; ++ks) {
+                        const int kk = KPS * s + ks;
+                        if (kk < kst) {
+#pragma unroll
+                            for (int mb = 0; mb < NMB; ++mb)
+                                mma_bf16_ss(d2 + mb * (2 * NTOK), desc_mn_a | desc_addr(st + mb * (2 * SPS * 128) + ks * 2048),
+                                            desc_mn_b | desc_addr(sH + kk * 2048), IDESC_D, !(k.i == 0 && kk == 0));
+                        }
                     }
                     mma_commit(w_empty(ws));
                     ++wcnt;
+                    ++stage;
                 }
                 mma_commit_mc(h_free, 0xff);
-                if (k.i == k.run.ntiles - 1) mma_commit(d2_full(d2b));
+                if (k.i == k.run.ntiles - 1) { mma_commit(d2_full(d2b)); RM_PS(k.item, 25); }
             };
             Cur g, d;
             cur_init(g, env);
             d = g;
             if (g.valid) { issue_g(g); cur_next(g, env); }
             while (d.valid && !gave_up) {
-                const bool ahead = g.valid && (g.item == d.item || B >= 2);
+                const bool ahead = g.valid && may_run_ahead(g, d);
                 if (ahead) { issue_g(g); cur_next(g, env); }
                 issue_d(d);
                 cur_next(d, env);
                 if (!ahead && g.valid) { issue_g(g); cur_next(g, env); }
             }
         }
-    } else if (warp >= W_NORM0) {
-        // ================================================================ normalisation: this cluster's copy of x
-        const int nw = warp - W_NORM0;
-        int use = 0;
+    } else {
+        // ================================================================ epilogue (8 warps): GLU, h exchange, flush
+        const int et = tid;                                         // 0..255
+        const int q4 = warp & 3, ch = warp >> 2;                    // tensor-memory lane quarter; token half
+        // D1 (M = 128): lane m < 64 holds row m's sum over the first half of H (token columns 0..63), lane 64 + m the
+        // same row's sum over the second half (token columns 64..127).  Row 2 i is neuron i's gate, row 2 i + 1 its up.
+        const bool fin = q4 < 2;                                    // lanes with a first-half sum (the others: second half)
+        const int m_row = (q4 & 1) * 32 + lane;                     // row 0..63 of this lane
+        const int ni_loc = m_row >> 1;                              // neuron of this lane among the CTA's 32
+        const bool isup = lane & 1;
+        float* sEx = reinterpret_cast<float*>(gbase + G::OFF_EX);   // [direction][token half][16 tokens][64 rows] fp32
+        unsigned char* gH = gbase + G::OFF_HX;
+        int seq = 0, ni = 0;
         bool stop = false;
-        for (int item = 0; item < n_items && !stop; ++item) {
+        // Normalisation of an item's input into this cluster's copy of x: CTA j takes the token rows j, j + 8, ...,
+        // one row per warp.  With one episode it runs right before the item's tiles (it has to wait for the previous
+        // layer's adds anyway); with several episodes it runs one item ahead, so that the next item's gate/up
+        // products can start while this item's tiles are finished.
+        int next_norm = 0, use = 0;
+        auto norm_item = [&](int item) {
             const int l = item / B, b = item - l * B;
-            const Run run = cluster_run(sK[item], c, NC);
-            if (run.ntiles == 0 || item_ext(env, l)) continue;
             const int slot = use & 1, nu = use >> 1;
             ++use;
-            if (nu >= 1) WAIT(x_free(slot), (nu - 1) & 1);
+            const bool xf_ok = nu >= 1 ? mbar_test_wait(x_free(slot), (nu - 1) & 1) : true;     // looked at before the stores
             if (l > 0) {
                 // every CTA has added its part of layer l-1 to this episode's rows
                 const int target = n_ctas * l;
@@ -515,23 +699,30 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 }
                 __syncwarp();
             }
-            if (nw == 0 && lane == 0) RM_PS(item, 8);
-            const float* rb = a.r + (size_t)b * T * H;
-            __nv_bfloat16* xb = a.xbuf + (size_t)(c * 2 + slot) * NTOK * H;
-            for (int row = j + 8 * nw; row < T; row += 32) {
-                const float4* src = reinterpret_cast<const float4*>(rb + (size_t)row * H);
+            if (et == 0) RM_PS(item, 8);
+            const long long n0 = RM_CLK();
+            long long n1 = n0, n2 = n0, n3 = n0;
+            const int row = j + 8 * warp;
+            if (row < T) {
+                const float4* src = reinterpret_cast<const float4*>(a.r + ((size_t)b * T + row) * H);
                 float4 v[H / 128];
                 float ss = 0.f;
 #pragma unroll
+                for (int q = 0; q < H / 128; ++q) v[q] = __ldcg(src + lane + 32 * q);
+#pragma unroll
                 for (int q = 0; q < H / 128; ++q) {
-                    v[q] = __ldcg(src + lane + 32 * q);
                     ss = fmaf(v[q].x, v[q].x, ss); ss = fmaf(v[q].y, v[q].y, ss);
                     ss = fmaf(v[q].z, v[q].z, ss); ss = fmaf(v[q].w, v[q].w, ss);
                 }
 #pragma unroll
                 for (int dd = 16; dd > 0; dd >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, dd);
                 const float inv = 1.0f / sqrtf(ss / (float)H + 1e-6f);
-                uint2* dst = reinterpret_cast<uint2*>(xb + (size_t)row * H);
+                n1 = RM_CLK();
+                if (!xf_ok) WAIT(x_free(slot), (nu - 1) & 1);          // the products that read this copy's previous contents are complete
+                // columns 4 (lane + 32 q) .. + 3 of this row: block q * 2 + lane / 16, 16-byte piece (lane % 16) / 2 of the
+                // row's 128 bytes in that block, swizzled by the row
+                unsigned char* img = reinterpret_cast<unsigned char*>(a.xbuf) + (size_t)(c * 2 + slot) * (H / 64) * X_BYTES +
+                                     row * 128 + ((((lane & 15) >> 1) ^ (row & 7)) << 4) + (lane & 1) * 8;
 #pragma unroll
                 for (int q = 0; q < H / 128; ++q) {
                     const __nv_bfloat162 lo = __floats2bfloat162_rn(v[q].x * inv, v[q].y * inv);
@@ -539,25 +730,27 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     uint2 u;
                     u.x = *reinterpret_cast<const uint32_t*>(&lo);
                     u.y = *reinterpret_cast<const uint32_t*>(&hi);
-                    dst[lane + 32 * q] = u;
+                    *reinterpret_cast<uint2*>(img + (size_t)(2 * q + (lane >> 4)) * X_BYTES) = u;
                 }
+                n2 = RM_CLK();
+                // the readers are copy-engine reads issued by this cluster's CTAs after the cluster-scope arrivals below
+                fence_proxy_async();
+                n3 = RM_CLK();
             }
-            __threadfence();
-            fence_proxy_async();
-            stop = named_barrier_or(2, 128, gave_up || *sAbort);
-            if (nw == 0 && lane < CS) mbar_arrive_remote(map_to_rank(x_ready(slot), lane));
-            if (nw == 0 && lane == 0) RM_PS(item, 9);
-        }
-    } else {
-        // ================================================================ epilogue (8 warps): GLU, h exchange, flush
-        const int et = tid;                                         // 0..255
-        const int q4 = warp & 3, ch = warp >> 2;                    // tensor-memory lane quarter; token half
-        const bool act = lane < 16;                                 // rows of D1 (M = 64) sit in lanes 0..15 of a quarter
-        const int ni_loc = 8 * q4 + (lane >> 1);                    // neuron of this lane among the CTA's 32
-        const bool isup = lane & 1;
-        int seq = 0, ni = 0;
-        bool stop = false;
+            stop = named_barrier_or(1, 256, gave_up || *sAbort);
+            const long long n4 = RM_CLK();
+            if (warp == 0 && lane < CS) mbar_arrive_remote(map_to_rank(x_ready(slot), lane));
+            if (et == 0) { RM_PS(item, 9); RM_PC(item, 26, n1 - n0); RM_PC(item, 27, n2 - n1); RM_PC(item, 28, n3 - n2); RM_PC(item, 29, n4 - n3); RM_PC(item, 30, RM_CLK() - n4); }
+        };
+        auto prepare_up_to = [&](int last) {
+            for (; next_norm <= last && next_norm < n_items && !stop; ++next_norm) {
+                const Run r = cluster_run(sK[next_norm], c, NC);
+                if (r.ntiles > 0 && !item_ext(env, next_norm / B)) norm_item(next_norm);
+            }
+        };
         for (int item = 0; item < n_items && !stop; ++item) {
+            prepare_up_to(item + (B >= 2 ? 1 : 0));
+            if (stop) break;
             const int l = item / B, b = item - l * B;
             const Run run = cluster_run(sK[item], c, NC);
             const int32_t* list = a.idx ? a.idx + (size_t)b * a.idx_b_stride + (size_t)l * a.idx_l_stride : nullptr;
@@ -567,86 +760,113 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 cta_span(ts, j, off, nj);
                 const int buf = seq & 1;
                 int n = -1;
-                if (act && ni_loc < nj) {
+                if (ni_loc < nj) {
                     n = list ? __ldg(list + t0 + off + ni_loc) : t0 + off + ni_loc;
                     if (n < 0 || n >= I) n = -1;
                 }
                 WAIT(d1_full(buf), (seq >> 1) & 1);
                 tc_fence_after();
                 if (et == 0 && i == 0) RM_PS(item, 2);
+                const long long e0 = RM_CLK();
+                // the test of "every CTA is done with the previous tile's h" takes ~300 clocks to come back even when the
+                // phase is long complete: start it now, look at the result when the h values are ready to be written
+                const bool hf_ok = seq >= 1 ? mbar_test_wait(h_free, (seq - 1) & 1) : true;
                 float v[32];
-                tmem_ld32(tmem + buf * NTOK + ch * 32 + ((uint32_t)(q4 * 32) << 16), v);
+                tmem_ld32(tmem + buf * (2 * NTOK) + (fin ? 0 : NTOK) + ch * 32 + ((uint32_t)(q4 * 32) << 16), v);
                 tc_fence_before();
-                // lane pair (2m, 2m+1) holds the gate and the up row of one neuron for tokens 32 ch .. 32 ch + 31;
-                // the even lane finishes the first 16 of them, the odd lane the last 16
-                float hv[16];
+                // This lane holds one half's sum of row m_row for tokens 32 ch .. 32 ch + 31.  Of these the first-half
+                // lane finishes tokens 0..15 and the second-half lane tokens 16..31: each passes the other 16 values.
                 {
-                    float gg[16], uu[16], e[16];
+                    float* out = sEx + (((fin ? 0 : 1) * 2 + ch) * 16) * 64 + m_row;
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) {
-                        const float mine = isup ? v[r] : v[16 + r];
+                    for (int r = 0; r < 16; ++r) out[r * 64] = fin ? v[16 + r] : v[r];
+                }
+                const long long e1 = RM_CLK();
+                named_barrier(1, 256);
+                const long long e2 = RM_CLK();
+                float s16[16];
+                {
+                    const float* in = sEx + (((fin ? 1 : 0) * 2 + ch) * 16) * 64 + m_row;
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) s16[r] = (fin ? v[r] : v[16 + r]) + in[r * 64];
+                }
+                // lane pair (2 i, 2 i + 1) = (gate row, up row) of neuron i for these 16 tokens: the even lane finishes
+                // the first 8 of them, the odd lane the last 8
+                float hv[8];
+                {
+                    float gg[8], uu[8], e[8];
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) {
+                        const float mine = isup ? s16[r] : s16[8 + r];
                         const float got = __shfl_xor_sync(0xffffffffu, mine, 1);
-                        gg[r] = isup ? got : v[r];
-                        uu[r] = isup ? v[16 + r] : got;
+                        gg[r] = isup ? got : s16[r];
+                        uu[r] = isup ? s16[8 + r] : got;
                     }
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) e[r] = __expf(-1.5957691216057308f * (gg[r] + 0.044715f * gg[r] * gg[r] * gg[r]));
+                    for (int r = 0; r < 8; ++r) e[r] = __expf(-1.5957691216057308f * (gg[r] + 0.044715f * gg[r] * gg[r] * gg[r]));
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) e[r] = __fdividef(gg[r], 1.0f + e[r]);
+                    for (int r = 0; r < 8; ++r) e[r] = __fdividef(gg[r], 1.0f + e[r]);
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) hv[r] = n >= 0 ? e[r] * uu[r] : 0.f;
+                    for (int r = 0; r < 8; ++r) hv[r] = n >= 0 ? e[r] * uu[r] : 0.f;
                 }
                 if (a.record) {
                     float rec = 0.f;
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) rec += fabsf(hv[r]);
+                    for (int r = 0; r < 8; ++r) rec += fabsf(hv[r]);
                     rec += __shfl_xor_sync(0xffffffffu, rec, 1);
-                    if (ch == 1 && act && !isup) sRec[ni_loc] = rec;
+                    const int grp = ch * 2 + (fin ? 0 : 1);                  // the four token quarters of a neuron
+                    if (grp != 0 && !isup) sRec[grp * NT + ni_loc] = rec;
                     named_barrier(1, 256);
-                    if (ch == 0 && act && !isup && n >= 0) {
-                        rec += sRec[ni_loc];
+                    if (grp == 0 && !isup && n >= 0) {
+                        rec += sRec[NT + ni_loc] + sRec[2 * NT + ni_loc] + sRec[3 * NT + ni_loc];
                         const float sc = a.record_scale ? a.record_scale[(size_t)l * I + n] : 1.f;
                         a.record[(size_t)b * a.rec_b_stride + (size_t)l * I + n] = a.record_scale ? rec * sc : rec;
                     }
                 }
-                if (seq >= 1) WAIT(h_free, (seq - 1) & 1);           // every CTA's down products of the previous tile are complete
-                if (act && ni_loc < nj) {
+                const long long e3 = RM_CLK();
+                if (!hf_ok) WAIT(h_free, (seq - 1) & 1);             // every CTA's down products of the previous tile are complete
+                const long long e4 = RM_CLK();
+                if (ni_loc < nj) {
                     const int kslot = off + ni_loc;
-                    const int p0 = ch * 4 + (isup ? 2 : 0);          // first 16-byte piece (8 tokens) of this lane's 16 tokens
-                    unsigned char* rowp = gbase + G::OFF_H + kslot * 128;
+                    const int p0 = ch * 4 + (fin ? 0 : 2) + (isup ? 1 : 0);   // 16-byte piece (8 tokens) of the row's 128 bytes
+                    uint32_t hi[4], lo[4];
 #pragma unroll
-                    for (int pp = 0; pp < 2; ++pp) {
-                        uint32_t hi[4], lo[4];
-#pragma unroll
-                        for (int e2 = 0; e2 < 4; ++e2) {
-                            const float f0 = hv[pp * 8 + 2 * e2], f1 = hv[pp * 8 + 2 * e2 + 1];
-                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(f0, f1);
-                            const float2 hf = __bfloat1622float2(h2);
-                            const __nv_bfloat162 l2 = __floats2bfloat162_rn(f0 - hf.x, f1 - hf.y);
-                            hi[e2] = *reinterpret_cast<const uint32_t*>(&h2);
-                            lo[e2] = *reinterpret_cast<const uint32_t*>(&l2);
-                        }
-                        const int o = ((p0 + pp) ^ (kslot & 7)) << 4;
-                        *reinterpret_cast<uint4*>(rowp + o) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                        *reinterpret_cast<uint4*>(rowp + H_HALF + o) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    for (int e2i = 0; e2i < 4; ++e2i) {
+                        const float f0 = hv[2 * e2i], f1 = hv[2 * e2i + 1];
+                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(f0, f1);
+                        const float2 hf = __bfloat1622float2(h2);
+                        const __nv_bfloat162 l2 = __floats2bfloat162_rn(f0 - hf.x, f1 - hf.y);
+                        hi[e2i] = *reinterpret_cast<const uint32_t*>(&h2);
+                        lo[e2i] = *reinterpret_cast<const uint32_t*>(&l2);
                     }
+                    unsigned char* rowp = gH + kslot * 128 + ((p0 ^ (kslot & 7)) << 4);
+                    *reinterpret_cast<uint4*>(rowp) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4*>(rowp + h_half) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                 }
                 {
                     // slots from ts to the end of the last product step: zeros (their weight rows are zeros too)
                     const int prow = ts + (et >> 4), pp = et & 15;
                     if (prow < (((ts + 15) >> 4) << 4))
-                        *reinterpret_cast<uint4*>(gbase + G::OFF_H + (pp >> 3) * H_HALF + prow * 128 + ((pp & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                        *reinterpret_cast<uint4*>(gH + (pp >> 3) * h_half + prow * 128 + ((pp & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
                 }
+                const long long e5 = RM_CLK();
                 fence_proxy_async_smem();
+                const long long e6 = RM_CLK();
                 stop = named_barrier_or(1, 256, gave_up || *sAbort);
+                const long long e7 = RM_CLK();
                 if (et == 0) mbar_arrive_expect_tx(h_full, (uint32_t)(ts - nj) * 256u);
                 if (et < 2 * (CS - 1) && nj > 0) {
                     int peer = et >> 1;
                     if (peer >= j) ++peer;
-                    const uint32_t src = sH + (et & 1) * H_HALF + off * 128;
+                    const uint32_t src = sH + (et & 1) * h_half + off * 128;
                     bulk_copy_to_peer(map_to_rank(src, peer), src, (uint32_t)nj * 128u, map_to_rank(h_full, peer));
                 }
-                if (et == 0 && i == 0) RM_PS(item, 3);
+                if (et == 0 && i == 0) {
+                    const long long e8 = RM_CLK();
+                    RM_PS(item, 3);
+                    RM_PC(item, 16, e1 - e0); RM_PC(item, 17, e2 - e1); RM_PC(item, 18, e3 - e2); RM_PC(item, 19, e4 - e3);
+                    RM_PC(item, 20, e5 - e4); RM_PC(item, 21, e6 - e5); RM_PC(item, 22, e7 - e6); RM_PC(item, 23, e8 - e7);
+                }
             }
             if (stop) break;
             if (run.ntiles > 0) {
@@ -737,7 +957,7 @@ int query_clusters(int* out) {
 }
 
 template <int HS8>
-int launch(rm_ctx* ctx, const PArgs& a, const CUtensorMap& tmX, const CUtensorMap& tmXext, int n_clusters, cudaStream_t s) {
+int launch(rm_ctx* ctx, const PArgs& a, const CUtensorMap& tmXext, int n_clusters, cudaStream_t s) {
     static rm_smem_configured configured = {};
     if (!configured.covers(ctx->device, Geo<HS8>::TOTAL)) {
         RM_CUDA_TRY(cudaFuncSetAttribute(step_kernel<HS8>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<HS8>::TOTAL));
@@ -755,7 +975,7 @@ int launch(rm_ctx* ctx, const PArgs& a, const CUtensorMap& tmX, const CUtensorMa
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, step_kernel<HS8>, a, tmX, tmXext));
+    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, step_kernel<HS8>, a, tmXext));
     ctx->launches++;
     return RM_OK;
 }
@@ -789,7 +1009,7 @@ size_t rm_persist_workspace_bytes(const rm_ctx* ctx) {
 
 int rm_persist_debug_stamps(long long* host_out, int n) {
 #ifdef RM_PHASE_TIMING
-    if (n > 64 * 128 * 16) n = 64 * 128 * 16;
+    if (n > 64 * 128 * 32) n = 64 * 128 * 32;
     return cudaMemcpyFromSymbol(host_out, g_ps_stamps, sizeof(long long) * n) == cudaSuccess ? RM_OK : RM_ERR_CUDA;
 #else
     (void)host_out; (void)n;
@@ -819,11 +1039,13 @@ int rm_launch_step_persist(rm_ctx* ctx, const rm_step_args& sa, void* ws, cudaSt
     a.T = sa.T;
     a.I = g.I;
     a.x_ext = sa.x_ext ? 1 : 0;
+    a.pf_bytes = ctx->persist_prefetch_kb * 1024;
     int nc = ctx->persist_clusters;
     if (ctx->max_clusters_override > 0 && ctx->max_clusters_override < nc) nc = ctx->max_clusters_override;
-    if (ctx->persist_xbuf != a.xbuf) {
-        const int rc = make_x_map(reinterpret_cast<CUtensorMap*>(ctx->persist_tm), a.xbuf,
-                                  (uint64_t)ctx->persist_clusters * 2 * NTOK, (uint64_t)g.H);
+    // the caller's x (single-layer entry) as a tensor map; otherwise any valid map (the kernel does not use it): one over
+    // the workspace, made once per workspace
+    if (!sa.x_ext && ctx->persist_xbuf != a.xbuf) {
+        const int rc = make_x_map(reinterpret_cast<CUtensorMap*>(ctx->persist_tm), a.xbuf, (uint64_t)NTOK, (uint64_t)g.H);
         if (rc != RM_OK) return rc;
         ctx->persist_xbuf = a.xbuf;
     }
@@ -835,6 +1057,5 @@ int rm_launch_step_persist(rm_ctx* ctx, const rm_step_args& sa, void* ws, cudaSt
         tm_ext = *reinterpret_cast<const CUtensorMap*>(ctx->persist_tm);
     }
     RM_CUDA_TRY(cudaMemsetAsync(a.sync, 0, 256, s));
-    const CUtensorMap& tmX = *reinterpret_cast<const CUtensorMap*>(ctx->persist_tm);
-    return g.H == 1024 ? launch<128>(ctx, a, tmX, tm_ext, nc, s) : launch<256>(ctx, a, tmX, tm_ext, nc, s);
+    return g.H == 1024 ? launch<128>(ctx, a, tm_ext, nc, s) : launch<256>(ctx, a, tm_ext, nc, s);
 }

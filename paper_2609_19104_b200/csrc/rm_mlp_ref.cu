@@ -185,6 +185,29 @@ size_t rm_ref_workspace_bytes(const rm_ctx* ctx, int B, int T) {
     return x_bytes + h_bytes;
 }
 
+namespace {
+// The gate/up kernel's dynamic shared-memory limit, per device: only ever raised, so that two users of the kernel
+// with different H (a context's portable path and the allocation-free entry point) cannot lower it under each other.
+constexpr int RM_MAX_DEVICES = 64;
+std::mutex g_gateup_mutex;
+int g_gateup_smem[RM_MAX_DEVICES] = {};
+constexpr size_t RM_GATEUP_SMEM_LIMIT = 227 * 1024;               // opt-in shared memory of one CTA on sm_100
+
+int ensure_gateup_smem(size_t smem) {
+    if (smem <= 48 * 1024) return RM_OK;
+    if (smem > RM_GATEUP_SMEM_LIMIT) return RM_ERR_SHAPE;
+    int dev = -1;
+    RM_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= RM_MAX_DEVICES) return RM_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_gateup_mutex);
+    if (g_gateup_smem[dev] < (int)smem) {
+        RM_CUDA_TRY(cudaFuncSetAttribute(ref_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        g_gateup_smem[dev] = (int)smem;
+    }
+    return RM_OK;
+}
+}  // namespace
+
 int rm_launch_layer_ref(rm_ctx* ctx, const rm_layer_args& a, void* ws, cudaStream_t s) {
     const rm_geom& g = ctx->g;
     if (a.B <= 0 || a.T <= 0) return RM_OK;
@@ -198,8 +221,10 @@ int rm_launch_layer_ref(rm_ctx* ctx, const rm_layer_args& a, void* ws, cudaStrea
         x = xbuf;
     }
     size_t smem = (size_t)GU_WARPS * 2 * g.H * sizeof(__nv_bfloat16);
-    if (smem > 48 * 1024)
-        RM_CUDA_TRY(cudaFuncSetAttribute(ref_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    {
+        const int rc = ensure_gateup_smem(smem);
+        if (rc != RM_OK) return rc == RM_ERR_SHAPE ? RM_ERR_UNSUPPORTED : rc;      // H beyond what this kernel can stage
+    }
     int kcap = a.count ? (int)(a.list_cap < (int64_t)g.I ? a.list_cap : (int64_t)g.I) : g.I;
     dim3 g1((kcap + GU_WARPS - 1) / GU_WARPS, a.B);
     ref_gateup_kernel<<<g1, GU_WARPS * 32, smem, s>>>(a, g, x, h, ctx->d_status);
@@ -226,7 +251,6 @@ static __device__ __align__(256) float g_static_h[RM_STATIC_H_FLOATS];
 constexpr int RM_STATIC_MAX_DEVICES = 64;
 std::mutex g_static_mutex;
 float* g_static_h_addr[RM_STATIC_MAX_DEVICES] = {};             // device address of g_static_h, per device
-int g_static_smem_set[RM_STATIC_MAX_DEVICES] = {};              // dynamic shared memory already enabled up to here
 
 }  // namespace
 
@@ -245,6 +269,10 @@ extern "C" int rm_sparse_mlp_static(const void* packed_layer, const void* x, con
     RM_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= RM_STATIC_MAX_DEVICES) return RM_ERR_UNSUPPORTED;
     const size_t smem = (size_t)GU_WARPS * 2 * H * sizeof(__nv_bfloat16);
+    {
+        const int rc = ensure_gateup_smem(smem);                  // RM_ERR_SHAPE: H above 7232 does not fit a CTA's shared memory
+        if (rc != RM_OK) return rc;
+    }
     float* h = nullptr;
     {
         // Once per device, with that device current: ask the runtime where the array lives on this device.  In host
@@ -254,10 +282,6 @@ extern "C" int rm_sparse_mlp_static(const void* packed_layer, const void* x, con
             float* p = nullptr;
             if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_h) != cudaSuccess || !p) return RM_ERR_CUDA;
             g_static_h_addr[dev] = p;
-        }
-        if (smem > 48 * 1024 && g_static_smem_set[dev] < (int)smem) {
-            RM_CUDA_TRY(cudaFuncSetAttribute(ref_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            g_static_smem_set[dev] = (int)smem;
         }
         h = g_static_h_addr[dev];
     }
@@ -273,7 +297,7 @@ extern "C" int rm_sparse_mlp_static(const void* packed_layer, const void* x, con
     a.r_in = residual;
     a.r_out = y;
     a.idx = idx;
-    a.count = idx ? count_dev : nullptr;
+    a.count = count_dev;                                           // with idx NULL: the leading count neurons, as in rm_sparse_mlp
     a.idx_stride = I;
     a.list_cap = I;
     a.count_stride = 1;

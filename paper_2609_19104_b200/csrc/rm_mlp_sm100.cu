@@ -1655,7 +1655,7 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
     const bool two_per_sm = ctx->g.H == 1024 && 2 * (lean_bytes + 1024) <= 228 * 1024;
     int cap = two_per_sm ? 2 * ctx->fused_clusters + 2 : ctx->fused_clusters;
     if (ctx->max_clusters_override > 0) cap = ctx->max_clusters_override;
-    int variant = ctx->variant_override;
+    int variant = ctx->variant_override == 5 ? 0 : ctx->variant_override;    // 5: a call the whole-step kernel does not cover
     if (variant == 0) variant = (ctx->g.H == 1024 || (tiles > 0 && tiles <= cap)) ? 1 : 3;
     if (variant == 3) {
         const int fits_t = ctx->g.H == 1024 ? SmemWS<64, 128>::total_bytes(la.T) : SmemWS<64, 256>::total_bytes(la.T);

@@ -78,3 +78,28 @@ def test_gather_read_microbenchmark_runs_and_reports_bad_counts(lib):
     ctx.rm_debug_gather_read(model.packed[0], dev(idx[0]), dev(np.array([I + 7], np.int32)), I)
     assert ctx.rm_device_status() != 0                                             # count above the capacity
     model.close()
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable(lib):
+    """Failure detection without a fault: a one-CTA kernel waits on a barrier nobody arrives at, with a few thousand
+    polls; the wait gives up, records RM_ERR_TIMEOUT with the place, and the kernel returns."""
+    import torch
+    ctx = lib.Context(1, 128, 64, 4)
+    assert ctx.rm_device_status() == 0
+    ctx.rm_debug_wait_timeout(4096)
+    assert ctx.rm_device_status() == lib.RM_ERR_TIMEOUT
+    detail = ctx.rm_get_info("status_detail")
+    assert detail != 0 and (detail >> 12) > 0 and (detail & 0xfff) == 0          # source line of the wait, CTA 0
+    assert ctx.rm_get_info("status_log_count") == 1
+    assert ctx.rm_device_status() == 0                                           # cleared by the read
+    assert ctx.rm_get_info("status_detail") == 0
+    # the context still works
+    w = wl.Workload(96, "after-timeout", 1, 128, 64, 4, 0.1, 1, 0.5)
+    model = Model(lib, w)
+    x, r = wl.step_input(w, 0), wl.residual_input(w)
+    y = torch.empty(4, 128, dtype=torch.float32, device="cuda")
+    from harness import dev_bf16
+    model.ctx.rm_sparse_mlp(model.packed[0], dev_bf16(x), dev(r), None, None, y)
+    assert_close(y.cpu().numpy(), oracle.dense_mlp(x, model.Wg[0], model.Wu[0], model.Wd[0], r), "after a timeout")
+    model.close()
+    ctx.close()

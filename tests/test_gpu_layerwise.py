@@ -1,0 +1,126 @@
+"""The deep dense stacks, layer by layer, at the UNRELAXED per-element bound.
+
+A dense (or anchored) step through all 18 layers is ill-conditioned as a whole: every layer re-quantises x to bf16,
+and a one-ulp difference early in the stack is carried to the output (test_oracle_pins.py::
+test_dense_stack_amplifies_one_ulp shows the oracle doing it to itself).  The free-running step outputs are therefore
+judged with a small allowance for outliers (harness.assert_close(deep_dense=True)).  What is well conditioned is a
+single layer: here every layer of those stacks gets the ORACLE's own x_l and r_l as its input, runs through
+rm_sparse_mlp (or a one-layer rm_action_expert_step_ex for the anchored schedule), and must meet
+|err| <= 2e-2 + 1e-2 |ref| on every element and 5e-3 in relative L2, with no allowance.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_19104_b200 import workloads as wl
+from harness import Model, assert_close, dev, dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def f32_of(bits):
+    return wl.bf16_bits_to_f32(bits)
+
+
+@pytest.fixture(scope="module")
+def pi0(lib):
+    w = wl.config1()
+    model = Model(lib, w, B_max=1)
+    yield model
+    model.close()
+
+
+def layer_by_layer(lib, model, r0, what, idx_lists=None, T=None):
+    """Walks the oracle through the stack; every layer's GPU result on the oracle's inputs is compared strictly."""
+    import torch
+    w = model.w
+    T = w.T if T is None else T
+    r = np.ascontiguousarray(r0, dtype=np.float32)
+    y = torch.empty(T, w.H, dtype=torch.float32, device="cuda")
+    worst_rel = 0.0
+    for l in range(w.L):
+        x = oracle.rmsnorm_bf16(r)
+        if idx_lists is None:
+            want = oracle.dense_mlp(x, model.Wg[l], model.Wu[l], model.Wd[l], r)
+            model.ctx.rm_sparse_mlp(model.packed[l], dev_bf16(x), dev(r), None, None, y, T=T)
+        else:
+            sel = np.ascontiguousarray(idx_lists[l], dtype=np.int32)
+            want = oracle.masked_mlp(x, model.Wg[l], model.Wu[l], model.Wd[l], r, sel)
+            buf = np.zeros(w.I, np.int32)
+            buf[:sel.size] = sel
+            model.ctx.rm_sparse_mlp(model.packed[l], dev_bf16(x), dev(r), dev(buf), dev(np.array([sel.size], np.int32)), y, T=T)
+        worst_rel = max(worst_rel, assert_close(y.cpu().numpy(), want, f"{what}, layer {l}"))
+        r = want                                                     # the oracle's own r_{l+1} feeds the next layer
+    assert model.ctx.rm_device_status() == 0
+    return worst_rel
+
+
+def test_dense_reference_pass_layer_by_layer(lib, pi0):
+    """The dense reference step of configs 1 and 3 (rho = 1.0 with idx = NULL)."""
+    w = pi0.w
+    rel = layer_by_layer(lib, pi0, f32_of(wl.reference_input(w)), "dense reference pass")
+    print(f"dense reference pass, per layer: worst rel_l2 {rel:.2e}")
+    rel = layer_by_layer(lib, pi0, f32_of(wl.step_input(w, 3)), "config 3 rho=1.0 (idx NULL)")
+    print(f"config 3 rho=1.0, per layer: worst rel_l2 {rel:.2e}")
+
+
+def test_full_list_layer_by_layer(lib, pi0):
+    """Config 3 at density 1.0 as a full index list (the gathering loaders on every neuron)."""
+    w = pi0.w
+    full = [np.arange(w.I, dtype=np.int32)] * w.L
+    layer_by_layer(lib, pi0, f32_of(wl.step_input(w, 3)), "config 3 rho=1.0 (full list)", idx_lists=full)
+
+
+def test_config4_dense_reference_layer_by_layer(lib, pi0):
+    """The dense reference passes of config 4 (T = 32) on the same weights."""
+    import paper_2609_19104_b200 as rm
+    w4 = wl.config4()
+
+    class View:
+        pass
+    m = View()
+    m.w, m.packed, m.Wg, m.Wu, m.Wd = w4, pi0.packed, pi0.Wg, pi0.Wu, pi0.Wd
+    m.ctx = rm.Context(w4.L, w4.H, w4.I, T_max=w4.T)
+    layer_by_layer(lib, m, f32_of(wl.reference_input(w4, record=0)), "config 4 dense reference", T=w4.T)
+    m.ctx.close()
+
+
+def test_anchor_schedule_layer_by_layer(lib, pi0):
+    """Config 5 (Eq. 4 with the output gate): the anchor step and one update step of each group, every layer on the
+    oracle's own inputs and anchor state through a one-layer rm_action_expert_step_ex."""
+    import torch
+    w = wl.config5()
+    L, T, H, I, K, G = w.L, w.T, w.H, w.I, w.K, w.extra["group"]
+    ctx1 = lib.Context(1, H, I, T_max=T)                            # one-layer stacks on the shared packed layers
+    h_stride = 52
+    y_an = torch.zeros(1, 1, T, H, dtype=torch.float32, device="cuda")
+    h_an = torch.zeros(1, 1, I, h_stride, dtype=torch.float32, device="cuda")
+    out = torch.empty(1, T, H, dtype=torch.float32, device="cuda")
+    # group masks from the oracle's own records of a reference execution (any valid lists serve here)
+    for s_anchor, s_update in ((0, 2), (5, 9)):
+        r_a = f32_of(wl.step_input(w, s_anchor))
+        r_u = f32_of(wl.step_input(w, s_update))
+        gate_a, gate_u = wl.output_gate(w, s_anchor), wl.output_gate(w, s_update)
+        for l in range(L):
+            # anchor layer on the oracle's r_a
+            x = oracle.rmsnorm_bf16(r_a)
+            ya, ha, rec = oracle.dense_mlp(x, pi0.Wg[l], pi0.Wu[l], pi0.Wd[l], None, return_h=True, return_record=True)
+            want_a = (r_a.astype(np.float64) + gate_a[l][None, :].astype(np.float64) * ya.astype(np.float64)).astype(np.float32)
+            ctx1.rm_action_expert_step_ex([pi0.packed[l]], dev(r_a[None]), None, None, 0, out, lib.RM_ANCHOR_WRITE, y_an, h_an,
+                                          h_stride, out_gate=dev(gate_a[l][None, None, :]), B=1, T=T)
+            assert_close(out.cpu().numpy()[0], want_a, f"config 5 anchor step {s_anchor}, layer {l}")
+            assert_close(y_an.cpu().numpy()[0, 0], ya, f"config 5 y_anchor, step {s_anchor}, layer {l}")
+            # update layer: mask = the layer's top-K by this anchor's record; anchor state = the GPU's own (just checked)
+            sel = oracle.compact_scores(rec, oracle.RULE_TOPK, k=K)
+            x_u = oracle.rmsnorm_bf16(r_u)
+            want_u = oracle.anchor_mlp(x_u, pi0.Wg[l], pi0.Wu[l], pi0.Wd[l], r_u, sel, ya, np.ascontiguousarray(ha[:, sel]),
+                                       gate_u[l])
+            buf = np.zeros(I, np.int32)
+            buf[:sel.size] = sel
+            ctx1.rm_action_expert_step_ex([pi0.packed[l]], dev(r_u[None]), dev(buf[None]), dev(np.array([sel.size], np.int32)),
+                                          I, out, lib.RM_ANCHOR_UPDATE, y_an, h_an, h_stride,
+                                          out_gate=dev(gate_u[l][None, None, :]), B=1, T=T)
+            assert_close(out.cpu().numpy()[0], want_u, f"config 5 update step {s_update}, layer {l}")
+            r_a, r_u = want_a, want_u
+    assert ctx1.rm_device_status() == 0
+    ctx1.close()

@@ -117,6 +117,19 @@ def test_group_mask(lib, W, k):
     check_lists(out_idx, out_cnt, [oracle.compact_group([r[i] for r in recs], k) for i in range(n_lists)])
 
 
+def test_group_mask_tie_at_the_cut(lib):
+    """Hand-built records whose union members have equal summed scores on both sides of the cut: the expected lists
+    are written out here (lower index kept), not taken from the oracle."""
+    cases = [([[9, 0, 0, 4, 1, 0, 0, 0], [0, 0, 0, 1, 4, 0, 0, 0]], 2, [0, 3]),
+             ([[9, 0, 0, 1, 4, 0, 0, 0], [0, 0, 0, 4, 1, 0, 0, 0]], 2, [0, 3]),
+             ([[0, 7, 3, 0, 0, 0, 0, 0], [0, 0, 0, 0, 0, 3, 3, 3]], 3, [1, 2, 5])]
+    for recs, k, want in cases:
+        recs = [np.array(r, np.float32)[None] for r in recs]
+        out_idx, out_cnt, status = run_compact(lib, 8, recs, lib.RM_SRC_SCORE_F32, lib.RM_REDUCE_GROUP, 1, k=k)
+        assert status == 0 and out_cnt[0] == len(want) and out_idx[0, :len(want)].tolist() == want
+        assert np.array_equal(oracle.compact_group([r[0] for r in recs], k), np.array(want, np.int32))
+
+
 def test_truncation_is_reported_not_fatal(lib):
     I = 512
     m = np.ones((1, I), dtype=np.uint8)

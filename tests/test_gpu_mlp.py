@@ -183,7 +183,7 @@ def test_step_host_variant_matches_device_variant(lib):
     model.close()
 
 
-@pytest.mark.parametrize("variant", [1, 2, 3, 4])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4, 5])
 @pytest.mark.parametrize("H,I,T,B", [(1024, 2048, 51, 2), (1024, 1024, 32, 1), (2048, 1024, 51, 1),
                                      (2048, 1024, 32, 1), (1024, 1024, 64, 1), (2048, 1024, 64, 1)])
 def test_every_tensor_core_variant_and_the_portable_path_agree_with_the_oracle(lib, variant, H, I, T, B):
@@ -256,7 +256,7 @@ def test_repeated_dense_stacks_agree_across_runs_and_variants(lib, H, I, T, mask
     ref = run(1)
     assert_close(ref, oracle.step(model.Wg, model.Wu, model.Wd, wl.bf16_bits_to_f32(wl.step_input(w, 0)), idx, cnt),
                  "lean kernel")
-    for variant in (1, 2, 3, 4):
+    for variant in (1, 2, 3, 4, 5):
         for rep in range(60):
             got = run(variant)
             worst = float(np.max(np.abs(got - ref)))

@@ -37,7 +37,7 @@ def test_batched_masked_stacks_repeat(lib, H, I, T, L, B, max_clusters):
     for b in range(B):
         i_b, c_b = lists_to_padded(lists[b], I)
         want.append(oracle.step(model.Wg, model.Wu, model.Wd, r0[b], i_b, c_b))
-    for variant in (1, 2, 3, 4):
+    for variant in (1, 2, 3, 4, 5):
         ctx.rm_set_option("path", 2)
         ctx.rm_set_option("variant", variant)
         ctx.rm_set_option("max_clusters", max_clusters)

@@ -339,6 +339,30 @@ def test_group_mask_identities():
     assert total[g].min() >= total[rest].max()
 
 
+def hand_built_group_ties():
+    """Two records whose per-record top-2 sets are {0, 3} and {3, 4}: the union {0, 3, 4} has the summed scores 9, 5, 5,
+    so the cut of the group's top-2 falls between two members with EQUAL sums -- the lower index (3) stays.  In the
+    second pair the two records swap which of 3 / 4 they favour: the kept member must still be 3 (the rule looks at
+    the sum and the index, not at which record brought the neuron in)."""
+    a0 = np.array([9, 0, 0, 4, 1, 0, 0, 0], np.float32)
+    a1 = np.array([0, 0, 0, 1, 4, 0, 0, 0], np.float32)
+    return [([a0, a1], 2, np.array([0, 3], np.int32)),
+            ([np.array([9, 0, 0, 1, 4, 0, 0, 0], np.float32), np.array([0, 0, 0, 4, 1, 0, 0, 0], np.float32)], 2,
+             np.array([0, 3], np.int32))]
+
+
+def test_group_mask_tie_at_the_cut_keeps_the_lower_index():
+    for recs, k, want in hand_built_group_ties():
+        for r in recs:                                   # the premise: per-record sets as the docstring says
+            assert oracle.compact_scores(r, oracle.RULE_TOPK, k=k).size == k
+        got = oracle.compact_group(recs, k)
+        assert np.array_equal(got, want), (got, want)
+    # a longer tie run across the cut: sums 7, 3, 3, 3, 3 over members 1, 2, 5, 6, 7 and k = 3 -> {1, 2, 5}
+    r0 = np.array([0, 7, 3, 0, 0, 0, 0, 0], np.float32)
+    r1 = np.array([0, 0, 0, 0, 0, 3, 3, 3], np.float32)
+    assert np.array_equal(oracle.compact_group([r0, r1], 3), np.array([1, 2, 5], np.int32))
+
+
 # ------------------------------------------------------------------ Eq. 4 and the stack
 def test_eq4_special_cases():
     x, Wg, Wu, Wd, r = small_problem(19)
