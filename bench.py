@@ -30,9 +30,15 @@ from paper_2609_19104_b200 import workloads as wl  # noqa: E402
 METRIC = "masked_mlp_us_per_denoise_step"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one fused layer launch, from the ncu capture summarised in
-# profiles/fused_layer_kernel_config1.md
-TRAFFIC_BYTES_PER_LAUNCH = {"pi0-stack-top25": 6.794e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per layer of a step, from ncu captures of the kernels that run these
+# workloads (one layer launch of the lean per-layer kernel; the whole-step kernel's figure divided by its layers)
+TRAFFIC_BYTES_PER_LAYER = {"pi0-stack-top25": 6.794e6}
+KERNEL_FAMILY = {0: "portable CUDA-core kernels (norm, gate/up, down)",
+                 1: "fused_layer_kernel (lean per-layer cluster kernel, dependent-launch chained)",
+                 2: "fused_layer_kernel, two tiles in flight",
+                 3: "fused_layer_ws_kernel (warp-specialised per-layer cluster kernel)",
+                 4: "stream_prep_kernel + stream_tile_kernel (per-layer streaming kernel)",
+                 5: "step_kernel (whole step in one launch)"}
 
 
 def measured_hbm_peak():
@@ -334,6 +340,161 @@ def run_context(args, w: wl.Workload):
     print(json.dumps(line))
 
 
+
+# ------------------------------------------------------------------------------------------------ the other workloads
+def side_configs(rm, ctx1, packed1, w1, flush, stream, args):
+    """The workloads besides the headline one, measured in the same run and reported in the line's "configs" object:
+    us per step (cold L2, CUDA events on the launching stream, median), algorithmic bytes per layer of a step,
+    achieved GB/s and fraction of the measured copy bandwidth, and the kernel family the library chose by itself
+    (read back from the library).  For batches the fraction is computed on the bytes that must leave HBM at least
+    once -- the UNION of the episodes' lists -- and the sum over the episodes is given beside it."""
+    import torch
+    peak, _ = measured_hbm_peak()
+    reps = max(5, min(args.steps, 20))
+    f32 = lambda bits: torch.from_numpy(wl.bf16_bits_to_f32(bits))
+
+    def timed_us(fn):
+        evs = []
+        for i in range(3 + reps):
+            flush.fill_(i & 0xFF)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn(i)
+            b.record(stream)
+            if i >= 3:
+                evs.append((a, b))
+        torch.cuda.synchronize()
+        return float(np.median([a.elapsed_time(b) for a, b in evs])) * 1e3
+
+    def entry(ctx, w, us, K, B=1, union_rows=None, layers=None, note=None):
+        L = w.L if layers is None else layers
+        per_layer_sum = wl.algorithmic_bytes_per_layer(w.H, w.T, int(round(K))) * B
+        e = {"us_per_step": us / B, "us_per_layer": us / L, "K_per_layer": K, "B": B, "T": w.T, "H": w.H, "I": w.I, "L": L,
+             "kernel_family": ctx.rm_get_info("last_variant"), "kernel": KERNEL_FAMILY.get(ctx.rm_get_info("last_variant"))}
+        if union_rows is None:
+            e["bytes_per_layer"] = per_layer_sum
+        else:
+            act = per_layer_sum - int(round(K)) * 3 * w.H * 2 * B              # activations, residuals, indices of all episodes
+            e["bytes_per_layer"] = int(union_rows * 3 * w.H * 2) + act
+            e["bytes_per_layer_sum_over_episodes"] = per_layer_sum
+            e["union_neurons_per_layer"] = union_rows
+        e["achieved_gbs"] = e["bytes_per_layer"] * L / (us * 1e-6) / 1e9
+        e["frac"] = e["achieved_gbs"] / peak
+        if union_rows is not None:
+            e["frac_on_sum_over_episodes"] = per_layer_sum * L / (us * 1e-6) / 1e9 / peak
+        status = ctx.rm_device_status()
+        if status != 0:
+            raise RuntimeError(f"device status {status} in side workload {w.name}")
+        if note:
+            e["note"] = note
+        return e
+
+    def topk_lists(ctx, w, rec, K, n_lists):
+        idx = torch.zeros(n_lists, w.I, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros(n_lists, dtype=torch.int32, device="cuda")
+        ctx.rm_mask_compact([rec.view(n_lists, w.I)], rm.RM_SRC_SCORE_F32, rm.RM_REDUCE_TOPK, idx, cnt, w.I, n_lists=n_lists, k=K)
+        return idx, cnt
+
+    out = {}
+    # ---- config 3: density sweep and the batch of 8 on the headline model
+    rec1 = torch.zeros(1, w1.L, w1.I, dtype=torch.float32, device="cuda")
+    r_out = torch.empty(1, w1.T, w1.H, dtype=torch.float32, device="cuda")
+    ref1 = f32(wl.reference_input(w1))[None].cuda()
+    x1 = f32(wl.step_input(w1, 3))[None].cuda()
+    ctx1.rm_action_expert_step(packed1, ref1, None, None, 0, r_out, records_out=rec1, B=1, T=w1.T)
+    for rho in (0.2, 0.4, 1.0):
+        w3 = wl.config3(rho)
+        idx, cnt = topk_lists(ctx1, w3, rec1, w3.K, w3.L)
+        ctx1.rm_set_option("count_hint", w3.K)
+        us = timed_us(lambda i: ctx1.rm_action_expert_step(packed1, x1, idx, cnt, w3.I, r_out, B=1, T=w3.T))
+        out[f"config3_rho{rho:g}"] = entry(ctx1, w3, us, w3.K)
+    us = timed_us(lambda i: ctx1.rm_action_expert_step(packed1, x1, None, None, 0, r_out, records_out=rec1, B=1, T=w1.T))
+    out["config1_dense_reference_step"] = entry(ctx1, w1, us, w1.I, note="idx = NULL, activation records emitted")
+    B = 8
+    w3b = wl.config3(0.25, B=B)
+    ctxb = rm.Context(w3b.L, w3b.H, w3b.I, T_max=w3b.T, B_max=B)
+    refs = torch.stack([f32(wl.reference_input(w3b, episode=b)) for b in range(B)]).cuda()
+    xs = torch.stack([f32(wl.step_input(w3b, 2, episode=b)) for b in range(B)]).cuda()
+    recb = torch.zeros(B, w3b.L, w3b.I, dtype=torch.float32, device="cuda")
+    outb = torch.empty(B, w3b.T, w3b.H, dtype=torch.float32, device="cuda")
+    ctxb.rm_action_expert_step(packed1, refs, None, None, 0, outb, records_out=recb, B=B, T=w3b.T)
+    idxb, cntb = topk_lists(ctxb, w3b, recb, w3b.K, B * w3b.L)
+    ctxb.rm_set_option("count_hint", w3b.K)
+    h_idx = idxb.cpu().numpy().reshape(B, w3b.L, -1)
+    union = float(np.mean([len(set().union(*[set(h_idx[b, l, :w3b.K].tolist()) for b in range(B)])) for l in range(w3b.L)]))
+    us = timed_us(lambda i: ctxb.rm_action_expert_step(packed1, xs, idxb, cntb, w3b.I, outb, B=B, T=w3b.T))
+    out["config3_rho0.25_B8"] = entry(ctxb, w3b, us, w3b.K, B=B, union_rows=union,
+                                      note="us_per_step is per episode (one call runs 8 episodes); frac on the union of the lists")
+    ctxb.close()
+    # ---- config 4: T = 32, vote over a window of 4 records with a run-structured score scale
+    w4 = wl.config4()
+    ctx4 = rm.Context(w4.L, w4.H, w4.I, T_max=w4.T)
+    scale = torch.from_numpy(np.stack([wl.run_structure(w4, l)[1] for l in range(w4.L)])).cuda()
+    recs4 = []
+    out4 = torch.empty(1, w4.T, w4.H, dtype=torch.float32, device="cuda")
+    for i in range(w4.extra["window"]):
+        rec = torch.zeros(1, w4.L, w4.I, dtype=torch.float32, device="cuda")
+        ctx4.rm_action_expert_step(packed1, f32(wl.reference_input(w4, record=i))[None].cuda(), None, None, 0, out4,
+                                   records_out=rec, record_scale=scale, B=1, T=w4.T)
+        recs4.append(rec.view(w4.L, w4.I))
+    idx4 = torch.zeros(w4.L, w4.I, dtype=torch.int32, device="cuda")
+    cnt4 = torch.zeros(w4.L, dtype=torch.int32, device="cuda")
+    ctx4.rm_mask_compact(recs4, rm.RM_SRC_SCORE_F32, rm.RM_REDUCE_TOPK, idx4, cnt4, w4.I, n_lists=w4.L, k=w4.K,
+                         min_votes=w4.extra["min_votes"])
+    K4 = float(cnt4.float().mean().item())
+    ctx4.rm_set_option("count_hint", int(round(K4)))
+    x4 = f32(wl.step_input(w4, 3))[None].cuda()
+    us = timed_us(lambda i: ctx4.rm_action_expert_step(packed1, x4, idx4, cnt4, w4.I, out4, B=1, T=w4.T))
+    out["config4"] = entry(ctx4, w4, us, K4, note="lists: 3-of-4 vote over per-record top-615 sets of run-structured records")
+    ctx4.close()
+    # ---- config 0: one layer, Bernoulli(0.30) mask, through rm_sparse_mlp
+    w0 = wl.config0()
+    ctx0 = rm.Context(1, w0.H, w0.I, T_max=w0.T)
+    to = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    # eight copies of the layer in turn, so that consecutive timed calls do not find their weights in L2 either way
+    g0, u0, d0 = wl.layer_weights(w0, 0)
+    copies = [ctx0.rm_pack_weights(to(g0), to(u0), to(d0)) for _ in range(8)]
+    mask = torch.from_numpy(wl.bernoulli_mask(w0)).cuda()
+    idx0 = torch.zeros(w0.I, dtype=torch.int32, device="cuda")
+    cnt0 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx0.rm_mask_compact([mask], rm.RM_SRC_BOOL_U8, rm.RM_REDUCE_NONE, idx0, cnt0, w0.I, n_lists=1)
+    K0 = int(cnt0.item())
+    ctx0.rm_set_option("count_hint", K0)
+    x0, r0 = to(wl.step_input(w0, 0)), torch.from_numpy(wl.residual_input(w0)).cuda()
+    y0 = torch.empty(w0.T, w0.H, dtype=torch.float32, device="cuda")
+    us = timed_us(lambda i: ctx0.rm_sparse_mlp(copies[i % 8], x0, r0, idx0, cnt0, y0, T=w0.T))
+    out["config0_single_layer"] = entry(ctx0, w0, us, K0, layers=1, note="one rm_sparse_mlp call")
+    ctx0.close()
+    del copies
+    # ---- config 2: H = 2048, I = 16384 (weights drawn on the device: 1.8 G values)
+    w2 = wl.config2()
+    ctx2 = rm.Context(w2.L, w2.H, w2.I, T_max=w2.T)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w2.seed)
+    mk = lambda shape: (torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32) * w2.sigma).to(torch.bfloat16)
+    packed2 = [ctx2.rm_pack_weights(mk((w2.I, w2.H)), mk((w2.I, w2.H)), mk((w2.H, w2.I))) for _ in range(w2.L)]
+    rec2 = torch.zeros(1, w2.L, w2.I, dtype=torch.float32, device="cuda")
+    out2 = torch.empty(1, w2.T, w2.H, dtype=torch.float32, device="cuda")
+    xd = f32(wl.step_input(w2, 0))[None].cuda()
+    xsp = f32(wl.step_input(w2, 1))[None].cuda()
+    us_dense = timed_us(lambda i: ctx2.rm_action_expert_step(packed2, xd, None, None, 0, out2, records_out=rec2, B=1, T=w2.T))
+    out["config2_dense_step"] = entry(ctx2, w2, us_dense, w2.I, note="even steps of the schedule: dense, activation records emitted")
+    idx2, cnt2 = topk_lists(ctx2, w2, rec2, w2.K, w2.L)
+    ctx2.rm_set_option("count_hint", w2.K)
+    us_sparse = timed_us(lambda i: ctx2.rm_action_expert_step(packed2, xsp, idx2, cnt2, w2.I, out2, B=1, T=w2.T))
+    e = entry(ctx2, w2, us_sparse, w2.K, note="odd steps of the schedule: masked with the previous step's top-20 % lists")
+    e["traffic_bytes_per_layer"] = TRAFFIC_BYTES_PER_LAYER.get(w2.name)
+    us_g = timed_us(lambda i: ctx2.rm_debug_gather_read_step(packed2, idx2, cnt2, w2.I))
+    e["gather_read_microbench_us_per_step"] = us_g
+    e["gather_read_microbench_gbs"] = w2.K * 3 * w2.H * 2 * w2.L / (us_g * 1e-6) / 1e9
+    out["config2_sparse_step"] = e
+    us_c = timed_us(lambda i: ctx2.rm_mask_compact([rec2.view(w2.L, w2.I)], rm.RM_SRC_SCORE_F32, rm.RM_REDUCE_TOPK, idx2, cnt2,
+                                                   w2.I, n_lists=w2.L, k=w2.K))
+    out["config2_schedule_10_steps"] = {"us_total": 5 * (us_dense + us_c + us_sparse), "mask_compact_us": us_c,
+                                        "note": "5 x (dense step + top-k on the GPU + sparse step)"}
+    ctx2.close()
+    return out
+
 # ------------------------------------------------------------------------------------------------ GPU arm
 def run_gpu(args, w: wl.Workload):
     import torch
@@ -476,6 +637,7 @@ def run_gpu(args, w: wl.Workload):
         dist.barrier()
     torch.cuda.synchronize()
     launches = ctx.launch_count() - launches0
+    step_variant = ctx.rm_get_info("last_variant")          # the kernel family the library chose for the timed steps
     status = ctx.rm_device_status()
     if status != 0:
         log = [ctx.rm_get_info(f"status_log:{i}") for i in range(ctx.rm_get_info("status_log_count"))]
@@ -507,7 +669,7 @@ def run_gpu(args, w: wl.Workload):
                          3, True)
         compact()                                           # the lists again, from the records just rewritten
     # the same lists through the gather-read microbenchmark (layer by layer, cold L2): how fast they can leave HBM at all
-    gather_us = timed(lambda i: [ctx.rm_debug_gather_read(packed[l], idx[l], cnt[l:l + 1], w.I) for l in range(w.L)], 5, True)
+    gather_us = timed(lambda i: ctx.rm_debug_gather_read_step(packed, idx, cnt, w.I), 5, True)
     union_rows = None
     if B > 1 and not anchored:
         h_idx, h_cnt = idx.cpu().numpy().reshape(B, w.L, -1), cnt.cpu().numpy().reshape(B, w.L)
@@ -556,6 +718,10 @@ def run_gpu(args, w: wl.Workload):
 
     total_ms, e2e_total_ms = max_over_ranks([total_ms, e2e_total_ms], world, device="cuda")
 
+    side = None
+    if rank == 0 and world == 1 and w.config == 1 and not args.no_configs and not args.variant:
+        side = side_configs(rm, ctx, packed, w, flush, stream, args)
+
     if rank == 0:
         us_per_step = job_us_per_step(total_ms, args.steps, world, B)   # per denoising step of one episode, whole job
         e2e_us = job_us_per_step(e2e_total_ms, args.steps, world, B)
@@ -568,15 +734,7 @@ def run_gpu(args, w: wl.Workload):
             bytes_layer = wl.algorithmic_bytes_per_layer(w.H, w.T, int(round(K_mean))) * B
         bytes_step = bytes_layer * w.L
         launches_per_step = launches / args.steps                 # fused layer launches + mask compaction share
-        # the kernel the library picks for this launch shape (see the variant selection in the library)
-        tiles_per_launch = (int(round(K_mean)) + 63) // 64 * B
-        stream_from = 48 if w.H == 1024 else 64                   # the library's default crossover ("stream_min_tiles")
-        if args.variant == 4 or (args.variant == 0 and tiles_per_launch >= stream_from):
-            kernel_name = "stream_prep_kernel + stream_tile_kernel"
-        elif w.H == 1024:
-            kernel_name = "fused_layer_kernel<NTOK,128,false,*>" if args.variant in (0, 1) else f"variant {args.variant}"
-        else:
-            kernel_name = "fused_layer_ws_kernel<NTOK,256,*>" if args.variant in (0, 3) else f"variant {args.variant}"
+        kernel_name = KERNEL_FAMILY.get(step_variant, f"variant {step_variant}")
         in_step_layer_us = us_per_step * B / w.L                  # average duration of a layer launch inside the step
         achieved = bytes_layer / (in_step_layer_us * 1e-6) / 1e9
         io_bytes = B * w.T * w.H * 4
@@ -595,8 +753,8 @@ def run_gpu(args, w: wl.Workload):
                        "l2": "flushed before every timed step (512 MB fill, outside the timed interval)",
                        "multi_gpu": "replicas: each rank runs its own episodes, no collective on the data path"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name), "peak_kind": f"{peak_kind} copy bandwidth",
-                         "kernel": kernel_name + " (one launch per layer, dependent-launch chained)",
+                         "traffic": TRAFFIC_BYTES_PER_LAYER.get(w.name) if step_variant == 1 else None,
+                         "peak_kind": f"{peak_kind} copy bandwidth", "kernel": kernel_name, "kernel_family": step_variant,
                          "bytes_per_launch": bytes_layer, "us_per_launch": in_step_layer_us,
                          "us_per_launch_isolated_cold": layer_us, "launches_per_step": launches_per_step,
                          "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
@@ -609,10 +767,10 @@ def run_gpu(args, w: wl.Workload):
             "warm_l2_us_per_step": float(np.median(warm_us)) / B,
             "mask_compact_us": {"value": float(np.median(compact_us)), "lists": int(n_lists)},
             "gather_read_microbench": {
-                "us_per_layer": float(np.median(gather_us)) / w.L,
-                "gbs": int(round(K_mean)) * 3 * w.H * 2 / (float(np.median(gather_us)) / w.L * 1e-6) / 1e9,
-                "note": "episode 0's lists read with the kernels' access pattern (8 slices per neuron, 16-byte cp.async into "
-                        "two shared-memory stages) and discarded; one plain launch per layer, cold L2"},
+                "us_per_step": float(np.median(gather_us)),
+                "gbs": int(round(K_mean)) * 3 * w.H * 2 * w.L / (float(np.median(gather_us)) * 1e-6) / 1e9,
+                "note": "episode 0's lists of all layers read in ONE launch and discarded: one CTA per SM, whole 6H-byte rows by "
+                        "16-byte cp.async, 12 rows in flight per CTA, cold L2: the rate at which these lists can leave HBM"},
         }
         if dense_us is not None:
             line["dense_step_us"] = float(np.median(dense_us)) / B
@@ -620,6 +778,8 @@ def run_gpu(args, w: wl.Workload):
             line["roofline"]["union_weight_bytes_per_launch"] = int(union_rows * 3 * w.H * 2)
             line["roofline"]["note"] = ("bytes_per_launch is the sum over the episodes' lists; the union of the lists (rows that "
                                         "must leave HBM at least once) is given beside it")
+        if side is not None:
+            line["configs"] = side
         if cpu_us is not None:
             line["cpu_baseline"] = {"value": cpu_us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}
             us0, k0 = time_oracle_config0_single_thread()
@@ -646,9 +806,15 @@ def main():
     ap.add_argument("--variant", type=int, default=0,
                     help="kernel variant override (library option \"variant\": 0 = chosen per launch)")
     ap.add_argument("--max-clusters", type=int, default=0, help="library option \"max_clusters\" (0 = default)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="run the first N layers of the workload only (small cases for profiler captures; not a bench value)")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the side measurements of the other workloads (the \"configs\" object of the line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = pick_workload(args.workload)
+    if args.layers > 0:
+        w = wl.scaled(w, L=args.layers)
     if args.impl == "reference":
         run_reference(args, w)
     elif w.config == 6:

@@ -22,18 +22,25 @@ inline bool use_fused(const rm_ctx* ctx, int B, int T) {
     return ctx->path != 1 && rm_fused_supported(ctx, B, T);
 }
 
-// The whole-step kernel (variant 5).  Chosen by itself where it is measured ahead of the per-layer kernels: masked
-// steps of single episodes at H = 2048 (config 2: 395 against 509 us per step); it adapts to the counts on the device,
-// so it needs no hint.  At H = 1024 the lean per-layer kernel, which overlaps consecutive layers with two CTAs per SM,
-// is still ahead on masked steps (210 against 236 us at config 1), and the streaming kernel on dense passes (341 / 1151
-// against 360 / 1256 us at H = 1024 / 2048) and on batches.  `steps`: a whole stack (false: the one-layer entry, which
-// pays the kernel's set-up for a single layer).
+// The whole-step kernel (variant 5).  Chosen by itself where it is measured ahead of the per-layer kernels (single
+// episodes, masked steps; us per step, cold L2, per-layer kernels first):
+//   H = 2048, I = 16384:  K =  820: 321 / 320 (it is what runs)   3277: 509 / 393   9831: 1098 / 848   13108: 1148 / 1074
+//                         16384 (every neuron listed): 1170 / 1300 -> streaming kernel
+//   H = 1024, I = 4096:   K =  205: 169 / 226   1024: 198 / 241   1639: 248 / 246   2048: 269 / 258   3072: 347 / 277
+//                         4096: 355 / 365
+// It adapts to the counts on the device, so at H = 2048 it needs no hint; at H = 1024 the lean per-layer kernel (two
+// CTAs per SM, consecutive layers overlap) stays ahead on short lists, so the whole-step kernel is chosen only when
+// the caller's count hint says that the lists hold 35 % to 90 % of the neurons.  Dense passes (no list) and batches
+// stay with the streaming kernel.  `steps`: a whole stack (false: the one-layer entry, which would pay the kernel's
+// set-up for a single layer).
 inline bool use_persist(const rm_ctx* ctx, int B, int T, bool masked, bool steps) {
     if (ctx->path == 1 || !rm_persist_supported(ctx, B, T)) return false;
     if (ctx->variant_override == 5) return true;
     if (ctx->variant_override != 0 || B > ctx->persist_max_b || !steps || !masked) return false;
-    if (ctx->count_hint > 0 && (long long)ctx->count_hint * 10 > (long long)ctx->g.I * 6) return false;   // nearly dense lists
-    return ctx->g.H == 2048;
+    const long long hint = ctx->count_hint, I = ctx->g.I;
+    if (hint > 0 && hint * 10 > I * 9) return false;              // nearly every neuron listed
+    if (ctx->g.H == 2048) return true;
+    return hint > 0 && hint * 100 >= I * 35;
 }
 
 inline void* persist_ws(const rm_ctx* ctx, void* ws, int B, int T) {

@@ -28,27 +28,46 @@ struct GatherArgs {
     int* status;
 };
 
+constexpr int MAX_ROWS_PER_CTA = 512;  // list positions one CTA takes per layer (I / CTAs, rounded up)
+
 __global__ void __launch_bounds__(GT) gather_read_kernel(const __grid_constant__ GatherArgs a) {
     extern __shared__ unsigned char smem[];
+    __shared__ int ids[2][MAX_ROWS_PER_CTA];
+    __shared__ int cnts[2];
     const uint32_t base = (smem_u32(smem) + 127u) & ~127u;
     const int row_bytes = 6 * a.H, pieces = row_bytes / 16;
-    int k = 0;
-    for (int l = 0; l < a.L; ++l) {
+    // the neuron ids of this CTA's list positions, one layer ahead of the reads (an id fetched right before its row
+    // would put an L2 round trip in front of every row)
+    auto fetch_ids = [&](int l) {
         int c = a.idx ? a.count[l] : a.I;
         if (c < 0 || c > a.cap || c > a.I) {
             if (blockIdx.x == 0 && threadIdx.x == 0) rm_set_status(a.status, RM_ERR_INDEX);
             c = c < 0 ? 0 : (int)(a.cap < (int64_t)a.I ? a.cap : (int64_t)a.I);
         }
         const int32_t* list = a.idx ? a.idx + (size_t)l * a.stride : nullptr;
-        for (int p = blockIdx.x; p < c; p += gridDim.x, ++k) {
+        const int mine = c > (int)blockIdx.x ? (c - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+        for (int k = threadIdx.x; k < mine && k < MAX_ROWS_PER_CTA; k += GT) {
+            const int p = blockIdx.x + k * gridDim.x;
             int n = list ? list[p] : p;
-            if (n < 0 || n >= a.I) n = -1;
+            ids[l & 1][k] = (n < 0 || n >= a.I) ? -1 : n;
+        }
+        if (threadIdx.x == 0) cnts[l & 1] = mine < MAX_ROWS_PER_CTA ? mine : MAX_ROWS_PER_CTA;
+    };
+    fetch_ids(0);
+    __syncthreads();
+    int k = 0;
+    for (int l = 0; l < a.L; ++l) {
+        if (l + 1 < a.L) fetch_ids(l + 1);
+        const int mine = cnts[l & 1];
+        for (int r = 0; r < mine; ++r, ++k) {
+            const int n = ids[l & 1][r];
             const uint32_t st = base + (k % DEPTH) * row_bytes;
             if (k >= DEPTH) cp_async_wait<DEPTH - 1>();        // the stage's previous row has landed
             const __nv_bfloat16* src = a.packed[l] + (size_t)(n < 0 ? 0 : n) * 3 * a.H;
             for (int e = threadIdx.x; e < pieces; e += GT) cp_async16(st + e * 16, src + e * 8, n >= 0);
             cp_async_commit();
         }
+        __syncthreads();
     }
     cp_async_wait<0>();
 }
