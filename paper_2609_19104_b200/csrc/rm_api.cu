@@ -114,6 +114,9 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->persist_max_b = 1;
     c->persist_prefetch_kb = 0;
     c->persist_xbuf = nullptr;
+    c->persist_sync = nullptr;
+    c->persist_sync_dirty = 0;
+    for (int b = 0; b < 16; ++b) c->persist_sync_base[b] = c->persist_copy_base[b] = 0;
     if (prop.major == 10) { rm_fused_init(c); rm_persist_init(c); }   // failure leaves the portable path in charge
     cudaGetLastError();
     *out = c;
@@ -319,12 +322,12 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
     const size_t r_bytes = align_up(n_bytes, 256);
     char* layer_ws = static_cast<char*>(ws) + 4 * r_bytes;
     if (use_persist(ctx, B, T, count_dev != nullptr, true) && an.mode == RM_ANCHOR_NONE && !an.gate) {
-        // the whole step in one launch: the layers add into r_out in place
-        if (r_out != r_in) RM_CUDA_TRY(cudaMemcpyAsync(r_out, r_in, n_bytes, cudaMemcpyDeviceToDevice, s));
+        // the whole step in one launch: the layers add into r_out in place (the kernel starts it as a copy of r_in)
         rm_step_args sa{};
         sa.packed_layers = packed_layers;
         sa.L = g.L;
         sa.r = r_out;
+        sa.r_in = r_out != r_in ? r_in : nullptr;
         sa.idx = idx;
         sa.count = count_dev;
         sa.idx_b_stride = (int64_t)g.L * stride;
@@ -492,6 +495,7 @@ int rm_device_status(rm_ctx* ctx, int* host_out, rm_stream_t stream) {
     RM_CUDA_TRY(cudaMemsetAsync(ctx->d_status, 0, sizeof(v), s));
     RM_CUDA_TRY(cudaStreamSynchronize(s));
     *host_out = v[0];
+    if (v[0] != 0) ctx->persist_sync_dirty = 1;                 // a whole-step launch may have stopped half way
     ctx->status_detail = v[0] ? v[1] : 0;
     std::memcpy(ctx->status_log, v, sizeof(v));
     return RM_OK;

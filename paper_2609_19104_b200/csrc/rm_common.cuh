@@ -49,6 +49,10 @@ struct rm_ctx {
     int persist_prefetch_kb;               // weight KB a CTA of the whole-step kernel may ask into L2 ahead of its loaders
     int persist_max_b;                     // largest batch the whole-step kernel is chosen for when the variant is automatic
     const void* persist_xbuf;              // buffer the cached tensor map below describes
+    const int* persist_sync;               // the workspace's arrival counters this context has been counting on
+    int persist_sync_base[16];             // their values after the launches so far
+    int persist_copy_base[16];             // the same for the counters of the r_in -> r copies
+    int persist_sync_dirty;                // a launch may have left them at an unknown count: clear before the next one
     alignas(64) unsigned char persist_tm[128];   // CUtensorMap of the clusters' x copies in the workspace
 };
 
@@ -146,7 +150,8 @@ int rm_launch_layer_stream(rm_ctx* ctx, const rm_layer_args& a, __nv_bfloat16* x
 struct rm_step_args {
     const void* const* packed_layers;      // host array of L device pointers
     int L;
-    float* r;                              // [B,T,H] fp32: r_0 on entry, r_L on exit
+    float* r;                              // [B,T,H] fp32: r_L on exit (r_0 on entry when r_in is NULL)
+    const float* r_in;                     // [B,T,H] fp32 r_0 in another buffer (the kernel starts r as its copy), or NULL
     const int32_t* idx;                    // list (b, l) at idx + b * idx_b_stride + l * idx_l_stride; NULL: positions
     const int32_t* count;                  // count (b, l) at count[b * count_b_stride + l]; NULL: every neuron
     int64_t idx_b_stride, idx_l_stride, list_cap, count_b_stride;

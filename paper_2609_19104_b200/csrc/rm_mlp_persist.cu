@@ -46,16 +46,20 @@ constexpr int XSB = 2 * X_BYTES;       // x ring stage: the blocks of columns c 
 constexpr int XS_MAX = 8;
 constexpr int SB = 16384;              // weight ring stage: 128 rows x 128 bytes
 constexpr int EXCH = 16384;            // second-half partial sums of a tile on their way to the threads that finish them
-constexpr int MAXL = 64, MAXB = 16;
+constexpr int MAXL = 64, MAXB = 16, MAX_ITEMS = 512;   // layers, episodes, layers x episodes of one launch
 constexpr int NXW = 4;                 // warps that issue the x copies (copies of one issuing thread do not overlap much)
 constexpr int NTHREADS = 608;          // warps: 0-7 epilogue and normalisation, 8-11 loaders, 12 issuer, 13-16 x copies, 17 L2 prefetch,
                                        // 18 stage watcher
 constexpr int W_LOAD0 = 8, W_MMA = 12, W_X0 = 13, W_PF = 17, W_WATCH = 18;
 constexpr int SYNC_ABORT = MAXB;       // sync[0..MAXB): per-episode arrival counters; sync[MAXB]: abort flag
+constexpr int SYNC_COPY = 32;          // sync[32..32+MAXB): per-episode counters of the CTAs that have copied r_in into r
+constexpr int SYNC_ITEM = 64;          // sync[64..64+MAX_ITEMS): batches count the arrivals of every (layer, episode) by itself
+constexpr int SYNC_BYTES = (SYNC_ITEM + 512) * 4;
 
 struct PArgs {
     const __nv_bfloat16* packed[MAXL];
-    float* r;                          // [B,T,H] fp32: holds r_0 on entry and r_L on exit (layers add in place)
+    float* r;                          // [B,T,H] fp32: r_L on exit; the layers add into it in place
+    const float* r_in;                 // [B,T,H] fp32: r_0.  When it is another buffer than r, the kernel starts r as a copy of it
     __nv_bfloat16* xbuf;               // [clusters][2][H/64][64 rows x 128 bytes]: the clusters' own copies of x, stored as
                                        // the shared-memory image of each 64-column block (128-byte swizzle)
     const int32_t* idx;                // list (b, l) at idx + b * idx_b_stride + l * idx_l_stride; NULL: positions
@@ -64,9 +68,14 @@ struct PArgs {
     float* record;                     // record (b, l, n) at record[b * rec_b_stride + l * I + n]; NULL: none
     int64_t rec_b_stride;
     const float* record_scale;         // [L, I] or NULL
-    int* sync;
+    int* sync;                         // [0..MAXB): per-episode arrival counters, never reset between launches; [MAXB]: abort flag
+    int sync_base[MAXB];               // value of each counter when this launch starts (the host keeps count)
+    int copy_base[MAXB];               // the same for the copy counters
     int* status;
     int L, B, T, I;
+    int per_item;                      // arrivals are counted per (layer, episode) on counters cleared before the launch (batches:
+                                       // a cluster that takes no part in an episode runs ahead of those that do, so one
+                                       // counter per episode could not tell the layers apart); else per episode, never cleared
     int x_ext;                         // layer 0 takes x from the caller's buffer (single-layer entry): no normalisation
     int pf_bytes;                      // weight bytes a CTA may have asked into L2 ahead of its loaders (0: no prefetch)
 };
@@ -135,15 +144,22 @@ __device__ __forceinline__ bool named_barrier_or(int id, int count, bool pred) {
 
 // ---- the split of an item over clusters, tiles and CTAs (every role computes it the same way)
 struct Run { int start, n, ntiles; };
-__device__ __forceinline__ Run cluster_run(int K, int c, int NC) {
+// The lists of a layer's episodes, laid end to end, are cut evenly over the clusters: cluster c takes positions
+// [S c / NC, S (c + 1) / NC) of the S = sum of the counts.  Its run in episode b's list (which starts at position P
+// of the concatenation and holds K neurons) is the overlap.  One episode: its list is cut evenly over all clusters.
+// Several episodes: every cluster gets the same number of neurons per layer, from one or two episodes.
+__device__ __forceinline__ Run cluster_run(int K, int P, int S, int c, int NC) {
     Run r;
-    r.start = (int)((long long)K * c / NC);
-    r.n = (int)((long long)K * (c + 1) / NC) - r.start;
+    const int lo = (int)((long long)S * c / NC), hi = (int)((long long)S * (c + 1) / NC);
+    const int a = lo > P ? lo : P, b = hi < P + K ? hi : P + K;
+    r.start = a - P;
+    r.n = b > a ? b - a : 0;
     r.ntiles = (r.n + CT - 1) / CT;
     return r;
 }
 __device__ __forceinline__ void tile_span(const Run& r, int i, int& t0, int& ts) {
-    const int a = (int)((long long)r.n * i / r.ntiles), b = (int)((long long)r.n * (i + 1) / r.ntiles);
+    if (r.ntiles == 1) { t0 = r.start; ts = r.n; return; }
+    const int a = r.n * i / r.ntiles, b = r.n * (i + 1) / r.ntiles;               // (n <= I < 2^24, i < 2^7: no overflow)
     t0 = r.start + a;
     ts = b - a;                                                    // <= 256
 }
@@ -161,14 +177,22 @@ struct Cur {
     int use;                           // uses of the cluster's x buffer before this item
     bool valid;
 };
-struct Env { const int* sK; int L, B, c, NC, x_ext; };
+struct Env { const int* sRunStart; const int* sRunN; int L, B, c, NC, x_ext; };   // this cluster's run in every item's list,
+                                                                                  // worked out once at the start of the kernel
+__device__ __forceinline__ Run item_run(const Env& e, int item) {
+    Run r;
+    r.start = e.sRunStart[item];
+    r.n = e.sRunN[item];
+    r.ntiles = (r.n + CT - 1) / CT;
+    return r;
+}
 __device__ __forceinline__ bool item_ext(const Env& e, int l) { return e.x_ext && l == 0; }
 __device__ __forceinline__ void cur_seek(Cur& k, const Env& e) {      // to the first non-empty item at or after k.item
     const int n_items = e.L * e.B;
     while (k.item < n_items) {
         k.l = k.item / e.B;
         k.b = k.item - k.l * e.B;
-        k.run = cluster_run(e.sK[k.item], e.c, e.NC);
+        k.run = item_run(e, k.item);
         if (k.run.ntiles > 0) { k.valid = true; k.i = 0; return; }
         ++k.item;
     }
@@ -179,10 +203,13 @@ __device__ __forceinline__ void cur_init(Cur& k, const Env& e) {
     cur_seek(k, e);
 }
 // The gate/up products of tile g may be issued before the down products of tile d (the tile in front of it) when g
-// does not need d's result: the same item, or another episode.  (The next layer of the same episode does: its input is
-// normalised from the residual stream that d's item adds into.  With empty lists in between, the next non-empty item
-// can be that even when several episodes are in the batch.)
-__device__ __forceinline__ bool may_run_ahead(const Cur& g, const Cur& d) { return g.item == d.item || g.b != d.b; }
+// does not need d's result: the same item, or an item fewer than B places further on in the (layer, episode) order --
+// that is another episode, and the layer of that episode that it depends on lies before d's item.  (An item B or more
+// places on can be the next layer of d's own episode, or depend on an item this cluster has not finished yet: with empty
+// lists, or clusters that take no part in some episodes, the next non-empty item can be that far away.)  The epilogue
+// warps prepare the input x of the next item one item ahead under exactly the same rule.
+__device__ __forceinline__ bool item_may_run_ahead(int g_item, int d_item, int B) { return g_item == d_item || g_item < d_item + B; }
+__device__ __forceinline__ bool may_run_ahead(const Cur& g, const Cur& d, int B) { return item_may_run_ahead(g.item, d.item, B); }
 __device__ __forceinline__ void cur_next(Cur& k, const Env& e) {
     ++k.seq;
     if (++k.i < k.run.ntiles) return;
@@ -208,7 +235,8 @@ struct Geo {
     static constexpr int ND2 = NMB == 1 ? 2 : 1;       // down accumulators (an item's flush overlaps the next item's products)
     static constexpr int D2_COL = 4 * NTOK;            // tensor memory: D1[2] at 0 and 128 (128 columns each), D2 from 256
     static constexpr int OFF_K = 0;                    // counts of the items
-    static constexpr int OFF_IDX = OFF_K + MAXL * MAXB * 4;     // neuron ids of three tiles in turn
+    static constexpr int OFF_P = OFF_K + MAX_ITEMS * 4;         // (OFF_K: the items' counts, then this cluster's run lengths; OFF_P: run starts)
+    static constexpr int OFF_IDX = OFF_P + MAX_ITEMS * 4;       // neuron ids of three tiles in turn
     static constexpr int OFF_REC = OFF_IDX + 3 * CT * 4;
     static constexpr int OFF_MISC = OFF_REC + 4 * NT * 4;
     static constexpr int OFF_BAR = OFF_MISC + 128;
@@ -231,6 +259,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     unsigned char* gbase = smem_dyn + (base - smem_u32(smem_dyn));
     const uint32_t sW = base + G::OFF_W, sH = base + G::OFF_HX;
     int* sK = reinterpret_cast<int*>(gbase + G::OFF_K);
+    int* sP = reinterpret_cast<int*>(gbase + G::OFF_P);
     int* sIdx = reinterpret_cast<int*>(gbase + G::OFF_IDX);
     float* sRec = reinterpret_cast<float*>(gbase + G::OFF_REC);
     volatile int* sMisc = reinterpret_cast<volatile int*>(gbase + G::OFF_MISC);
@@ -284,9 +313,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         *sLoaded = 0;
         *sReady = 0;
         int ts_max = 16;
-        for (int it = 0; it < n_items; ++it) {
-            const Run r = cluster_run(sK[it], c, NC);
-            if (r.ntiles > 0) { const int ts = (r.n + r.ntiles - 1) / r.ntiles; ts_max = ts > ts_max ? ts : ts_max; }
+        for (int l = 0; l < L; ++l) {
+            int S = 0;
+            for (int b = 0; b < B; ++b) S += sK[l * B + b];
+            int P = 0;
+            for (int b = 0; b < B; ++b) {
+                const int K = sK[l * B + b];
+                const Run r = cluster_run(K, P, S, c, NC);
+                sP[l * B + b] = r.start;                             // (sP then holds the run starts, sK the run lengths)
+                sK[l * B + b] = r.n;
+                P += K;
+                if (r.ntiles > 0) { const int ts = (r.n + r.ntiles - 1) / r.ntiles; ts_max = ts > ts_max ? ts : ts_max; }
+            }
         }
         *sHslots = (ts_max + 15) & ~15;
     }
@@ -309,11 +347,27 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     cluster_sync();
     tc_fence_after();
     const uint32_t tmem = *g_tmem;
+    // r starts as a copy of r_in: cluster 0's CTA j copies column slice j of every episode and counts itself on the
+    // episode's copy counter; nobody adds into r before the 8 copies are counted
+    const int pre = a.r_in != a.r ? CS : 0;
+    if (pre && c == 0 && warp < 8) {
+        for (int b = 0; b < B; ++b) {
+            const float4* src = reinterpret_cast<const float4*>(a.r_in + (size_t)b * T * H + j * HS8);
+            float4* dst = reinterpret_cast<float4*>(a.r + (size_t)b * T * H + j * HS8);
+            for (int e = tid; e < T * (HS8 / 4); e += 256) {
+                const int t = e / (HS8 / 4), q = e - t * (HS8 / 4);
+                dst[(size_t)t * (H / 4) + q] = src[(size_t)t * (H / 4) + q];
+            }
+            __threadfence();
+            named_barrier(1, 256);
+            if (tid == 0) red_release_gpu(a.sync + SYNC_COPY + b, 1);
+        }
+    }
     const int h_half = *sHslots * 128;                             // bytes of the hi block (= of the lo block) of the h tile
     const uint32_t sX = sH + 2 * h_half;
     int xs_n = (G::END - G::OFF_HX - 2 * h_half) / XSB;
     const int XS = xs_n > XS_MAX ? XS_MAX : xs_n;                    // >= 2
-    Env env{sK, L, B, c, NC, a.x_ext};
+    Env env{sP, sK, L, B, c, NC, a.x_ext};
 
     bool gave_up = false;
     auto timed_out = [&](int line) {
@@ -435,7 +489,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         d = g;
         if (g.valid) { load_g(g); cur_next(g, env); }
         while (d.valid && !stop) {
-            const bool ahead = g.valid && may_run_ahead(g, d);
+            const bool ahead = g.valid && may_run_ahead(g, d, B);
             if (ahead) { load_g(g); cur_next(g, env); }
             load_d(d);
             cur_next(d, env);
@@ -560,7 +614,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             d = g;
             if (g.valid) { watch_g(g); cur_next(g, env); }
             while (d.valid && !gave_up) {
-                const bool ahead = g.valid && may_run_ahead(g, d);
+                const bool ahead = g.valid && may_run_ahead(g, d, B);
                 if (ahead) { watch_g(g); cur_next(g, env); }
                 watch_d(d);
                 cur_next(d, env);
@@ -655,7 +709,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             d = g;
             if (g.valid) { issue_g(g); cur_next(g, env); }
             while (d.valid && !gave_up) {
-                const bool ahead = g.valid && may_run_ahead(g, d);
+                const bool ahead = g.valid && may_run_ahead(g, d, B);
                 if (ahead) { issue_g(g); cur_next(g, env); }
                 issue_d(d);
                 cur_next(d, env);
@@ -680,7 +734,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         // one row per warp.  With one episode it runs right before the item's tiles (it has to wait for the previous
         // layer's adds anyway); with several episodes it runs one item ahead, so that the next item's gate/up
         // products can start while this item's tiles are finished.
-        int next_norm = 0, use = 0;
+        int use = 0;
         auto norm_item = [&](int item) {
             const int l = item / B, b = item - l * B;
             const int slot = use & 1, nu = use >> 1;
@@ -688,11 +742,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             const bool xf_ok = nu >= 1 ? mbar_test_wait(x_free(slot), (nu - 1) & 1) : true;     // looked at before the stores
             if (l > 0) {
                 // every CTA has added its part of layer l-1 to this episode's rows
-                const int target = n_ctas * l;
+                const int target = a.per_item ? n_ctas : a.sync_base[b] + n_ctas * l;
+                const int* counter = a.per_item ? a.sync + SYNC_ITEM + (l - 1) * B + b : a.sync + b;
                 if (lane == 0 && !gave_up) {
                     bool ok = false;
                     for (uint32_t i = 0; i < (1u << 21); ++i) {
-                        if (ld_acquire_gpu(a.sync + b) >= target) { ok = true; break; }
+                        if (ld_acquire_gpu(counter) >= target) { ok = true; break; }
                         if ((i & 255u) == 255u && (*sAbort || ld_acquire_gpu(a.sync + SYNC_ABORT))) break;
                     }
                     if (!ok) { if (!*sAbort && !ld_acquire_gpu(a.sync + SYNC_ABORT)) timed_out(__LINE__); gave_up = true; *sAbort = 1; }
@@ -704,7 +759,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             long long n1 = n0, n2 = n0, n3 = n0;
             const int row = j + 8 * warp;
             if (row < T) {
-                const float4* src = reinterpret_cast<const float4*>(a.r + ((size_t)b * T + row) * H);
+                const float4* src = reinterpret_cast<const float4*>((l == 0 ? a.r_in : a.r) + ((size_t)b * T + row) * H);
                 float4 v[H / 128];
                 float ss = 0.f;
 #pragma unroll
@@ -742,17 +797,25 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             if (warp == 0 && lane < CS) mbar_arrive_remote(map_to_rank(x_ready(slot), lane));
             if (et == 0) { RM_PS(item, 9); RM_PC(item, 26, n1 - n0); RM_PC(item, 27, n2 - n1); RM_PC(item, 28, n3 - n2); RM_PC(item, 29, n4 - n3); RM_PC(item, 30, RM_CLK() - n4); }
         };
-        auto prepare_up_to = [&](int last) {
-            for (; next_norm <= last && next_norm < n_items && !stop; ++next_norm) {
-                const Run r = cluster_run(sK[next_norm], c, NC);
-                if (r.ntiles > 0 && !item_ext(env, next_norm / B)) norm_item(next_norm);
+        // x of a non-empty item is prepared right before the item's own tiles, or one non-empty item earlier when the
+        // issuer may run that item's gate/up products ahead (item_may_run_ahead)
+        int normed = -1;                                            // last item whose x has been prepared
+        auto prepare = [&](int q) {
+            if (q > normed) {
+                normed = q;
+                if (!item_ext(env, q / B)) norm_item(q);
             }
         };
         for (int item = 0; item < n_items && !stop; ++item) {
-            prepare_up_to(item + (B >= 2 ? 1 : 0));
+            if (item_run(env, item).ntiles > 0) {
+                prepare(item);
+                int q = item + 1;
+                while (q < n_items && q < item + B && item_run(env, q).ntiles == 0) ++q;
+                if (q < n_items && q < item + B && !stop) prepare(q);
+            }
             if (stop) break;
             const int l = item / B, b = item - l * B;
-            const Run run = cluster_run(sK[item], c, NC);
+            const Run run = item_run(env, item);
             const int32_t* list = a.idx ? a.idx + (size_t)b * a.idx_b_stride + (size_t)l * a.idx_l_stride : nullptr;
             for (int i = 0; i < run.ntiles && !stop; ++i, ++seq) {
                 int t0, ts, off, nj;
@@ -876,6 +939,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 WAIT(d2_full(d2b), nu & 1);
                 tc_fence_after();
                 if (et == 0) RM_PS(item, 5);
+                if (l == 0 && pre) {
+                    // r has to hold its copy of r_in before anything is added to it
+                    if (lane == 0 && !gave_up) {
+                        bool ok = false;
+                        for (uint32_t w8 = 0; w8 < (1u << 21); ++w8) {
+                            if (ld_acquire_gpu(a.sync + SYNC_COPY + b) >= a.copy_base[b] + pre) { ok = true; break; }
+                            if ((w8 & 255u) == 255u && (*sAbort || ld_acquire_gpu(a.sync + SYNC_ABORT))) break;
+                        }
+                        if (!ok) { if (!*sAbort && !ld_acquire_gpu(a.sync + SYNC_ABORT)) timed_out(__LINE__); gave_up = true; *sAbort = 1; }
+                    }
+                    __syncwarp();
+                }
                 float* rb = a.r + (size_t)b * T * H + j * HS8 + q4 * 32 + lane;
 #pragma unroll
                 for (int mb = 0; mb < NMB; ++mb) {
@@ -895,12 +970,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 __threadfence();
                 stop = named_barrier_or(1, 256, gave_up || *sAbort);
             }
-            if (et == 0) { red_release_gpu(a.sync + b, 1); RM_PS(item, 7); }
+            if (et == 0) { red_release_gpu(a.per_item ? a.sync + SYNC_ITEM + item : a.sync + b, 1); RM_PS(item, 7); }
         }
     }
 #undef WAIT
     tc_fence_before();
     __syncthreads();
+    if (*sAbort) {
+        // a wait gave up somewhere: copies into this CTA's shared memory (x blocks, peers' h rows) may still be in flight
+        // although nobody waits for them any more.  They land within microseconds; idle for longer than that.
+        for (int i = 0; i < 64; ++i) __nanosleep(4000);
+        __syncthreads();
+    }
     cluster_sync();                    // no CTA leaves while a peer may still write into its shared memory
     if (warp == W_MMA) tmem_dealloc(tmem, 512);
 }
@@ -998,13 +1079,13 @@ int rm_persist_init(rm_ctx* ctx) {
 
 bool rm_persist_supported(const rm_ctx* ctx, int B, int T) {
     const int H = ctx->g.H;
-    return (H == 1024 || H == 2048) && T >= 1 && T <= NTOK && B >= 1 && B <= MAXB && ctx->g.L <= MAXL &&
+    return (H == 1024 || H == 2048) && T >= 1 && T <= NTOK && B >= 1 && B <= MAXB && ctx->g.L <= MAXL && ctx->g.L * B <= MAX_ITEMS &&
            ctx->persist_clusters > 0 && encode_fn() != nullptr;
 }
 
 size_t rm_persist_workspace_bytes(const rm_ctx* ctx) {
     if (ctx->persist_clusters <= 0) return 0;
-    return 256 + (size_t)ctx->persist_clusters * 2 * NTOK * ctx->g.H * sizeof(__nv_bfloat16);
+    return SYNC_BYTES + (size_t)ctx->persist_clusters * 2 * NTOK * ctx->g.H * sizeof(__nv_bfloat16);
 }
 
 int rm_persist_debug_stamps(long long* host_out, int n) {
@@ -1022,8 +1103,10 @@ int rm_launch_step_persist(rm_ctx* ctx, const rm_step_args& sa, void* ws, cudaSt
     PArgs a{};
     for (int l = 0; l < sa.L; ++l) a.packed[l] = static_cast<const __nv_bfloat16*>(sa.packed_layers[l]);
     a.r = sa.r;
+    a.r_in = sa.r_in ? sa.r_in : sa.r;
     a.sync = reinterpret_cast<int*>(ws);
-    a.xbuf = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + 256);
+    a.xbuf = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + SYNC_BYTES);
+    a.per_item = sa.B > 1 ? 1 : 0;
     a.idx = sa.idx;
     a.count = sa.count;
     a.idx_b_stride = sa.idx_b_stride;
@@ -1056,6 +1139,22 @@ int rm_launch_step_persist(rm_ctx* ctx, const rm_step_args& sa, void* ws, cudaSt
     } else {
         tm_ext = *reinterpret_cast<const CUtensorMap*>(ctx->persist_tm);
     }
-    RM_CUDA_TRY(cudaMemsetAsync(a.sync, 0, 256, s));
-    return g.H == 1024 ? launch<128>(ctx, a, tm_ext, nc, s) : launch<256>(ctx, a, tm_ext, nc, s);
+    int nc_ctas = nc * CS;
+    const int pre = a.r_in != a.r ? CS : 0;
+    // The arrival counters live in the workspace and only ever count up; the host keeps their values.  They are cleared
+    // when the workspace is new to this context, after a launch whose status was not clean (its count is unknown), and
+    // long before they could wrap.
+    bool reset = ctx->persist_sync != a.sync || ctx->persist_sync_dirty || a.per_item;
+    for (int b = 0; b < MAXB; ++b) reset = reset || ctx->persist_sync_base[b] > (1 << 30);
+    if (reset) {
+        RM_CUDA_TRY(cudaMemsetAsync(a.sync, 0, a.per_item ? SYNC_BYTES : 256, s));
+        for (int b = 0; b < MAXB; ++b) ctx->persist_sync_base[b] = ctx->persist_copy_base[b] = 0;
+        ctx->persist_sync = a.sync;
+        ctx->persist_sync_dirty = 0;
+    }
+    for (int b = 0; b < MAXB; ++b) { a.sync_base[b] = ctx->persist_sync_base[b]; a.copy_base[b] = ctx->persist_copy_base[b]; }
+    for (int b = 0; b < sa.B; ++b) { ctx->persist_sync_base[b] += nc_ctas * sa.L; ctx->persist_copy_base[b] += pre; }
+    const int rc = g.H == 1024 ? launch<128>(ctx, a, tm_ext, nc, s) : launch<256>(ctx, a, tm_ext, nc, s);
+    if (rc != RM_OK) ctx->persist_sync_dirty = 1;               // nothing ran: the counters are behind the host's count
+    return rc;
 }
