@@ -967,7 +967,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 tc_fence_before();
                 mbar_arrive(d2_empty(d2b));
                 if (et == 0) RM_PS(item, 6);
-                __threadfence();
+                // no fence per thread: the barrier orders every thread's adds before thread 0's release on the counter
+                // below, and a release is cumulative (the pattern of a grid-wide barrier: sync, then one thread fences)
                 stop = named_barrier_or(1, 256, gave_up || *sAbort);
             }
             if (et == 0) { red_release_gpu(a.per_item ? a.sync + SYNC_ITEM + item : a.sync + b, 1); RM_PS(item, 7); }
