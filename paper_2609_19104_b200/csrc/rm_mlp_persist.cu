@@ -224,8 +224,9 @@ __device__ __forceinline__ void cur_next(Cur& k, const Env& e) {
 template <int HS8>
 struct Geo {
     static constexpr int H = 8 * HS8;
-    // weight ring stages: the wide model streams twice as much x per tile, so its x ring gets some of the space
-    static constexpr int NW = HS8 == 256 ? 5 : 6;
+    // weight ring stages (measured at H = 2048, top-20 % / full list: 4 stages 420 / 1344 us per step, 5: 401 / 1288,
+    // 6: 398 / 1264); the x ring takes what the h tile leaves
+    static constexpr int NW = 6;
     static constexpr int W_RING = NW * SB;
     static constexpr int NSB = HS8 / 64;               // 64-column boxes per column slice
     static constexpr int NMB = HS8 / 128;              // 128-column output blocks per slice
