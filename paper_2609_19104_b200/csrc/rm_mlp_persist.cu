@@ -269,6 +269,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     volatile int* sHslots = sMisc + 2;                             // [2] slots of the h tile (largest tile, rounded to 16)
     volatile int* sLoaded = sMisc + 3;                             // [3] neurons whose gate/up rows the loaders have started on
     int* sReady = const_cast<int*>(sMisc) + 4;                     // [4] ring stages (in consumption order) whose data has landed
+    volatile int* sAlias = sMisc + 5;                              // [5] the x ring lies over the h tile (see below)
     const uint32_t s_tmem = base + G::OFF_MISC;
     const uint32_t bar0 = base + G::OFF_BAR;
     auto w_full = [&](int s) { return bar0 + 8 * s; };              // NW <= 6
@@ -280,7 +281,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     auto d2_empty = [&](int s) { return bar0 + 480 + 8 * s; };
     auto x_ready = [&](int s) { return bar0 + 496 + 8 * s; };       // 2
     auto x_free = [&](int s) { return bar0 + 512 + 8 * s; };
-    const uint32_t h_full = bar0 + 528, h_free = bar0 + 536;
+    const uint32_t h_full = bar0 + 528, h_free = bar0 + 536, g_all = bar0 + 544;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int j = (int)cluster_ctarank(), c = (int)cluster_id_x(), NC = (int)cluster_count_x();
@@ -308,12 +309,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             mbar_init(d1_full(s), 1); mbar_init(d2_full(s), 1); mbar_init(d2_empty(s), 256);
             mbar_init(x_ready(s), CS); mbar_init(x_free(s), CS);
         }
-        mbar_init(h_full, 1); mbar_init(h_free, CS);
+        mbar_init(h_full, 1); mbar_init(h_free, CS); mbar_init(g_all, CS);
         fence_mbar_init();
         *sAbort = 0;
         *sLoaded = 0;
         *sReady = 0;
-        int ts_max = 16;
+        int ts_max = 16, tiles_max = 0;
         for (int l = 0; l < L; ++l) {
             int S = 0;
             for (int b = 0; b < B; ++b) S += sK[l * B + b];
@@ -325,12 +326,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 sK[l * B + b] = r.n;
                 P += K;
                 if (r.ntiles > 0) { const int ts = (r.n + r.ntiles - 1) / r.ntiles; ts_max = ts > ts_max ? ts : ts_max; }
+                tiles_max = r.ntiles > tiles_max ? r.ntiles : tiles_max;
             }
         }
         *sHslots = (ts_max + 15) & ~15;
+        // One episode and at most one tile per layer in this cluster: a layer's h is written after its gate/up products
+        // and dead before the next layer's x exists, so the x ring may lie over the h tile and be twice as deep.
+        *sAlias = B == 1 && tiles_max <= 1;
     }
     if (warp == W_MMA) tmem_alloc(s_tmem, 512);
-    // the x copies bring token rows 0..T-1 only: the other rows of every ring stage stay zero from here on
+    // the x copies bring token rows 0..T-1 only: the other rows of every ring stage stay zero from here on (when the ring
+    // lies over the h tile they hold old h values instead: the sums of the token columns T..63 are never used, the
+    // epilogue writes zeros for them)
     for (int e = tid; e < (G::END - G::OFF_HX) / 16; e += NTHREADS)
         reinterpret_cast<uint4*>(gbase + G::OFF_HX)[e] = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
@@ -365,8 +372,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         }
     }
     const int h_half = *sHslots * 128;                             // bytes of the hi block (= of the lo block) of the h tile
-    const uint32_t sX = sH + 2 * h_half;
-    int xs_n = (G::END - G::OFF_HX - 2 * h_half) / XSB;
+    const bool alias = *sAlias != 0;
+    const uint32_t sX = alias ? sH : sH + 2 * h_half;
+    int xs_n = (G::END - G::OFF_HX - (alias ? 0 : 2 * h_half)) / XSB;
     const int XS = xs_n > XS_MAX ? XS_MAX : xs_n;                    // >= 2
     Env env{sP, sK, L, B, c, NC, a.x_ext};
 
@@ -670,6 +678,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     ++stage;
                 }
                 mma_commit(d1_full(buf));
+                if (alias) mma_commit_mc(g_all, 0xff);                // this CTA's x ring (which lies over its h tile) is read out
                 if (k.i == 0) { RM_PS(k.item, 24); RM_PC(k.item, 10, c_n); RM_PC(k.item, 11, c_m); RM_PC(k.item, 12, c_c); }
                 if (k.i == k.run.ntiles - 1 && !item_ext(env, k.l)) mma_commit_mc(x_free(k.use & 1), 0xff);
             };
@@ -857,6 +866,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 // lane pair (2 i, 2 i + 1) = (gate row, up row) of neuron i for these 16 tokens: the even lane finishes
                 // the first 8 of them, the odd lane the last 8
                 float hv[8];
+                const int tok0 = 8 * (ch * 4 + (fin ? 0 : 2) + (isup ? 1 : 0));     // first of this lane's 8 tokens
                 {
                     float gg[8], uu[8], e[8];
 #pragma unroll
@@ -871,7 +881,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
 #pragma unroll
                     for (int r = 0; r < 8; ++r) e[r] = __fdividef(gg[r], 1.0f + e[r]);
 #pragma unroll
-                    for (int r = 0; r < 8; ++r) hv[r] = n >= 0 ? e[r] * uu[r] : 0.f;
+                    for (int r = 0; r < 8; ++r) hv[r] = n >= 0 && tok0 + r < T ? e[r] * uu[r] : 0.f;
                 }
                 if (a.record) {
                     float rec = 0.f;
@@ -920,6 +930,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 const long long e7 = RM_CLK();
                 if (et == 0) mbar_arrive_expect_tx(h_full, (uint32_t)(ts - nj) * 256u);
                 if (et < 2 * (CS - 1) && nj > 0) {
+                    // (x ring over the h tile: a peer's h tile is free only once its own gate/up products are complete)
+                    if (alias) WAIT(g_all, seq & 1);
                     int peer = et >> 1;
                     if (peer >= j) ++peer;
                     const uint32_t src = sH + (et & 1) * h_half + off * 128;
