@@ -89,11 +89,21 @@ __device__ __forceinline__ long long ps_now() {
 }
 #define RM_PS(item, slot) do { if ((item) < 64 && blockIdx.x < 128) g_ps_stamps[((item) * 128 + blockIdx.x) * 32 + (slot)] = ps_now(); } while (0)
 #define RM_PC(item, slot, v) do { if ((item) < 64 && blockIdx.x < 128) g_ps_stamps[((item) * 128 + blockIdx.x) * 32 + (slot)] = (v); } while (0)
+// -DRM_PHASE_TIMING=1: the phase stamps only (a handful per layer); =2 adds clock deltas around every wait and the
+// per-stage clocks of one item's gate/up stream (row 32 + who of the stamp array, one value per ring stage)
+#if RM_PHASE_TIMING + 0 >= 2
 #define RM_CLK() clock64()
+#define RM_TRACE_ITEM 5
+#define RM_TR(item, who, stage) do { if ((item) == RM_TRACE_ITEM && (stage) < 32) RM_PC(32 + (who), (stage), clock64()); } while (0)
+#else
+#define RM_CLK() 0ll
+#define RM_TR(item, who, stage) do { } while (0)
+#endif
 #else
 #define RM_PS(item, slot) do { } while (0)
 #define RM_PC(item, slot, v) do { } while (0)
 #define RM_CLK() 0ll
+#define RM_TR(item, who, stage) do { } while (0)
 #endif
 
 __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
@@ -105,6 +115,30 @@ __device__ __forceinline__ int ld_acquire_cta(const int* p) {          // shared
     int v;
     asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
     return v;
+}
+// The issuer's read of the landed-stage count: a relaxed load.  An acquire load holds back the product instructions
+// behind it for ~160 clocks; here the order is kept by the branch on the value, by tcgen05.fence::after_thread_sync
+// before the products, and by the watcher's proxy fence before its release store.
+__device__ __forceinline__ int ld_relaxed_cta(const int* p) {          // shared memory
+    int v;
+    asm volatile("ld.relaxed.cta.shared::cta.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    return v;
+}
+// The issuer's wait for more landed stages, kept out of line so that the loop that issues the products holds no wait
+// loop: returns the count once it exceeds `stage`, or what it last read when the bounded wait ran out or the CTA aborts.
+__device__ __noinline__ uint32_t landed_stages(const int* count, uint32_t stage, const int* abort_flag) {
+    uint32_t ready = 0;
+    for (uint32_t i = 0; i < (1u << 24); ++i) {
+        ready = (uint32_t)ld_relaxed_cta(count);
+        if (stage < ready) break;
+        if ((i & 4095u) == 4095u && *reinterpret_cast<const volatile int*>(abort_flag)) break;
+    }
+    return ready;
+}
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 __device__ __forceinline__ void st_release_cta(int* p, int v) {         // shared memory
     asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
@@ -455,6 +489,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             // stage cc: the rows over the 64-column blocks cc (first 8 KB) and cc + NCH/2 (second 8 KB)
             for (int cc = 0; cc < NCH / 2; ++cc) {
                 const uint32_t st = acquire();
+                if (lt == 0) RM_TR(k.item, 0, cc);
                 const int c1 = cc + NCH / 2;
                 const int so0 = (cc / NSB) * 3 * HS8 + (cc % NSB) * 64, so1 = (c1 / NSB) * 3 * HS8 + (c1 % NSB) * 64;
 #pragma unroll
@@ -466,6 +501,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                         cp_async16(d + 8192, src[q] + so1, true);
                     }
                 }
+                if (lt == 0) RM_TR(k.item, 1, cc);
                 cp_async_arrive_noinc(w_full(wcnt % NW));
                 ++wcnt;
             }
@@ -567,6 +603,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 const unsigned char* img = reinterpret_cast<const unsigned char*>(a.xbuf) + (size_t)(c * 2 + slot) * NCH * X_BYTES;
                 for (int cc = xq >> 1; cc < NCH / 2; cc += 2) {
                     if (n >= (uint32_t)XS) WAIT(x_empty(xs), ph ^ 1);
+                    if (half == 0) RM_TR(k.item, 2, cc);
                     const int blk = cc + half * (NCH / 2);
                     const uint32_t dst = sX + xs * XSB + half * X_BYTES;
                     if (ext) {
@@ -596,8 +633,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     const long long q0 = RM_CLK();
                     WAIT(w_full(wcnt % NW), (wcnt / NW) & 1);
                     const long long q1 = RM_CLK();
+                    RM_TR(k.item, 3, cc);
                     WAIT(x_full(xs), xph);
                     const long long q2 = RM_CLK();
+                    RM_TR(k.item, 4, cc);
                     fence_proxy_async_smem();
                     st_release_cta(sReady, (int)++stage);
                     const long long q3 = RM_CLK();
@@ -631,56 +670,53 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             }
         }
     } else if (warp == W_MMA) {
-        // ================================================================ issuer (one thread)
-        if (lane == 0) {
-            uint32_t wcnt = 0;
-            int xs = 0;
-            // Testing an mbarrier costs ~170 clocks even when its phase is long complete, which is more than the ~140
-            // clocks of a stage's two product instructions.  So the watcher thread does the waiting (and the proxy fence
-            // for the cp.async data) and publishes how many stages of the stream have landed; the issuer only reads that
-            // count, and reads it again only when it has used up what it knows of.
+        // ================================================================ issuer (one warp; an elected lane issues)
+        // Issuing is the scarce resource here: the tensor pipe idles while the issuing thread executes anything else
+        // (4 products of a stage keep it busy for ~256 clocks; a commit adds ~30-50, an acquire load ~160, a test of an
+        // mbarrier ~170, and in a loop that only lane 0 of a warp runs every branch around a wait loop cost another
+        // ~100-170 per stage).  Hence: the whole warp runs the control flow and one elected lane issues (measured 100-150
+        // clocks per stage cheaper than a one-lane loop); the watcher thread does the waiting and the proxy fence and
+        // publishes how many stages of the stream have landed; the issuer reads that count with a relaxed load (in a
+        // function of its own, off the hot path) only when it has used up what it knows of.
+        {
+            int ws = 0, xs = 0;                                    // ring slots of the next weight stage and x stage
+            const uint64_t dW0 = desc_k | desc_addr(sW), dX0 = desc_k | desc_addr(sX), dA0 = desc_mn_a | desc_addr(sW);
             uint32_t stage = 0, ready = 0;                         // stages issued; stages known to have landed
-            int ready_next = 0;                                    // a read of the count started before the last products
-            auto peek = [&]() { if (stage + 1 >= ready) ready_next = ld_acquire_cta(sReady); };
             auto need = [&](int line) {
-                if (stage >= ready) ready = (uint32_t)ready_next > ready ? (uint32_t)ready_next : ready;
                 if (stage < ready || gave_up) return;
-                for (uint32_t i = 0; i < (1u << 24); ++i) {
-                    ready = (uint32_t)ld_acquire_cta(sReady);
-                    if (stage < ready) return;
-                    if ((i & 4095u) == 4095u && *sAbort) { gave_up = true; return; }
-                }
-                timed_out(line);
+                ready = landed_stages(sReady, stage, const_cast<const int*>(sAbort));
+                if (stage < ready) return;
+                if (*sAbort) { gave_up = true; return; }
+                if (lane == 0) timed_out(line);
+                gave_up = true;
             };
             auto issue_g = [&](const Cur& k) {
-                const int buf = k.seq & 1;
-                long long c_n = 0, c_m = 0, c_c = 0;
+                const uint32_t d1 = tmem + (k.seq & 1) * (2 * NTOK);
                 for (int cc = 0; cc < NCH / 2; ++cc) {
-                    const int ws = wcnt % NW;
-                    const uint32_t st = sW + ws * SB, xt = sX + xs * XSB;
-                    const long long q0 = RM_CLK();
                     need(__LINE__);
-                    if (cc == 0 && k.i == 0) RM_PS(k.item, 1);
+                    if (cc == 0 && k.i == 0 && lane == 0) RM_PS(k.item, 1);
                     tc_fence_after();
-                    peek();
-                    const long long q1 = RM_CLK();
+                    const uint64_t da = dW0 + (uint64_t)(ws * (SB >> 4)), db = dX0 + (uint64_t)(xs * (XSB >> 4));
+                    if (elect_one()) {
+                        RM_TR(k.item, 5, cc);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        mma_bf16_ss(tmem + buf * (2 * NTOK), desc_k | desc_addr(st + ks * 32), desc_k | desc_addr(xt + ks * 32),
-                                    IDESC_G, (cc | ks) != 0);
-                    const long long q2 = RM_CLK();
-                    mma_commit(x_empty(xs));
-                    mma_commit(w_empty(ws));
-                    const long long q3 = RM_CLK();
-                    if (cc > 0) { c_n += q1 - q0; c_m += q2 - q1; c_c += q3 - q2; }
+                        for (int ks = 0; ks < 4; ++ks) mma_bf16_ss(d1, da + 2 * ks, db + 2 * ks, IDESC_G, (cc | ks) != 0);
+                        mma_commit(x_empty(xs));
+                        mma_commit(w_empty(ws));
+                        RM_TR(k.item, 6, cc);
+                    }
+                    __syncwarp();
                     if (++xs == XS) xs = 0;
-                    ++wcnt;
+                    if (++ws == NW) ws = 0;
                     ++stage;
                 }
-                mma_commit(d1_full(buf));
-                if (alias) mma_commit_mc(g_all, 0xff);                // this CTA's x ring (which lies over its h tile) is read out
-                if (k.i == 0) { RM_PS(k.item, 24); RM_PC(k.item, 10, c_n); RM_PC(k.item, 11, c_m); RM_PC(k.item, 12, c_c); }
-                if (k.i == k.run.ntiles - 1 && !item_ext(env, k.l)) mma_commit_mc(x_free(k.use & 1), 0xff);
+                if (elect_one()) {
+                    mma_commit(d1_full(k.seq & 1));
+                    if (alias) mma_commit_mc(g_all, 0xff);            // this CTA's x ring (which lies over its h tile) is read out
+                    if (k.i == 0) RM_PS(k.item, 24);
+                    if (k.i == k.run.ntiles - 1 && !item_ext(env, k.l)) mma_commit_mc(x_free(k.use & 1), 0xff);
+                }
+                __syncwarp();
             };
             auto issue_d = [&](const Cur& k) {
                 int t0, ts;
@@ -689,30 +725,35 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 const int d2b = ND2 == 2 ? (k.ni & 1) : 0, nu = ND2 == 2 ? (k.ni >> 1) : k.ni;
                 if (k.i == 0 && nu >= 1) WAIT(d2_empty(d2b), (nu - 1) & 1);
                 WAIT(h_full, k.seq & 1);
-                RM_PS(k.item, 4);
+                if (lane == 0) RM_PS(k.item, 4);
                 const uint32_t d2 = tmem + G::D2_COL + d2b * (2 * NTOK);
+                uint64_t dh = desc_mn_b | desc_addr(sH);             // 16 slots of h per product step
                 for (int s = 0; s < nst; ++s) {
-                    const int ws = wcnt % NW;
-                    const uint32_t st = sW + ws * SB;
                     need(__LINE__);
                     tc_fence_after();
-                    peek();
+                    const uint64_t da = dA0 + (uint64_t)(ws * (SB >> 4));
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < KPS; ++ks) {
-                        const int kk = KPS * s + ks;
-                        if (kk < kst) {
+                        for (int ks = 0; ks < KPS; ++ks) {
+                            if (KPS * s + ks < kst) {
 #pragma unroll
-                            for (int mb = 0; mb < NMB; ++mb)
-                                mma_bf16_ss(d2 + mb * (2 * NTOK), desc_mn_a | desc_addr(st + mb * (2 * SPS * 128) + ks * 2048),
-                                            desc_mn_b | desc_addr(sH + kk * 2048), IDESC_D, !(k.i == 0 && kk == 0));
+                                for (int mb = 0; mb < NMB; ++mb)
+                                    mma_bf16_ss(d2 + mb * (2 * NTOK), da + (uint64_t)((mb * (2 * SPS * 128) + ks * 2048) >> 4),
+                                                dh + (uint64_t)(ks * (2048 >> 4)), IDESC_D, !(k.i == 0 && s == 0 && ks == 0));
+                            }
                         }
+                        mma_commit(w_empty(ws));
                     }
-                    mma_commit(w_empty(ws));
-                    ++wcnt;
+                    __syncwarp();
+                    dh += KPS * (2048 >> 4);
+                    if (++ws == NW) ws = 0;
                     ++stage;
                 }
-                mma_commit_mc(h_free, 0xff);
-                if (k.i == k.run.ntiles - 1) { mma_commit(d2_full(d2b)); RM_PS(k.item, 25); }
+                if (elect_one()) {
+                    mma_commit_mc(h_free, 0xff);
+                    if (k.i == k.run.ntiles - 1) { mma_commit(d2_full(d2b)); RM_PS(k.item, 25); }
+                }
+                __syncwarp();
             };
             Cur g, d;
             cur_init(g, env);
