@@ -840,7 +840,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 }
                 n2 = RM_CLK();
                 // the readers are copy-engine reads issued by this cluster's CTAs after the cluster-scope arrivals below
-                fence_proxy_async();
+                fence_proxy_async_global();
                 n3 = RM_CLK();
             }
             stop = named_barrier_or(1, 256, gave_up || *sAbort);
@@ -973,8 +973,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 if (et < 2 * (CS - 1) && nj > 0) {
                     // (x ring over the h tile: a peer's h tile is free only once its own gate/up products are complete)
                     if (alias) WAIT(g_all, seq & 1);
-                    int peer = et >> 1;
-                    if (peer >= j) ++peer;
+                    // CTA j sends to j + 1, j + 2, ... in turn: the copies of a CTA leave one after the other (~0.13 us
+                    // each), and with every CTA starting at rank 0 the high ranks had their h 1-2 us after the low ones
+                    const int peer = (j + 1 + (et >> 1)) & (CS - 1);
                     const uint32_t src = sH + (et & 1) * h_half + off * 128;
                     bulk_copy_to_peer(map_to_rank(src, peer), src, (uint32_t)nj * 128u, map_to_rank(h_full, peer));
                 }

@@ -138,6 +138,8 @@ __device__ __forceinline__ void named_barrier(int id, int count) {
 // make generic-proxy writes to shared memory visible to the async proxy (tcgen05.mma reads operands through it)
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 // the same for this CTA's shared memory only (cheaper; enough when the reader is this CTA's own copy engine or MMA)
+// (restricted to global memory: for generic-proxy stores to global memory that a bulk copy reads afterwards)
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---------------------------------------------------------------- mbarrier
