@@ -202,6 +202,33 @@ __device__ __forceinline__ void cta_span(int ts, int j, int& off, int& nj) {
     nj = ts * (j + 1) / CS - off;                                  // <= 32
 }
 
+// Down stages of a tile are taken in an order that follows the arrival of the h pieces.  CTA p sends its piece to
+// p + 1, p + 2, ... in turn, so CTA j receives the pieces j - 1, j - 2, ..., j + 1 in that order (ranks mod 8, ~0.13 us
+// apart); it starts with the highest stage that lies entirely below the end of its own piece (that stage needs its own
+// piece and the one or two below it) and goes downwards, wrapping round, so that the stage that reaches into piece
+// j + 1 comes last.  Stage number k of that order:
+__device__ __forceinline__ int d_stage_first(int ts, int j, int sps, int nst) {
+    const int end = ts * (j + 1) / CS;                             // end of CTA j's piece
+    int s0 = end / sps - 1;
+    if (s0 >= nst) s0 = nst - 1;
+    return s0 < 0 ? nst - 1 : s0;
+}
+__device__ __forceinline__ int d_stage(int s0, int k, int nst) {
+    const int s = s0 - k;
+    return s < 0 ? s + nst : s;
+}
+// The pieces whose slots a stage reads, as a bit mask over the CTA ranks
+__device__ __forceinline__ uint32_t d_stage_pieces(int ts, int s, int sps) {
+    const int lo = s * sps, hi = (s + 1) * sps < ts ? (s + 1) * sps : ts;
+    uint32_t m = 0;
+#pragma unroll
+    for (int p = 0; p < CS; ++p) {
+        const int a = ts * p / CS, b = ts * (p + 1) / CS;
+        if (a < hi && b > lo) m |= 1u << p;
+    }
+    return m;
+}
+
 // Cursor over the tiles this cluster walks during the step, in order.
 struct Cur {
     int item, l, b, i;
@@ -315,7 +342,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     auto d2_empty = [&](int s) { return bar0 + 480 + 8 * s; };
     auto x_ready = [&](int s) { return bar0 + 496 + 8 * s; };       // 2
     auto x_free = [&](int s) { return bar0 + 512 + 8 * s; };
-    const uint32_t h_full = bar0 + 528, h_free = bar0 + 536, g_all = bar0 + 544;
+    const uint32_t h_free = bar0 + 536, g_all = bar0 + 544;
+    auto h_arr = [&](int p) { return bar0 + 552 + 8 * p; };        // CS: piece p of the tile's h has arrived in this CTA
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int j = (int)cluster_ctarank(), c = (int)cluster_id_x(), NC = (int)cluster_count_x();
@@ -343,7 +371,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             mbar_init(d1_full(s), 1); mbar_init(d2_full(s), 1); mbar_init(d2_empty(s), 256);
             mbar_init(x_ready(s), CS); mbar_init(x_free(s), CS);
         }
-        mbar_init(h_full, 1); mbar_init(h_free, CS); mbar_init(g_all, CS);
+        for (int p2 = 0; p2 < CS; ++p2) mbar_init(h_arr(p2), 1);
+        mbar_init(h_free, CS); mbar_init(g_all, CS);
         fence_mbar_init();
         *sAbort = 0;
         *sLoaded = 0;
@@ -515,7 +544,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             constexpr int SPW = 32 / PPS;                          // slots one warp instruction covers
             const int piece = lane % PPS;
             const __nv_bfloat16* wl = a.packed[k.l] + j * 3 * HS8 + 2 * HS8 + piece * 8;
-            for (int s = 0; s < nst; ++s) {
+            const int s0 = d_stage_first(ts, j, SPS, nst);
+            for (int ks0 = 0; ks0 < nst; ++ks0) {
+                const int s = d_stage(s0, ks0, nst);
                 const uint32_t st = acquire();
 #pragma unroll
                 for (int m = 0; m < 8; ++m) {
@@ -631,10 +662,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 long long c_w = 0, c_x = 0, c_f = 0;
                 for (int cc = 0; cc < NCH / 2; ++cc) {
                     const long long q0 = RM_CLK();
-                    WAIT(w_full(wcnt % NW), (wcnt / NW) & 1);
+                    const uint32_t both = mbar_test_wait_2(w_full(wcnt % NW), (wcnt / NW) & 1, x_full(xs), xph);
+                    if (!(both & 1u)) WAIT(w_full(wcnt % NW), (wcnt / NW) & 1);
                     const long long q1 = RM_CLK();
                     RM_TR(k.item, 3, cc);
-                    WAIT(x_full(xs), xph);
+                    if (!(both & 2u)) WAIT(x_full(xs), xph);
                     const long long q2 = RM_CLK();
                     RM_TR(k.item, 4, cc);
                     fence_proxy_async_smem();
@@ -650,8 +682,25 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 int t0, ts;
                 tile_span(k.run, k.i, t0, ts);
                 const int nst = (ts + SPS - 1) / SPS;
-                for (int s = 0; s < nst; ++s) {
-                    WAIT(w_full(wcnt % NW), (wcnt / NW) & 1);
+                const int s0 = d_stage_first(ts, j, SPS, nst);
+                uint32_t arrived = 0;                              // pieces of this tile's h known to be here
+                for (int ks0 = 0; ks0 < nst; ++ks0) {
+                    const uint32_t want = d_stage_pieces(ts, d_stage(s0, ks0, nst), SPS);
+                    bool w_ok;
+                    if (want & ~arrived) {
+                        // the stage's weights and all eight pieces in one round of tests
+                        const uint32_t m = mbar_test_wait_8_1(h_arr(0), k.seq & 1, w_full(wcnt % NW), (wcnt / NW) & 1);
+                        arrived |= m & 0xffu;
+                        w_ok = (m >> 8) & 1u;
+                    } else {
+                        w_ok = mbar_test_wait(w_full(wcnt % NW), (wcnt / NW) & 1);
+                    }
+                    if (!w_ok) WAIT(w_full(wcnt % NW), (wcnt / NW) & 1);
+                    for (uint32_t i = 0; (want & ~arrived) && i < (1u << 20) && !gave_up; ++i) {
+                        arrived |= mbar_test_wait_8_1(h_arr(0), k.seq & 1, w_full(wcnt % NW), (wcnt / NW) & 1) & 0xffu;
+                        if ((i & 255u) == 255u && *sAbort) gave_up = true;
+                    }
+                    if ((want & ~arrived) && !gave_up) timed_out(__LINE__);
                     fence_proxy_async_smem();
                     st_release_cta(sReady, (int)++stage);
                     ++wcnt;
@@ -724,14 +773,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 const int kst = (ts + 15) >> 4, nst = (ts + SPS - 1) / SPS;
                 const int d2b = ND2 == 2 ? (k.ni & 1) : 0, nu = ND2 == 2 ? (k.ni >> 1) : k.ni;
                 if (k.i == 0 && nu >= 1) WAIT(d2_empty(d2b), (nu - 1) & 1);
-                WAIT(h_full, k.seq & 1);
-                if (lane == 0) RM_PS(k.item, 4);
                 const uint32_t d2 = tmem + G::D2_COL + d2b * (2 * NTOK);
-                uint64_t dh = desc_mn_b | desc_addr(sH);             // 16 slots of h per product step
-                for (int s = 0; s < nst; ++s) {
+                const uint64_t dh0 = desc_mn_b | desc_addr(sH);      // 16 slots of h per product step
+                // (the watcher publishes a down stage only when the h pieces it reads have arrived; the stages come in
+                // the order of d_stage)
+                const int s0 = d_stage_first(ts, j, SPS, nst);
+                for (int ks0 = 0; ks0 < nst; ++ks0) {
+                    const int s = d_stage(s0, ks0, nst);
                     need(__LINE__);
+                    if (ks0 == 0 && lane == 0) RM_PS(k.item, 4);
                     tc_fence_after();
-                    const uint64_t da = dA0 + (uint64_t)(ws * (SB >> 4));
+                    const uint64_t da = dA0 + (uint64_t)(ws * (SB >> 4)), dh = dh0 + (uint64_t)(s * (KPS * (2048 >> 4)));
                     if (elect_one()) {
 #pragma unroll
                         for (int ks = 0; ks < KPS; ++ks) {
@@ -739,13 +791,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
 #pragma unroll
                                 for (int mb = 0; mb < NMB; ++mb)
                                     mma_bf16_ss(d2 + mb * (2 * NTOK), da + (uint64_t)((mb * (2 * SPS * 128) + ks * 2048) >> 4),
-                                                dh + (uint64_t)(ks * (2048 >> 4)), IDESC_D, !(k.i == 0 && s == 0 && ks == 0));
+                                                dh + (uint64_t)(ks * (2048 >> 4)), IDESC_D, !(k.i == 0 && ks0 == 0 && ks == 0));
                             }
                         }
                         mma_commit(w_empty(ws));
                     }
                     __syncwarp();
-                    dh += KPS * (2048 >> 4);
                     if (++ws == NW) ws = 0;
                     ++stage;
                 }
@@ -969,7 +1020,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 const long long e6 = RM_CLK();
                 stop = named_barrier_or(1, 256, gave_up || *sAbort);
                 const long long e7 = RM_CLK();
-                if (et == 0) mbar_arrive_expect_tx(h_full, (uint32_t)(ts - nj) * 256u);
+                // every piece barrier completes once per tile: a peer's piece by its two copies (hi and lo rows), this
+                // CTA's own piece (written above, fenced, behind the barrier) and empty pieces by the arrival alone
+                if (et < CS) {
+                    int poff, pn;
+                    cta_span(ts, et, poff, pn);
+                    if (et == j || pn == 0) mbar_arrive(h_arr(et));
+                    else mbar_arrive_expect_tx(h_arr(et), (uint32_t)pn * 256u);
+                }
                 if (et < 2 * (CS - 1) && nj > 0) {
                     // (x ring over the h tile: a peer's h tile is free only once its own gate/up products are complete)
                     if (alias) WAIT(g_all, seq & 1);
@@ -977,7 +1035,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     // each), and with every CTA starting at rank 0 the high ranks had their h 1-2 us after the low ones
                     const int peer = (j + 1 + (et >> 1)) & (CS - 1);
                     const uint32_t src = sH + (et & 1) * h_half + off * 128;
-                    bulk_copy_to_peer(map_to_rank(src, peer), src, (uint32_t)nj * 128u, map_to_rank(h_full, peer));
+                    bulk_copy_to_peer(map_to_rank(src, peer), src, (uint32_t)nj * 128u, map_to_rank(h_arr(j), peer));
                 }
                 if (et == 0 && i == 0) {
                     const long long e8 = RM_CLK();

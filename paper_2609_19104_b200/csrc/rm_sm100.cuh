@@ -170,6 +170,47 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Tests of several phases whose answers come back together: one test takes ~200 clocks to return even when the phase
+// is long complete, and a thread that looks at each answer before it starts the next test pays that once per test.
+// Bit i of the result: the phase with parity `parity` of the mbarrier at base + 8 i has completed (i < 8); bit 8: the
+// phase with parity `parity_x` of the mbarrier `extra`.
+__device__ __forceinline__ uint32_t mbar_test_wait_8_1(uint32_t base, uint32_t parity, uint32_t extra, uint32_t parity_x) {
+    uint32_t m;
+    asm volatile(
+        "{\n\t.reg .pred p0, p1, p2, p3, p4, p5, p6, p7, p8;\n\t.reg .b32 t;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p8, [%3], %4;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p0, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p1, [%1+8], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p2, [%1+16], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p3, [%1+24], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p4, [%1+32], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p5, [%1+40], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p6, [%1+48], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p7, [%1+56], %2;\n\t"
+        "selp.u32 %0, 256, 0, p8;\n\t"
+        "selp.u32 t, 1, 0, p0;\n\tor.b32 %0, %0, t;\n\t"
+        "selp.u32 t, 2, 0, p1;\n\tor.b32 %0, %0, t;\n\t"
+        "selp.u32 t, 4, 0, p2;\n\tor.b32 %0, %0, t;\n\t"
+        "selp.u32 t, 8, 0, p3;\n\tor.b32 %0, %0, t;\n\t"
+        "selp.u32 t, 16, 0, p4;\n\tor.b32 %0, %0, t;\n\t"
+        "selp.u32 t, 32, 0, p5;\n\tor.b32 %0, %0, t;\n\t"
+        "selp.u32 t, 64, 0, p6;\n\tor.b32 %0, %0, t;\n\t"
+        "selp.u32 t, 128, 0, p7;\n\tor.b32 %0, %0, t;\n\t}"
+        : "=&r"(m) : "r"(base), "r"(parity), "r"(extra), "r"(parity_x) : "memory");
+    return m;
+}
+// The same for two phases: bit 0 for (a, parity_a), bit 1 for (b, parity_b)
+__device__ __forceinline__ uint32_t mbar_test_wait_2(uint32_t a, uint32_t parity_a, uint32_t b, uint32_t parity_b) {
+    uint32_t m;
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b32 t;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p0, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p1, [%3], %4;\n\t"
+        "selp.u32 %0, 1, 0, p0;\n\t"
+        "selp.u32 t, 2, 0, p1;\n\tor.b32 %0, %0, t;\n\t}"
+        : "=&r"(m) : "r"(a), "r"(parity_a), "r"(b), "r"(parity_b) : "memory");
+    return m;
+}
 // Bounded wait: returns false when the phase did not complete within the budget (the caller records a status
 // code and carries on; nothing spins forever).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t max_polls = 1u << 22) {
