@@ -846,7 +846,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 // every CTA has added its part of layer l-1 to this episode's rows
                 const int target = a.per_item ? n_ctas : a.sync_base[b] + n_ctas * l;
                 const int* counter = a.per_item ? a.sync + SYNC_ITEM + (l - 1) * B + b : a.sync + b;
-                if (lane == 0 && !gave_up) {
+                // one thread per CTA watches the counter (with every warp's lane 0 polling, ~1000 threads read the line
+                // that the last arrivals have to get through); the barrier passes its acquire on to the others
+                if (et == 0 && !gave_up) {
                     bool ok = false;
                     for (uint32_t i = 0; i < (1u << 21); ++i) {
                         if (ld_acquire_gpu(counter) >= target) { ok = true; break; }
@@ -854,7 +856,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     }
                     if (!ok) { if (!*sAbort && !ld_acquire_gpu(a.sync + SYNC_ABORT)) timed_out(__LINE__); gave_up = true; *sAbort = 1; }
                 }
-                __syncwarp();
+                named_barrier(1, 256);
             }
             if (et == 0) RM_PS(item, 8);
             const long long n0 = RM_CLK();
@@ -992,6 +994,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 const long long e3 = RM_CLK();
                 if (!hf_ok) WAIT(h_free, (seq - 1) & 1);             // every CTA's down products of the previous tile are complete
                 const long long e4 = RM_CLK();
+                // The piece barriers complete once per tile: a peer's piece by its two copies (hi and lo rows), armed here
+                // (the previous tile's pieces have all arrived: its down products are complete); this CTA's own piece
+                // and empty pieces by an arrival alone (the own one further down, behind the writes).
+                if (et < CS && et != j) {
+                    int poff, pn;
+                    cta_span(ts, et, poff, pn);
+                    if (pn == 0) mbar_arrive(h_arr(et));
+                    else mbar_arrive_expect_tx(h_arr(et), (uint32_t)pn * 256u);
+                }
+                // (x ring over the h tile: a peer's h tile is free only once its own gate/up products are complete; the
+                // test is started here and looked at when the copies are ready to go)
+                const bool ga_ok = alias && et < 2 * (CS - 1) ? mbar_test_wait(g_all, seq & 1) : true;
                 if (ni_loc < nj) {
                     const int kslot = off + ni_loc;
                     const int p0 = ch * 4 + (fin ? 0 : 2) + (isup ? 1 : 0);   // 16-byte piece (8 tokens) of the row's 128 bytes
@@ -1020,17 +1034,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 const long long e6 = RM_CLK();
                 stop = named_barrier_or(1, 256, gave_up || *sAbort);
                 const long long e7 = RM_CLK();
-                // every piece barrier completes once per tile: a peer's piece by its two copies (hi and lo rows), this
-                // CTA's own piece (written above, fenced, behind the barrier) and empty pieces by the arrival alone
-                if (et < CS) {
-                    int poff, pn;
-                    cta_span(ts, et, poff, pn);
-                    if (et == j || pn == 0) mbar_arrive(h_arr(et));
-                    else mbar_arrive_expect_tx(h_arr(et), (uint32_t)pn * 256u);
-                }
+                if (et == 0) mbar_arrive(h_arr(j));                  // this CTA's own piece: written, fenced, behind the barrier
                 if (et < 2 * (CS - 1) && nj > 0) {
-                    // (x ring over the h tile: a peer's h tile is free only once its own gate/up products are complete)
-                    if (alias) WAIT(g_all, seq & 1);
+                    if (!ga_ok) WAIT(g_all, seq & 1);
                     // CTA j sends to j + 1, j + 2, ... in turn: the copies of a CTA leave one after the other (~0.13 us
                     // each), and with every CTA starting at rank 0 the high ranks had their h 1-2 us after the low ones
                     const int peer = (j + 1 + (et >> 1)) & (CS - 1);
