@@ -23,24 +23,31 @@ inline bool use_fused(const rm_ctx* ctx, int B, int T) {
 }
 
 // The whole-step kernel (variant 5).  Chosen by itself where it is measured ahead of the per-layer kernels (single
-// episodes, masked steps; us per step, cold L2, per-layer kernels first):
-//   H = 2048, I = 16384:  K =  820: 321 / 320 (it is what runs)   3277: 509 / 393   9831: 1098 / 848   13108: 1148 / 1074
-//                         16384 (every neuron listed): 1170 / 1300 -> streaming kernel
-//   H = 1024, I = 4096:   K =  205: 169 / 226   1024: 198 / 241   1639: 248 / 246   2048: 269 / 258   3072: 347 / 277
-//                         4096: 355 / 365
-// It adapts to the counts on the device, so at H = 2048 it needs no hint; at H = 1024 the lean per-layer kernel (two
-// CTAs per SM, consecutive layers overlap) stays ahead on short lists, so the whole-step kernel is chosen only when
-// the caller's count hint says that the lists hold 35 % to 90 % of the neurons.  Dense passes (no list) and batches
-// stay with the streaming kernel.  `steps`: a whole stack (false: the one-layer entry, which would pay the kernel's
-// set-up for a single layer).
+// episodes; us per step, cold L2: lean per-layer kernel / streaming kernel / whole-step kernel):
+//   H = 2048, I = 16384:  K =  820: 265 / 572 / 299    1639: 377 / 577 / 308    3277: 603 / 577 / 342
+//                         4916: 827 / 587 / 522    8192: 1179 / 648 / 732    12288: 1641 / 1130 / 967
+//                         16384 (every neuron listed): 2160 / 1173 / 1192
+//   H = 1024, I = 4096:   K =  205: 170 / 341 / 210    820: 176 / 343 / 215    1024: 199 / 343 / 223
+//                         1229: 231 / 345 / 225    2048: 269 / 345 / 236    3072: 376 / 347 / 240    4096: 404 / 355 / 330
+// The streaming kernel's time steps up with every wave of 64-neuron tiles over the SMs (148 tiles per wave); the
+// whole-step kernel grows evenly with K and has a fixed cost of ~11-16 us per layer.  So, with K the caller's count
+// hint (the whole layer for a dense pass): at H = 1024 from 28 % of the neurons upwards; at H = 2048 from 7 % up to
+// 42 %, and again where the streaming kernel needs a second wave, up to 95 %.  Without a hint at H = 2048 it is
+// chosen as well (it adapts to the counts on the device), at H = 1024 the lean kernel.  Batches stay with the
+// streaming kernel.  `steps`: a whole stack (false: the one-layer entry, which would pay the kernel's set-up for a
+// single layer).
 inline bool use_persist(const rm_ctx* ctx, int B, int T, bool masked, bool steps) {
     if (ctx->path == 1 || !rm_persist_supported(ctx, B, T)) return false;
     if (ctx->variant_override == 5) return true;
-    if (ctx->variant_override != 0 || B > ctx->persist_max_b || !steps || !masked) return false;
-    const long long hint = ctx->count_hint, I = ctx->g.I;
-    if (hint > 0 && hint * 10 > I * 9) return false;              // nearly every neuron listed
-    if (ctx->g.H == 2048) return true;
-    return hint > 0 && hint * 100 >= I * 35;
+    if (ctx->variant_override != 0 || B > ctx->persist_max_b || !steps) return false;
+    const long long I = ctx->g.I, K = masked ? ctx->count_hint : I;
+    if (ctx->g.H == 2048) {
+        if (K <= 0) return true;
+        if (K * 100 < I * 7) return false;
+        if (K * 100 <= I * 42) return true;
+        return (K + 63) / 64 > ctx->sm_count && K * 100 <= I * 95;
+    }
+    return K > 0 && K * 100 >= I * 28;
 }
 
 inline void* persist_ws(const rm_ctx* ctx, void* ws, int B, int T) {
