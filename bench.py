@@ -32,7 +32,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per layer of a step, from ncu captures of the kernels that run these
 # workloads (one layer launch of the lean per-layer kernel; the whole-step kernel's figure divided by its layers)
-TRAFFIC_BYTES_PER_LAYER = {"pi0-stack-top25": 6.794e6}
+TRAFFIC_BYTES_PER_LAYER = {("pi0-stack-top25", 1): 6.794e6, ("large-stack-top20-refresh2", 5): 43.1e6}
 KERNEL_FAMILY = {0: "portable CUDA-core kernels (norm, gate/up, down)",
                  1: "fused_layer_kernel (lean per-layer cluster kernel, dependent-launch chained)",
                  2: "fused_layer_kernel, two tiles in flight",
@@ -483,7 +483,7 @@ def side_configs(rm, ctx1, packed1, w1, flush, stream, args):
     ctx2.rm_set_option("count_hint", w2.K)
     us_sparse = timed_us(lambda i: ctx2.rm_action_expert_step(packed2, xsp, idx2, cnt2, w2.I, out2, B=1, T=w2.T))
     e = entry(ctx2, w2, us_sparse, w2.K, note="odd steps of the schedule: masked with the previous step's top-20 % lists")
-    e["traffic_bytes_per_layer"] = TRAFFIC_BYTES_PER_LAYER.get(w2.name)
+    e["traffic_bytes_per_layer"] = TRAFFIC_BYTES_PER_LAYER.get((w2.name, e["kernel_family"]))
     us_g = timed_us(lambda i: ctx2.rm_debug_gather_read_step(packed2, idx2, cnt2, w2.I))
     e["gather_read_microbench_us_per_step"] = us_g
     e["gather_read_microbench_gbs"] = w2.K * 3 * w2.H * 2 * w2.L / (us_g * 1e-6) / 1e9
@@ -617,6 +617,9 @@ def run_gpu(args, w: wl.Workload):
         if timed_events is not None:
             timed_events[1].record(stream)
 
+    if args.phase_timeline:
+        phase_timeline(ctx, w, lambda s: one_step(s))
+        return
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -753,7 +756,7 @@ def run_gpu(args, w: wl.Workload):
                        "l2": "flushed before every timed step (512 MB fill, outside the timed interval)",
                        "multi_gpu": "replicas: each rank runs its own episodes, no collective on the data path"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": TRAFFIC_BYTES_PER_LAYER.get(w.name) if step_variant == 1 else None,
+                         "traffic": TRAFFIC_BYTES_PER_LAYER.get((w.name, step_variant)),
                          "peak_kind": f"{peak_kind} copy bandwidth", "kernel": kernel_name, "kernel_family": step_variant,
                          "bytes_per_launch": bytes_layer, "us_per_launch": in_step_layer_us,
                          "us_per_launch_isolated_cold": layer_us, "launches_per_step": launches_per_step,
@@ -790,6 +793,46 @@ def run_gpu(args, w: wl.Workload):
         dist.destroy_process_group()
 
 
+PHASES = ["x ready (cluster barrier)", "first x stage landed, first gate/up product", "gate/up products complete",
+          "h pieces sent", "first down product", "down products complete", "adds issued", "arrival on the counter",
+          "counter complete: normalisation starts", "normalisation done"]
+PHASE_ORDER = [8, 9, 0, 1, 2, 3, 4, 5, 6, 7]
+
+
+def phase_timeline(ctx, w, step):
+    """Profiling aid for a library built with -DRM_PHASE_TIMING=1 (python -m paper_2609_19104_b200.build with
+    RM_EXTRA_NVCC_FLAGS set): runs three cold steps through the whole-step kernel and prints, per layer, when its
+    phases were reached in the fastest and the slowest CTA (us after the first CTA saw the layer's counter complete)."""
+    import ctypes
+    import torch
+    for s in range(1, 4):                                   # (step 0 of a schedule rebuilds the masks: skip it)
+        step(s)
+    torch.cuda.synchronize()
+    if ctx.rm_get_info("last_variant") != 5:
+        print(json.dumps({"phase_timeline": "the whole-step kernel did not run this workload"}))
+        return
+    n = 64 * 128 * 32
+    buf = (ctypes.c_longlong * n)()
+    rc = ctx.lib.rm_debug_phase_times(ctx._h, buf, -(1 << 20) - n)
+    if rc != 0:
+        print(json.dumps({"phase_timeline": f"unavailable (rm_debug_phase_times returned {rc}: build with -DRM_PHASE_TIMING=1)"}))
+        return
+    st = np.frombuffer(buf, dtype=np.int64).reshape(64, 128, 32).astype(np.float64)
+    ncta = ctx.rm_get_info("persist_clusters") * 8
+    t_first = None
+    for it in range(min(w.L, 64)):
+        s0 = st[it, :ncta, :10]
+        go = s0[:, 8][s0[:, 8] > 0]
+        ref = go.min() if go.size else s0[:, 1][s0[:, 1] > 0].min()
+        t_first = ref if t_first is None else t_first
+        row = {"layer": it, "starts_at_us": round((ref - t_first) / 1e3, 2)}
+        for k in PHASE_ORDER:
+            v = s0[:, k][s0[:, k] > 0]
+            if v.size:
+                row[PHASES[k]] = [round((v.min() - ref) / 1e3, 2), round((v.max() - ref) / 1e3, 2)]
+        print(json.dumps(row))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -808,6 +851,9 @@ def main():
     ap.add_argument("--max-clusters", type=int, default=0, help="library option \"max_clusters\" (0 = default)")
     ap.add_argument("--layers", type=int, default=0,
                     help="run the first N layers of the workload only (small cases for profiler captures; not a bench value)")
+    ap.add_argument("--phase-timeline", action="store_true",
+                    help="profiling aid (library built with -DRM_PHASE_TIMING=1): print when each layer's phases were "
+                         "reached inside the whole-step kernel, then exit; not a bench value")
     ap.add_argument("--no-configs", action="store_true",
                     help="skip the side measurements of the other workloads (the \"configs\" object of the line)")
     args = ap.parse_args()

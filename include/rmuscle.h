@@ -42,7 +42,7 @@ typedef enum {
     RM_ERR_UNSUPPORTED = -8        /* valid request that this build does not implement                    */
 } rm_status;
 
-enum { RM_ACT_GELU_TANH = 0 };     /* the gated unit's activation ("post-GeGLU activation", Eq. 1)        */
+enum { RM_ACT_GELU_TANH = 0 };     /* the gated unit's activation (Eq. 1 takes it after the GeGLU)     */
 
 /* Model geometry fixed at context creation.  H must be a multiple of 64, I >= 1, L >= 1.
  * T_max / B_max bound the T and B of later calls (they size rm_workspace_bytes). */
@@ -100,22 +100,21 @@ typedef struct {
 int rm_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32_t* count_out, int64_t stride,
                     rm_stream_t stream);
 
-/* ---- rm_gather_weights: the paper's own preparation of the selected weights (Sec. 4.1: "Selected weights are
- * prepared in shared compact buffers and reused across each group's steps"; Sec. 5 "Overlapping Retrieval and Weight
- * Gathering"), as a comparison variant to gathering inside the products.  Copies the packed rows of the listed
- * neurons to the front of compact_out: compact row p = packed row idx[p] for p < count; the rows from count up to the
- * next multiple of 64 (where the buffer has them) are cleared, because a kernel may fetch the last 64-neuron tile whole
- * and multiply its unused rows by zero -- a compact layer built by other means must hold finite values there too.
- * compact_out holds at least
- * min(list_cap, I) rows of 3*H bf16 (rm_packed_layer_bytes is always enough) and is itself a packed layer: pass it to
- * rm_sparse_mlp / rm_action_expert_step with idx = NULL and the same count_dev ("the leading count neurons"), and the
+/* ---- rm_gather_weights: the paper's own preparation of the selected weights (Sec. 4.1, last
+ * paragraph: the rows a group's mask selects are copied once into compact buffers that all steps of the group read;
+ * Sec. 5 "Overlapping Retrieval and Weight Gathering"), as a comparison variant to gathering inside the products.
+ * Copies the packed rows of the listed neurons to the front of compact_out: compact row p = packed row idx[p] for
+ * p < count; the rows from count up to the next multiple of 64 (where the buffer has them) are cleared, because a
+ * kernel may fetch the last 64-neuron tile whole and multiply its unused rows by zero -- a compact layer built by
+ * other means must hold finite values there too.  compact_out holds at least min(list_cap, I) rows of 3*H bf16 (rm_packed_layer_bytes is always enough) and is itself a packed layer: pass it to
+ * rm_sparse_mlp / rm_action_expert_step with idx = NULL and the same count_dev (the leading count neurons), and the
  * result is the masked layer over the listed neurons.  Activation records and anchor activations of such a call are
  * indexed by compact position.  Call it on a side stream to overlap it with other work; ordering is the caller's. */
 int rm_gather_weights(rm_ctx* ctx, const void* packed_layer, const int32_t* idx, const int32_t* count_dev,
                       int64_t list_cap, void* compact_out, rm_stream_t stream);
 
-/* ---- rm_sparse_mlp: one layer, zero-fill form of the masked evaluation (Sec. 4.1: "compute only the selected
- * neurons' hidden activations and update the output using their down-projection weights"):
+/* ---- rm_sparse_mlp: one layer, zero-fill form of the masked evaluation (Sec. 4.1: hidden activations are computed
+ * for the selected neurons only, and only their down-projection columns update the output):
  *     y[t,:] = residual[t,:] + sum_{n in S} gelu_tanh(<x_t, Wg_n>) * <x_t, Wu_n> * Wd[:,n]
  *   packed_layer: output of rm_pack_weights.   x [T,H] bf16.   residual [T,H] fp32, nullable (=> 0).
  *   idx [>= count] int32 ascending, nullable => every neuron (dense);  count_dev [1] int32 on the device.
@@ -149,8 +148,8 @@ int rm_action_expert_step_host(rm_ctx* ctx, const void* const* packed_layers, co
                                int B, int T, void* ws, size_t ws_bytes, rm_stream_t stream);
 
 /* ---- rm_action_expert_step_ex: the same stack with the anchor-relative local update of the Action Cache (Sec. 4.1
- * "Anchors with Mask Recomputation", Eq. 4) and the output gate that follows it ("the output follows the normal
- * adaptive gate and residual addition").  Per layer l and episode:
+ * "Anchors with Mask Recomputation", Eq. 4) and the output gate that follows it (after Eq. 4 the paper applies the model's
+ * usual adaptive gate and then adds the residual).  Per layer l and episode:
  *   RM_ANCHOR_WRITE  (the group's anchor step; normally dense, idx = NULL):
  *       y_a = sum_{n in S} h_n Wd[:,n]   (S = every neuron when idx is NULL),   r_{l+1} = r_l + gate * y_a,
  *       and the call retains y_a in y_anchor and h_n[t] (n in S) in h_anchor.
@@ -283,7 +282,10 @@ int rm_get_info(const rm_ctx* ctx, const char* name, int* out);
 
 /* Profiling aid, available only in builds made with -DRM_PHASE_TIMING (RM_ERR_UNSUPPORTED otherwise): copies the
  * per-CTA clock stamps the fused layer kernel took at its phase boundaries (host_out: n int64 values, 32 per CTA).
- * Host-synchronous. */
+ * n = -(1 << 20) - m with m > 0 copies m values of the whole-step kernel's stamps instead, laid out
+ * [item < 64][CTA < 128][32 slots]: slots 0-9 are globaltimer values in ns (x ready, first gate/up product, gate/up
+ * complete, h sent, first down product, down complete, adds issued, arrival, normalisation start, normalisation done),
+ * the others clock counts of a -DRM_PHASE_TIMING=2 build.  Host-synchronous. */
 int rm_debug_phase_times(rm_ctx* ctx, long long* host_out, int n);
 
 const char* rm_status_string(int status);

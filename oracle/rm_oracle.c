@@ -7,7 +7,7 @@
  * table or helper with the CUDA sources.
  *
  * Conventions (all sizes in elements):
- *   x      [T,H]  bf16 bit patterns (uint16), the FFN input after RMSNorm (Sec. 4.1, "FFN input after RMSNorm")
+ *   x      [T,H]  bf16 bit patterns (uint16), the FFN input after RMSNorm (as Sec. 4.1 defines x)
  *   Wg, Wu [I,H]  bf16, row n = gate / up weights of intermediate neuron n
  *   Wd     [H,I]  bf16, column n = down-projection weights of neuron n
  *   r      [T,H]  fp32 residual (nullable => 0);  y [T,H] fp32
@@ -45,14 +45,14 @@ static inline uint16_t f32_to_bf16(float f) {
     return (uint16_t)(u >> 16);
 }
 
-/* GeLU, tanh form: 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3))).  The paper only says "post-GeGLU
- * activation" (Eq. 1); the tanh form is the reading fixed by the workload definition. */
+/* GeLU, tanh form: 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3))).  The paper names the activation only as the
+ * output of the GeGLU unit (Eq. 1); the tanh form is the reading fixed by the workload definition. */
 double orc_gelu_tanh(double g) {
     return 0.5 * g * (1.0 + tanh(0.7978845608028654 * (g + 0.044715 * g * g * g)));
 }
 
 /* One neuron's hidden activation for one token: h = gelu_tanh(g) * u with g = <x_t, Wg_n>, u = <x_t, Wu_n>
- * (Sec. 4.1: "compute only the selected neurons' hidden activations").  g and u are rounded to fp32 once,
+ * (Sec. 4.1: hidden activations of the selected neurons only).  g and u are rounded to fp32 once,
  * the activation is evaluated in double on those, and h is rounded to fp32 once. */
 static float hidden_one(const uint16_t* xt, const uint16_t* wg, const uint16_t* wu, int H) {
     double g = 0.0, u = 0.0;
@@ -126,8 +126,8 @@ void orc_dense_mlp(const uint16_t* x, const uint16_t* Wg, const uint16_t* Wu, co
 }
 
 /* Anchor-relative local update (Eq. 4): y_hat = y_anchor + (h_t^M - h_anchor^M) W_down[:,M], followed by the
- * output gate and the residual addition (Sec. 4.1: "the output follows the normal adaptive gate and residual
- * addition"): out = r + gate * y_hat, gate [H] per output channel, NULL = 1.  y_anchor [T,H] is the anchor step's
+ * output gate and the residual addition (Sec. 4.1, after Eq. 4: the model's usual adaptive gate, then the residual
+ * addition): out = r + gate * y_hat, gate [H] per output channel, NULL = 1.  y_anchor [T,H] is the anchor step's
  * FFN output before gate and residual, h_anchor [T,K] its activations on the mask.  With y_anchor = 0 and
  * h_anchor = 0 this is the zero-fill form. */
 void orc_anchor_mlp(const uint16_t* x, const uint16_t* Wg, const uint16_t* Wu, const uint16_t* Wd,
@@ -205,7 +205,7 @@ int orc_compact_bool(const uint8_t* m, int I, int32_t* idx_out) {
 }
 
 /* Selection flags of one record under a rule.  rule 1: score > threshold (strict).  rule 2: the k neurons with
- * the largest score, ties going to the lower index ("rank all neurons by c in descending order", Eq. 1 text;
+ * the largest score, ties going to the lower index (the text after Eq. 1 ranks the neurons by c, largest first;
  * K_l = ceil(rho_n * I) is computed by the caller).  score = record[n] * scale[n] (one fp32 multiply) when a
  * scale is given.  NaN ranks below every number; -0 equals +0. */
 typedef struct { float s; int32_t n; } orc_pair;
