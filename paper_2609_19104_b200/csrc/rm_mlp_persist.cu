@@ -399,15 +399,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     for (int e = tid; e < (G::END - G::OFF_HX) / 16; e += NTHREADS)
         reinterpret_cast<uint4*>(gbase + G::OFF_HX)[e] = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
-    if (warp < 8) {
-        // token rows T..63 of the cluster's x copies stay zero for the whole step (CTA j clears every 8th block)
-        for (int blk = j + CS * warp; blk < 2 * (H / 64); blk += CS * 8) {
-            unsigned char* img = reinterpret_cast<unsigned char*>(a.xbuf) + ((size_t)c * 2 * (H / 64) + blk) * X_BYTES;
-            for (int e = T * 8 + lane; e < NTOK * 8; e += 32) reinterpret_cast<uint4*>(img)[e] = make_uint4(0u, 0u, 0u, 0u);
-        }
-        __threadfence();
-        fence_proxy_async();
-    }
+    // (the cluster's x copies in global memory need no clearing: a copy brings token rows 0..T-1 only)
     tc_fence_before();
     __syncthreads();
     cluster_sync();
