@@ -135,6 +135,26 @@ __device__ __noinline__ uint32_t landed_stages(const int* count, uint32_t stage,
     }
     return ready;
 }
+__device__ __noinline__ void report_timeout(int* status, volatile int* abort_flag, int* sync, int line) {
+    rm_set_status_at(status, RM_ERR_TIMEOUT, (line << 12) | (int)(blockIdx.x & 0xfffu));
+    *abort_flag = 1;
+    atomicExch(sync + SYNC_ABORT, 1);
+}
+// The part of a bounded wait that runs when the phase was not complete at the first look.  Returns true when the waiter
+// has to give up: the wait ran out (status RM_ERR_TIMEOUT with the wait's source line and the CTA), or this CTA or the
+// grid is aborting.
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, int line, volatile int* abort_flag, int* sync, int* status) {
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(bar, parity)) return false;
+        if (i > 64) __nanosleep(32);
+        if ((i & 1023u) == 1023u && (*abort_flag || ((i & 16383u) == 16383u && ld_acquire_gpu(sync + SYNC_ABORT)))) {
+            *abort_flag = 1;
+            return true;
+        }
+    }
+    report_timeout(status, abort_flag, sync, line);
+    return true;
+}
 __device__ __forceinline__ void st_release_cta(int* p, int v) {         // shared memory
     asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
@@ -273,6 +293,27 @@ __device__ __forceinline__ void cur_next(Cur& k, const Env& e) {
     ++k.ni;
     ++k.item;
     cur_seek(k, e);
+}
+
+// The order in which every role takes a cluster's tiles: the gate/up part of the first tile, then per tile its down
+// part, with the next tile's gate/up part before it when that may run ahead and after it otherwise.  Written as a state
+// machine so that each part's code exists once per role (inlined at one call site).
+template <class FS, class FG, class FD>
+__device__ __forceinline__ void walk_tiles(const Env& env, int B, FS stop, FG gate_up, FD down) {
+    Cur g, d;
+    cur_init(g, env);
+    d = g;
+    int st = g.valid ? 3 : 0;                                      // 3: the very first gate/up part; 0: start of a round
+    for (;;) {
+        bool is_g;
+        if (st == 3) { is_g = true; st = 0; }
+        else if (st == 0) {
+            if (!d.valid || stop()) break;
+            if (g.valid && may_run_ahead(g, d, B)) { is_g = true; st = 1; } else { is_g = false; st = 2; }
+        } else if (st == 1) { is_g = false; st = 0; }               // the down part behind a gate/up part that ran ahead
+        else { st = 0; if (!g.valid) continue; is_g = true; }       // the gate/up part behind the down part
+        if (is_g) { gate_up(g); cur_next(g, env); } else { down(d); cur_next(d, env); }
+    }
 }
 
 // Shared memory: a fixed head (item counts, the tiles' neuron ids, barriers), the weight ring, then the h tile and the x
@@ -428,26 +469,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     const int XS = xs_n > XS_MAX ? XS_MAX : xs_n;                    // >= 2
     Env env{sP, sK, L, B, c, NC, a.x_ext};
 
+    // The kernel is large (every role is its own code) and the instruction caches are small: a wait's slow path and the
+    // error report live in functions of their own, and every role calls its per-tile code from one place, so that the
+    // loops that run all the time stay compact.
     bool gave_up = false;
     auto timed_out = [&](int line) {
-        rm_set_status_at(a.status, RM_ERR_TIMEOUT, (line << 12) | (int)(blockIdx.x & 0xfffu));
+        report_timeout(a.status, sAbort, a.sync, line);
         gave_up = true;
-        *sAbort = 1;
-        atomicExch(a.sync + SYNC_ABORT, 1);
     };
     auto wait_at = [&](uint32_t bar, uint32_t parity, int line) {
         if (gave_up) return;
         if (mbar_test_wait(bar, parity)) return;
-        for (uint32_t i = 0; i < (1u << 22); ++i) {
-            if (mbar_try_wait(bar, parity)) return;
-            if (i > 64) __nanosleep(32);
-            if ((i & 1023u) == 1023u && (*sAbort || ((i & 16383u) == 16383u && ld_acquire_gpu(a.sync + SYNC_ABORT)))) {
-                gave_up = true;
-                *sAbort = 1;
-                return;
-            }
-        }
-        timed_out(line);
+        gave_up = wait_slow(bar, parity, line, sAbort, a.sync, a.status);
     };
 #define WAIT(bar, parity) wait_at((bar), (parity), __LINE__)
 
@@ -547,17 +580,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 ++wcnt;
             }
         };
-        Cur g, d;
-        cur_init(g, env);
-        d = g;
-        if (g.valid) { load_g(g); cur_next(g, env); }
-        while (d.valid && !stop) {
-            const bool ahead = g.valid && may_run_ahead(g, d, B);
-            if (ahead) { load_g(g); cur_next(g, env); }
-            load_d(d);
-            cur_next(d, env);
-            if (!ahead && g.valid) { load_g(g); cur_next(g, env); }
-        }
+        walk_tiles(env, B, [&]() { return stop; }, load_g, load_d);
         cp_async_wait<0>();
     } else if (warp == W_PF) {
         // ================================================================ L2 prefetch: while the loaders wait for ring
@@ -693,17 +716,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     ++wcnt;
                 }
             };
-            Cur g, d;
-            cur_init(g, env);
-            d = g;
-            if (g.valid) { watch_g(g); cur_next(g, env); }
-            while (d.valid && !gave_up) {
-                const bool ahead = g.valid && may_run_ahead(g, d, B);
-                if (ahead) { watch_g(g); cur_next(g, env); }
-                watch_d(d);
-                cur_next(d, env);
-                if (!ahead && g.valid) { watch_g(g); cur_next(g, env); }
-            }
+            walk_tiles(env, B, [&]() { return gave_up; }, watch_g, watch_d);
         }
     } else if (warp == W_MMA) {
         // ================================================================ issuer (one warp; an elected lane issues)
@@ -729,9 +742,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             auto issue_g = [&](const Cur& k) {
                 const uint32_t d1 = tmem + (k.seq & 1) * (2 * NTOK);
                 for (int cc = 0; cc < NCH / 2; ++cc) {
+                    if (lane == 0) RM_TR(k.item, 7, cc);
                     need(__LINE__);
+                    if (lane == 0) RM_TR(k.item, 8, cc);
                     if (cc == 0 && k.i == 0 && lane == 0) RM_PS(k.item, 1);
                     tc_fence_after();
+                    if (lane == 0) RM_TR(k.item, 9, cc);
                     const uint64_t da = dW0 + (uint64_t)(ws * (SB >> 4)), db = dX0 + (uint64_t)(xs * (XSB >> 4));
                     if (elect_one()) {
                         RM_TR(k.item, 5, cc);
@@ -742,6 +758,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                         RM_TR(k.item, 6, cc);
                     }
                     __syncwarp();
+                    if (lane == 0) RM_TR(k.item, 10, cc);
                     if (++xs == XS) xs = 0;
                     if (++ws == NW) ws = 0;
                     ++stage;
@@ -793,17 +810,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 }
                 __syncwarp();
             };
-            Cur g, d;
-            cur_init(g, env);
-            d = g;
-            if (g.valid) { issue_g(g); cur_next(g, env); }
-            while (d.valid && !gave_up) {
-                const bool ahead = g.valid && may_run_ahead(g, d, B);
-                if (ahead) { issue_g(g); cur_next(g, env); }
-                issue_d(d);
-                cur_next(d, env);
-                if (!ahead && g.valid) { issue_g(g); cur_next(g, env); }
-            }
+            walk_tiles(env, B, [&]() { return gave_up; }, issue_g, issue_d);
         }
     } else {
         // ================================================================ epilogue (8 warps): GLU, h exchange, flush
@@ -891,18 +898,21 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         // x of a non-empty item is prepared right before the item's own tiles, or one non-empty item earlier when the
         // issuer may run that item's gate/up products ahead (item_may_run_ahead)
         int normed = -1;                                            // last item whose x has been prepared
-        auto prepare = [&](int q) {
-            if (q > normed) {
-                normed = q;
-                if (!item_ext(env, q / B)) norm_item(q);
-            }
-        };
         for (int item = 0; item < n_items && !stop; ++item) {
             if (item_run(env, item).ntiles > 0) {
-                prepare(item);
-                int q = item + 1;
-                while (q < n_items && q < item + B && item_run(env, q).ntiles == 0) ++q;
-                if (q < n_items && q < item + B && !stop) prepare(q);
+                // (one call site for the normalisation: first this item, then the look-ahead item if there is one)
+                int q = item;
+                for (int pass = 0; pass < 2 && !stop; ++pass) {
+                    if (pass == 1) {
+                        q = item + 1;
+                        while (q < n_items && q < item + B && item_run(env, q).ntiles == 0) ++q;
+                        if (!(q < n_items && q < item + B)) break;
+                    }
+                    if (q > normed) {
+                        normed = q;
+                        if (!item_ext(env, q / B)) norm_item(q);
+                    }
+                }
             }
             if (stop) break;
             const int l = item / B, b = item - l * B;
