@@ -733,6 +733,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             uint32_t stage = 0, ready = 0;                         // stages issued; stages known to have landed
             auto need = [&](int line) {
                 if (stage < ready || gave_up) return;
+                ready = (uint32_t)ld_relaxed_cta(sReady);            // (a call costs ~200 clocks here: look once before it)
+                if (stage < ready) return;
                 ready = landed_stages(sReady, stage, const_cast<const int*>(sAbort));
                 if (stage < ready) return;
                 if (*sAbort) { gave_up = true; return; }
