@@ -413,25 +413,36 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         *sAbort = 0;
         *sLoaded = 0;
         *sReady = 0;
-        int ts_max = 16, tiles_max = 0;
-        for (int l = 0; l < L; ++l) {
-            int S = 0;
-            for (int b = 0; b < B; ++b) S += sK[l * B + b];
-            int P = 0;
-            for (int b = 0; b < B; ++b) {
-                const int K = sK[l * B + b];
-                const Run r = cluster_run(K, P, S, c, NC);
-                sP[l * B + b] = r.start;                             // (sP then holds the run starts, sK the run lengths)
-                sK[l * B + b] = r.n;
-                P += K;
-                if (r.ntiles > 0) { const int ts = (r.n + r.ntiles - 1) / r.ntiles; ts_max = ts > ts_max ? ts : ts_max; }
-                tiles_max = r.ntiles > tiles_max ? r.ntiles : tiles_max;
+        sMisc[8] = 16;                                             // [8] largest tile of the step; [9] most tiles of an item
+        sMisc[9] = 0;
+    }
+    __syncthreads();
+    {
+        // This cluster's run in every item's list: one thread per item (sK holds the counts; afterwards sP the run starts
+        // and sK the run lengths).  One thread doing all of them took ~3 us of every launch.
+        Run r{0, 0, 0};
+        const bool mine = tid < n_items;
+        if (mine) {
+            const int l = tid / B, b = tid - l * B;
+            int S = 0, P = 0;
+            for (int b2 = 0; b2 < B; ++b2) {
+                const int K2 = sK[l * B + b2];
+                S += K2;
+                if (b2 < b) P += K2;
             }
+            r = cluster_run(sK[tid], P, S, c, NC);
+            if (r.ntiles > 0) atomicMax(const_cast<int*>(sMisc) + 8, (r.n + r.ntiles - 1) / r.ntiles);
+            atomicMax(const_cast<int*>(sMisc) + 9, r.ntiles);
         }
-        *sHslots = (ts_max + 15) & ~15;
+        __syncthreads();
+        if (mine) { sP[tid] = r.start; sK[tid] = r.n; }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        *sHslots = (sMisc[8] + 15) & ~15;
         // One episode and at most one tile per layer in this cluster: a layer's h is written after its gate/up products
         // and dead before the next layer's x exists, so the x ring may lie over the h tile and be twice as deep.
-        *sAlias = B == 1 && tiles_max <= 1;
+        *sAlias = B == 1 && sMisc[9] <= 1;
     }
     if (warp == W_MMA) tmem_alloc(s_tmem, 512);
     // the x copies bring token rows 0..T-1 only: the other rows of every ring stage stay zero from here on (when the ring
