@@ -32,7 +32,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per layer of a step, from ncu captures of the kernels that run these
 # workloads (one layer launch of the lean per-layer kernel; the whole-step kernel's figure divided by its layers)
-TRAFFIC_BYTES_PER_LAYER = {("pi0-stack-top25", 1): 6.794e6, ("large-stack-top20-refresh2", 5): 43.1e6}
+TRAFFIC_BYTES_PER_LAYER = {("pi0-stack-top25", 1): 6.794e6, ("pi0-stack-top25", 5): 6.62e6,
+                           ("large-stack-top20-refresh2", 5): 42.7e6}
 KERNEL_FAMILY = {0: "portable CUDA-core kernels (norm, gate/up, down)",
                  1: "fused_layer_kernel (lean per-layer cluster kernel, dependent-launch chained)",
                  2: "fused_layer_kernel, two tiles in flight",

@@ -24,18 +24,18 @@ inline bool use_fused(const rm_ctx* ctx, int B, int T) {
 
 // The whole-step kernel (variant 5).  Chosen by itself where it is measured ahead of the per-layer kernels (single
 // episodes; us per step, cold L2: lean per-layer kernel / streaming kernel / whole-step kernel):
-//   H = 2048, I = 16384:  K =  820: 265 / 572 / 299    1639: 377 / 577 / 308    3277: 603 / 577 / 342
-//                         4916: 827 / 587 / 522    8192: 1179 / 648 / 732    12288: 1641 / 1130 / 967
-//                         16384 (every neuron listed): 2160 / 1173 / 1192
-//   H = 1024, I = 4096:   K =  205: 170 / 341 / 210    820: 176 / 343 / 215    1024: 199 / 343 / 223
-//                         1229: 231 / 345 / 225    2048: 269 / 345 / 236    3072: 376 / 347 / 240    4096: 404 / 355 / 330
-// The streaming kernel's time steps up with every wave of 64-neuron tiles over the SMs (148 tiles per wave); the
-// whole-step kernel grows evenly with K and has a fixed cost of ~11-16 us per layer.  So, with K the caller's count
-// hint (the whole layer for a dense pass): at H = 1024 from 28 % of the neurons upwards; at H = 2048 from 7 % up to
-// 42 %, and again where the streaming kernel needs a second wave, up to 95 %.  Without a hint at H = 2048 it is
-// chosen as well (it adapts to the counts on the device), at H = 1024 the lean kernel.  Batches stay with the
-// streaming kernel.  `steps`: a whole stack (false: the one-layer entry, which would pay the kernel's set-up for a
-// single layer).
+//   H = 2048, I = 16384:  K =  492: 236 / 572 / 275    820: 266 / 572 / 279    1147: 362 / 572 / 279
+//                         1639: 377 / 577 / 287    3277: 604 / 577 / 330    4916: 828 / 586 / 516
+//                         8192: 1180 / 645 / 727    12288: 1640 / 1131 / 968    16384 (every neuron listed): 2170 / 1173 / 1198
+//   H = 1024, I = 4096:   K =  820: 176 / 343 / 193    902: 178 / 345 / 193    984: 201 / 344 / 197
+//                         1024: 199 / 343 / 197    1229: 231 / 345 / 199    2048: 269 / 345 / 209    4096: 410 / 355 / 303
+// The streaming kernel's time steps up with every wave of 64-neuron tiles over the SMs (148 tiles per wave), the lean
+// kernel's with every 64-neuron tile beyond 15; the whole-step kernel grows evenly with K and has a fixed cost of
+// ~10-15 us per layer.  So, with K the caller's count hint (the whole layer for a dense pass): at H = 1024 from 23.5 %
+// of the neurons upwards; at H = 2048 from 6 % up to 42 %, and again where the streaming kernel needs a second wave,
+// up to 95 %.  Without a hint at H = 2048 it is chosen as well (it adapts to the counts on the device), at H = 1024
+// the lean kernel.  Batches stay with the streaming kernel.  `steps`: a whole stack (false: the one-layer entry, which
+// would pay the kernel's set-up for a single layer).
 inline bool use_persist(const rm_ctx* ctx, int B, int T, bool masked, bool steps) {
     if (ctx->path == 1 || !rm_persist_supported(ctx, B, T)) return false;
     if (ctx->variant_override == 5) return true;
@@ -43,11 +43,11 @@ inline bool use_persist(const rm_ctx* ctx, int B, int T, bool masked, bool steps
     const long long I = ctx->g.I, K = masked ? ctx->count_hint : I;
     if (ctx->g.H == 2048) {
         if (K <= 0) return true;
-        if (K * 100 < I * 7) return false;
+        if (K * 100 < I * 6) return false;
         if (K * 100 <= I * 42) return true;
         return (K + 63) / 64 > ctx->sm_count && K * 100 <= I * 95;
     }
-    return K > 0 && K * 100 >= I * 28;
+    return K > 0 && K * 1000 >= I * 235;
 }
 
 inline void* persist_ws(const rm_ctx* ctx, void* ws, int B, int T) {
