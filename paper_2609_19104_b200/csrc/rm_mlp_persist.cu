@@ -1081,17 +1081,19 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     __syncwarp();
                 }
                 float* rb = a.r + (size_t)b * T * H + j * HS8 + q4 * 32 + lane;
+                // (rolled loops over 8 token columns at a time: this code runs once per layer, and the smaller it is the
+                // less of the other roles' loops it pushes out of the instruction cache)
+#pragma unroll 1
+                for (int q8 = 0; q8 < NMB * 4; ++q8) {
+                    const int mb = q8 >> 2, c8 = (q8 & 3) * 8;
+                    float hi[8], lo[8];
+                    const uint32_t col = tmem + G::D2_COL + d2b * (2 * NTOK) + mb * (2 * NTOK) + ch * 32 + c8 + ((uint32_t)(q4 * 32) << 16);
+                    tmem_ld8(col, hi);
+                    tmem_ld8(col + NTOK, lo);
+                    float* dst = rb + (size_t)(ch * 32 + c8) * H + mb * 128;
 #pragma unroll
-                for (int mb = 0; mb < NMB; ++mb) {
-                    float hi[32], lo[32];
-                    const uint32_t col = tmem + G::D2_COL + d2b * (2 * NTOK) + mb * (2 * NTOK) + ch * 32 + ((uint32_t)(q4 * 32) << 16);
-                    tmem_ld32(col, hi);
-                    tmem_ld32(col + NTOK, lo);
-#pragma unroll
-                    for (int r = 0; r < 32; ++r) {
-                        const int t = ch * 32 + r;
-                        if (t < T) red_add_f32(rb + (size_t)t * H + mb * 128, hi[r] + lo[r]);
-                    }
+                    for (int r = 0; r < 8; ++r)
+                        if (ch * 32 + c8 + r < T) red_add_f32(dst + (size_t)r * H, hi[r] + lo[r]);
                 }
                 tc_fence_before();
                 mbar_arrive(d2_empty(d2b));
