@@ -724,6 +724,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     if ((want & ~arrived) && !gave_up) timed_out(__LINE__);
                     fence_proxy_async_smem();
                     st_release_cta(sReady, (int)++stage);
+                    RM_TR(k.item, 11, ks0);
                     ++wcnt;
                 }
             };
@@ -797,9 +798,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 const int s0 = d_stage_first(ts, j, SPS, nst);
                 for (int ks0 = 0; ks0 < nst; ++ks0) {
                     const int s = d_stage(s0, ks0, nst);
+                    if (lane == 0) RM_TR(k.item, 14, ks0);
                     need(__LINE__);
                     if (ks0 == 0 && lane == 0) RM_PS(k.item, 4);
                     tc_fence_after();
+                    if (lane == 0) RM_TR(k.item, 12, ks0);
                     const uint64_t da = dA0 + (uint64_t)(ws * (SB >> 4)), dh = dh0 + (uint64_t)(s * (KPS * (2048 >> 4)));
                     if (elect_one()) {
 #pragma unroll
@@ -814,6 +817,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                         mma_commit(w_empty(ws));
                     }
                     __syncwarp();
+                    if (lane == 0) RM_TR(k.item, 13, ks0);
                     if (++ws == NW) ws = 0;
                     ++stage;
                 }
@@ -1055,6 +1059,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 }
                 if (et == 0 && i == 0) {
                     const long long e8 = RM_CLK();
+                    RM_TR(item, 15, 0);
                     RM_PS(item, 3);
                     RM_PC(item, 16, e1 - e0); RM_PC(item, 17, e2 - e1); RM_PC(item, 18, e3 - e2); RM_PC(item, 19, e4 - e3);
                     RM_PC(item, 20, e5 - e4); RM_PC(item, 21, e6 - e5); RM_PC(item, 22, e7 - e6); RM_PC(item, 23, e8 - e7);
