@@ -321,10 +321,10 @@ __device__ __forceinline__ void walk_tiles(const Env& env, int B, FS stop, FG ga
 template <int HS8>
 struct Geo {
     static constexpr int H = 8 * HS8;
-    // weight ring stages (measured at H = 2048, top-20 % / full list: 4 stages 420 / 1344 us per step, 5: 401 / 1288,
-    // 6: 398 / 1264); the x ring takes what the h tile leaves
-    static constexpr int NW = 6;
-    static constexpr int W_RING = NW * SB;
+    // weight ring stages: six, or eight when the x ring lies over the h tile (one episode, one tile per layer) and can
+    // spare the room.  (Measured at H = 2048, top-20 % / full list, before that mode existed: 4 stages 420 / 1344 us per
+    // step, 5: 401 / 1288, 6: 398 / 1264.)  The x ring takes what the weight ring and the h tile leave.
+    static constexpr int NW_MIN = 6, NW_MAX = 8;
     static constexpr int NSB = HS8 / 64;               // 64-column boxes per column slice
     static constexpr int NMB = HS8 / 128;              // 128-column output blocks per slice
     static constexpr int NCH = H / 64;                 // 64-column blocks of H
@@ -338,12 +338,11 @@ struct Geo {
     static constexpr int OFF_REC = OFF_IDX + 3 * CT * 4;
     static constexpr int OFF_MISC = OFF_REC + 4 * NT * 4;
     static constexpr int OFF_BAR = OFF_MISC + 128;
-    static constexpr int OFF_W = 9 * 1024;
-    static constexpr int OFF_EX = OFF_W + W_RING;
-    static constexpr int OFF_HX = OFF_EX + EXCH;
+    static constexpr int OFF_EX = 9 * 1024;
+    static constexpr int OFF_W = OFF_EX + EXCH;                // weight ring, then the h tile and the x ring up to END
     static constexpr int END = 231424;
     static constexpr int TOTAL = END + 1024;           // + slack for the 1024-byte alignment
-    static_assert(OFF_BAR + 640 <= OFF_W, "fixed head overflows");
+    static_assert(OFF_BAR + 640 <= OFF_EX, "fixed head overflows");
     static_assert(TOTAL <= 232448, "buffers exceed the shared memory of a CTA");
 };
 
@@ -351,11 +350,11 @@ template <int HS8>
 __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant__ PArgs a,
                                                           const __grid_constant__ CUtensorMap tmXext) {
     using G = Geo<HS8>;
-    constexpr int H = G::H, NSB = G::NSB, NMB = G::NMB, SPS = G::SPS, KPS = G::KPS, ND2 = G::ND2, NCH = G::NCH, NW = G::NW;
+    constexpr int H = G::H, NSB = G::NSB, NMB = G::NMB, SPS = G::SPS, KPS = G::KPS, ND2 = G::ND2, NCH = G::NCH;
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* gbase = smem_dyn + (base - smem_u32(smem_dyn));
-    const uint32_t sW = base + G::OFF_W, sH = base + G::OFF_HX;
+    const uint32_t sW = base + G::OFF_W;
     int* sK = reinterpret_cast<int*>(gbase + G::OFF_K);
     int* sP = reinterpret_cast<int*>(gbase + G::OFF_P);
     int* sIdx = reinterpret_cast<int*>(gbase + G::OFF_IDX);
@@ -401,7 +400,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     }
     __syncthreads();
     if (tid == 0) {
-        for (int s = 0; s < NW; ++s) { mbar_init(w_full(s), 128); mbar_init(w_empty(s), 1); }
+        for (int s = 0; s < G::NW_MAX; ++s) { mbar_init(w_full(s), 128); mbar_init(w_empty(s), 1); }
         for (int s = 0; s < XS_MAX; ++s) { mbar_init(x_full(s), 2); mbar_init(x_empty(s), 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(d1_full(s), 1); mbar_init(d2_full(s), 1); mbar_init(d2_empty(s), 256);
@@ -448,8 +447,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     // the x copies bring token rows 0..T-1 only: the other rows of every ring stage stay zero from here on (when the ring
     // lies over the h tile they hold old h values instead: the sums of the token columns T..63 are never used, the
     // epilogue writes zeros for them)
-    for (int e = tid; e < (G::END - G::OFF_HX) / 16; e += NTHREADS)
-        reinterpret_cast<uint4*>(gbase + G::OFF_HX)[e] = make_uint4(0u, 0u, 0u, 0u);
+    for (int e = tid; e < (G::END - G::OFF_W - G::NW_MIN * SB) / 16; e += NTHREADS)
+        reinterpret_cast<uint4*>(gbase + G::OFF_W + G::NW_MIN * SB)[e] = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
     // (the cluster's x copies in global memory need no clearing: a copy brings token rows 0..T-1 only)
     tc_fence_before();
@@ -475,8 +474,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     }
     const int h_half = *sHslots * 128;                             // bytes of the hi block (= of the lo block) of the h tile
     const bool alias = *sAlias != 0;
+    const int NW = alias ? G::NW_MAX : G::NW_MIN;       // (nine with three x stages: 2-5 % slower than eight with four)
+    const int OFF_HX = G::OFF_W + NW * SB;
+    const uint32_t sH = base + OFF_HX;
     const uint32_t sX = alias ? sH : sH + 2 * h_half;
-    int xs_n = (G::END - G::OFF_HX - (alias ? 0 : 2 * h_half)) / XSB;
+    int xs_n = (G::END - OFF_HX - (alias ? 0 : 2 * h_half)) / XSB;
     const int XS = xs_n > XS_MAX ? XS_MAX : xs_n;                    // >= 2
     Env env{sP, sK, L, B, c, NC, a.x_ext};
 
@@ -506,14 +508,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         // order in which the issuer consumes them
         const int lt = tid - W_LOAD0 * 32, lw = lt >> 5;
         const int pc = lt & 7, r0 = lt >> 3;                       // gate/up: 16-byte piece, rows r0 + 16 q
-        uint32_t wcnt = 0;
+        int ws = 0;                                                // ring slot of the next stage; its pass over the ring
+        uint32_t wpass = 0;
+        auto advance = [&]() { if (++ws == NW) { ws = 0; ++wpass; } };
         int loaded = 0;
         bool stop = false;                                         // agreed by all loader threads at the start of a tile
         // one lane per warp waits for the stage (128 threads testing one mbarrier take several hundred clocks)
         auto acquire = [&]() {
-            const int ws = wcnt % NW;
-            if (wcnt >= (uint32_t)NW) {
-                if (lane == 0) WAIT(w_empty(ws), ((wcnt / NW) - 1) & 1);
+            if (wpass >= 1) {
+                if (lane == 0) WAIT(w_empty(ws), (wpass - 1) & 1);
                 __syncwarp();
             }
             return sW + ws * SB;
@@ -562,8 +565,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     }
                 }
                 if (lt == 0) RM_TR(k.item, 1, cc);
-                cp_async_arrive_noinc(w_full(wcnt % NW));
-                ++wcnt;
+                cp_async_arrive_noinc(w_full(ws));
+                advance();
             }
         };
         auto load_d = [&](const Cur& k) {
@@ -587,8 +590,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     const uint32_t d = st + (piece >> 3) * (SPS * 128) + slot * 128 + (((piece & 7) ^ (slot & 7)) << 4);
                     cp_async16(d, wl + (size_t)(n < 0 ? 0 : n) * 3 * H, n >= 0);      // unused slots of the last step: zeros
                 }
-                cp_async_arrive_noinc(w_full(wcnt % NW));
-                ++wcnt;
+                cp_async_arrive_noinc(w_full(ws));
+                advance();
             }
         };
         walk_tiles(env, B, [&]() { return stop; }, load_g, load_d);
@@ -677,14 +680,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         // stages in the order in which the issuer consumes them, fences their cp.async data for the tensor core, and
         // publishes the count
         if (lane == 0) {
-            uint32_t wcnt = 0, xph = 0, stage = 0;
+            uint32_t wph = 0, xph = 0, stage = 0;                  // parities of the ring passes; stages published
+            int ws = 0;
             int xs = 0;
             auto watch_g = [&](const Cur& k) {
                 long long c_w = 0, c_x = 0, c_f = 0;
                 for (int cc = 0; cc < NCH / 2; ++cc) {
                     const long long q0 = RM_CLK();
-                    const uint32_t both = mbar_test_wait_2(w_full(wcnt % NW), (wcnt / NW) & 1, x_full(xs), xph);
-                    if (!(both & 1u)) WAIT(w_full(wcnt % NW), (wcnt / NW) & 1);
+                    const uint32_t both = mbar_test_wait_2(w_full(ws), wph, x_full(xs), xph);
+                    if (!(both & 1u)) WAIT(w_full(ws), wph);
                     const long long q1 = RM_CLK();
                     RM_TR(k.item, 3, cc);
                     if (!(both & 2u)) WAIT(x_full(xs), xph);
@@ -695,7 +699,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     const long long q3 = RM_CLK();
                     if (cc > 0) { c_w += q1 - q0; c_x += q2 - q1; c_f += q3 - q2; }
                     if (++xs == XS) { xs = 0; xph ^= 1; }
-                    ++wcnt;
+                    if (++ws == NW) { ws = 0; wph ^= 1; }
                 }
                 if (k.i == 0) { RM_PC(k.item, 13, c_w); RM_PC(k.item, 14, c_x); RM_PC(k.item, 15, c_f); }
             };
@@ -710,22 +714,22 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     bool w_ok;
                     if (want & ~arrived) {
                         // the stage's weights and all eight pieces in one round of tests
-                        const uint32_t m = mbar_test_wait_8_1(h_arr(0), k.seq & 1, w_full(wcnt % NW), (wcnt / NW) & 1);
+                        const uint32_t m = mbar_test_wait_8_1(h_arr(0), k.seq & 1, w_full(ws), wph);
                         arrived |= m & 0xffu;
                         w_ok = (m >> 8) & 1u;
                     } else {
-                        w_ok = mbar_test_wait(w_full(wcnt % NW), (wcnt / NW) & 1);
+                        w_ok = mbar_test_wait(w_full(ws), wph);
                     }
-                    if (!w_ok) WAIT(w_full(wcnt % NW), (wcnt / NW) & 1);
+                    if (!w_ok) WAIT(w_full(ws), wph);
                     for (uint32_t i = 0; (want & ~arrived) && i < (1u << 20) && !gave_up; ++i) {
-                        arrived |= mbar_test_wait_8_1(h_arr(0), k.seq & 1, w_full(wcnt % NW), (wcnt / NW) & 1) & 0xffu;
+                        arrived |= mbar_test_wait_8_1(h_arr(0), k.seq & 1, w_full(ws), wph) & 0xffu;
                         if ((i & 255u) == 255u && *sAbort) gave_up = true;
                     }
                     if ((want & ~arrived) && !gave_up) timed_out(__LINE__);
                     fence_proxy_async_smem();
                     st_release_cta(sReady, (int)++stage);
                     RM_TR(k.item, 11, ks0);
-                    ++wcnt;
+                    if (++ws == NW) { ws = 0; wph ^= 1; }
                 }
             };
             walk_tiles(env, B, [&]() { return gave_up; }, watch_g, watch_d);
@@ -840,7 +844,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
         const int ni_loc = m_row >> 1;                              // neuron of this lane among the CTA's 32
         const bool isup = lane & 1;
         float* sEx = reinterpret_cast<float*>(gbase + G::OFF_EX);   // [direction][token half][16 tokens][64 rows] fp32
-        unsigned char* gH = gbase + G::OFF_HX;
+        unsigned char* gH = gbase + OFF_HX;
         int seq = 0, ni = 0;
         bool stop = false;
         // Normalisation of an item's input into this cluster's copy of x: CTA j takes the token rows j, j + 8, ...,
