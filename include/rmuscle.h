@@ -251,8 +251,11 @@ int64_t rm_launch_count(const rm_ctx* ctx);
  *                         cluster kernel or RM_ERR_UNSUPPORTED
  *   "pdl"                 1 = chain the layers of a step with programmatic dependent launch (default)
  *   "neurons_per_cluster" active neurons a cluster should get before another cluster is used (default 64)
- *   "count_hint"          expected active neurons per layer and episode; lets a launch use only as many clusters
- *                         as that needs, so that the next layer's CTAs can become resident early (0 = unknown)
+ *   "count_hint"          expected active neurons per layer and episode: the kernel family is chosen by it, and a
+ *                         per-layer launch uses only as many clusters as it needs, so that the next layer's CTAs can
+ *                         become resident early.  0 (default) = the k of the last top-k or group rm_mask_compact call
+ *                         made through this context, if there was one, else unknown (the counts themselves stay on the
+ *                         device and are never read by the host)
  *   "max_clusters"        cap on the clusters per launch (0 = none)
  *   "l2_prefetch"         warp-specialised kernel: number of tiles ahead for which the weights are pulled into L2
  *                         (0 = off, the default)

@@ -40,7 +40,7 @@ inline bool use_persist(const rm_ctx* ctx, int B, int T, bool masked, bool steps
     if (ctx->path == 1 || !rm_persist_supported(ctx, B, T)) return false;
     if (ctx->variant_override == 5) return true;
     if (ctx->variant_override != 0 || B > ctx->persist_max_b || !steps) return false;
-    const long long I = ctx->g.I, K = masked ? ctx->count_hint : I;
+    const long long I = ctx->g.I, K = masked ? rm_effective_count_hint(ctx) : I;
     if (ctx->g.H == 2048) {
         if (K <= 0) return true;
         if (K * 100 < I * 5) return false;
@@ -66,7 +66,7 @@ inline bool use_stream(const rm_ctx* ctx, bool masked, int B, int T, bool anchor
     if (ctx->path == 1 || !rm_stream_supported(ctx, B, T)) return false;
     if (ctx->variant_override == 4) return true;
     if (ctx->variant_override != 0 && ctx->variant_override != 5) return false;   // 5: a call the whole-step kernel does not cover
-    const int per_episode = masked ? ctx->count_hint : ctx->g.I;
+    const int per_episode = masked ? rm_effective_count_hint(ctx) : ctx->g.I;
     if (per_episode <= 0) return false;
     const long long tiles = (long long)((per_episode + 63) / 64) * B;
     return tiles >= (anchor_write && ctx->stream_min_tiles < 112 ? 112 : ctx->stream_min_tiles);
@@ -111,6 +111,7 @@ int rm_create(rm_ctx** out, const rm_model_desc* desc) {
     c->use_pdl = 1;
     c->npc_target = 64;
     c->count_hint = 0;
+    c->count_hint_seen = 0;
     c->max_clusters_override = 0;
     c->variant_override = 0;
     c->l2_prefetch = 0;
@@ -240,6 +241,8 @@ int rm_mask_compact(rm_ctx* ctx, const rm_mask_src* src, int32_t* idx_out, int32
     }
     if (!all_aligned({idx_out, src->scale})) return RM_ERR_ALIGN;
     if (src->scale && src->kind != RM_SRC_SCORE_F32) return RM_ERR_INVALID_ARG;
+    if ((src->reduce == RM_REDUCE_TOPK || src->reduce == RM_REDUCE_GROUP) && src->I == ctx->g.I)
+        ctx->count_hint_seen = src->k < src->I ? src->k : src->I;
     return rm_launch_mask_compact(ctx, src, idx_out, count_out, stride, static_cast<cudaStream_t>(stream));
 }
 

@@ -39,6 +39,7 @@ struct rm_ctx {
     int use_pdl;                           // chain layers with programmatic dependent launch
     int npc_target;                        // neurons per cluster aimed for when spreading a layer
     int count_hint;                        // expected active neurons per layer and episode (0: unknown)
+    int count_hint_seen;                   // k of the last top-k / group compaction through this context (0: none yet)
     int max_clusters_override;             // > 0: cap on clusters per launch
     int l2_prefetch;                       // L2 prefetch distance (tiles) of the warp-specialised kernel
     int stream_min_tiles;                  // launches with at least this many 64-neuron tiles use the streaming variant
@@ -55,6 +56,10 @@ struct rm_ctx {
     int persist_sync_dirty;                // a launch may have left them at an unknown count: clear before the next one
     alignas(64) unsigned char persist_tm[128];   // CUtensorMap of the clusters' x copies in the workspace
 };
+
+// The count the kernel selection works with: the caller's hint, else what the last compaction through this context
+// was asked to keep (the counts themselves stay on the device; the host never reads them).
+inline int rm_effective_count_hint(const rm_ctx* ctx) { return ctx->count_hint > 0 ? ctx->count_hint : ctx->count_hint_seen; }
 
 extern int rm_last_cuda_error;            // cudaError_t of the last failed runtime call (diagnostics; "last_cuda_error")
 #define RM_CUDA_TRY(expr)                                  \

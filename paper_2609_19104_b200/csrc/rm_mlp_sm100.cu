@@ -1643,7 +1643,7 @@ int rm_launch_layer_fused(rm_ctx* ctx, const rm_layer_args& la, float* zero_buf,
     a.gate = la.gate;
     // Tiles of 64 neurons in this launch, when the host knows the number of active neurons (dense calls, or the
     // caller's hint); 0 = unknown.
-    const int per_episode = la.count ? ctx->count_hint : ctx->g.I;
+    const int per_episode = la.count ? rm_effective_count_hint(ctx) : ctx->g.I;
     const long long tiles = per_episode > 0 ? (long long)((per_episode + NT - 1) / NT) * la.B : 0;
     // Variant.  H = 1024: the lean kernel for every launch (112 KB and 107 registers: two CTAs per SM, so a cluster's
     // exchange waits are covered by its SM-mate and consecutive layers overlap); measured, 33 of its clusters are

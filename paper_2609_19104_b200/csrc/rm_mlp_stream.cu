@@ -692,7 +692,7 @@ int rm_launch_layer_stream(rm_ctx* ctx, const rm_layer_args& la, __nv_bfloat16* 
     a.h_anchor = la.h_anchor;
     a.h_stride = la.h_stride;
     a.gate = la.gate;
-    const int per_episode = la.count ? ctx->count_hint : g.I;
+    const int per_episode = la.count ? rm_effective_count_hint(ctx) : g.I;
     long long tiles = per_episode > 0 ? (long long)((per_episode + NT - 1) / NT) * la.B : 0;
     int n_ctas = ctx->sm_count;
     if (tiles > 0 && tiles < n_ctas) n_ctas = (int)tiles;

@@ -103,3 +103,28 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable(l
     assert_close(y.cpu().numpy(), oracle.dense_mlp(x, model.Wg[0], model.Wu[0], model.Wd[0], r), "after a timeout")
     model.close()
     ctx.close()
+
+
+def test_without_a_hint_the_kernel_family_follows_the_last_compaction(lib):
+    """count_hint = 0: the k of the last top-k rm_mask_compact call through the context stands in for the hint, so a
+    caller who never sets the option gets the same kernel family as one who does (the result is checked too)."""
+    import torch
+    w = wl.scaled(wl.config1(), L=2)
+    L, H, I, T = w.L, w.H, w.I, w.T
+    model = Model(lib, w, B_max=8)
+    ctx = model.ctx
+    for B, k, family in ((8, I // 4, 4), (1, I // 2, 5), (1, I // 10, 1)):
+        rec = torch.rand(B * L, I, dtype=torch.float32, device="cuda")
+        idx = torch.zeros(B * L, I, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros(B * L, dtype=torch.int32, device="cuda")
+        ctx.rm_mask_compact([rec], lib.RM_SRC_SCORE_F32, lib.RM_REDUCE_TOPK, idx, cnt, I, n_lists=B * L, k=k)
+        r0 = np.stack([wl.bf16_bits_to_f32(wl.step_input(w, 1, episode=b)) for b in range(B)])
+        out = torch.empty(B, T, H, dtype=torch.float32, device="cuda")
+        ctx.rm_action_expert_step(model.packed, dev(r0), idx, cnt, I, out, B=B, T=T)
+        assert ctx.rm_get_info("last_variant") == family, (B, k, ctx.rm_get_info("last_variant"))
+        h_idx, h_cnt = idx.cpu().numpy().reshape(B, L, I), cnt.cpu().numpy().reshape(B, L)
+        for b in range(B):
+            want = oracle.step(model.Wg, model.Wu, model.Wd, r0[b], h_idx[b], h_cnt[b])
+            assert_close(out.cpu().numpy()[b], want, f"B={B}, k={k}, episode {b}")
+    assert ctx.rm_device_status() == 0
+    model.close()
