@@ -485,9 +485,19 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
             if (m == 0) bulk_wait_read_all();
             named_barrier(1, 128);                                 // the exchange area is free for the next tile
         }
-    } else if (warp == 8 && lane == 0) {
-        // ================================================================ issuer (one thread)
+    } else if (warp == 8) {
+        // ================================================================ issuer: the whole warp runs the loop and one
+        // elected lane issues (a loop that only lane 0 runs costs 100-150 clocks more per stage, and the tensor pipe
+        // idles while the issuing thread does anything else).  The test of the next stage's barrier (~200 clocks even
+        // when the data is there) is started behind the products of the current stage, so that it runs while they do.
         uint32_t blk = 0, mbc = 0;
+        bool next_ok = false;                                      // the stage about to be used is known to have landed
+        auto stage_ready = [&]() {
+            if (!next_ok) wait_bar(full(blk % NSTAGE), (blk / NSTAGE) & 1);
+        };
+        auto look_ahead = [&]() {
+            next_ok = __all_sync(0xffffffffu, mbar_test_wait(full((blk + 1) % NSTAGE), ((blk + 1) / NSTAGE) & 1));
+        };
         for (int k = 0;; ++k) {
             const int g = (int)blockIdx.x + k * (int)gridDim.x;
             if (g >= tiles_total) break;
@@ -495,39 +505,51 @@ __global__ void __launch_bounds__(SE, 1) stream_tile_kernel(const StreamArgs a, 
             tc_fence_after();
             for (int kb = 0; kb < KBN; ++kb, ++blk) {
                 const uint32_t st = sRing + (blk % NSTAGE) * STAGE;
-                wait_bar(full(blk % NSTAGE), (blk / NSTAGE) & 1);
-                if (kb == 0) RM_ST(3);
-                if (kb == KBN - 1) RM_ST(4);
+                stage_ready();
+                if (lane == 0) {
+                    if (kb == 0) RM_ST(3);
+                    if (kb == KBN - 1) RM_ST(4);
+                }
                 if (GATHER) fence_proxy_async_smem();
                 tc_fence_after();
+                if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    mma_bf16_ss(tmem_d1, desc_k | desc_addr(st + ks * 32), desc_k | desc_addr(st + W_BYTES + ks * 32),
-                                IDESC_GU, (kb | ks) != 0);
-                mma_commit(empty(blk % NSTAGE));
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_bf16_ss(tmem_d1, desc_k | desc_addr(st + ks * 32), desc_k | desc_addr(st + W_BYTES + ks * 32),
+                                    IDESC_GU, (kb | ks) != 0);
+                    mma_commit(empty(blk % NSTAGE));
+                }
+                __syncwarp();
+                look_ahead();
             }
-            mma_commit(d1_full);
-            RM_ST(5);
+            if (elect_one()) mma_commit(d1_full);
+            __syncwarp();
+            if (lane == 0) RM_ST(5);
             wait_bar(h_full, k & 1);
-            RM_ST(6);
+            if (lane == 0) RM_ST(6);
             for (int mb = 0; mb < MBN; ++mb, ++blk, ++mbc) {
                 const int slot = mbc & 1;
                 const uint32_t st = sRing + (blk % NSTAGE) * STAGE;
                 if (mbc >= 2) wait_bar(d2_free(slot), ((mbc >> 1) - 1) & 1);
-                wait_bar(full(blk % NSTAGE), (blk / NSTAGE) & 1);
+                stage_ready();
                 if (GATHER) fence_proxy_async_smem();
                 tc_fence_after();
+                if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t aa = desc_mn | desc_addr(st + ks * 2048);
-                    mma_bf16_ss(tmem_d1 + NTOK * (1 + slot), aa, desc_mn | desc_addr(sHT + ks * 2048), IDESC_DN, ks != 0);
-                    mma_bf16_ss(tmem_d1 + NTOK * (1 + slot), aa, desc_mn | desc_addr(sHT + NT * 128 + ks * 2048), IDESC_DN, true);
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t aa = desc_mn | desc_addr(st + ks * 2048);
+                        mma_bf16_ss(tmem_d1 + NTOK * (1 + slot), aa, desc_mn | desc_addr(sHT + ks * 2048), IDESC_DN, ks != 0);
+                        mma_bf16_ss(tmem_d1 + NTOK * (1 + slot), aa, desc_mn | desc_addr(sHT + NT * 128 + ks * 2048), IDESC_DN, true);
+                    }
+                    mma_commit(empty(blk % NSTAGE));
+                    mma_commit(d2_full(slot));
                 }
-                mma_commit(empty(blk % NSTAGE));
-                mma_commit(d2_full(slot));
+                __syncwarp();
+                look_ahead();
             }
-            mma_commit(h_free);
-            RM_ST(7);
+            if (elect_one()) mma_commit(h_free);
+            __syncwarp();
+            if (lane == 0) RM_ST(7);
         }
     }
     tc_fence_before();
