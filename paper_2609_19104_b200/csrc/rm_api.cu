@@ -25,15 +25,16 @@ inline bool use_fused(const rm_ctx* ctx, int B, int T) {
 // The whole-step kernel (variant 5).  Chosen by itself where it is measured ahead of the per-layer kernels (single
 // episodes; us per step, cold L2: lean per-layer kernel / streaming kernel / whole-step kernel):
 //   H = 2048, I = 16384:  K =  492: 236 / 572 / 262    820: 265 / 571 / 262    1147: 360 / 571 / 266
-//                         1639: 377 / 577 / 275    3277: 604 / 577 / 320    4916: 829 / 586 / 496
-//                         8192: 1180 / 645 / 703    12288: 1637 / 1134 / 942    16384 (every neuron listed): 2162 / 1173 / 1169
+//                         1639: 377 / 577 / 273    3277: 605 / 577 / 308    4916: 829 / 554 / 495
+//                         6554: 957 / 577 / 548    7373: 1064 / 605 / 625    8192: 1181 / 626 / 706
+//                         12288: 1632 / 1139 / 949    14746: 1964 / 1115 / 1125    16384 (every neuron listed): 2159 / 1130 / 1178
 //   H = 1024, I = 4096:   K =  820: 176 / 344 / 188    902: 178 / 345 / 190    984: 200 / 343 / 193
 //                         1024: 199 / 345 / 193    1229: 231 / 345 / 195    2048: 270 / 346 / 203    4096: 404 / 355 / 291
 // The streaming kernel's time steps up with every wave of 64-neuron tiles over the SMs (148 tiles per wave), the lean
 // kernel's with every 64-neuron tile beyond 15; the whole-step kernel grows evenly with K and has a fixed cost of
 // ~10-15 us per layer.  So, with K the caller's count hint (the whole layer for a dense pass): at H = 1024 from 23.5 %
 // of the neurons upwards; at H = 2048 from 5 % up to 42 %, and again where the streaming kernel needs a second wave,
-// up to 95 %.  Without a hint at H = 2048 it is chosen as well (it adapts to the counts on the device), at H = 1024
+// up to 88 %.  Without a hint at H = 2048 it is chosen as well (it adapts to the counts on the device), at H = 1024
 // the lean kernel.  Batches stay with the streaming kernel.  `steps`: a whole stack (false: the one-layer entry, which
 // would pay the kernel's set-up for a single layer).
 inline bool use_persist(const rm_ctx* ctx, int B, int T, bool masked, bool steps) {
@@ -45,7 +46,7 @@ inline bool use_persist(const rm_ctx* ctx, int B, int T, bool masked, bool steps
         if (K <= 0) return true;
         if (K * 100 < I * 5) return false;
         if (K * 100 <= I * 42) return true;
-        return (K + 63) / 64 > ctx->sm_count && K * 100 <= I * 95;
+        return (K + 63) / 64 > ctx->sm_count && K * 100 <= I * 88;
     }
     return K > 0 && K * 1000 >= I * 235;
 }
