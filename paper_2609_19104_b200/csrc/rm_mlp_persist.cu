@@ -253,7 +253,7 @@ struct Cur {
     int use;                           // uses of the cluster's x buffer before this item
     bool valid;
 };
-struct Env { const int* sRunStart; const int* sRunN; int L, B, c, NC, x_ext; };   // this cluster's run in every item's list,
+struct Env { const int* sRunStart; const int* sRunN; int L, B, c, NC, x_ext, serial; };   // this cluster's run in every item's list,
                                                                                   // worked out once at the start of the kernel
 __device__ __forceinline__ Run item_run(const Env& e, int item) {
     Run r;
@@ -309,7 +309,7 @@ __device__ __forceinline__ void walk_tiles(const Env& env, int B, FS stop, FG ga
         if (st == 3) { is_g = true; st = 0; }
         else if (st == 0) {
             if (!d.valid || stop()) break;
-            if (g.valid && may_run_ahead(g, d, B)) { is_g = true; st = 1; } else { is_g = false; st = 2; }
+            if (g.valid && !env.serial && may_run_ahead(g, d, B)) { is_g = true; st = 1; } else { is_g = false; st = 2; }
         } else if (st == 1) { is_g = false; st = 0; }               // the down part behind a gate/up part that ran ahead
         else { st = 0; if (!g.valid) continue; is_g = true; }       // the gate/up part behind the down part
         if (is_g) { gate_up(g); cur_next(g, env); } else { down(d); cur_next(d, env); }
@@ -379,6 +379,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     auto x_free = [&](int s) { return bar0 + 512 + 8 * s; };
     const uint32_t h_free = bar0 + 536, g_all = bar0 + 544;
     auto h_arr = [&](int p) { return bar0 + 552 + 8 * p; };        // CS: piece p of the tile's h has arrived in this CTA
+    const uint32_t d_local = bar0 + 616;                           // this CTA's down products of a tile are complete
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int j = (int)cluster_ctarank(), c = (int)cluster_id_x(), NC = (int)cluster_count_x();
@@ -407,7 +408,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             mbar_init(x_ready(s), CS); mbar_init(x_free(s), CS);
         }
         for (int p2 = 0; p2 < CS; ++p2) mbar_init(h_arr(p2), 1);
-        mbar_init(h_free, CS); mbar_init(g_all, CS);
+        mbar_init(h_free, CS); mbar_init(g_all, CS); mbar_init(d_local, 1);
         fence_mbar_init();
         *sAbort = 0;
         *sLoaded = 0;
@@ -439,9 +440,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     }
     if (tid == 0) {
         *sHslots = (sMisc[8] + 15) & ~15;
-        // One episode and at most one tile per layer in this cluster: a layer's h is written after its gate/up products
-        // and dead before the next layer's x exists, so the x ring may lie over the h tile and be twice as deep.
-        *sAlias = B == 1 && sMisc[9] <= 1;
+        // One episode and the tiles taken strictly one after the other (gate/up, GLU, down): a tile's h is written after
+        // its gate/up products and dead before the next tile's x copies start (they wait for this CTA's down products), so
+        // the x ring lies over the h tile, and the room that saves goes to the weight ring.  With one tile per layer and
+        // cluster nothing is lost by that order.  With several it gives up running the next tile's gate/up products under
+        // this tile's GLU and down products: at H = 2048 the deeper rings are worth more (full lists: 1177 -> 1076 us per
+        // step), at H = 1024, where a tile's gate/up part is half as long, less (292 -> 320).
+        *sAlias = B == 1 && (sMisc[9] <= 1 || HS8 == 256);
     }
     if (warp == W_MMA) tmem_alloc(s_tmem, 512);
     // the x copies bring token rows 0..T-1 only: the other rows of every ring stage stay zero from here on (when the ring
@@ -480,7 +485,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     const uint32_t sX = alias ? sH : sH + 2 * h_half;
     int xs_n = (G::END - OFF_HX - (alias ? 0 : 2 * h_half)) / XSB;
     const int XS = xs_n > XS_MAX ? XS_MAX : xs_n;                    // >= 2
-    Env env{sP, sK, L, B, c, NC, a.x_ext};
+    Env env{sP, sK, L, B, c, NC, a.x_ext, alias ? 1 : 0};
 
     // The kernel is large (every role is its own code) and the instruction caches are small: a wait's slow path and the
     // error report live in functions of their own, and every role calls its per-tile code from one place, so that the
@@ -656,6 +661,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     }
                 }
                 const unsigned char* img = reinterpret_cast<const unsigned char*>(a.xbuf) + (size_t)(c * 2 + slot) * NCH * X_BYTES;
+                // (x ring over the h tile: the previous tile's h is read until this CTA's down products are complete)
+                if (alias && k.seq >= 1) WAIT(d_local, (k.seq - 1) & 1);
                 for (int cc = xq >> 1; cc < NCH / 2; cc += 2) {
                     if (n >= (uint32_t)XS) WAIT(x_empty(xs), ph ^ 1);
                     if (half == 0) RM_TR(k.item, 2, cc);
@@ -826,6 +833,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     ++stage;
                 }
                 if (elect_one()) {
+                    if (alias) mma_commit(d_local);
                     mma_commit_mc(h_free, 0xff);
                     if (k.i == k.run.ntiles - 1) { mma_commit(d2_full(d2b)); RM_PS(k.item, 25); }
                 }
@@ -1111,7 +1119,24 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 // below, and a release is cumulative (the pattern of a grid-wide barrier: sync, then one thread fences)
                 stop = named_barrier_or(1, 256, gave_up || *sAbort);
             }
-            if (et == 0) { red_release_gpu(a.per_item ? a.sync + SYNC_ITEM + item : a.sync + b, 1); RM_PS(item, 7); }
+            if (et == 0) {
+                // The episode's counter adds up the arrivals of all layers, and "n_ctas (l + 1) arrivals" means "every CTA has
+                // added its part of layer l" only if nobody arrives for layer l before every CTA has arrived for layer l - 1.
+                // A CTA with tiles in layer l has waited for exactly that before normalising; a CTA whose cluster has none
+                // (lists shorter than the number of clusters) would otherwise run through its empty layers at once, and its
+                // early arrivals would stand in for a slower CTA's.
+                if (run.ntiles == 0 && !a.per_item && l > 0 && !gave_up) {
+                    const int target = a.sync_base[b] + n_ctas * l;
+                    bool ok = false;
+                    for (uint32_t i = 0; i < (1u << 21); ++i) {
+                        if (ld_acquire_gpu(a.sync + b) >= target) { ok = true; break; }
+                        if ((i & 255u) == 255u && (*sAbort || ld_acquire_gpu(a.sync + SYNC_ABORT))) break;
+                    }
+                    if (!ok) { if (!*sAbort && !ld_acquire_gpu(a.sync + SYNC_ABORT)) timed_out(__LINE__); gave_up = true; *sAbort = 1; }
+                }
+                red_release_gpu(a.per_item ? a.sync + SYNC_ITEM + item : a.sync + b, 1);
+                RM_PS(item, 7);
+            }
         }
     }
 #undef WAIT

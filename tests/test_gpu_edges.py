@@ -128,3 +128,14 @@ def test_without_a_hint_the_kernel_family_follows_the_last_compaction(lib):
             assert_close(out.cpu().numpy()[b], want, f"B={B}, k={k}, episode {b}")
     assert ctx.rm_device_status() == 0
     model.close()
+
+
+@pytest.mark.parametrize("shape", [dict(H=1024, I=64, T=7, L=5, density=0.05, config=206),
+                                   dict(H=2048, I=520, T=64, L=5, density=0.01, config=229),
+                                   dict(H=1024, I=200, T=33, L=5, density=0.02, config=231)])
+def test_lists_shorter_than_the_number_of_clusters_through_a_deep_stack(lib, shape):
+    """A handful of active neurons per layer: most clusters of the whole-step kernel have nothing to do in a layer and
+    must not arrive for it before every CTA has arrived for the layer before (their early arrivals stood in for slower
+    CTAs' once; a randomised sweep found it)."""
+    for rep in range(3):
+        step_case(lib, B=1, variant=5, **shape)
