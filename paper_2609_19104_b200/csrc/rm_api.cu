@@ -25,18 +25,19 @@ inline bool use_fused(const rm_ctx* ctx, int B, int T) {
 // The whole-step kernel (variant 5).  Chosen by itself where it is measured ahead of the per-layer kernels (single
 // episodes; us per step, cold L2: lean per-layer kernel / streaming kernel / whole-step kernel):
 //   H = 2048, I = 16384:  K =  492: 236 / 572 / 262    820: 265 / 571 / 262    1147: 360 / 571 / 266
-//                         1639: 377 / 577 / 273    3277: 605 / 577 / 308    4916: 829 / 554 / 495
-//                         6554: 957 / 577 / 548    7373: 1064 / 605 / 625    8192: 1181 / 626 / 706
-//                         12288: 1632 / 1139 / 949    14746: 1964 / 1115 / 1125    16384 (every neuron listed): 2159 / 1130 / 1178
+//                         1639: 377 / 577 / 273    3277: 605 / 577 / 308    4916: 829 / 554 / 462
+//                         6882: 1058 / 584 / 532    7373: 1066 / 605 / 544    8192: 1183 / 624 / 652
+//                         9012: 1279 / 665 / 687    9503: 1301 / 1039 / 701    12288: 1632 / 1139 / 871
+//                         14746: 1962 / 1114 / 960    16384 (every neuron listed): 2158 / 1130 / 1081
 //   H = 1024, I = 4096:   K =  820: 176 / 344 / 188    902: 178 / 345 / 190    984: 200 / 343 / 193
-//                         1024: 199 / 345 / 193    1229: 231 / 345 / 195    2048: 270 / 346 / 203    4096: 404 / 355 / 291
+//                         1024: 199 / 345 / 193    1229: 231 / 345 / 195    2048: 270 / 346 / 203    4096: 404 / 337 / 291
 // The streaming kernel's time steps up with every wave of 64-neuron tiles over the SMs (148 tiles per wave), the lean
 // kernel's with every 64-neuron tile beyond 15; the whole-step kernel grows evenly with K and has a fixed cost of
 // ~10-15 us per layer.  So, with K the caller's count hint (the whole layer for a dense pass): at H = 1024 from 23.5 %
-// of the neurons upwards; at H = 2048 from 5 % up to 42 %, and again where the streaming kernel needs a second wave,
-// up to 88 %.  Without a hint at H = 2048 it is chosen as well (it adapts to the counts on the device), at H = 1024
-// the lean kernel.  Batches stay with the streaming kernel.  `steps`: a whole stack (false: the one-layer entry, which
-// would pay the kernel's set-up for a single layer).
+// of the neurons upwards; at H = 2048 from 5 % upwards, except where the streaming kernel's single wave is nearly full
+// (47 % of the neurons up to 148 tiles).  Without a hint at H = 2048 it is chosen as well (it adapts to the counts on
+// the device), at H = 1024 the lean kernel.  Batches stay with the streaming kernel.  `steps`: a whole stack (false:
+// the one-layer entry, which would pay the kernel's set-up for a single layer).
 inline bool use_persist(const rm_ctx* ctx, int B, int T, bool masked, bool steps) {
     if (ctx->path == 1 || !rm_persist_supported(ctx, B, T)) return false;
     if (ctx->variant_override == 5) return true;
@@ -45,8 +46,7 @@ inline bool use_persist(const rm_ctx* ctx, int B, int T, bool masked, bool steps
     if (ctx->g.H == 2048) {
         if (K <= 0) return true;
         if (K * 100 < I * 5) return false;
-        if (K * 100 <= I * 42) return true;
-        return (K + 63) / 64 > ctx->sm_count && K * 100 <= I * 88;
+        return !(K * 100 > I * 47 && (K + 63) / 64 <= ctx->sm_count);
     }
     return K > 0 && K * 1000 >= I * 235;
 }

@@ -155,6 +155,16 @@ __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, int line, 
     report_timeout(status, abort_flag, sync, line);
     return true;
 }
+// A bounded wait for a counter in global memory, out of line (for the path that is rarely taken).  Returns true when
+// the waiter has to give up.
+__device__ __noinline__ bool counter_wait_slow(const int* counter, int target, int line, volatile int* abort_flag, int* sync, int* status) {
+    for (uint32_t i = 0; i < (1u << 21); ++i) {
+        if (ld_acquire_gpu(counter) >= target) return false;
+        if ((i & 255u) == 255u && (*abort_flag || ld_acquire_gpu(sync + SYNC_ABORT))) { *abort_flag = 1; return true; }
+    }
+    report_timeout(status, abort_flag, sync, line);
+    return true;
+}
 __device__ __forceinline__ void st_release_cta(int* p, int v) {         // shared memory
     asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
@@ -479,6 +489,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     }
     const int h_half = *sHslots * 128;                             // bytes of the hi block (= of the lo block) of the h tile
     const bool alias = *sAlias != 0;
+    const bool alias_multi = alias && sMisc[9] > 1;             // ... and some item has several tiles (see d_local)
     const int NW = alias ? G::NW_MAX : G::NW_MIN;       // (nine with three x stages: 2-5 % slower than eight with four)
     const int OFF_HX = G::OFF_W + NW * SB;
     const uint32_t sH = base + OFF_HX;
@@ -661,8 +672,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     }
                 }
                 const unsigned char* img = reinterpret_cast<const unsigned char*>(a.xbuf) + (size_t)(c * 2 + slot) * NCH * X_BYTES;
-                // (x ring over the h tile: the previous tile's h is read until this CTA's down products are complete)
-                if (alias && k.seq >= 1) WAIT(d_local, (k.seq - 1) & 1);
+                // (x ring over the h tile: the previous tile's h is read until this CTA's down products are complete.  With one
+                // tile per layer the next tile's x exists only after every CTA's adds of this layer, so nothing to wait for.)
+                if (alias_multi && k.seq >= 1) WAIT(d_local, (k.seq - 1) & 1);
                 for (int cc = xq >> 1; cc < NCH / 2; cc += 2) {
                     if (n >= (uint32_t)XS) WAIT(x_empty(xs), ph ^ 1);
                     if (half == 0) RM_TR(k.item, 2, cc);
@@ -833,7 +845,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     ++stage;
                 }
                 if (elect_one()) {
-                    if (alias) mma_commit(d_local);
+                    if (alias_multi) mma_commit(d_local);
                     mma_commit_mc(h_free, 0xff);
                     if (k.i == k.run.ntiles - 1) { mma_commit(d2_full(d2b)); RM_PS(k.item, 25); }
                 }
@@ -1125,15 +1137,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 // A CTA with tiles in layer l has waited for exactly that before normalising; a CTA whose cluster has none
                 // (lists shorter than the number of clusters) would otherwise run through its empty layers at once, and its
                 // early arrivals would stand in for a slower CTA's.
-                if (run.ntiles == 0 && !a.per_item && l > 0 && !gave_up) {
-                    const int target = a.sync_base[b] + n_ctas * l;
-                    bool ok = false;
-                    for (uint32_t i = 0; i < (1u << 21); ++i) {
-                        if (ld_acquire_gpu(a.sync + b) >= target) { ok = true; break; }
-                        if ((i & 255u) == 255u && (*sAbort || ld_acquire_gpu(a.sync + SYNC_ABORT))) break;
-                    }
-                    if (!ok) { if (!*sAbort && !ld_acquire_gpu(a.sync + SYNC_ABORT)) timed_out(__LINE__); gave_up = true; *sAbort = 1; }
-                }
+                if (run.ntiles == 0 && !a.per_item && l > 0 && !gave_up)
+                    gave_up = counter_wait_slow(a.sync + b, a.sync_base[b] + n_ctas * l, __LINE__, sAbort, a.sync, a.status);
                 red_release_gpu(a.per_item ? a.sync + SYNC_ITEM + item : a.sync + b, 1);
                 RM_PS(item, 7);
             }
