@@ -326,8 +326,9 @@ __device__ __forceinline__ void walk_tiles(const Env& env, int B, FS stop, FG ga
     }
 }
 
-// Shared memory: a fixed head (item counts, the tiles' neuron ids, barriers), the weight ring, then the h tile and the x
-// ring, which share what is left: the h tile is sized for the largest tile of the step, the x ring takes the rest.
+// Shared memory: a fixed head (item counts, the tiles' neuron ids, barriers), the exchange area of the GLU, the weight
+// ring (six or eight stages, decided at the start of the launch), then the h tile and the x ring, which share what is
+// left: the h tile is sized for the largest tile of the step; the x ring takes the rest, or lies over the h tile.
 template <int HS8>
 struct Geo {
     static constexpr int H = 8 * HS8;
