@@ -53,8 +53,10 @@ constexpr int NTHREADS = 608;          // warps: 0-7 epilogue and normalisation,
 constexpr int W_LOAD0 = 8, W_MMA = 12, W_X0 = 13, W_PF = 17, W_WATCH = 18;
 constexpr int SYNC_ABORT = MAXB;       // sync[0..MAXB): per-episode arrival counters; sync[MAXB]: abort flag
 constexpr int SYNC_COPY = 32;          // sync[32..32+MAXB): per-episode counters of the CTAs that have copied r_in into r
+constexpr int SYNC_READ = 48;          // sync[48..48+MAXB): per-episode counters of the CTAs that have read r for a layer's normalisation
 constexpr int SYNC_ITEM = 64;          // sync[64..64+MAX_ITEMS): batches count the arrivals of every (layer, episode) by itself
-constexpr int SYNC_BYTES = (SYNC_ITEM + 512) * 4;
+constexpr int SYNC_RITEM = SYNC_ITEM + MAX_ITEMS;      // ... and the CTAs that have read the item's input rows
+constexpr int SYNC_BYTES = (SYNC_RITEM + MAX_ITEMS) * 4;
 
 struct PArgs {
     const __nv_bfloat16* packed[MAXL];
@@ -935,6 +937,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
             stop = named_barrier_or(1, 256, gave_up || *sAbort);
             const long long n4 = RM_CLK();
             if (warp == 0 && lane < CS) mbar_arrive_remote(map_to_rank(x_ready(slot), lane));
+            // This CTA's reads of the item's input rows are complete (their values went into the sums above).  The adds
+            // of the item's OWN results go into the same rows, and a faster cluster's adds wait for this count.
+            if (et == 32) red_release_gpu(a.per_item ? a.sync + SYNC_RITEM + item : a.sync + SYNC_READ + b, 1);
             if (et == 0) { RM_PS(item, 9); RM_PC(item, 26, n1 - n0); RM_PC(item, 27, n2 - n1); RM_PC(item, 28, n3 - n2); RM_PC(item, 29, n4 - n3); RM_PC(item, 30, RM_CLK() - n4); }
         };
         // x of a non-empty item is prepared right before the item's own tiles, or one non-empty item earlier when the
@@ -1095,9 +1100,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 // the item's down products are complete: add this CTA's [T x H/8] part to the residual stream
                 const int d2b = ND2 == 2 ? (ni & 1) : 0, nu = ND2 == 2 ? (ni >> 1) : ni;
                 ++ni;
+                // The adds below go into the rows that every cluster has read for this item's normalisation.  Nothing else
+                // orders a slower cluster's reads before them: wait for the count of the CTAs that have read.  (The
+                // load is issued before the wait for the products, so its round trip is over by then.)
+                const bool ext = item_ext(env, l);
+                const int* rctr = a.per_item ? a.sync + SYNC_RITEM + item : a.sync + SYNC_READ + b;
+                const int rtarget = a.per_item ? n_ctas : a.sync_base[b] + n_ctas * (l + 1);
+                const int rseen = lane == 0 && !ext ? ld_acquire_gpu(rctr) : rtarget;
                 WAIT(d2_full(d2b), nu & 1);
                 tc_fence_after();
                 if (et == 0) RM_PS(item, 5);
+                if (rseen < rtarget && !gave_up) gave_up = counter_wait_slow(rctr, rtarget, __LINE__, sAbort, a.sync, a.status);
+                __syncwarp();
                 if (l == 0 && pre) {
                     // r has to hold its copy of r_in before anything is added to it
                     if (lane == 0 && !gave_up) {
@@ -1140,6 +1154,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 // early arrivals would stand in for a slower CTA's.
                 if (run.ntiles == 0 && !a.per_item && l > 0 && !gave_up)
                     gave_up = counter_wait_slow(a.sync + b, a.sync_base[b] + n_ctas * l, __LINE__, sAbort, a.sync, a.status);
+                // (CTAs that have not normalised this item -- no tiles, or x from the caller -- count as readers here)
+                if (run.ntiles == 0 || item_ext(env, l))
+                    red_release_gpu(a.per_item ? a.sync + SYNC_RITEM + item : a.sync + SYNC_READ + b, 1);
                 red_release_gpu(a.per_item ? a.sync + SYNC_ITEM + item : a.sync + b, 1);
                 RM_PS(item, 7);
             }
