@@ -332,7 +332,7 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
     const size_t n_bytes = (size_t)B * T * g.H * sizeof(float);
     const size_t r_bytes = align_up(n_bytes, 256);
     char* layer_ws = static_cast<char*>(ws) + 4 * r_bytes;
-    if (use_persist(ctx, B, T, count_dev != nullptr, true) && an.mode == RM_ANCHOR_NONE && !an.gate) {
+    if (use_persist(ctx, B, T, count_dev != nullptr, true)) {
         // the whole step in one launch: the layers add into r_out in place (the kernel starts it as a copy of r_in)
         rm_step_args sa{};
         sa.packed_layers = packed_layers;
@@ -350,6 +350,11 @@ static int step_device(rm_ctx* ctx, const void* const* packed_layers, const floa
         sa.record_scale = record_scale;
         sa.B = B;
         sa.T = T;
+        sa.anchor_mode = an.mode;
+        sa.y_anchor = an.y;
+        sa.h_anchor = an.h;
+        sa.h_stride = an.h_stride;
+        sa.gate = an.gate;
         ctx->last_variant = 5;
         return rm_launch_step_persist(ctx, sa, persist_ws(ctx, ws, B, T), s);
     }

@@ -165,6 +165,11 @@ struct rm_step_args {
     const float* record_scale;             // [L, I] or NULL
     int B, T;
     const void* x_ext;                     // [T,H] bf16: layer 0 takes this as its input instead of normalising r (L = 1 calls)
+    int anchor_mode;                       // Eq. 4: RM_ANCHOR_NONE / _WRITE / _UPDATE, with the whole stack's state
+    float* y_anchor;                       // [L,B,T,H]
+    float* h_anchor;                       // [L,B,I,h_stride]
+    int64_t h_stride;
+    const float* gate;                     // [L,B,H] output gate, or NULL
 };
 int rm_persist_init(rm_ctx* ctx);
 bool rm_persist_supported(const rm_ctx* ctx, int B, int T);

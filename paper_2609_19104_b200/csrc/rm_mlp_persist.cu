@@ -80,6 +80,12 @@ struct PArgs {
                                        // counter per episode could not tell the layers apart); else per episode, never cleared
     int x_ext;                         // layer 0 takes x from the caller's buffer (single-layer entry): no normalisation
     int pf_bytes;                      // weight bytes a CTA may have asked into L2 ahead of its loaders (0: no prefetch)
+    // Anchor-relative update (Eq. 4) and output gate; read by the EQ4 instantiation only
+    int anchor_mode;                   // RM_ANCHOR_NONE / _WRITE / _UPDATE
+    float* y_anchor;                   // [L,B,T,H] fp32, pre-gate: accumulated (from zeros) in a write step, read in an update step
+    float* h_anchor;                   // [L,B,I,h_stride] fp32, neuron-major: written in a write step, read in an update step
+    int64_t h_stride;
+    const float* gate;                 // [L,B,H] fp32 or NULL (= 1)
 };
 
 #ifdef RM_PHASE_TIMING
@@ -359,7 +365,7 @@ struct Geo {
     static_assert(TOTAL <= 232448, "buffers exceed the shared memory of a CTA");
 };
 
-template <int HS8>
+template <int HS8, bool EQ4>
 __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant__ PArgs a,
                                                           const __grid_constant__ CUtensorMap tmXext) {
     using G = Geo<HS8>;
@@ -399,6 +405,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
     const int T = a.T, L = a.L, B = a.B, I = a.I;
     const int n_ctas = (int)gridDim.x;
     const int n_items = L * B;
+    const int anchor_mode = EQ4 ? a.anchor_mode : (int)RM_ANCHOR_NONE;
 
     {
         const int cap = (int)(a.list_cap < (int64_t)I ? a.list_cap : (int64_t)I);
@@ -975,6 +982,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     n = list ? __ldg(list + t0 + off + ni_loc) : t0 + off + ni_loc;
                     if (n < 0 || n >= I) n = -1;
                 }
+                const int tok0 = 8 * (ch * 4 + (fin ? 0 : 2) + (isup ? 1 : 0));     // first of this lane's 8 tokens (see below)
+                // update steps: the neuron's anchor values for this lane's tokens, asked for before the products are waited for
+                float4 ha0 = make_float4(0.f, 0.f, 0.f, 0.f), ha1 = ha0;
+                float* hap = nullptr;
+                if (EQ4 && anchor_mode != RM_ANCHOR_NONE && n >= 0) {
+                    hap = a.h_anchor + (((size_t)l * B + b) * I + n) * a.h_stride + tok0;
+                    if (anchor_mode == RM_ANCHOR_UPDATE) {
+                        if (tok0 < T) ha0 = __ldcg(reinterpret_cast<const float4*>(hap));
+                        if (tok0 + 4 < T) ha1 = __ldcg(reinterpret_cast<const float4*>(hap) + 1);
+                    }
+                }
                 WAIT(d1_full(buf), (seq >> 1) & 1);
                 tc_fence_after();
                 if (et == 0 && i == 0) RM_PS(item, 2);
@@ -1004,7 +1022,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 // lane pair (2 i, 2 i + 1) = (gate row, up row) of neuron i for these 16 tokens: the even lane finishes
                 // the first 8 of them, the odd lane the last 8
                 float hv[8];
-                const int tok0 = 8 * (ch * 4 + (fin ? 0 : 2) + (isup ? 1 : 0));     // first of this lane's 8 tokens
                 {
                     float gg[8], uu[8], e[8];
 #pragma unroll
@@ -1033,6 +1050,19 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                         rec += sRec[NT + ni_loc] + sRec[2 * NT + ni_loc] + sRec[3 * NT + ni_loc];
                         const float sc = a.record_scale ? a.record_scale[(size_t)l * I + n] : 1.f;
                         a.record[(size_t)b * a.rec_b_stride + (size_t)l * I + n] = a.record_scale ? rec * sc : rec;
+                    }
+                }
+                if (EQ4 && hap) {
+                    // Eq. 4: the anchor step retains h (fp32, before the split); an update step multiplies the down rows
+                    // with h - h_a.  (The record above is that of h itself.)
+                    if (anchor_mode == RM_ANCHOR_WRITE) {
+                        if (tok0 < T) *reinterpret_cast<float4*>(hap) = make_float4(hv[0], hv[1], hv[2], hv[3]);
+                        if (tok0 + 4 < T) *(reinterpret_cast<float4*>(hap) + 1) = make_float4(hv[4], hv[5], hv[6], hv[7]);
+                    } else {
+                        const float hs[8] = {ha0.x, ha0.y, ha0.z, ha0.w, ha1.x, ha1.y, ha1.z, ha1.w};
+#pragma unroll
+                        for (int r = 0; r < 8; ++r)
+                            if (tok0 + r < T) hv[r] -= hs[r];
                     }
                 }
                 const long long e3 = RM_CLK();
@@ -1096,6 +1126,24 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 }
             }
             if (stop) break;
+            // Eq. 4, update step: the layer's output also holds gate * y_a.  The token rows c, c + NC, ... are this cluster's
+            // share of that term, the columns of slice j this CTA's; it is added next to the CTA's own partial sums.
+            const bool upd = EQ4 && anchor_mode == RM_ANCHOR_UPDATE;
+            const bool ext = item_ext(env, l);
+            const int* rctr = a.per_item ? a.sync + SYNC_RITEM + item : a.sync + SYNC_READ + b;
+            const int rtarget = a.per_item ? n_ctas : a.sync_base[b] + n_ctas * (l + 1);
+            if (run.ntiles == 0 && upd) {
+                // no tiles, yet rows to add to: the same order of events as for a CTA with tiles (see the arrival below)
+                if (et == 0 && !gave_up) {
+                    if (!a.per_item && l > 0)
+                        gave_up = counter_wait_slow(a.sync + b, a.sync_base[b] + n_ctas * l, __LINE__, sAbort, a.sync, a.status);
+                    red_release_gpu(const_cast<int*>(rctr), 1);
+                    if (!gave_up) gave_up = counter_wait_slow(rctr, rtarget, __LINE__, sAbort, a.sync, a.status);
+                    if (l == 0 && pre && !gave_up)                 // r holds its copy of r_in
+                        gave_up = counter_wait_slow(a.sync + SYNC_COPY + b, a.copy_base[b] + pre, __LINE__, sAbort, a.sync, a.status);
+                }
+                stop = named_barrier_or(1, 256, gave_up || *sAbort);
+            }
             if (run.ntiles > 0) {
                 // the item's down products are complete: add this CTA's [T x H/8] part to the residual stream
                 const int d2b = ND2 == 2 ? (ni & 1) : 0, nu = ND2 == 2 ? (ni >> 1) : ni;
@@ -1103,9 +1151,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                 // The adds below go into the rows that every cluster has read for this item's normalisation.  Nothing else
                 // orders a slower cluster's reads before them: wait for the count of the CTAs that have read.  (The
                 // load is issued before the wait for the products, so its round trip is over by then.)
-                const bool ext = item_ext(env, l);
-                const int* rctr = a.per_item ? a.sync + SYNC_RITEM + item : a.sync + SYNC_READ + b;
-                const int rtarget = a.per_item ? n_ctas : a.sync_base[b] + n_ctas * (l + 1);
                 const int rseen = lane == 0 && !ext ? ld_acquire_gpu(rctr) : rtarget;
                 WAIT(d2_full(d2b), nu & 1);
                 tc_fence_after();
@@ -1124,7 +1169,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     }
                     __syncwarp();
                 }
-                float* rb = a.r + (size_t)b * T * H + j * HS8 + q4 * 32 + lane;
+                const size_t col0 = (size_t)j * HS8 + q4 * 32 + lane;
+                float* rb = a.r + (size_t)b * T * H + col0;
+                // Eq. 4: the sum is scaled by the output gate of its column on the way into r; the anchor step also
+                // accumulates the sum as it is into y_a (cleared by the host before the launch)
+                float gt0 = 1.f, gt1 = 1.f;
+                if (EQ4 && a.gate) {
+                    const float* gp = a.gate + ((size_t)l * B + b) * H + col0;
+                    gt0 = __ldg(gp);
+                    if (NMB == 2) gt1 = __ldg(gp + 128);
+                }
+                float* yb = EQ4 && anchor_mode == RM_ANCHOR_WRITE ? a.y_anchor + ((size_t)l * B + b) * T * H + col0 : nullptr;
                 // (rolled loops over 8 token columns at a time: this code runs once per layer, and the smaller it is the
                 // less of the other roles' loops it pushes out of the instruction cache)
 #pragma unroll 1
@@ -1134,29 +1189,45 @@ __global__ void __launch_bounds__(NTHREADS, 1) step_kernel(const __grid_constant
                     const uint32_t col = tmem + G::D2_COL + d2b * (2 * NTOK) + mb * (2 * NTOK) + ch * 32 + c8 + ((uint32_t)(q4 * 32) << 16);
                     tmem_ld8(col, hi);
                     tmem_ld8(col + NTOK, lo);
-                    float* dst = rb + (size_t)(ch * 32 + c8) * H + mb * 128;
+                    const size_t o = (size_t)(ch * 32 + c8) * H + mb * 128;
+                    const float gt = EQ4 ? (mb ? gt1 : gt0) : 1.f;
 #pragma unroll
                     for (int r = 0; r < 8; ++r)
-                        if (ch * 32 + c8 + r < T) red_add_f32(dst + (size_t)r * H, hi[r] + lo[r]);
+                        if (ch * 32 + c8 + r < T) {
+                            const float y = hi[r] + lo[r];
+                            red_add_f32(rb + o + (size_t)r * H, EQ4 ? gt * y : y);
+                            if (EQ4 && yb) red_add_f32(yb + o + (size_t)r * H, y);
+                        }
                 }
                 tc_fence_before();
                 mbar_arrive(d2_empty(d2b));
                 if (et == 0) RM_PS(item, 6);
-                // no fence per thread: the barrier orders every thread's adds before thread 0's release on the counter
-                // below, and a release is cumulative (the pattern of a grid-wide barrier: sync, then one thread fences)
-                stop = named_barrier_or(1, 256, gave_up || *sAbort);
             }
+            if (upd && !stop) {
+                const int nrows = c < T ? (T - c + NC - 1) / NC : 0;
+                const float* ya = a.y_anchor + ((size_t)l * B + b) * T * H + (size_t)j * HS8;
+                const float* gp = a.gate ? a.gate + ((size_t)l * B + b) * H + (size_t)j * HS8 : nullptr;
+                float* rr = a.r + (size_t)b * T * H + (size_t)j * HS8;
+                for (int e = et; e < nrows * HS8; e += 256) {
+                    const int ri = e / HS8, cc = e - ri * HS8;
+                    const size_t o = (size_t)(c + ri * NC) * H + cc;
+                    red_add_f32(rr + o, (gp ? __ldg(gp + cc) : 1.f) * __ldcg(ya + o));
+                }
+            }
+            // no fence per thread: the barrier orders every thread's adds before thread 0's release on the counter
+            // below, and a release is cumulative (the pattern of a grid-wide barrier: sync, then one thread fences)
+            if (run.ntiles > 0 || upd) stop = named_barrier_or(1, 256, gave_up || *sAbort);
             if (et == 0) {
                 // The episode's counter adds up the arrivals of all layers, and "n_ctas (l + 1) arrivals" means "every CTA has
                 // added its part of layer l" only if nobody arrives for layer l before every CTA has arrived for layer l - 1.
                 // A CTA with tiles in layer l has waited for exactly that before normalising; a CTA whose cluster has none
                 // (lists shorter than the number of clusters) would otherwise run through its empty layers at once, and its
                 // early arrivals would stand in for a slower CTA's.
-                if (run.ntiles == 0 && !a.per_item && l > 0 && !gave_up)
+                const bool empty = run.ntiles == 0 && !upd;
+                if (empty && !a.per_item && l > 0 && !gave_up)
                     gave_up = counter_wait_slow(a.sync + b, a.sync_base[b] + n_ctas * l, __LINE__, sAbort, a.sync, a.status);
                 // (CTAs that have not normalised this item -- no tiles, or x from the caller -- count as readers here)
-                if (run.ntiles == 0 || item_ext(env, l))
-                    red_release_gpu(a.per_item ? a.sync + SYNC_RITEM + item : a.sync + SYNC_READ + b, 1);
+                if (empty || (ext && run.ntiles > 0)) red_release_gpu(const_cast<int*>(rctr), 1);
                 red_release_gpu(a.per_item ? a.sync + SYNC_ITEM + item : a.sync + b, 1);
                 RM_PS(item, 7);
             }
@@ -1209,7 +1280,7 @@ int make_x_map(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t cols) {
 
 template <int HS8>
 int query_clusters(int* out) {
-    auto kern = step_kernel<HS8>;
+    auto kern = step_kernel<HS8, false>;
     RM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<HS8>::TOTAL));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CS * 32);
@@ -1226,11 +1297,11 @@ int query_clusters(int* out) {
     return RM_OK;
 }
 
-template <int HS8>
+template <int HS8, bool EQ4>
 int launch(rm_ctx* ctx, const PArgs& a, const CUtensorMap& tmXext, int n_clusters, cudaStream_t s) {
     static rm_smem_configured configured = {};
     if (!configured.covers(ctx->device, Geo<HS8>::TOTAL)) {
-        RM_CUDA_TRY(cudaFuncSetAttribute(step_kernel<HS8>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<HS8>::TOTAL));
+        RM_CUDA_TRY(cudaFuncSetAttribute(step_kernel<HS8, EQ4>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<HS8>::TOTAL));
         configured.set(ctx->device, Geo<HS8>::TOTAL);
     }
     cudaLaunchConfig_t cfg = {};
@@ -1245,7 +1316,7 @@ int launch(rm_ctx* ctx, const PArgs& a, const CUtensorMap& tmXext, int n_cluster
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, step_kernel<HS8>, a, tmXext));
+    RM_CUDA_TRY(cudaLaunchKernelEx(&cfg, step_kernel<HS8, EQ4>, a, tmXext));
     ctx->launches++;
     return RM_OK;
 }
@@ -1343,7 +1414,18 @@ int rm_launch_step_persist(rm_ctx* ctx, const rm_step_args& sa, void* ws, cudaSt
     }
     for (int b = 0; b < MAXB; ++b) { a.sync_base[b] = ctx->persist_sync_base[b]; a.copy_base[b] = ctx->persist_copy_base[b]; }
     for (int b = 0; b < sa.B; ++b) { ctx->persist_sync_base[b] += nc_ctas * sa.L; ctx->persist_copy_base[b] += pre; }
-    const int rc = g.H == 1024 ? launch<128>(ctx, a, tm_ext, nc, s) : launch<256>(ctx, a, tm_ext, nc, s);
+    // (the instantiation without Eq. 4 and gate is the one the plain steps run: it carries none of their code)
+    const bool eq4 = sa.anchor_mode != RM_ANCHOR_NONE || sa.gate != nullptr;
+    a.anchor_mode = sa.anchor_mode;
+    a.y_anchor = sa.y_anchor;
+    a.h_anchor = sa.h_anchor;
+    a.h_stride = sa.h_stride;
+    a.gate = sa.gate;
+    // the anchor step's sums are accumulated by the CTAs' atomics: start them from zero
+    if (sa.anchor_mode == RM_ANCHOR_WRITE)
+        RM_CUDA_TRY(cudaMemsetAsync(sa.y_anchor, 0, (size_t)sa.L * sa.B * sa.T * g.H * sizeof(float), s));
+    const int rc = g.H == 1024 ? (eq4 ? launch<128, true>(ctx, a, tm_ext, nc, s) : launch<128, false>(ctx, a, tm_ext, nc, s))
+                               : (eq4 ? launch<256, true>(ctx, a, tm_ext, nc, s) : launch<256, false>(ctx, a, tm_ext, nc, s));
     if (rc != RM_OK) ctx->persist_sync_dirty = 1;               // nothing ran: the counters are behind the host's count
     return rc;
 }

@@ -51,8 +51,8 @@ def lib_const(name):
     return getattr(rm, name)
 
 
-@pytest.mark.parametrize("path,variant,max_clusters", [(1, 0, 0), (2, 0, 0), (2, 1, 3), (2, 2, 3), (2, 3, 3), (2, 4, 0), (2, 4, 3)])
-@pytest.mark.parametrize("H,I,T,L,B", [(1024, 1024, 51, 3, 2), (2048, 512, 32, 2, 1)])
+@pytest.mark.parametrize("path,variant,max_clusters", [(1, 0, 0), (2, 0, 0), (2, 1, 3), (2, 2, 3), (2, 3, 3), (2, 4, 0), (2, 4, 3), (2, 5, 0), (2, 5, 3)])
+@pytest.mark.parametrize("H,I,T,L,B", [(1024, 1024, 51, 3, 2), (2048, 512, 32, 2, 1), (1024, 600, 51, 4, 1)])
 def test_anchor_write_then_update_matches_the_oracle(lib, path, variant, max_clusters, H, I, T, L, B):
     import torch
     w, model, r_a, r_t, gate, lists = make_case(lib, H, I, T, L, B)
@@ -93,6 +93,37 @@ def test_anchor_write_then_update_matches_the_oracle(lib, path, variant, max_clu
     ctx.rm_action_expert_step_ex(model.packed, dev(r_a), dev(idx), dev(cnt), I, out_same, lib_const("RM_ANCHOR_UPDATE"),
                                  y_an, h_an, h_stride, out_gate=dev(gate), B=B, T=T)
     assert_close(out_same.cpu().numpy(), out_a.cpu().numpy(), "update on the anchor's input")
+    if variant:
+        assert ctx.rm_get_info("last_variant") == variant      # the kernel family asked for is the one that ran
+    assert ctx.rm_device_status() == 0
+    model.close()
+
+
+@pytest.mark.parametrize("B", [1, 2])
+def test_update_with_lists_shorter_than_the_number_of_clusters(lib, B):
+    """Whole-step kernel, update steps whose lists give most clusters nothing to compute in most layers (some lists
+    empty): every cluster still adds its share of gate * y_a, in layer order."""
+    import torch
+    H, I, T, L = 1024, 256, 51, 6
+    w, model, r_a, r_t, gate, _ = make_case(lib, H, I, T, L, B)
+    ctx = model.ctx
+    ctx.rm_set_option("variant", 5)
+    h_stride = 52
+    out_a, y_an, h_an, _ = run_write(model, w, r_a, gate, B, h_stride)
+    lists = [[np.flatnonzero(wl.uniform(wl.tensor_key(7, 94, l, 2, b), I) < (0.0 if (l + b) % 3 == 1 else 0.02)).astype(np.int32)
+              for l in range(L)] for b in range(B)]
+    assert max(len(s) for per_b in lists for s in per_b) < 15
+    idx, cnt = lists_to_padded([s for per_b in lists for s in per_b], I)
+    out_t = torch.empty(B, T, H, dtype=torch.float32, device="cuda")
+    for _ in range(3):                                    # the counters carry over from launch to launch
+        ctx.rm_action_expert_step_ex(model.packed, dev(r_t), dev(idx), dev(cnt), I, out_t, lib_const("RM_ANCHOR_UPDATE"),
+                                     y_an, h_an, h_stride, out_gate=dev(gate), B=B, T=T)
+    assert ctx.rm_get_info("last_variant") == 5
+    for b in range(B):
+        _, want_y, want_h, _ = oracle.anchor_step_write(model.Wg, model.Wu, model.Wd, r_a[b], gate[:, b])
+        i_b, c_b = lists_to_padded(lists[b], I)
+        want = oracle.anchor_step_update(model.Wg, model.Wu, model.Wd, r_t[b], i_b, c_b, want_y, want_h, gate[:, b])
+        assert_close(out_t.cpu().numpy()[b], want, f"update step with short lists, episode {b}")
     assert ctx.rm_device_status() == 0
     model.close()
 
