@@ -24,6 +24,9 @@
 // into the cluster's own copy of x in global memory, tell one another through remote mbarrier arrivals, and
 // stream x from there.
 //
+// The EQ4 instantiation adds the anchor-relative update (Eq. 4) and the output gate: the anchor step retains h per neuron
+// and the ungated sums y_a; an update step multiplies the down rows with h - h_a and adds gate * y_a.
+//
 // Every wait is bounded; a wait that runs out records RM_ERR_TIMEOUT (with its source line), raises the launch's
 // abort flag, and every role leaves its loop at the next check.  CTAs leave together (cluster barrier at the end).
 #include <cuda.h>
