@@ -124,6 +124,12 @@ def test_update_with_lists_shorter_than_the_number_of_clusters(lib, B):
         i_b, c_b = lists_to_padded(lists[b], I)
         want = oracle.anchor_step_update(model.Wg, model.Wu, model.Wd, r_t[b], i_b, c_b, want_y, want_h, gate[:, b])
         assert_close(out_t.cpu().numpy()[b], want, f"update step with short lists, episode {b}")
+    # the same step in place (input and output in one buffer), compared within the parity bound: the order of the adds
+    # differs from run to run, so the rows are not bit-identical
+    buf = torch.from_numpy(r_t).cuda()
+    ctx.rm_action_expert_step_ex(model.packed, buf, dev(idx), dev(cnt), I, buf, lib_const("RM_ANCHOR_UPDATE"),
+                                 y_an, h_an, h_stride, out_gate=dev(gate), B=B, T=T)
+    assert_close(buf.cpu().numpy(), out_t.cpu().numpy(), "update step in place")
     assert ctx.rm_device_status() == 0
     model.close()
 
