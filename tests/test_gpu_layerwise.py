@@ -3,7 +3,7 @@
 A dense (or anchored) step through all 18 layers is ill-conditioned as a whole: every layer re-quantises x to bf16,
 and a one-ulp difference early in the stack is carried to the output (test_oracle_pins.py::
 test_dense_stack_amplifies_one_ulp shows the oracle doing it to itself).  The free-running step outputs are therefore
-judged with a small allowance for outliers (harness.assert_close(deep_dense=True)).  What is well conditioned is a
+compared with a small allowance for outliers (harness.assert_close(deep_dense=True)).  What is well conditioned is a
 single layer: here every layer of those stacks gets the ORACLE's own x_l and r_l as its input, runs through
 rm_sparse_mlp (or a one-layer rm_action_expert_step_ex for the anchored schedule), and must meet
 |err| <= 2e-2 + 1e-2 |ref| on every element and 5e-3 in relative L2, with no allowance.
